@@ -1,0 +1,224 @@
+"""ctypes marshalling for the C++ checker in ``aq_oracle.cpp`` (no arithmetic here)."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from typing import Optional, Tuple
+
+import numpy as np
+
+_DIR = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_DIR, "aq_oracle.cpp")
+_LIB = os.path.join(_DIR, "libaq_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the checker with g++ (-O3, OpenMP); returns the library path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["g++", "-O3", "-march=native", "-fopenmp", "-std=c++17", "-shared",
+                               "-fPIC", _SRC, "-o", tmp])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        L = _lib
+        L.orc_half_to_float.restype = C.c_float
+        L.orc_half_to_float.argtypes = [C.c_uint16]
+        L.orc_double_to_half.restype = C.c_uint16
+        L.orc_double_to_half.argtypes = [C.c_double]
+        L.orc_float_to_half.restype = C.c_uint16
+        L.orc_float_to_half.argtypes = [C.c_float]
+        L.orc_pow2_exponent.restype = C.c_int
+        L.orc_pow2_exponent.argtypes = [C.c_float, C.c_int]
+        L.orc_absmax.restype = C.c_float
+        L.orc_layer_exponent.restype = C.c_int
+        L.orc_token_select.restype = C.c_int
+        L.orc_int_gemm.restype = C.c_longlong
+        L.orc_linear.restype = C.c_longlong
+        L.orc_progressive_ratio.restype = C.c_double
+        L.orc_progressive_ratio.argtypes = [C.c_double, C.c_int]
+        L.orc_num_threads.restype = C.c_int
+    return _lib
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _c(a, dtype) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    assert a.dtype == dtype, (a.dtype, dtype)
+    return a
+
+
+def _half_bits(a) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.float16
+    return a.view(np.uint16)
+
+
+def num_groups(K: int, group: int) -> int:
+    return 1 if group == 0 else K // group
+
+
+def half_to_float(bits: int) -> float:
+    return float(lib().orc_half_to_float(int(bits)))
+
+
+def double_to_half(d: float) -> int:
+    return int(lib().orc_double_to_half(float(d)))
+
+
+def float_to_half(f: float) -> int:
+    return int(lib().orc_float_to_half(float(f)))
+
+
+def pow2_exponent(a: float, bits: int) -> int:
+    return int(lib().orc_pow2_exponent(C.c_float(a), bits))
+
+
+def progressive_ratio(beta: float, m: int) -> float:
+    return float(lib().orc_progressive_ratio(beta, m))
+
+
+def num_threads() -> int:
+    return int(lib().orc_num_threads())
+
+
+def quantize_weights(w: np.ndarray, group: int) -> Tuple[np.ndarray, np.ndarray]:
+    """fp16 [N,K] -> (int8 codes [N,K], fp16 scales [N,G])."""
+    N, K = w.shape
+    G = num_groups(K, group)
+    codes = np.empty((N, K), np.int8)
+    scales = np.empty((N, G), np.float16)
+    lib().orc_quantize_weights(_p(_half_bits(w)), N, K, group, _p(codes), _p(scales.view(np.uint16)))
+    return codes, scales
+
+
+def pack_w4(codes: np.ndarray) -> np.ndarray:
+    codes = _c(codes, np.int8)
+    N, K = codes.shape
+    out = np.empty((N, K // 2), np.uint8)
+    lib().orc_pack_w4(_p(codes), N, K, _p(out))
+    return out
+
+
+def unpack_w4(packed: np.ndarray) -> np.ndarray:
+    packed = _c(packed, np.uint8)
+    N, K2 = packed.shape
+    out = np.empty((N, K2 * 2), np.int8)
+    lib().orc_unpack_w4(_p(packed), N, K2 * 2, _p(out))
+    return out
+
+
+def token_select(scores: np.ndarray, n_keep: int) -> np.ndarray:
+    scores = _c(scores, np.float32)
+    idx = np.empty((n_keep,), np.int32)
+    rc = lib().orc_token_select(_p(scores), scores.shape[0], n_keep, _p(idx))
+    if rc != 0:
+        raise ValueError("n_keep out of range")
+    return idx
+
+
+def token_compact(x: np.ndarray, idx: np.ndarray) -> np.ndarray:
+    idx = _c(idx, np.int32)
+    M, K = x.shape
+    out = np.empty((idx.shape[0], K), np.float16)
+    lib().orc_token_compact(_p(_half_bits(x)), K, _p(idx), idx.shape[0], _p(out.view(np.uint16)))
+    return out
+
+
+def absmax(x: np.ndarray, row_idx: Optional[np.ndarray] = None) -> float:
+    M_in, K = x.shape
+    ri = None if row_idx is None else _c(row_idx, np.int32)
+    M = M_in if ri is None else ri.shape[0]
+    return float(lib().orc_absmax(_p(_half_bits(x)), K, _p(ri), M))
+
+
+def layer_exponent(x: np.ndarray, bits: int, row_idx: Optional[np.ndarray] = None) -> int:
+    M_in, K = x.shape
+    ri = None if row_idx is None else _c(row_idx, np.int32)
+    M = M_in if ri is None else ri.shape[0]
+    return int(lib().orc_layer_exponent(_p(_half_bits(x)), K, _p(ri), M, bits))
+
+
+def quantize_act(x: np.ndarray, bits: int, e: int, row_idx: Optional[np.ndarray] = None) -> np.ndarray:
+    M_in, K = x.shape
+    ri = None if row_idx is None else _c(row_idx, np.int32)
+    M = M_in if ri is None else ri.shape[0]
+    q = np.empty((M, K), np.int8)
+    lib().orc_quantize_act(_p(_half_bits(x)), K, _p(ri), M, bits, e, _p(q))
+    return q
+
+
+def int_gemm(q: np.ndarray, c: np.ndarray, group: int) -> np.ndarray:
+    """int8 [M,K] x int8 [N,K] -> int32 [M,N,G]; raises if an int32 sum overflowed."""
+    q = _c(q, np.int8)
+    c = _c(c, np.int8)
+    M, K = q.shape
+    N = c.shape[0]
+    G = num_groups(K, group)
+    acc = np.empty((M, N, G), np.int32)
+    ovf = lib().orc_int_gemm(_p(q), _p(c), M, N, K, group, _p(acc))
+    if ovf:
+        raise OverflowError(f"{ovf} int32 accumulators overflowed")
+    return acc
+
+
+def dequant(acc: np.ndarray, scales: np.ndarray, e: int) -> np.ndarray:
+    acc = _c(acc, np.int32)
+    M, N, G = acc.shape
+    scales = np.ascontiguousarray(scales)
+    assert scales.shape == (N, G) and scales.dtype == np.float16
+    y = np.empty((M, N), np.float16)
+    lib().orc_dequant(_p(acc), _p(scales.view(np.uint16)), e, M, N, G, _p(y.view(np.uint16)))
+    return y
+
+
+def linear_sampled(q, c, scales, e: int, group: int, rows, cols):
+    """(int32 acc [count,G], fp16 y [count]) at the given output positions."""
+    q = _c(q, np.int8)
+    c = _c(c, np.int8)
+    rows = _c(rows, np.int32)
+    cols = _c(cols, np.int32)
+    M, K = q.shape
+    N = c.shape[0]
+    G = num_groups(K, group)
+    scales = np.ascontiguousarray(scales)
+    assert scales.shape == (N, G) and scales.dtype == np.float16
+    cnt = rows.shape[0]
+    acc = np.empty((cnt, G), np.int32)
+    y = np.empty((cnt,), np.float16)
+    lib().orc_linear_sampled(_p(q), _p(c), _p(scales.view(np.uint16)), e, N, K, group, _p(rows),
+                             _p(cols), cnt, _p(acc), _p(y.view(np.uint16)))
+    return acc, y
+
+
+def linear(x, codes, scales, bits: int, group: int, scale_mode: int = 0, clip_shift_or_exp: int = 0,
+           row_idx=None, want_acc: bool = False):
+    """Whole layer. Returns dict(y fp16 [M,N], q int8 [M,K], e int, acc int32 [M,N,G] or None)."""
+    M_in, K = x.shape
+    ri = None if row_idx is None else _c(row_idx, np.int32)
+    M = M_in if ri is None else ri.shape[0]
+    codes = _c(codes, np.int8)
+    N = codes.shape[0]
+    G = num_groups(K, group)
+    scales = np.ascontiguousarray(scales)
+    assert scales.shape == (N, G) and scales.dtype == np.float16
+    y = np.empty((M, N), np.float16)
+    q = np.empty((M, K), np.int8)
+    acc = np.empty((M, N, G), np.int32) if want_acc else None
+    e = C.c_int32(0)
+    ovf = lib().orc_linear(_p(_half_bits(x)), K, _p(ri), M, bits, scale_mode, clip_shift_or_exp,
+                           _p(codes), _p(scales.view(np.uint16)), N, group, _p(y.view(np.uint16)),
+                           _p(q), _p(acc), C.byref(e))
+    if ovf:
+        raise OverflowError(f"{ovf} int32 accumulators overflowed")
+    return {"y": y, "q": q, "e": int(e.value), "acc": acc}

@@ -1,0 +1,406 @@
+"""Pins for the CPU checker: it is compared with things other than itself.
+
+Hand-worked fixtures (tests/golden), closed forms, invariants the quantizers must
+satisfy, brute force in Python integers on tiny inputs, library routines that the
+special cases reduce to (numpy's fp16 casts, torch's int64 matmul, numpy sorting), and
+a restatement of the packed-lane product of Algorithm 1 as a third route to the same
+integer sums.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2312_05693_b200 import inputs
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rows(name):
+    out = []
+    with open(os.path.join(GOLDEN, name)) as f:
+        for line in f:
+            line = line.strip()
+            if line and not line.startswith("#"):
+                out.append(line.split())
+    return out
+
+
+# ----------------------------------------------------------------------------- fp16
+def test_half_to_float_all_patterns_match_numpy():
+    bits = np.arange(65536, dtype=np.uint32).astype(np.uint16)
+    ref = bits.view(np.float16).astype(np.float32)
+    got = np.array([oracle.half_to_float(int(b)) for b in bits], dtype=np.float32)
+    nan = np.isnan(ref)
+    assert np.array_equal(np.isnan(got), nan)
+    assert np.array_equal(got[~nan].view(np.uint32), ref[~nan].view(np.uint32))
+
+
+def test_double_to_half_matches_numpy_rne():
+    rng = np.random.default_rng(7)
+    vals = np.concatenate([
+        rng.standard_normal(20000) * 10.0 ** rng.integers(-9, 6, 20000),
+        # exact ties between neighbouring halves, subnormals, overflow boundary
+        np.array([1.00048828125, 1.00146484375, 2047.5, 2048.5, 65504.0, 65519.999, 65520.0,
+                  65536.0, 1e9, 5.960464477539063e-08, 2.9802322387695312e-08,
+                  2.98023223876953e-08, 8.940696716308594e-08, 6.097555160522461e-05,
+                  6.103515625e-05, 0.0, -0.0, float("inf"), -float("inf")]),
+    ])
+    vals = np.concatenate([vals, -vals])
+    with np.errstate(over="ignore"):
+        ref = vals.astype(np.float64).astype(np.float16).view(np.uint16)
+    got = np.array([oracle.double_to_half(float(v)) for v in vals], dtype=np.uint16)
+    assert np.array_equal(got, ref)
+
+
+def test_half_round_trip_identity():
+    for b in list(range(0, 0x7C01)) + list(range(0x8000, 0xFC01)):
+        assert oracle.float_to_half(oracle.half_to_float(b)) == b
+
+
+# ------------------------------------------------------------------- layer exponent
+def test_pow2_exponent_hand_worked():
+    for bits, a, e in _rows("pow2_exponent_hand_worked.txt"):
+        assert oracle.pow2_exponent(float(a), int(bits)) == int(e), (bits, a, e)
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_pow2_exponent_is_smallest_covering_power(bits):
+    rng = np.random.default_rng(1)
+    qmax = 2 ** (bits - 1) - 1
+    a = (rng.random(20000) * 10.0 ** rng.integers(-6, 5, 20000)).astype(np.float32)
+    a = np.minimum(a, np.float32(65504.0))
+    for v in a:
+        if v == 0:
+            continue
+        e = oracle.pow2_exponent(float(v), bits)
+        assert math.ldexp(qmax, e) >= float(v) > math.ldexp(qmax, e - 1)
+
+
+def test_layer_exponent_ignores_nan_and_uses_kept_rows_only():
+    x = np.zeros((6, 32), np.float16)
+    x[1, 3] = 200.0       # dropped row
+    x[2, 5] = -3.0
+    x[4, 7] = np.nan
+    rows = np.array([0, 2, 4, 5], np.int32)
+    assert oracle.absmax(x, rows) == 3.0
+    assert oracle.layer_exponent(x, 8, rows) == oracle.pow2_exponent(3.0, 8) == -5
+    assert oracle.layer_exponent(x, 8) == 1
+
+
+# ---------------------------------------------------------------- activation quantizer
+def test_quantize_act_hand_worked():
+    for bits, e, x, code in _rows("quantizer_hand_worked.txt"):
+        xs = np.array([[float(x)]], np.float16)
+        q = oracle.quantize_act(xs, int(bits), int(e))
+        assert int(q[0, 0]) == int(code), (bits, e, x, code, int(q[0, 0]))
+
+
+@pytest.mark.parametrize("bits,e", [(8, 0), (8, -3), (8, 2), (4, 1), (4, -2), (4, 0)])
+def test_quantize_act_invariants(bits, e):
+    rng = np.random.default_rng(bits * 100 + e + 50)
+    s = 2.0 ** e
+    lo, hi = -(2 ** (bits - 1)), 2 ** (bits - 1) - 1
+    x = (rng.standard_normal((64, 96)) * s * (hi / 2.0)).astype(np.float16)
+    q = oracle.quantize_act(x, bits, e).astype(np.int64)
+    xf = x.astype(np.float64)
+    assert q.min() >= lo and q.max() <= hi
+    inside = (xf >= lo * s) & (xf <= hi * s)
+    assert inside.any() and (~inside).any()
+    # half a step inside the range (Eq. 2 rounds to the nearest code)
+    assert np.all(np.abs(xf[inside] - q[inside] * s) <= s / 2)
+    # exact saturation outside
+    assert np.all(q[xf > hi * s] == hi)
+    assert np.all(q[xf < lo * s] == lo)
+    # idempotent: quantizing the dequantized value reproduces the code
+    dq = (q * s).astype(np.float16)
+    assert np.array_equal(oracle.quantize_act(dq, bits, e).astype(np.int64), q)
+    # monotone in x
+    order = np.argsort(xf.ravel(), kind="stable")
+    assert np.all(np.diff(q.ravel()[order]) >= 0)
+
+
+def test_quantize_act_ties_go_to_even_and_nonfinite():
+    e = -1
+    js = np.arange(-20, 20)
+    x = ((js + 0.5) * 2.0 ** e).astype(np.float16)[None, :]
+    q = oracle.quantize_act(x, 8, e)[0].astype(np.int64)
+    expect = np.where(js % 2 == 0, js, js + 1)
+    assert np.array_equal(q, expect)
+    x = np.array([[np.nan, np.inf, -np.inf]], np.float16)
+    assert oracle.quantize_act(x, 8, 0)[0].tolist() == [0, 127, -128]
+    assert oracle.quantize_act(x, 4, 3)[0].tolist() == [0, 7, -8]
+
+
+def test_dynamic_scale_never_clips_and_uses_the_range():
+    for seed, bits in [(0, 8), (1, 4), (2, 8)]:
+        x = inputs.activations(32, 256, seed, 0.01, 20.0)
+        e = oracle.layer_exponent(x, bits)
+        q = oracle.quantize_act(x, bits, e).astype(np.int64)
+        hi = 2 ** (bits - 1) - 1
+        assert np.abs(q).max() <= hi          # -2^(b-1) is never produced without clip_shift
+        assert np.abs(q).max() > hi // 2      # one exponent lower would have clipped
+        err = np.abs(x.astype(np.float64) - q * 2.0 ** e)
+        assert err.max() <= 2.0 ** e / 2
+
+
+# -------------------------------------------------------------------- weight quantizer
+@pytest.mark.parametrize("group", [0, 128])
+def test_weight_quantizer_invariants(group):
+    w = inputs.weights(24, 384, seed=3)
+    w[5, :] = 0                         # an all-zero channel
+    w[7, 128:256] = 0                   # an all-zero group
+    codes, scales = oracle.quantize_weights(w, group)
+    G = 1 if group == 0 else 384 // group
+    assert codes.shape == (24, 384) and scales.shape == (24, G)
+    assert codes.min() >= -8 and codes.max() <= 7
+    gs = 384 // G
+    wf = w.astype(np.float64).reshape(24, G, gs)
+    cf = codes.astype(np.float64).reshape(24, G, gs)
+    sf = scales.astype(np.float64)[:, :, None]
+    # every weight is within half a step of its code (the scale is a/7 rounded to fp16,
+    # so the largest weight can land a hair beyond code 7 before rounding: allow the
+    # clip at 7 to cost at most that rounding)
+    amax = np.abs(wf).max(axis=2, keepdims=True)
+    slack = np.maximum(amax - 7 * sf, 0)
+    assert np.all(np.abs(wf - cf * sf) <= sf / 2 + slack + 1e-12)
+    # scale is fp16(absmax/7); the extreme code is used in every non-zero group
+    nz = amax[:, :, 0] > 0
+    exp_scale = (amax[:, :, 0].astype(np.float32) / np.float32(7.0)).astype(np.float16)
+    assert np.array_equal(scales[nz], exp_scale[nz])
+    assert np.all(np.abs(cf).max(axis=2)[nz] == 7)
+    assert np.all(cf[~nz] == 0) and np.all(scales[~nz] == np.float16(1.0))
+
+
+def test_weight_codes_match_numpy_rint_of_ieee_division():
+    w = inputs.weights(16, 256, seed=11)
+    codes, scales = oracle.quantize_weights(w, 128)
+    s = np.repeat(scales.astype(np.float32), 128, axis=1)
+    ref = np.clip(np.rint(w.astype(np.float32) / s), -8, 7).astype(np.int8)
+    assert np.array_equal(codes, ref)
+
+
+def test_pack_unpack_identity_and_nibble_order():
+    allb = np.arange(256, dtype=np.uint8).reshape(1, 256)
+    codes = oracle.unpack_w4(allb)
+    assert codes.min() == -8 and codes.max() == 7
+    assert np.array_equal(oracle.pack_w4(codes), allb)
+    # byte 0x8F: low nibble 0xF = -1 is the even k, high nibble 0x8 = -8 the odd k
+    assert oracle.unpack_w4(np.array([[0x8F]], np.uint8))[0].tolist() == [-1, -8]
+    rng = np.random.default_rng(5)
+    c = rng.integers(-8, 8, size=(9, 64)).astype(np.int8)
+    assert np.array_equal(oracle.unpack_w4(oracle.pack_w4(c)), c)
+
+
+# --------------------------------------------------------------------- integer product
+def _brute(q, c, group):
+    M, K = q.shape
+    N = c.shape[0]
+    gs = K if group == 0 else group
+    G = K // gs
+    out = np.zeros((M, N, G), dtype=object)
+    for g in range(G):
+        for k in range(g * gs, (g + 1) * gs):      # k outermost: an unrelated loop order
+            for n in range(N):
+                for m in range(M):
+                    out[m, n, g] += int(q[m, k]) * int(c[n, k])
+    return out.astype(np.int64)
+
+
+@pytest.mark.parametrize("M,N,K,group", [(3, 5, 32, 0), (4, 2, 128, 0), (5, 3, 256, 128),
+                                         (1, 4, 384, 128), (2, 5, 160, 0)])
+def test_int_gemm_brute_force(M, N, K, group):
+    rng = np.random.default_rng(M * 1000 + N * 10 + K)
+    q = rng.integers(-128, 128, size=(M, K)).astype(np.int8)
+    c = rng.integers(-8, 8, size=(N, K)).astype(np.int8)
+    assert np.array_equal(oracle.int_gemm(q, c, group).astype(np.int64), _brute(q, c, group))
+
+
+def test_int_gemm_closed_forms():
+    K = 256
+    ones_q = np.ones((3, K), np.int8)
+    ones_c = np.ones((4, K), np.int8)
+    assert np.all(oracle.int_gemm(ones_q, ones_c, 0) == K)
+    assert np.all(oracle.int_gemm(ones_q, ones_c, 128) == 128)
+    # c[n,k] = [k == n] picks column n of q
+    rng = np.random.default_rng(2)
+    q = rng.integers(-128, 128, size=(5, K)).astype(np.int8)
+    eye = np.zeros((7, K), np.int8)
+    eye[np.arange(7), np.arange(7)] = 1
+    assert np.array_equal(oracle.int_gemm(q, eye, 0)[:, :, 0], q[:, :7].astype(np.int32))
+    # extremes: (-128)(-8)K, and the largest supported reduction stays inside int32
+    lo_q = np.full((1, 13824), -128, np.int8)
+    lo_c = np.full((1, 13824), -8, np.int8)
+    assert oracle.int_gemm(lo_q, lo_c, 0)[0, 0, 0] == 128 * 8 * 13824
+    # transposition would be caught: asymmetric operands
+    q2 = np.zeros((2, 32), np.int8)
+    c2 = np.zeros((3, 32), np.int8)
+    q2[1, 4] = 9
+    c2[2, 4] = -3
+    acc = oracle.int_gemm(q2, c2, 0)
+    assert acc[1, 2, 0] == -27 and np.count_nonzero(acc) == 1
+
+
+def test_int_gemm_linearity_and_library_matmul():
+    rng = np.random.default_rng(9)
+    M, N, K = 17, 33, 384
+    q1 = rng.integers(-60, 60, size=(M, K)).astype(np.int8)
+    q2 = rng.integers(-60, 60, size=(M, K)).astype(np.int8)
+    c = rng.integers(-8, 8, size=(N, K)).astype(np.int8)
+    a1, a2 = oracle.int_gemm(q1, c, 128), oracle.int_gemm(q2, c, 128)
+    assert np.array_equal(oracle.int_gemm((q1 + q2).astype(np.int8), c, 128), a1 + a2)
+    # textbook integer matmul from a library, per group and over all of K
+    tq, tc = torch.from_numpy(q1).long(), torch.from_numpy(c).long()
+    for g in range(3):
+        ref = tq[:, g * 128:(g + 1) * 128] @ tc[:, g * 128:(g + 1) * 128].T
+        assert np.array_equal(a1[:, :, g].astype(np.int64), ref.numpy())
+    assert np.array_equal(oracle.int_gemm(q1, c, 0)[:, :, 0].astype(np.int64), (tq @ tc.T).numpy())
+    assert np.array_equal(a1.sum(axis=2), oracle.int_gemm(q1, c, 0)[:, :, 0])
+
+
+def test_int_gemm_agrees_with_packed_lane_products():
+    """Sec. 4.4 'INT4 Multiplier' / Algorithm 1: two unsigned 4-bit weights sit in one
+    16-bit lane (8 bits each), one multiply by the shared activation gives both products,
+    a shift-or-mask (0x00FF00FF) spreads them into the two 16-bit halves of a 32-bit word,
+    and up to 2^8 such words are summed without overflow. Restated here on unsigned 4-bit
+    operands as an independent route to the same integer sums."""
+    rng = np.random.default_rng(4)
+    K = 256                                   # the paper's overflow-free limit
+    a = rng.integers(0, 16, size=(3, K))      # unsigned 4-bit activations
+    w0 = rng.integers(0, 16, size=(K,))       # two adjacent output channels
+    w1 = rng.integers(0, 16, size=(K,))
+    w0[:8] = 15
+    a[0, :8] = 15                             # largest product 225 fits its 8-bit field
+    c = np.stack([w0, w1]).astype(np.int8)
+    for m in range(3):
+        acc32 = 0
+        for k in range(K):
+            lane = int(w0[k]) | (int(w1[k]) << 8)
+            p = (lane * int(a[m, k])) & 0xFFFF            # one multiply, two products
+            p = (p | (p << 8)) & 0x00FF00FF               # rearrangement + mask
+            acc32 = (acc32 + p) & 0xFFFFFFFF              # 32-bit accumulation
+        ref = oracle.int_gemm(a[m:m + 1].astype(np.int8), c, 0)[0, :, 0]
+        assert int(ref[0]) == (acc32 & 0xFFFF) and int(ref[1]) == (acc32 >> 16)
+
+
+# ----------------------------------------------------------------------------- dequant
+def test_dequant_per_channel_is_one_rounding_of_the_exact_value():
+    rng = np.random.default_rng(12)
+    acc = rng.integers(-200000, 200000, size=(6, 10, 1)).astype(np.int32)
+    scales = (rng.random((10, 1)) * 0.01 + 1e-4).astype(np.float16)
+    for e in (-3, 0, 2):
+        y = oracle.dequant(acc, scales, e)
+        exact = acc[:, :, 0].astype(np.float64) * scales[:, 0].astype(np.float64)[None, :] * 2.0 ** e
+        with np.errstate(over="ignore"):
+            assert np.array_equal(y.view(np.uint16), exact.astype(np.float16).view(np.uint16))
+
+
+def test_dequant_groups_sum_in_double():
+    rng = np.random.default_rng(13)
+    acc = rng.integers(-100000, 100000, size=(4, 8, 5)).astype(np.int32)
+    scales = (rng.random((8, 5)) * 0.02 + 1e-4).astype(np.float16)
+    y = oracle.dequant(acc, scales, -1)
+    exact = np.einsum("mng,ng->mn", acc.astype(np.float64), scales.astype(np.float64)) * 0.5
+    assert np.array_equal(y.view(np.uint16), exact.astype(np.float16).view(np.uint16))
+
+
+@pytest.mark.parametrize("group,bits", [(0, 8), (128, 8), (128, 4)])
+def test_layer_output_within_quantization_error_bound_of_fp_linear(group, bits):
+    """With nothing clipped, |y - x w^T| <= sum_k (2^(e-1)|w_k| + (s_w/2)|x_k| + 2^(e-1) s_w/2)
+    plus the final fp16 rounding."""
+    M, K, N = 8, 256, 12
+    x = inputs.activations(M, K, 21, 0.01, 20.0)
+    w = inputs.weights(N, K, 21)
+    codes, scales = oracle.quantize_weights(w, group)
+    out = oracle.linear(x, codes, scales, bits, group)
+    e = out["e"]
+    xf, wf = x.astype(np.float64), w.astype(np.float64)
+    ref = xf @ wf.T
+    G = scales.shape[1]
+    sw = np.repeat(scales.astype(np.float64), K // G, axis=1)            # [N,K]
+    # the scale a/7 is rounded to fp16, so the largest weight of a group may clip by a hair
+    werr = np.maximum(sw / 2, np.abs(wf - codes * sw))
+    bound = (2.0 ** (e - 1)) * np.abs(wf).sum(axis=1)[None, :] + np.abs(xf) @ werr.T \
+        + (2.0 ** (e - 1)) * werr.sum(axis=1)[None, :]
+    y = out["y"].astype(np.float64)
+    assert np.all(np.abs(y - ref) <= bound + np.abs(ref) * 2.0 ** -10 + 1e-6)
+    # and it is not vacuous: the layer tracks the fp result
+    assert np.corrcoef(y.ravel(), ref.ravel())[0, 1] > (0.99 if bits == 8 else 0.8)
+
+
+def test_linear_composite_equals_its_steps():
+    M, K, N = 5, 256, 7
+    x = inputs.activations(M, K, 31, 0.01, 20.0)
+    w = inputs.weights(N, K, 31)
+    codes, scales = oracle.quantize_weights(w, 128)
+    out = oracle.linear(x, codes, scales, 4, 128, 0, 2, want_acc=True)
+    e = oracle.layer_exponent(x, 4) - 2
+    q = oracle.quantize_act(x, 4, e)
+    acc = oracle.int_gemm(q, codes, 128)
+    assert out["e"] == e and np.array_equal(out["q"], q) and np.array_equal(out["acc"], acc)
+    assert np.array_equal(out["y"].view(np.uint16), oracle.dequant(acc, scales, e).view(np.uint16))
+    assert q.min() == -8 and q.max() == 7      # clip_shift makes the outlier channels saturate
+    rows = np.array([0, 4, 2], np.int32)
+    cols = np.array([6, 0, 3], np.int32)
+    sa, sy = oracle.linear_sampled(q, codes, scales, e, 128, rows, cols)
+    assert np.array_equal(sa, acc[rows, cols]) and np.array_equal(sy, out["y"][rows, cols])
+    st = oracle.linear(x, codes, scales, 4, 128, 1, e)
+    assert np.array_equal(st["y"].view(np.uint16), out["y"].view(np.uint16))
+
+
+# ----------------------------------------------------------------------- token pruning
+def test_token_select_brute_force_with_ties():
+    rng = np.random.default_rng(8)
+    for M in (1, 2, 7, 33, 64):
+        scores = rng.integers(0, 6, size=M).astype(np.float32) / 4      # many duplicates
+        for n_keep in sorted({0, 1, M // 2, max(M - 1, 0), M}):
+            idx = oracle.token_select(scores, n_keep)
+            # brute force: rank = how many tokens beat token i
+            rank = [sum(1 for j in range(M) if scores[j] > scores[i] or
+                        (scores[j] == scores[i] and j < i)) for i in range(M)]
+            ref = [i for i in range(M) if rank[i] < n_keep]
+            assert idx.tolist() == ref
+
+
+def test_token_select_invariants_and_gather():
+    M, K = 257, 64
+    scores = inputs.token_scores(M, 4)
+    n_keep = int(math.ceil(0.6 * M))
+    idx = oracle.token_select(scores, n_keep)
+    assert len(idx) == n_keep and np.all(np.diff(idx) > 0)
+    dropped = np.setdiff1d(np.arange(M), idx)
+    assert scores[idx].min() >= scores[dropped].max()
+    # numpy's sort as the library routine: same kept set
+    ref = np.sort(np.argsort(-scores, kind="stable")[:n_keep])
+    assert np.array_equal(idx, ref.astype(np.int32))
+    x = inputs.activations(M, K, 4)
+    xp = oracle.token_compact(x, idx)
+    assert np.array_equal(xp.view(np.uint16), x[idx].view(np.uint16))
+    with pytest.raises(ValueError):
+        oracle.token_select(scores, M + 1)
+
+
+def test_progressive_ratio_closed_form():
+    # Eq. 9: applying gamma at each of the m pruning layers leaves (1-beta) of the tokens
+    for beta, m in [(0.4, 4), (0.16, 8), (0.5, 1), (0.0, 3)]:
+        g = oracle.progressive_ratio(beta, m)
+        assert abs((1 - g) ** m - (1 - beta)) < 1e-12
+    assert abs(oracle.progressive_ratio(0.75, 2) - 0.5) < 1e-15
+
+
+# ------------------------------------------------------------------------ input recipe
+def test_inputs_are_seeded_and_structured():
+    a = inputs.activations(64, 512, 1, 0.005, 30.0)
+    b = inputs.activations(64, 512, 1, 0.005, 30.0)
+    assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
+    ch = inputs.outlier_channels(512, 0.005, 1)
+    assert len(ch) == 3
+    body = np.delete(a.astype(np.float32), ch, axis=1)
+    assert 0.9 < body.std() < 1.1 and a.astype(np.float32)[:, ch].std() > 20
+    w = inputs.weights(32, 512, 1)
+    assert 0.018 < w.astype(np.float32).std() < 0.022
+    s = inputs.token_scores(100, 1)
+    assert s.min() >= 0 and s.max() < 1 and s.dtype == np.float32
