@@ -1,0 +1,154 @@
+/*
+ * agileq: the quantized linear layer of Agile-Quant (arXiv 2312.05693) for NVIDIA B200
+ * (sm_100a). C ABI, plain pointers and sizes.
+ *
+ * What the layer computes (paper Sec. 4.4, "Efficient TRIP Matrix Multiplication"):
+ * activations are quantized layer-wise (one scale for the whole matrix), weights per
+ * output channel (optionally per 128-wide group along K), products are summed as
+ * integers and the sums are mapped back to floating point:
+ *
+ *     e    = layer exponent, scale 2^e               (Eq. 6, symmetric, alpha = 0)
+ *     q    = clip(round(x / 2^e), -2^(b-1), 2^(b-1)-1)      (Eq. 1, Eq. 2 / Eq. 5, zp = 0)
+ *     acc  = sum_k q[m,k] * c[n,k]                   (int32; Sec. 4.4, Algorithm 1)
+ *     y    = fp16( 2^e * sum_g s_w[n,g] * acc[m,n,g] )
+ *
+ * Conventions
+ *  - Every tensor pointer is a DEVICE pointer owned by the caller unless its name ends
+ *    in "_host". The library never allocates or frees device memory; scratch comes from
+ *    a caller-provided workspace. Pointers must be 16-byte aligned (256 for workspaces).
+ *  - Calls enqueue work on the CUDA stream passed as `stream` (a cudaStream_t cast to
+ *    void*, NULL = default stream) and return without synchronizing, except the calls
+ *    documented as synchronizing.
+ *  - Return value: AQ_OK (0) or a negative aq_status. On error nothing was enqueued.
+ *  - Shapes: K % 128 == 0, 128 <= K <= 65536; N >= 1; M >= 1. group_size is 0 (one scale
+ *    per output channel) or 128. Activation bits is 8 or 4 (4-bit codes are stored one
+ *    per int8, values -8..7).
+ *  - Rounding is to nearest, ties to even.
+ *  - Requires a device of compute capability 10.0 (B200); anything else is refused with
+ *    AQ_ERR_UNSUPPORTED_DEVICE. There is no CPU or other fallback.
+ */
+#ifndef AGILEQ_H_
+#define AGILEQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct aq_context* aq_handle_t;
+
+typedef enum aq_status {
+    AQ_OK = 0,
+    AQ_ERR_INVALID_ARG = -1,        /* NULL pointer, bad enum value, bad bit width */
+    AQ_ERR_SHAPE = -2,              /* unsupported M / K / N / group_size / n_keep */
+    AQ_ERR_ALIGNMENT = -3,          /* a pointer is not aligned as required */
+    AQ_ERR_WORKSPACE = -4,          /* workspace NULL or smaller than aq_workspace_bytes() */
+    AQ_ERR_UNSUPPORTED_DEVICE = -5, /* not compute capability 10.0 */
+    AQ_ERR_CUDA = -6,               /* a CUDA call failed; see aq_last_cuda_error() */
+    AQ_ERR_DEVICE_TIMEOUT = -7      /* a bounded wait inside a kernel gave up */
+} aq_status;
+
+/* How the layer exponent e is chosen (paper Eq. 6 read as a symmetric power-of-two
+ * scale). DYNAMIC: e0 = smallest integer with (2^(b-1)-1) * 2^e0 >= max|x| over the rows
+ * used, e = e0 - clip_shift (clip_shift >= 0 lets outliers saturate). STATIC: e is given. */
+enum { AQ_SCALE_DYNAMIC = 0, AQ_SCALE_STATIC = 1 };
+
+/* Which matrix-product kernel aq_linear_* / aq_gemm_w4 uses. AUTO picks the decode kernel
+ * for M <= 16 and the tensor-core kernel otherwise; the others force one (for tests and
+ * measurements). All give identical integer sums. */
+enum { AQ_KERNEL_AUTO = 0, AQ_KERNEL_TENSOR = 1, AQ_KERNEL_DECODE = 2 };
+
+const char* aq_status_string(int status);
+int aq_version(void);
+
+/* Handle: host-side state only (device properties, driver entry points). `device` is a
+ * CUDA device ordinal; it must be the current device whenever the handle is used. */
+int aq_create(aq_handle_t* out, int device);
+int aq_destroy(aq_handle_t h);
+/* The cudaError_t value of the last failed CUDA call made through this handle. */
+int aq_last_cuda_error(aq_handle_t h);
+/* Force a kernel choice for subsequent calls on this handle (AQ_KERNEL_*). */
+int aq_set_kernel(aq_handle_t h, int kernel);
+
+/* ---- sizes -------------------------------------------------------------------------- */
+/* Bytes of the packed 4-bit weight buffer (rows are padded to a multiple of 128). */
+size_t aq_packed_w4_bytes(int N, int K);
+/* Bytes of the fp16 scale buffer: [G][Npad], G = 1 (group_size 0) or K/128, Npad = N
+ * rounded up to 128; element (g, n) at index g*Npad + n. */
+size_t aq_scales_bytes(int N, int K, int group_size);
+/* Bytes of scratch that aq_quantize_act / aq_linear_* / aq_gemm_w4 / aq_token_select need
+ * for these sizes (M = rows actually multiplied). Always a multiple of 256. */
+size_t aq_workspace_bytes(int M, int K, int N, int group_size);
+
+/* ---- weights (offline; paper Sec. 4.4 last paragraph, Sec. 5.1: 4-bit per-channel weights)
+ * Round-to-nearest symmetric quantization of w_fp16 [N,K] row-major:
+ *   a = max|w| over the channel (or 128-wide group), s = fp16(a/7) (1 if a == 0, the
+ *   smallest positive fp16 if a/7 underflows), c = clip(round(w/s), -8, 7).
+ * Writes the codes in the library's device-native packed layout (opaque; read it back
+ * with aq_unpack_w4) and the scales as described at aq_scales_bytes(). Weights must be
+ * finite. */
+int aq_pack_w4(aq_handle_t h, const void* w_fp16, int N, int K, int group_size,
+               void* w_packed, void* w_scales, void* stream);
+/* Test utility: packed layout -> int8 codes [N,K] row-major. */
+int aq_unpack_w4(aq_handle_t h, const void* w_packed, int N, int K, int8_t* codes, void* stream);
+
+/* ---- activations (paper Eq. 1, Eq. 2 / Eq. 5 with zp = 0; layer-wise scale, Sec. 4.4)
+ * x_fp16 [M_in,K] row-major. row_idx == NULL: rows 0..M-1 are quantized; otherwise row
+ * row_idx[i] (i < M) is read, so pruned tokens (Eq. 4) never enter the scale or the codes.
+ * q [M,K] int8 row-major. scale_exp_out: one int32 on the device, receives e.
+ * bits 8 or 4. NaN -> code 0 and is ignored by the scale; +-Inf saturate. */
+int aq_quantize_act(aq_handle_t h, const void* x_fp16, int M, int K, int bits, int scale_mode,
+                    int clip_shift_or_exp, const int32_t* row_idx, int8_t* q,
+                    int32_t* scale_exp_out, void* workspace, size_t workspace_bytes,
+                    void* stream);
+
+/* ---- the layer (paper Sec. 4.4): quantize, integer product, floating-point output
+ * y_fp16 [M,N] row-major. acc_dump: NULL, or int32 [M][N][G] (G as in aq_scales_bytes)
+ * receiving the integer sums (test aid; slows the call). row_idx as above. */
+int aq_linear_w4a8(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed,
+                   const void* w_scales, int N, int group_size, int scale_mode,
+                   int clip_shift_or_exp, const int32_t* row_idx, void* y_fp16,
+                   int32_t* acc_dump, void* workspace, size_t workspace_bytes, void* stream);
+/* Same with 4-bit activation codes (paper Sec. 4.2: some activations take 4 bits). */
+int aq_linear_w4a4(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed,
+                   const void* w_scales, int N, int group_size, int scale_mode,
+                   int clip_shift_or_exp, const int32_t* row_idx, void* y_fp16,
+                   int32_t* acc_dump, void* workspace, size_t workspace_bytes, void* stream);
+
+/* The product and output steps alone, on codes q [M,K] that are already quantized;
+ * scale_exp: device int32 holding e. */
+int aq_gemm_w4(aq_handle_t h, const int8_t* q, int M, int K, const void* w_packed,
+               const void* w_scales, int N, int group_size, const int32_t* scale_exp,
+               void* y_fp16, int32_t* acc_dump, void* workspace, size_t workspace_bytes,
+               void* stream);
+
+/* ---- token pruning (paper Eq. 4: X^P = F^P(X), n < m tokens kept by importance)
+ * aq_token_select: idx [n_keep] = indices of the n_keep largest scores, equal scores
+ * resolved toward the lower index, in ascending order. scores fp32 [M], no NaN,
+ * M <= 65536. aq_token_compact: x_out[i,:] = x[idx[i],:] (fp16 rows of K). */
+int aq_token_select(aq_handle_t h, const float* scores, int M, int n_keep, int32_t* idx,
+                    void* workspace, size_t workspace_bytes, void* stream);
+int aq_token_compact(aq_handle_t h, const void* x_fp16, int M, int K, const int32_t* idx,
+                     int n_keep, void* x_out, void* stream);
+
+/* ---- host-buffer convenience (SYNCHRONIZES the stream before returning)
+ * x_host fp16 [M,K] and y_host fp16 [M,N] are HOST pointers (pinned memory gives the best
+ * rate). Copies x to the device scratch, runs the layer with `bits` (8 or 4), copies y
+ * back. device_scratch must hold aq_linear_host_scratch_bytes() bytes. */
+size_t aq_linear_host_scratch_bytes(int M, int K, int N, int group_size);
+int aq_linear_host(aq_handle_t h, int bits, const void* x_host, int M, int K,
+                   const void* w_packed, const void* w_scales, int N, int group_size,
+                   int scale_mode, int clip_shift_or_exp, void* y_host, void* device_scratch,
+                   size_t scratch_bytes, void* stream);
+
+/* SYNCHRONIZES the stream, then reports whether any kernel that used this workspace gave
+ * up on a bounded wait (AQ_ERR_DEVICE_TIMEOUT) since the workspace was last used by a
+ * call; AQ_OK otherwise. */
+int aq_check_workspace(aq_handle_t h, const void* workspace, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* AGILEQ_H_ */

@@ -1,0 +1,110 @@
+// Shared declarations for the agileq kernels (device-side helpers, layout constants,
+// the workspace control block and the launcher prototypes).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/agileq.h"
+
+namespace aq {
+
+// ---------------------------------------------------------------------------------------
+// Packed 4-bit weight layout (device-native; defined only here and in aq_pack.cu).
+//
+// Rows are padded to Npad = ceil(N/128)*128. The matrix is cut into blocks of 128 rows x
+// 128 k. Block (nt, kb) starts at byte ((nt * K/128 + kb) * 8192). Inside a block, the
+// 16-byte unit (j, r), j = 0..3, r = 0..127, sits at byte (j*128 + r)*16 and holds the 32
+// codes k = kb*128 + 32j .. +31 of row nt*128 + r. Inside a unit, byte b of 32-bit word i
+// (i = 0..3, little endian) holds code k0+b in its low nibble and code k0+4+b in its high
+// nibble, k0 = kb*128 + 32j + 8i, as two's-complement nibbles.
+//
+// Why: a warp reads 512 contiguous bytes per load; "(w << 4) & 0xF0F0F0F0" and
+// "w & 0xF0F0F0F0" turn one word into two words of four int8 values equal to 16*code in k
+// order, with no sign extension. Integer sums therefore come out multiplied by 16 and are
+// shifted right by 4 (exact) before use.
+// ---------------------------------------------------------------------------------------
+constexpr int kTileN = 128;          // rows per packed block
+constexpr int kTileK = 128;          // k per packed block (= the weight-scale group)
+constexpr int kBlockBytes = kTileN * kTileK / 2;   // 8192
+
+__host__ __device__ inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
+__host__ __device__ inline size_t packed_unit_offset(int KB, int nt, int kb, int j, int r) {
+    return ((size_t)nt * KB + kb) * kBlockBytes + (size_t)(j * kTileN + r) * 16;
+}
+
+// ---------------------------------------------------------------------------------------
+// Workspace layout: [control block 256 B][activation codes M*K int8, padded to 256 B]
+// [kernel scratch].
+// ---------------------------------------------------------------------------------------
+struct Control {
+    unsigned int absmax_bits;   // fp16 bit pattern of max|x| (atomicMax target), cleared per call
+    int scale_exp;              // layer exponent e
+    unsigned int status;        // non-zero: a bounded wait gave up
+    unsigned int counter;       // scratch counter
+    unsigned int reserved[60];
+};
+static_assert(sizeof(Control) == 256, "control block is 256 bytes");
+
+// Layer exponent from max|x| (fp16 bits): the smallest e with qmax * 2^e >= a, qmax =
+// 2^(bits-1)-1 (Eq. 6 read as a symmetric power-of-two scale). Uses the binary expansion
+// a = m * 2^ex, m in [0.5, 1): qmax = mq * 2^xq with mq = 127/128 (xq = 7) or 7/8 (xq = 3),
+// so e = ex - xq, plus one if m > mq. a == 0 gives 0; +Inf counts as 65504.
+__device__ inline int layer_exponent_from_bits(unsigned int absmax_bits, int bits) {
+    unsigned int hb = absmax_bits & 0x7FFFu;
+    if (hb == 0) return 0;
+    if (hb >= 0x7C00u) hb = 0x7BFFu;
+    const float a = __half2float(__ushort_as_half((unsigned short)hb));
+    int ex;
+    const float m = frexpf(a, &ex);
+    const float mq = bits == 8 ? 0.9921875f : 0.875f;
+    const int xq = bits == 8 ? 7 : 3;
+    return ex - xq + (m > mq ? 1 : 0);
+}
+
+// ---------------------------------------------------------------------------------------
+// Launchers (implemented one per .cu file). All enqueue on `stream` and return the CUDA
+// launch status.
+// ---------------------------------------------------------------------------------------
+struct DeviceInfo {
+    int device;
+    int sm_count;
+    int cc_major, cc_minor;
+    size_t smem_optin;
+    void* encode_tiled;   // cuTensorMapEncodeTiled, resolved through the runtime
+};
+
+cudaError_t launch_pack_w4(const __half* w, int N, int K, int group, uint8_t* packed, __half* scales,
+                           cudaStream_t stream);
+cudaError_t launch_unpack_w4(const uint8_t* packed, int N, int K, int8_t* codes, cudaStream_t stream);
+
+cudaError_t launch_absmax(const __half* x, int M, int K, const int32_t* row_idx, Control* ctl,
+                          const DeviceInfo& dev, cudaStream_t stream);
+cudaError_t launch_quantize(const __half* x, int M, int K, const int32_t* row_idx, int bits,
+                            int scale_mode, int clip_shift_or_exp, Control* ctl, int8_t* q,
+                            int32_t* scale_exp_out, const DeviceInfo& dev, cudaStream_t stream);
+
+cudaError_t launch_token_select(const float* scores, int M, int n_keep, int32_t* idx, void* scratch,
+                                cudaStream_t stream);
+cudaError_t launch_token_compact(const __half* x, int K, const int32_t* idx, int n_keep, __half* out,
+                                 const DeviceInfo& dev, cudaStream_t stream);
+
+// Integer product + floating-point output on quantized codes.
+struct GemmArgs {
+    const int8_t* q;        // [M][K]
+    int M, K, N, group;     // group: 0 or 128
+    const uint8_t* w_packed;
+    const __half* w_scales; // [G][Npad]
+    const int32_t* scale_exp;
+    __half* y;              // [M][N]
+    int32_t* acc_dump;      // NULL or [M][N][G]
+    Control* ctl;
+    void* scratch;          // beyond control block + codes
+    size_t scratch_bytes;
+};
+cudaError_t launch_gemm_tensor(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream);
+cudaError_t launch_gemm_decode(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream);
+
+}  // namespace aq

@@ -1,0 +1,110 @@
+// Offline weight quantization and packing (4-bit, per output channel or per 128-wide
+// group; paper Sec. 4.4 last paragraph and Sec. 5.1), and the inverse of the packing.
+#include "aq_common.cuh"
+
+namespace aq {
+
+namespace {
+
+__device__ inline float block_max_128(float v, float* red) {
+    // 128 threads = 4 warps
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    const float r = fmaxf(fmaxf(red[0], red[1]), fmaxf(red[2], red[3]));
+    __syncthreads();
+    return r;
+}
+
+// Stored scale for a group whose largest magnitude is a: fp16(a/7); 1 for an all-zero
+// group; the smallest positive fp16 when a/7 underflows.
+__device__ inline __half group_scale(float a) {
+    __half s = __float2half_rn(__fdiv_rn(a, 7.0f));
+    if ((__half_as_ushort(s) & 0x7FFFu) == 0)
+        s = __ushort_as_half(a == 0.0f ? (unsigned short)0x3C00u : (unsigned short)0x0001u);
+    return s;
+}
+
+// One CTA of 128 threads per (padded) output channel.
+__global__ void __launch_bounds__(128)
+pack_w4_kernel(const __half* __restrict__ w, int N, int K, int group, uint8_t* __restrict__ packed,
+               __half* __restrict__ scales) {
+    __shared__ float red[4];
+    __shared__ int8_t codes[kTileK];
+    const int n = blockIdx.x;
+    const int Npad = gridDim.x;
+    const int KB = K / kTileK;
+    const int t = threadIdx.x;
+    const int nt = n / kTileN, r = n % kTileN;
+    const bool live = n < N;
+    const __half* row = w + (size_t)n * K;
+
+    float s_row = 1.0f;
+    if (group == 0) {
+        float a = 0.0f;
+        if (live)
+            for (int k = t; k < K; k += 128) a = fmaxf(a, fabsf(__half2float(row[k])));
+        a = block_max_128(a, red);
+        const __half sh = group_scale(a);
+        if (t == 0) scales[n] = live ? sh : __ushort_as_half((unsigned short)0);
+        s_row = __half2float(sh);
+    }
+    for (int kb = 0; kb < KB; ++kb) {
+        const float wv = live ? __half2float(row[kb * kTileK + t]) : 0.0f;
+        float s = s_row;
+        if (group != 0) {
+            const float a = block_max_128(fabsf(wv), red);
+            const __half sh = group_scale(a);
+            if (t == 0) scales[(size_t)kb * Npad + n] = live ? sh : __ushort_as_half((unsigned short)0);
+            s = __half2float(sh);
+        }
+        float c = rintf(__fdiv_rn(wv, s));
+        c = fminf(fmaxf(c, -8.0f), 7.0f);
+        codes[t] = (int8_t)(int)c;
+        __syncthreads();
+        if (t < 16) {
+            const int j = t >> 2, i = t & 3;
+            const int8_t* c8 = codes + 32 * j + 8 * i;
+            uint32_t word = 0;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                word |= ((uint32_t)c8[b] & 0xFu) << (8 * b);
+                word |= ((uint32_t)c8[4 + b] & 0xFu) << (8 * b + 4);
+            }
+            *reinterpret_cast<uint32_t*>(packed + packed_unit_offset(KB, nt, kb, j, r) + 4 * i) = word;
+        }
+        __syncthreads();
+    }
+}
+
+__global__ void unpack_w4_kernel(const uint8_t* __restrict__ packed, int N, int K,
+                                 int8_t* __restrict__ codes) {
+    const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (size_t)N * K) return;
+    const int n = (int)(idx / K), k = (int)(idx % K);
+    const int KB = K / kTileK;
+    const int kb = k / kTileK, kl = k % kTileK;
+    const int j = kl >> 5, i = (kl & 31) >> 3, p = kl & 7;
+    const uint8_t byte = packed[packed_unit_offset(KB, n / kTileN, kb, j, n % kTileN) + 4 * i + (p & 3)];
+    const int nib = (p & 4) ? (byte >> 4) : (byte & 0xF);
+    codes[idx] = (int8_t)(nib >= 8 ? nib - 16 : nib);
+}
+
+}  // namespace
+
+cudaError_t launch_pack_w4(const __half* w, int N, int K, int group, uint8_t* packed, __half* scales,
+                           cudaStream_t stream) {
+    const int Npad = round_up(N, kTileN);
+    pack_w4_kernel<<<Npad, 128, 0, stream>>>(w, N, K, group, packed, scales);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_unpack_w4(const uint8_t* packed, int N, int K, int8_t* codes, cudaStream_t stream) {
+    const size_t total = (size_t)N * K;
+    const unsigned int blocks = (unsigned int)((total + 255) / 256);
+    unpack_w4_kernel<<<blocks, 256, 0, stream>>>(packed, N, K, codes);
+    return cudaGetLastError();
+}
+
+}  // namespace aq

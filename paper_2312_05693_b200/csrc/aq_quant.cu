@@ -1,0 +1,199 @@
+// Activation side: layer-wise absolute maximum, power-of-two quantization to int8 / int4
+// codes (paper Eq. 1, Eq. 2 / Eq. 5 with zp = 0, layer-wise scale of Sec. 4.4), and the
+// token selection / gather of Eq. 4.
+#include "aq_common.cuh"
+
+namespace aq {
+
+namespace {
+
+constexpr int kQuantThreads = 256;
+
+// ---- layer absmax: 16-byte loads, warp-shuffle reduction, one atomic per warp ----------
+__global__ void __launch_bounds__(kQuantThreads)
+absmax_kernel(const uint4* __restrict__ x, int M, int vec_per_row, const int32_t* __restrict__ row_idx,
+              Control* __restrict__ ctl) {
+    const size_t total = (size_t)M * vec_per_row;
+    __half2 m2 = __float2half2_rn(0.0f);
+    for (size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v < total;
+         v += (size_t)gridDim.x * blockDim.x) {
+        const int m = (int)(v / vec_per_row), c = (int)(v % vec_per_row);
+        const size_t src = (size_t)(row_idx ? row_idx[m] : m) * vec_per_row + c;
+        const uint4 d = __ldg(x + src);
+        const __half2* h = reinterpret_cast<const __half2*>(&d);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) m2 = __hmax2(m2, __habs2(h[i]));   // NaN operands are dropped
+    }
+    unsigned int bits = max((unsigned int)__half_as_ushort(__low2half(m2)),
+                            (unsigned int)__half_as_ushort(__high2half(m2)));
+    if (bits > 0x7C00u) bits = 0;                                       // never publish NaN
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) bits = max(bits, __shfl_xor_sync(0xFFFFFFFFu, bits, o));
+    if ((threadIdx.x & 31) == 0 && bits != 0) atomicMax(&ctl->absmax_bits, bits);
+}
+
+__device__ inline int quantize_one(float v, float inv, float lo, float hi) {
+    const float t = v * inv;                 // exact: inv is a power of two
+    if (t != t) return 0;                    // NaN
+    return (int)fminf(fmaxf(rintf(t), lo), hi);
+}
+
+// ---- quantize: 16 halves in (two 16-byte loads), 16 codes out (one 16-byte store) -----
+__global__ void __launch_bounds__(kQuantThreads)
+quantize_kernel(const uint4* __restrict__ x, int M, int vec_per_row /* 16-element units */,
+                const int32_t* __restrict__ row_idx, int bits, int scale_mode, int clip_shift_or_exp,
+                Control* __restrict__ ctl, uint4* __restrict__ q, int32_t* __restrict__ scale_exp_out) {
+    const int e = scale_mode == AQ_SCALE_DYNAMIC
+                      ? layer_exponent_from_bits(ctl->absmax_bits, bits) - clip_shift_or_exp
+                      : clip_shift_or_exp;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        ctl->scale_exp = e;
+        if (scale_exp_out) *scale_exp_out = e;
+    }
+    const float inv = __int_as_float((127 - e) << 23);      // 2^-e, |e| <= 40
+    const float lo = -(float)(1 << (bits - 1)), hi = (float)((1 << (bits - 1)) - 1);
+    const size_t total = (size_t)M * vec_per_row;
+    const size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (v >= total) return;
+    const int m = (int)(v / vec_per_row), c = (int)(v % vec_per_row);
+    const size_t src = ((size_t)(row_idx ? row_idx[m] : m) * vec_per_row + c) * 2;
+    const uint4 d0 = __ldg(x + src), d1 = __ldg(x + src + 1);
+    const __half* h0 = reinterpret_cast<const __half*>(&d0);
+    const __half* h1 = reinterpret_cast<const __half*>(&d1);
+    uint32_t out[4];
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+        uint32_t word = 0;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int i = 4 * w + b;
+            const float f = __half2float(i < 8 ? h0[i] : h1[i - 8]);
+            word |= ((uint32_t)quantize_one(f, inv, lo, hi) & 0xFFu) << (8 * b);
+        }
+        out[w] = word;
+    }
+    q[v] = make_uint4(out[0], out[1], out[2], out[3]);
+}
+
+// ---- token selection: rank every score, keep rank < n_keep, then compact the flags ------
+// rank(i) = #{ j : s_j > s_i  or (s_j == s_i and j < i) }, so equal scores resolve toward
+// the lower index and exactly n_keep tokens have rank < n_keep.
+__global__ void __launch_bounds__(256)
+token_rank_kernel(const float* __restrict__ scores, int M, int n_keep, uint8_t* __restrict__ keep) {
+    __shared__ float tile[1024];
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const float si = i < M ? scores[i] : 0.0f;
+    int rank = 0;
+    for (int base = 0; base < M; base += 1024) {
+        for (int t = threadIdx.x; t < 1024; t += blockDim.x)
+            tile[t] = base + t < M ? scores[base + t] : -INFINITY;
+        __syncthreads();
+        const int lim = min(1024, M - base);
+        for (int t = 0; t < lim; ++t) {
+            const float sj = tile[t];
+            rank += (sj > si) || (sj == si && base + t < i);
+        }
+        __syncthreads();
+    }
+    if (i < M) keep[i] = rank < n_keep ? 1 : 0;
+}
+
+// One CTA of 1024 threads: exclusive scan of the keep flags, ascending indices out.
+__global__ void __launch_bounds__(1024)
+token_compact_idx_kernel(const uint8_t* __restrict__ keep, int M, int32_t* __restrict__ idx) {
+    __shared__ int warp_sums[32];
+    __shared__ int running;
+    if (threadIdx.x == 0) running = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    for (int base = 0; base < M; base += 1024) {
+        const int i = base + threadIdx.x;
+        const int f = i < M ? keep[i] : 0;
+        int incl = f;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) warp_sums[wid] = incl;
+        __syncthreads();
+        if (wid == 0) {
+            int ws = warp_sums[lane];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(0xFFFFFFFFu, ws, o);
+                if (lane >= o) ws += t;
+            }
+            warp_sums[lane] = ws;   // inclusive over warps
+        }
+        __syncthreads();
+        const int before = running + (wid ? warp_sums[wid - 1] : 0) + incl - f;
+        if (f) idx[before] = i;
+        __syncthreads();
+        if (threadIdx.x == 0) running += warp_sums[31];
+        __syncthreads();
+    }
+}
+
+__global__ void __launch_bounds__(256)
+gather_rows_kernel(const uint4* __restrict__ x, int vec_per_row, const int32_t* __restrict__ idx,
+                   int n_keep, uint4* __restrict__ out) {
+    const size_t total = (size_t)n_keep * vec_per_row;
+    for (size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v < total;
+         v += (size_t)gridDim.x * blockDim.x) {
+        const int m = (int)(v / vec_per_row), c = (int)(v % vec_per_row);
+        out[v] = __ldg(x + (size_t)idx[m] * vec_per_row + c);
+    }
+}
+
+}  // namespace
+
+cudaError_t launch_absmax(const __half* x, int M, int K, const int32_t* row_idx, Control* ctl,
+                          const DeviceInfo& dev, cudaStream_t stream) {
+    const int vec_per_row = K / 8;
+    const size_t total = (size_t)M * vec_per_row;
+    size_t blocks = (total + kQuantThreads - 1) / kQuantThreads;
+    const size_t cap = (size_t)dev.sm_count * 8;
+    if (blocks > cap) blocks = cap;
+    absmax_kernel<<<(unsigned int)blocks, kQuantThreads, 0, stream>>>(
+        reinterpret_cast<const uint4*>(x), M, vec_per_row, row_idx, ctl);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quantize(const __half* x, int M, int K, const int32_t* row_idx, int bits,
+                            int scale_mode, int clip_shift_or_exp, Control* ctl, int8_t* q,
+                            int32_t* scale_exp_out, const DeviceInfo& dev, cudaStream_t stream) {
+    (void)dev;
+    const int vec_per_row = K / 16;
+    const size_t total = (size_t)M * vec_per_row;
+    const size_t blocks = (total + kQuantThreads - 1) / kQuantThreads;
+    quantize_kernel<<<(unsigned int)blocks, kQuantThreads, 0, stream>>>(
+        reinterpret_cast<const uint4*>(x), M, vec_per_row, row_idx, bits, scale_mode, clip_shift_or_exp,
+        ctl, reinterpret_cast<uint4*>(q), scale_exp_out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_token_select(const float* scores, int M, int n_keep, int32_t* idx, void* scratch,
+                                cudaStream_t stream) {
+    uint8_t* keep = static_cast<uint8_t*>(scratch);
+    token_rank_kernel<<<(M + 255) / 256, 256, 0, stream>>>(scores, M, n_keep, keep);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+    token_compact_idx_kernel<<<1, 1024, 0, stream>>>(keep, M, idx);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_token_compact(const __half* x, int K, const int32_t* idx, int n_keep, __half* out,
+                                 const DeviceInfo& dev, cudaStream_t stream) {
+    if (n_keep == 0) return cudaSuccess;
+    const int vec_per_row = K / 8;
+    const size_t total = (size_t)n_keep * vec_per_row;
+    size_t blocks = (total + 255) / 256;
+    const size_t cap = (size_t)dev.sm_count * 16;
+    if (blocks > cap) blocks = cap;
+    gather_rows_kernel<<<(unsigned int)blocks, 256, 0, stream>>>(
+        reinterpret_cast<const uint4*>(x), vec_per_row, idx, n_keep, reinterpret_cast<uint4*>(out));
+    return cudaGetLastError();
+}
+
+}  // namespace aq
