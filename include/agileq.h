@@ -143,9 +143,9 @@ int aq_linear_host(aq_handle_t h, int bits, const void* x_host, int M, int K,
                    int scale_mode, int clip_shift_or_exp, void* y_host, void* device_scratch,
                    size_t scratch_bytes, void* stream);
 
-/* SYNCHRONIZES the stream, then reports whether any kernel that used this workspace gave
- * up on a bounded wait (AQ_ERR_DEVICE_TIMEOUT) since the workspace was last used by a
- * call; AQ_OK otherwise. */
+/* SYNCHRONIZES the stream, then reports whether a kernel of the most recent call that used
+ * this workspace gave up on a bounded wait (AQ_ERR_DEVICE_TIMEOUT); AQ_OK otherwise. Every
+ * aq_linear_* / aq_gemm_w4 / aq_quantize_act call clears the record when it starts. */
 int aq_check_workspace(aq_handle_t h, const void* workspace, void* stream);
 
 #ifdef __cplusplus

@@ -1,0 +1,327 @@
+// C ABI of the library: argument checks, workspace carving and kernel sequencing. Every
+// step of the layer runs in the kernels of the sibling files; nothing here computes.
+#include <new>
+
+#include "aq_common.cuh"
+
+struct aq_context {
+    aq::DeviceInfo dev;
+    int last_cuda_error;
+    int kernel_choice;
+};
+
+namespace {
+
+using namespace aq;
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) & (a - 1)) == 0; }
+inline size_t up256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+int cuda_fail(aq_handle_t h, cudaError_t e) {
+    if (h) h->last_cuda_error = (int)e;
+    return AQ_ERR_CUDA;
+}
+
+int check_shape(int M, int K, int N, int group) {
+    if (M < 1 || N < 1) return AQ_ERR_SHAPE;
+    if (K < 128 || K > 65536 || K % 128 != 0) return AQ_ERR_SHAPE;
+    if (group != 0 && group != 128) return AQ_ERR_SHAPE;
+    if ((size_t)M * (size_t)N > ((size_t)1 << 40)) return AQ_ERR_SHAPE;
+    return AQ_OK;
+}
+
+struct Workspace {
+    Control* ctl;
+    int8_t* codes;
+    void* scratch;
+    size_t scratch_bytes;
+};
+
+size_t workspace_bytes(int M, int K) {
+    return sizeof(Control) + up256((size_t)M * K) + up256((size_t)M);
+}
+
+Workspace carve(void* ws, int M, int K) {
+    Workspace w;
+    uint8_t* b = static_cast<uint8_t*>(ws);
+    w.ctl = reinterpret_cast<Control*>(b);
+    w.codes = reinterpret_cast<int8_t*>(b + sizeof(Control));
+    w.scratch = b + sizeof(Control) + up256((size_t)M * K);
+    w.scratch_bytes = up256((size_t)M);
+    return w;
+}
+
+int run_gemm(aq_handle_t h, const GemmArgs& g, cudaStream_t stream) {
+    int choice = h->kernel_choice;
+    if (choice == AQ_KERNEL_AUTO) choice = g.M <= 16 ? AQ_KERNEL_DECODE : AQ_KERNEL_TENSOR;
+    const cudaError_t e = choice == AQ_KERNEL_DECODE ? launch_gemm_decode(g, h->dev, stream)
+                                                     : launch_gemm_tensor(g, h->dev, stream);
+    return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
+int linear_impl(aq_handle_t h, int bits, const void* x, int M, int K, const void* w_packed,
+                const void* w_scales, int N, int group, int scale_mode, int clip_shift_or_exp,
+                const int32_t* row_idx, void* y, int32_t* acc_dump, void* workspace, size_t workspace_bytes_,
+                void* stream_) {
+    if (!h || !x || !w_packed || !w_scales || !y) return AQ_ERR_INVALID_ARG;
+    if (scale_mode != AQ_SCALE_DYNAMIC && scale_mode != AQ_SCALE_STATIC) return AQ_ERR_INVALID_ARG;
+    if (scale_mode == AQ_SCALE_DYNAMIC && (clip_shift_or_exp < 0 || clip_shift_or_exp > 16)) return AQ_ERR_INVALID_ARG;
+    if (scale_mode == AQ_SCALE_STATIC && (clip_shift_or_exp < -40 || clip_shift_or_exp > 40)) return AQ_ERR_INVALID_ARG;
+    const int s = check_shape(M, K, N, group);
+    if (s != AQ_OK) return s;
+    if (!workspace || workspace_bytes_ < workspace_bytes(M, K)) return AQ_ERR_WORKSPACE;
+    if (!aligned(x, 16) || !aligned(w_packed, 16) || !aligned(w_scales, 2) || !aligned(y, 2) ||
+        !aligned(workspace, 256) || (acc_dump && !aligned(acc_dump, 4)) || (row_idx && !aligned(row_idx, 4)))
+        return AQ_ERR_ALIGNMENT;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const Workspace w = carve(workspace, M, K);
+    cudaError_t e = cudaMemsetAsync(w.ctl, 0, sizeof(Control), stream);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    const __half* xh = static_cast<const __half*>(x);
+    if (scale_mode == AQ_SCALE_DYNAMIC) {
+        e = launch_absmax(xh, M, K, row_idx, w.ctl, h->dev, stream);
+        if (e != cudaSuccess) return cuda_fail(h, e);
+    }
+    e = launch_quantize(xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, w.ctl, w.codes, nullptr,
+                        h->dev, stream);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    GemmArgs g;
+    g.q = w.codes; g.M = M; g.K = K; g.N = N; g.group = group;
+    g.w_packed = static_cast<const uint8_t*>(w_packed);
+    g.w_scales = static_cast<const __half*>(w_scales);
+    g.scale_exp = &w.ctl->scale_exp;
+    g.y = static_cast<__half*>(y);
+    g.acc_dump = acc_dump;
+    g.ctl = w.ctl; g.scratch = w.scratch; g.scratch_bytes = w.scratch_bytes;
+    return run_gemm(h, g, stream);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* aq_status_string(int status) {
+    switch (status) {
+        case AQ_OK: return "ok";
+        case AQ_ERR_INVALID_ARG: return "invalid argument";
+        case AQ_ERR_SHAPE: return "unsupported shape";
+        case AQ_ERR_ALIGNMENT: return "misaligned pointer";
+        case AQ_ERR_WORKSPACE: return "workspace missing or too small";
+        case AQ_ERR_UNSUPPORTED_DEVICE: return "device is not compute capability 10.0";
+        case AQ_ERR_CUDA: return "CUDA call failed";
+        case AQ_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel gave up";
+        default: return "unknown status";
+    }
+}
+
+int aq_version(void) { return 100; }
+
+int aq_create(aq_handle_t* out, int device) {
+    if (!out) return AQ_ERR_INVALID_ARG;
+    *out = nullptr;
+    cudaDeviceProp prop;
+    cudaError_t e = cudaGetDeviceProperties(&prop, device);
+    if (e != cudaSuccess) return AQ_ERR_CUDA;
+    if (prop.major != 10 || prop.minor != 0) return AQ_ERR_UNSUPPORTED_DEVICE;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) return AQ_ERR_CUDA;
+    aq_context* c = new (std::nothrow) aq_context();
+    if (!c) return AQ_ERR_INVALID_ARG;
+    c->dev.device = device;
+    c->dev.sm_count = prop.multiProcessorCount;
+    c->dev.cc_major = prop.major;
+    c->dev.cc_minor = prop.minor;
+    c->dev.smem_optin = prop.sharedMemPerBlockOptin;
+    c->dev.encode_tiled = fn;
+    c->last_cuda_error = 0;
+    c->kernel_choice = AQ_KERNEL_AUTO;
+    *out = c;
+    return AQ_OK;
+}
+
+int aq_destroy(aq_handle_t h) {
+    delete h;
+    return AQ_OK;
+}
+
+int aq_last_cuda_error(aq_handle_t h) { return h ? h->last_cuda_error : 0; }
+
+int aq_set_kernel(aq_handle_t h, int kernel) {
+    if (!h || kernel < AQ_KERNEL_AUTO || kernel > AQ_KERNEL_DECODE) return AQ_ERR_INVALID_ARG;
+    h->kernel_choice = kernel;
+    return AQ_OK;
+}
+
+size_t aq_packed_w4_bytes(int N, int K) {
+    if (N < 1 || K < 128 || K % 128) return 0;
+    return (size_t)round_up(N, kTileN) * (size_t)K / 2;
+}
+
+size_t aq_scales_bytes(int N, int K, int group_size) {
+    if (N < 1 || K < 128 || K % 128 || (group_size != 0 && group_size != 128)) return 0;
+    const size_t G = group_size ? (size_t)K / 128 : 1;
+    return G * (size_t)round_up(N, kTileN) * sizeof(__half);
+}
+
+size_t aq_workspace_bytes(int M, int K, int N, int group_size) {
+    if (check_shape(M, K, N, group_size) != AQ_OK) return 0;
+    return workspace_bytes(M, K);
+}
+
+int aq_pack_w4(aq_handle_t h, const void* w_fp16, int N, int K, int group_size, void* w_packed,
+               void* w_scales, void* stream) {
+    if (!h || !w_fp16 || !w_packed || !w_scales) return AQ_ERR_INVALID_ARG;
+    const int s = check_shape(1, K, N, group_size);
+    if (s != AQ_OK) return s;
+    if (!aligned(w_fp16, 16) || !aligned(w_packed, 16) || !aligned(w_scales, 2)) return AQ_ERR_ALIGNMENT;
+    const cudaError_t e = launch_pack_w4(static_cast<const __half*>(w_fp16), N, K, group_size,
+                                         static_cast<uint8_t*>(w_packed), static_cast<__half*>(w_scales),
+                                         static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
+int aq_unpack_w4(aq_handle_t h, const void* w_packed, int N, int K, int8_t* codes, void* stream) {
+    if (!h || !w_packed || !codes) return AQ_ERR_INVALID_ARG;
+    const int s = check_shape(1, K, N, 0);
+    if (s != AQ_OK) return s;
+    const cudaError_t e = launch_unpack_w4(static_cast<const uint8_t*>(w_packed), N, K, codes,
+                                           static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
+int aq_quantize_act(aq_handle_t h, const void* x_fp16, int M, int K, int bits, int scale_mode,
+                    int clip_shift_or_exp, const int32_t* row_idx, int8_t* q, int32_t* scale_exp_out,
+                    void* workspace, size_t workspace_bytes_, void* stream_) {
+    if (!h || !x_fp16 || !q) return AQ_ERR_INVALID_ARG;
+    if (bits != 8 && bits != 4) return AQ_ERR_INVALID_ARG;
+    if (scale_mode != AQ_SCALE_DYNAMIC && scale_mode != AQ_SCALE_STATIC) return AQ_ERR_INVALID_ARG;
+    if (scale_mode == AQ_SCALE_DYNAMIC && (clip_shift_or_exp < 0 || clip_shift_or_exp > 16)) return AQ_ERR_INVALID_ARG;
+    if (scale_mode == AQ_SCALE_STATIC && (clip_shift_or_exp < -40 || clip_shift_or_exp > 40)) return AQ_ERR_INVALID_ARG;
+    const int s = check_shape(M, K, 1, 0);
+    if (s != AQ_OK) return s;
+    if (!workspace || workspace_bytes_ < sizeof(Control)) return AQ_ERR_WORKSPACE;
+    if (!aligned(x_fp16, 16) || !aligned(q, 16) || !aligned(workspace, 256) ||
+        (scale_exp_out && !aligned(scale_exp_out, 4)))
+        return AQ_ERR_ALIGNMENT;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    Control* ctl = static_cast<Control*>(workspace);
+    cudaError_t e = cudaMemsetAsync(ctl, 0, sizeof(Control), stream);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    const __half* xh = static_cast<const __half*>(x_fp16);
+    if (scale_mode == AQ_SCALE_DYNAMIC) {
+        e = launch_absmax(xh, M, K, row_idx, ctl, h->dev, stream);
+        if (e != cudaSuccess) return cuda_fail(h, e);
+    }
+    e = launch_quantize(xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, ctl, q, scale_exp_out, h->dev,
+                        stream);
+    return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
+int aq_linear_w4a8(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed,
+                   const void* w_scales, int N, int group_size, int scale_mode, int clip_shift_or_exp,
+                   const int32_t* row_idx, void* y_fp16, int32_t* acc_dump, void* workspace,
+                   size_t workspace_bytes_, void* stream) {
+    return linear_impl(h, 8, x_fp16, M, K, w_packed, w_scales, N, group_size, scale_mode, clip_shift_or_exp,
+                       row_idx, y_fp16, acc_dump, workspace, workspace_bytes_, stream);
+}
+
+int aq_linear_w4a4(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed,
+                   const void* w_scales, int N, int group_size, int scale_mode, int clip_shift_or_exp,
+                   const int32_t* row_idx, void* y_fp16, int32_t* acc_dump, void* workspace,
+                   size_t workspace_bytes_, void* stream) {
+    return linear_impl(h, 4, x_fp16, M, K, w_packed, w_scales, N, group_size, scale_mode, clip_shift_or_exp,
+                       row_idx, y_fp16, acc_dump, workspace, workspace_bytes_, stream);
+}
+
+int aq_gemm_w4(aq_handle_t h, const int8_t* q, int M, int K, const void* w_packed, const void* w_scales,
+               int N, int group_size, const int32_t* scale_exp, void* y_fp16, int32_t* acc_dump,
+               void* workspace, size_t workspace_bytes_, void* stream_) {
+    if (!h || !q || !w_packed || !w_scales || !scale_exp || !y_fp16) return AQ_ERR_INVALID_ARG;
+    const int s = check_shape(M, K, N, group_size);
+    if (s != AQ_OK) return s;
+    if (!workspace || workspace_bytes_ < workspace_bytes(M, K)) return AQ_ERR_WORKSPACE;
+    if (!aligned(q, 16) || !aligned(w_packed, 16) || !aligned(w_scales, 2) || !aligned(y_fp16, 2) ||
+        !aligned(workspace, 256) || !aligned(scale_exp, 4) || (acc_dump && !aligned(acc_dump, 4)))
+        return AQ_ERR_ALIGNMENT;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const Workspace w = carve(workspace, M, K);
+    const cudaError_t e = cudaMemsetAsync(w.ctl, 0, sizeof(Control), stream);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    GemmArgs g;
+    g.q = q; g.M = M; g.K = K; g.N = N; g.group = group_size;
+    g.w_packed = static_cast<const uint8_t*>(w_packed);
+    g.w_scales = static_cast<const __half*>(w_scales);
+    g.scale_exp = scale_exp;
+    g.y = static_cast<__half*>(y_fp16);
+    g.acc_dump = acc_dump;
+    g.ctl = w.ctl; g.scratch = w.scratch; g.scratch_bytes = w.scratch_bytes;
+    return run_gemm(h, g, stream);
+}
+
+int aq_token_select(aq_handle_t h, const float* scores, int M, int n_keep, int32_t* idx, void* workspace,
+                    size_t workspace_bytes_, void* stream) {
+    if (!h || !scores || (!idx && n_keep > 0)) return AQ_ERR_INVALID_ARG;
+    if (M < 1 || M > 65536 || n_keep < 0 || n_keep > M) return AQ_ERR_SHAPE;
+    if (!workspace || workspace_bytes_ < sizeof(Control) + up256((size_t)M)) return AQ_ERR_WORKSPACE;
+    if (!aligned(scores, 4) || !aligned(idx, 4) || !aligned(workspace, 256)) return AQ_ERR_ALIGNMENT;
+    const cudaError_t e = launch_token_select(scores, M, n_keep, idx,
+                                              static_cast<uint8_t*>(workspace) + sizeof(Control),
+                                              static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
+int aq_token_compact(aq_handle_t h, const void* x_fp16, int M, int K, const int32_t* idx, int n_keep,
+                     void* x_out, void* stream) {
+    if (!h || !x_fp16 || !idx || !x_out) return AQ_ERR_INVALID_ARG;
+    if (M < 1 || n_keep < 0 || n_keep > M || K < 8 || K % 8) return AQ_ERR_SHAPE;
+    if (!aligned(x_fp16, 16) || !aligned(x_out, 16) || !aligned(idx, 4)) return AQ_ERR_ALIGNMENT;
+    const cudaError_t e = launch_token_compact(static_cast<const __half*>(x_fp16), K, idx, n_keep,
+                                               static_cast<__half*>(x_out), h->dev,
+                                               static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
+size_t aq_linear_host_scratch_bytes(int M, int K, int N, int group_size) {
+    if (check_shape(M, K, N, group_size) != AQ_OK) return 0;
+    return up256((size_t)M * K * 2) + up256((size_t)M * N * 2) + workspace_bytes(M, K);
+}
+
+int aq_linear_host(aq_handle_t h, int bits, const void* x_host, int M, int K, const void* w_packed,
+                   const void* w_scales, int N, int group_size, int scale_mode, int clip_shift_or_exp,
+                   void* y_host, void* device_scratch, size_t scratch_bytes, void* stream_) {
+    if (!h || !x_host || !y_host) return AQ_ERR_INVALID_ARG;
+    if (bits != 8 && bits != 4) return AQ_ERR_INVALID_ARG;
+    const int s = check_shape(M, K, N, group_size);
+    if (s != AQ_OK) return s;
+    if (!device_scratch || scratch_bytes < aq_linear_host_scratch_bytes(M, K, N, group_size)) return AQ_ERR_WORKSPACE;
+    if (!aligned(device_scratch, 256)) return AQ_ERR_ALIGNMENT;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    uint8_t* b = static_cast<uint8_t*>(device_scratch);
+    void* x_dev = b;
+    void* y_dev = b + up256((size_t)M * K * 2);
+    void* ws = b + up256((size_t)M * K * 2) + up256((size_t)M * N * 2);
+    cudaError_t e = cudaMemcpyAsync(x_dev, x_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    const int rc = linear_impl(h, bits, x_dev, M, K, w_packed, w_scales, N, group_size, scale_mode,
+                               clip_shift_or_exp, nullptr, y_dev, nullptr, ws, workspace_bytes(M, K), stream_);
+    if (rc != AQ_OK) return rc;
+    e = cudaMemcpyAsync(y_host, y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, stream);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    e = cudaStreamSynchronize(stream);
+    return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
+int aq_check_workspace(aq_handle_t h, const void* workspace, void* stream_) {
+    if (!h || !workspace) return AQ_ERR_INVALID_ARG;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    cudaError_t e = cudaStreamSynchronize(stream);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    Control c;
+    e = cudaMemcpy(&c, workspace, sizeof(Control), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    return c.status ? AQ_ERR_DEVICE_TIMEOUT : AQ_OK;
+}
+
+}  // extern "C"

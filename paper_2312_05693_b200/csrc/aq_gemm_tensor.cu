@@ -1,0 +1,458 @@
+// Integer product on the 5th-generation tensor cores (tcgen05, kind::i8) with TMEM
+// accumulators, for the sums of Sec. 4.4 / Algorithm 1 and the floating-point output.
+//
+// Operand roles are swapped with respect to y = x w^T: the 128 output channels of a tile
+// are the MMA's M dimension and the tokens its N dimension, so that
+//   * the 4-bit weights never touch shared memory: four warps read the packed layout from
+//     global memory (512 contiguous bytes per warp load), widen each nibble to the int8
+//     value 16*code with two logic ops per word, and store the result straight into
+//     tensor memory, where the MMA reads it as its A operand;
+//   * every epilogue thread owns one output channel, so its weight scale(s) sit in a
+//     register and the per-128-k group rescaling costs one FMA per element;
+//   * the int8 activation tile (tokens x 128 k) is the only shared-memory operand, staged
+//     by TMA with the 128-byte swizzle and read through an MMA shared-memory descriptor.
+//
+// One persistent CTA per SM walks a static list of (channel tile, token tile) pairs.
+// Warp roles: 0 = TMA producer, 1 = MMA issue + TMEM allocation, 2-5 = weight unpack,
+// 6-9 = epilogue. Two accumulator stages in TMEM let the epilogue of one accumulation
+// overlap the MMAs of the next. Every wait is bounded; on expiry the CTA records a status
+// word, stops issuing work and leaves through the common exit that frees TMEM.
+#include <cuda.h>
+
+#include "aq_common.cuh"
+
+namespace aq {
+
+namespace {
+
+constexpr int kNumStages = 6;                 // ring depth: activation tiles (smem) and weight slices (TMEM)
+constexpr int kUnpackPrefetch = 4;            // packed 128-k blocks held in registers per unpack thread
+constexpr int kThreads = 320;
+constexpr int kAColsPerStage = 32;            // 128 k of int8 = 32 TMEM columns per lane
+constexpr unsigned long long kWaitCycles = 4000000000ull;   // ~2 s
+
+// ------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait. Returns false when the limit ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 0x3FFu) == 0) {
+            if (*abort_flag) return false;
+            if ((unsigned long long)(clock64() - t0) > kWaitCycles) {
+                *abort_flag = 1;
+                return false;
+            }
+        }
+    }
+    return true;
+}
+// The same for a whole warp: all lanes agree on the outcome before any warp-wide instruction.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+    return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag) ? 1 : 0) != 0;
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem descriptor]; int8 x int8 -> int32.
+__device__ __forceinline__ void tc_mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor for a K-major tile whose rows are 128 bytes, written by
+// TMA with the 128-byte swizzle: start address >> 4 in bits 0-13, stride between 8-row
+// groups (1024 B) >> 4 in bits 32-45, descriptor version 1 in bits 46-47, swizzle mode 2
+// (128 B) in bits 61-63. The leading-dimension field is not used for this layout.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+// Instruction descriptor for kind::i8: D = s32 (2) at bits 4-5, A and B signed 8-bit (1) at
+// bits 7-9 and 10-12, both K-major (bits 15, 16 = 0), N >> 3 at bits 17-22, M >> 4 at 24-28.
+__host__ __device__ constexpr uint32_t idesc_i8(int m, int n) {
+    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+template <int BM>
+struct SharedStorage {
+    alignas(1024) uint8_t x[kNumStages][BM * 128];   // activation tiles, 128-byte swizzled rows
+    alignas(8) uint64_t full[kNumStages];            // TMA bytes + 4 unpack warps -> MMA
+    uint64_t empty[kNumStages];                      // MMA done with the stage -> producers
+    uint64_t acc_full[2];                            // MMA -> epilogue
+    uint64_t acc_empty[2];                           // epilogue (4 warps) -> MMA
+    uint32_t tmem_base;
+    volatile uint32_t abort_flag;
+};
+
+struct TensorParams {
+    int M, K, N, Npad;
+    int n_tiles_m, n_tiles;        // token tiles; total tiles
+    const uint8_t* w_packed;
+    const __half* w_scales;
+    const int32_t* scale_exp;
+    __half* y;
+    int32_t* acc_dump;
+    Control* ctl;
+};
+
+template <int BM, bool GROUPED>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    using Smem = SharedStorage<BM>;
+    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+
+    constexpr int kAccCols = 2 * BM;
+    constexpr int kTmemColsUsed = kAccCols + kNumStages * kAColsPerStage;
+    constexpr int kTmemCols = kTmemColsUsed <= 128 ? 128 : kTmemColsUsed <= 256 ? 256 : 512;
+    static_assert(kTmemColsUsed <= 512, "tensor memory has 512 columns");
+    static_assert(BM % 32 == 0 && BM >= 32 && BM <= 256, "token tile");
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int KB = p.K / kTileK;
+    const int my_tiles = p.n_tiles > (int)blockIdx.x
+                             ? (p.n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+    const long long total_iters = (long long)my_tiles * KB;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kNumStages; ++s) {
+            mbar_init(&sm.full[s], 1 + 4);
+            mbar_init(&sm.empty[s], 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(&sm.acc_full[a], 1);
+            mbar_init(&sm.acc_empty[a], 4);
+        }
+        sm.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&sm.tmem_base)), "r"((uint32_t)kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+    const uint32_t tmem_acc = tmem;                 // columns [0, 2*BM)
+    const uint32_t tmem_a = tmem + kAccCols;        // columns [2*BM, 2*BM + stages*32)
+    volatile uint32_t* abort_flag = &sm.abort_flag;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            long long it = 0;
+            for (int tl = 0; tl < my_tiles; ++tl) {
+                const int tile = blockIdx.x + tl * gridDim.x;
+                const int mt = tile % p.n_tiles_m;
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    const int s = (int)(it % kNumStages);
+                    const uint32_t ph = (uint32_t)(it / kNumStages) & 1u;
+                    if (!mbar_wait(&sm.empty[s], ph ^ 1u, abort_flag)) goto role_done;
+                    mbar_arrive_expect_tx(&sm.full[s], BM * 128);
+                    tma_load_2d(sm.x[s], &x_map, kb * kTileK, mt * BM, &sm.full[s]);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_i8(128, BM);
+            long long it = 0;
+            long long unit = 0;      // accumulations handed to the epilogue so far
+            for (int tl = 0; tl < my_tiles; ++tl) {
+                for (int kb = 0; kb < KB; ++kb, ++it) {
+                    const bool first = GROUPED || kb == 0;
+                    const int a = (int)(unit & 1);
+                    if (first) {
+                        const uint32_t aph = (uint32_t)(unit >> 1) & 1u;
+                        if (!mbar_wait(&sm.acc_empty[a], aph ^ 1u, abort_flag)) goto role_done;
+                        tc_fence_after();
+                    }
+                    const int s = (int)(it % kNumStages);
+                    const uint32_t ph = (uint32_t)(it / kNumStages) & 1u;
+                    if (!mbar_wait(&sm.full[s], ph, abort_flag)) goto role_done;
+                    tc_fence_after();
+                    const uint32_t d_addr = tmem_acc + (uint32_t)(a * BM);
+                    const uint32_t a_addr = tmem_a + (uint32_t)(s * kAColsPerStage);
+                    const uint64_t bdesc = smem_desc_sw128(smem_u32(sm.x[s]));
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        // 32 k per instruction: 8 TMEM columns of A, 32 bytes along the swizzled row of B
+                        tc_mma_i8_ts(d_addr, a_addr + 8 * j, bdesc + (uint64_t)(2 * j), idesc,
+                                     (first && j == 0) ? 0u : 1u);
+                    }
+                    tc_commit(&sm.empty[s]);
+                    const bool last = GROUPED || kb == KB - 1;
+                    if (last) {
+                        tc_commit(&sm.acc_full[a]);
+                        ++unit;
+                    }
+                }
+            }
+        }
+    } else if (warp < 6) {
+        // --------------------------------------------------- weight unpack -> tensor memory
+        const int quarter = warp & 3;
+        const int r = quarter * 32 + lane;            // row inside the 128-channel tile = TMEM lane
+        const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        uint4 buf[kUnpackPrefetch][4];
+        auto block_ptr = [&](long long it) -> const uint4* {
+            const int tl = (int)(it / KB), kb = (int)(it % KB);
+            const int tile = blockIdx.x + tl * gridDim.x;
+            const int nt = tile / p.n_tiles_m;
+            return reinterpret_cast<const uint4*>(p.w_packed + ((size_t)nt * KB + kb) * kBlockBytes) + r;
+        };
+#pragma unroll
+        for (int d = 0; d < kUnpackPrefetch; ++d) {
+            if (d < total_iters) {
+                const uint4* src = block_ptr(d);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) buf[d][j] = __ldg(src + j * kTileN);
+            }
+        }
+        for (long long it0 = 0; it0 < total_iters; it0 += kUnpackPrefetch) {
+#pragma unroll
+            for (int d = 0; d < kUnpackPrefetch; ++d) {
+                const long long it = it0 + d;
+                if (it >= total_iters) break;
+                uint32_t v[32];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t w[4] = {buf[d][j].x, buf[d][j].y, buf[d][j].z, buf[d][j].w};
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        v[8 * j + 2 * i] = (w[i] << 4) & 0xF0F0F0F0u;
+                        v[8 * j + 2 * i + 1] = w[i] & 0xF0F0F0F0u;
+                    }
+                }
+                if (it + kUnpackPrefetch < total_iters) {
+                    const uint4* src = block_ptr(it + kUnpackPrefetch);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) buf[d][j] = __ldg(src + j * kTileN);
+                }
+                const int s = (int)(it % kNumStages);
+                const uint32_t ph = (uint32_t)(it / kNumStages) & 1u;
+                if (!mbar_wait_warp(&sm.empty[s], ph ^ 1u, abort_flag)) goto role_done;
+                tc_fence_after();
+                tc_st32(tmem_a + lane_addr + (uint32_t)(s * kAColsPerStage), v);
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.full[s]);
+            }
+        }
+    } else {
+        // ----------------------------------------------------------------------- epilogue
+        const int quarter = warp & 3;
+        const int r = quarter * 32 + lane;
+        const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        const float pe = __int_as_float((127 + *p.scale_exp) << 23);     // 2^e
+        const int G = GROUPED ? KB : 1;
+        long long unit = 0;
+        for (int tl = 0; tl < my_tiles; ++tl) {
+            const int tile = blockIdx.x + tl * gridDim.x;
+            const int mt = tile % p.n_tiles_m, nt = tile / p.n_tiles_m;
+            const int n = nt * kTileN + r;
+            const int m_base = mt * BM;
+            const bool n_ok = n < p.N;
+            if (!GROUPED) {
+                const int a = (int)(unit & 1);
+                const uint32_t aph = (uint32_t)(unit >> 1) & 1u;
+                const float sc = __half2float(p.w_scales[n]) * 0.0625f * pe;   // sums carry a factor 16
+                if (!mbar_wait_warp(&sm.acc_full[a], aph, abort_flag)) goto role_done;
+                tc_fence_after();
+#pragma unroll 1
+                for (int c0 = 0; c0 < BM; c0 += 32) {
+                    uint32_t v[32];
+                    tc_ld32(tmem_acc + lane_addr + (uint32_t)(a * BM + c0), v);
+                    tc_wait_ld();
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) {
+                        const int m = m_base + c0 + c;
+                        if (n_ok && m < p.M) {
+                            const int acc16 = (int)v[c];
+                            p.y[(size_t)m * p.N + n] = __float2half_rn((float)acc16 * sc);
+                            if (p.acc_dump) p.acc_dump[(size_t)m * p.N + n] = acc16 >> 4;
+                        }
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.acc_empty[a]);
+                ++unit;
+            } else {
+                float fsum[BM];
+#pragma unroll
+                for (int c = 0; c < BM; ++c) fsum[c] = 0.0f;
+                float s_next = __half2float(p.w_scales[n]) * 0.0625f;
+                for (int kb = 0; kb < KB; ++kb, ++unit) {
+                    const int a = (int)(unit & 1);
+                    const uint32_t aph = (uint32_t)(unit >> 1) & 1u;
+                    const float s = s_next;
+                    if (kb + 1 < KB) s_next = __half2float(p.w_scales[(size_t)(kb + 1) * p.Npad + n]) * 0.0625f;
+                    if (!mbar_wait_warp(&sm.acc_full[a], aph, abort_flag)) goto role_done;
+                    tc_fence_after();
+#pragma unroll
+                    for (int c0 = 0; c0 < BM; c0 += 32) {
+                        uint32_t v[32];
+                        tc_ld32(tmem_acc + lane_addr + (uint32_t)(a * BM + c0), v);
+                        tc_wait_ld();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            fsum[c0 + c] = fmaf((float)(int)v[c], s, fsum[c0 + c]);
+                            if (p.acc_dump) {
+                                const int m = m_base + c0 + c;
+                                if (n_ok && m < p.M)
+                                    p.acc_dump[((size_t)m * p.N + n) * G + kb] = (int)v[c] >> 4;
+                            }
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm.acc_empty[a]);
+                }
+#pragma unroll
+                for (int c = 0; c < BM; ++c) {
+                    const int m = m_base + c;
+                    if (n_ok && m < p.M) p.y[(size_t)m * p.N + n] = __float2half_rn(fsum[c] * pe);
+                }
+            }
+        }
+    }
+
+role_done:
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (sm.abort_flag) {
+        // Give copies that may still be in flight time to land before shared memory is released.
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+        if (threadIdx.x == 0) atomicOr(&p.ctl->status, 1u);
+    }
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kTmemCols)
+                     : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+template <int BM, bool GROUPED>
+cudaError_t launch_bm(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
+    using Smem = SharedStorage<BM>;
+    const size_t smem_bytes = sizeof(Smem) + 1024;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_tensor_kernel<BM, GROUPED>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    CUtensorMap map;
+    const cuuint64_t dims[2] = {(cuuint64_t)a.K, (cuuint64_t)a.M};
+    const cuuint64_t strides[1] = {(cuuint64_t)a.K};
+    const cuuint32_t box[2] = {128u, (cuuint32_t)BM};
+    const cuuint32_t estr[2] = {1u, 1u};
+    const CUresult r = reinterpret_cast<EncodeTiledFn>(dev.encode_tiled)(
+        &map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(a.q), dims, strides, box, estr,
+        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+
+    TensorParams p;
+    p.M = a.M; p.K = a.K; p.N = a.N; p.Npad = round_up(a.N, kTileN);
+    p.n_tiles_m = (a.M + BM - 1) / BM;
+    p.n_tiles = p.n_tiles_m * (p.Npad / kTileN);
+    p.w_packed = a.w_packed; p.w_scales = a.w_scales; p.scale_exp = a.scale_exp;
+    p.y = a.y; p.acc_dump = a.acc_dump; p.ctl = a.ctl;
+    const int grid = p.n_tiles < dev.sm_count ? p.n_tiles : dev.sm_count;
+    gemm_tensor_kernel<BM, GROUPED><<<grid, kThreads, smem_bytes, stream>>>(map, p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_gemm_tensor(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
+    if (a.M <= 32) return a.group ? launch_bm<32, true>(a, dev, stream) : launch_bm<32, false>(a, dev, stream);
+    if (a.M <= 64) return a.group ? launch_bm<64, true>(a, dev, stream) : launch_bm<64, false>(a, dev, stream);
+    return a.group ? launch_bm<128, true>(a, dev, stream) : launch_bm<128, false>(a, dev, stream);
+}
+
+}  // namespace aq
