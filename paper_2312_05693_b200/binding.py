@@ -1,0 +1,247 @@
+"""ctypes binding for libagileq.so: same names as the C ABI, argument marshalling only.
+
+Tensors are torch CUDA tensors used purely as device memory; every step of the layer runs
+in the library's kernels. Nothing here computes, and nothing falls back to another path:
+if the library is missing or the device is not a B200 the calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import re
+from typing import Optional, Tuple
+
+import torch
+
+_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_DIR, "libagileq.so")
+HEADER_PATH = os.path.join(os.path.dirname(_DIR), "include", "agileq.h")
+
+AQ_OK = 0
+AQ_ERR_INVALID_ARG, AQ_ERR_SHAPE, AQ_ERR_ALIGNMENT, AQ_ERR_WORKSPACE = -1, -2, -3, -4
+AQ_ERR_UNSUPPORTED_DEVICE, AQ_ERR_CUDA, AQ_ERR_DEVICE_TIMEOUT = -5, -6, -7
+AQ_SCALE_DYNAMIC, AQ_SCALE_STATIC = 0, 1
+AQ_KERNEL_AUTO, AQ_KERNEL_TENSOR, AQ_KERNEL_DECODE = 0, 1, 2
+
+_lib = None
+
+
+class AgileqError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {status_string(status)} ({status})")
+
+
+def declared_symbols() -> list:
+    """Names of the functions declared in include/agileq.h."""
+    text = open(HEADER_PATH).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(aq_[a-z0-9_]+)\s*\(", text)))
+
+
+def load():
+    """Loads the CUDA library; raises if it was not built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2312_05693_b200.build` "
+                          "(there is no fallback implementation)")
+    L = C.CDLL(LIB_PATH)
+    vp, i32, sz = C.c_void_p, C.c_int, C.c_size_t
+    L.aq_status_string.restype = C.c_char_p
+    L.aq_status_string.argtypes = [i32]
+    L.aq_version.restype = i32
+    L.aq_create.argtypes = [C.POINTER(vp), i32]
+    L.aq_destroy.argtypes = [vp]
+    L.aq_last_cuda_error.argtypes = [vp]
+    L.aq_set_kernel.argtypes = [vp, i32]
+    for f in ("aq_packed_w4_bytes",):
+        getattr(L, f).restype = sz
+        getattr(L, f).argtypes = [i32, i32]
+    L.aq_scales_bytes.restype = sz
+    L.aq_scales_bytes.argtypes = [i32, i32, i32]
+    L.aq_workspace_bytes.restype = sz
+    L.aq_workspace_bytes.argtypes = [i32, i32, i32, i32]
+    L.aq_linear_host_scratch_bytes.restype = sz
+    L.aq_linear_host_scratch_bytes.argtypes = [i32, i32, i32, i32]
+    L.aq_pack_w4.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
+    L.aq_unpack_w4.argtypes = [vp, vp, i32, i32, vp, vp]
+    L.aq_quantize_act.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, sz, vp]
+    lin = [vp, vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, sz, vp]
+    L.aq_linear_w4a8.argtypes = lin
+    L.aq_linear_w4a4.argtypes = lin
+    L.aq_gemm_w4.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, vp, vp, vp, vp, sz, vp]
+    L.aq_token_select.argtypes = [vp, vp, i32, i32, vp, vp, sz, vp]
+    L.aq_token_compact.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp]
+    L.aq_linear_host.argtypes = [vp, i32, vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, vp, sz, vp]
+    L.aq_check_workspace.argtypes = [vp, vp, vp]
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return load().aq_status_string(status).decode()
+
+
+def _check(status: int, what: str):
+    if status != AQ_OK:
+        raise AgileqError(status, what)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream() -> C.c_void_p:
+    return C.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def aq_packed_w4_bytes(N: int, K: int) -> int:
+    return load().aq_packed_w4_bytes(N, K)
+
+
+def aq_scales_bytes(N: int, K: int, group_size: int) -> int:
+    return load().aq_scales_bytes(N, K, group_size)
+
+
+def aq_workspace_bytes(M: int, K: int, N: int, group_size: int) -> int:
+    return load().aq_workspace_bytes(M, K, N, group_size)
+
+
+def aq_linear_host_scratch_bytes(M: int, K: int, N: int, group_size: int) -> int:
+    return load().aq_linear_host_scratch_bytes(M, K, N, group_size)
+
+
+class Handle:
+    """aq_create / aq_destroy. Methods mirror the C entry points and enqueue on torch's
+    current stream."""
+
+    def __init__(self, device: int = 0):
+        self._h = C.c_void_p()
+        self.device = device
+        _check(load().aq_create(C.byref(self._h), device), "aq_create")
+
+    def close(self):
+        if self._h:
+            load().aq_destroy(self._h)
+            self._h = C.c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- helpers: device memory only
+    def _dev(self):
+        return torch.device("cuda", self.device)
+
+    def alloc_workspace(self, M: int, K: int, N: int, group_size: int) -> torch.Tensor:
+        n = aq_workspace_bytes(M, K, N, group_size)
+        if n == 0:
+            raise AgileqError(AQ_ERR_SHAPE, "aq_workspace_bytes")
+        return torch.empty(n, dtype=torch.uint8, device=self._dev())
+
+    def aq_set_kernel(self, kernel: int):
+        _check(load().aq_set_kernel(self._h, kernel), "aq_set_kernel")
+
+    def aq_last_cuda_error(self) -> int:
+        return load().aq_last_cuda_error(self._h)
+
+    def aq_pack_w4(self, w: torch.Tensor, group_size: int) -> Tuple[torch.Tensor, torch.Tensor]:
+        """fp16 [N,K] -> (packed uint8 buffer, fp16 scales [G, Npad])."""
+        N, K = w.shape
+        nb, ns = aq_packed_w4_bytes(N, K), aq_scales_bytes(N, K, group_size)
+        if nb == 0 or ns == 0:
+            raise AgileqError(AQ_ERR_SHAPE, "aq_pack_w4")
+        packed = torch.empty(nb, dtype=torch.uint8, device=w.device)
+        G = K // 128 if group_size else 1
+        scales = torch.empty((G, ns // (2 * G)), dtype=torch.float16, device=w.device)
+        _check(load().aq_pack_w4(self._h, _ptr(w), N, K, group_size, _ptr(packed), _ptr(scales), _stream()),
+               "aq_pack_w4")
+        return packed, scales
+
+    def aq_unpack_w4(self, packed: torch.Tensor, N: int, K: int) -> torch.Tensor:
+        codes = torch.empty((N, K), dtype=torch.int8, device=packed.device)
+        _check(load().aq_unpack_w4(self._h, _ptr(packed), N, K, _ptr(codes), _stream()), "aq_unpack_w4")
+        return codes
+
+    def aq_quantize_act(self, x: torch.Tensor, bits: int, scale_mode: int = AQ_SCALE_DYNAMIC,
+                        clip_shift_or_exp: int = 0, row_idx: Optional[torch.Tensor] = None,
+                        workspace: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+        M_in, K = x.shape
+        M = M_in if row_idx is None else row_idx.shape[0]
+        q = torch.empty((M, K), dtype=torch.int8, device=x.device)
+        e = torch.empty(1, dtype=torch.int32, device=x.device)
+        ws = workspace if workspace is not None else torch.empty(256, dtype=torch.uint8, device=x.device)
+        _check(load().aq_quantize_act(self._h, _ptr(x), M, K, bits, scale_mode, clip_shift_or_exp,
+                                      _ptr(row_idx), _ptr(q), _ptr(e), _ptr(ws), ws.numel(), _stream()),
+               "aq_quantize_act")
+        return q, e
+
+    def _linear(self, fn, name, x, packed, scales, N, group_size, scale_mode, clip_shift_or_exp, row_idx,
+                y, acc_dump, workspace):
+        M_in, K = x.shape
+        M = M_in if row_idx is None else row_idx.shape[0]
+        if y is None:
+            y = torch.empty((M, N), dtype=torch.float16, device=x.device)
+        if workspace is None:
+            workspace = self.alloc_workspace(M, K, N, group_size)
+        _check(fn(self._h, _ptr(x), M, K, _ptr(packed), _ptr(scales), N, group_size, scale_mode,
+                  clip_shift_or_exp, _ptr(row_idx), _ptr(y), _ptr(acc_dump), _ptr(workspace),
+                  workspace.numel(), _stream()), name)
+        return y
+
+    def aq_linear_w4a8(self, x, packed, scales, N, group_size, scale_mode=AQ_SCALE_DYNAMIC,
+                       clip_shift_or_exp=0, row_idx=None, y=None, acc_dump=None, workspace=None):
+        return self._linear(load().aq_linear_w4a8, "aq_linear_w4a8", x, packed, scales, N, group_size,
+                            scale_mode, clip_shift_or_exp, row_idx, y, acc_dump, workspace)
+
+    def aq_linear_w4a4(self, x, packed, scales, N, group_size, scale_mode=AQ_SCALE_DYNAMIC,
+                       clip_shift_or_exp=0, row_idx=None, y=None, acc_dump=None, workspace=None):
+        return self._linear(load().aq_linear_w4a4, "aq_linear_w4a4", x, packed, scales, N, group_size,
+                            scale_mode, clip_shift_or_exp, row_idx, y, acc_dump, workspace)
+
+    def aq_gemm_w4(self, q, packed, scales, N, group_size, scale_exp, y=None, acc_dump=None, workspace=None):
+        M, K = q.shape
+        if y is None:
+            y = torch.empty((M, N), dtype=torch.float16, device=q.device)
+        if workspace is None:
+            workspace = self.alloc_workspace(M, K, N, group_size)
+        _check(load().aq_gemm_w4(self._h, _ptr(q), M, K, _ptr(packed), _ptr(scales), N, group_size,
+                                 _ptr(scale_exp), _ptr(y), _ptr(acc_dump), _ptr(workspace),
+                                 workspace.numel(), _stream()), "aq_gemm_w4")
+        return y
+
+    def aq_token_select(self, scores: torch.Tensor, n_keep: int, workspace=None) -> torch.Tensor:
+        M = scores.shape[0]
+        idx = torch.empty(max(n_keep, 1), dtype=torch.int32, device=scores.device)[:n_keep]
+        if workspace is None:
+            workspace = torch.empty(256 + ((M + 255) // 256) * 256, dtype=torch.uint8, device=scores.device)
+        _check(load().aq_token_select(self._h, _ptr(scores), M, n_keep, _ptr(idx), _ptr(workspace),
+                                      workspace.numel(), _stream()), "aq_token_select")
+        return idx
+
+    def aq_token_compact(self, x: torch.Tensor, idx: torch.Tensor, out=None) -> torch.Tensor:
+        M, K = x.shape
+        n_keep = idx.shape[0]
+        if out is None:
+            out = torch.empty((n_keep, K), dtype=torch.float16, device=x.device)
+        _check(load().aq_token_compact(self._h, _ptr(x), M, K, _ptr(idx), n_keep, _ptr(out), _stream()),
+               "aq_token_compact")
+        return out
+
+    def aq_linear_host(self, bits: int, x_host: torch.Tensor, packed, scales, N, group_size,
+                       y_host: torch.Tensor, device_scratch: torch.Tensor,
+                       scale_mode=AQ_SCALE_DYNAMIC, clip_shift_or_exp=0):
+        """x_host / y_host are CPU (ideally pinned) fp16 tensors; synchronizes the stream."""
+        M, K = x_host.shape
+        _check(load().aq_linear_host(self._h, bits, _ptr(x_host), M, K, _ptr(packed), _ptr(scales), N,
+                                     group_size, scale_mode, clip_shift_or_exp, _ptr(y_host),
+                                     _ptr(device_scratch), device_scratch.numel(), _stream()),
+               "aq_linear_host")
+        return y_host
+
+    def aq_check_workspace(self, workspace: torch.Tensor) -> int:
+        return load().aq_check_workspace(self._h, _ptr(workspace), _stream())

@@ -1,0 +1,219 @@
+"""GPU parity: the CUDA library against the CPU checker, element by element, through the
+C ABI. Integer results (weight codes, scales' bit patterns, the layer exponent, activation
+codes, int32 sums, token indices) must be bit-exact; fp16 outputs must satisfy
+max|y_gpu - y_ref| <= 1e-3 * max|y_ref|."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2312_05693_b200 import binding, inputs
+from gpu_util import assert_y_close, dev, handle, run_layer_both, scales_to_oracle_layout
+
+pytestmark = pytest.mark.gpu
+
+TENSOR, DECODE = binding.AQ_KERNEL_TENSOR, binding.AQ_KERNEL_DECODE
+KERNELS = [pytest.param(DECODE, id="decode"), pytest.param(TENSOR, id="tensor")]
+
+
+# ------------------------------------------------------------------------------ weights
+@pytest.mark.parametrize("N,K,group", [(768, 768, 0), (200, 384, 128), (128, 128, 0), (1, 256, 128),
+                                       (384, 1024, 128)])
+def test_pack_w4_codes_and_scales_bit_exact(N, K, group):
+    w = inputs.weights(N, K, seed=N + K)
+    if N > 5:
+        w[3, :] = 0
+        w[4, :128] = 0
+        w[5, 7] = np.float16(6e-8)       # a/7 underflows fp16 in its group when alone
+        w[5, :7] = 0
+        w[5, 8:128] = 0
+    h = handle()
+    packed, scales = h.aq_pack_w4(dev(w), group)
+    codes_gpu = h.aq_unpack_w4(packed, N, K).cpu().numpy()
+    codes, sc = oracle.quantize_weights(w, group)
+    assert np.array_equal(codes_gpu, codes)
+    assert np.array_equal(scales_to_oracle_layout(scales, N).view(np.uint16), sc.view(np.uint16))
+
+
+# -------------------------------------------------------------------------- activations
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("M,K", [(1, 128), (16, 768), (37, 1152), (300, 4096)])
+def test_quantize_act_dynamic(bits, M, K):
+    x = inputs.activations(M, K, seed=M + bits, outlier_frac=0.01, outlier_mult=20.0)
+    for clip in (0, 3):
+        q, e = handle().aq_quantize_act(dev(x), bits, binding.AQ_SCALE_DYNAMIC, clip)
+        e_ref = oracle.layer_exponent(x, bits) - clip
+        assert int(e.item()) == e_ref
+        assert np.array_equal(q.cpu().numpy(), oracle.quantize_act(x, bits, e_ref))
+
+
+def test_quantize_act_static_rowidx_and_nonfinite():
+    M, K = 40, 256
+    x = inputs.activations(M, K, seed=5, outlier_frac=0.01, outlier_mult=20.0)
+    x[3, 5] = np.nan
+    x[7, 9] = np.inf
+    x[8, 1] = -np.inf
+    x[0, 0] = 30000.0                     # dropped by row_idx below
+    rows = np.array([1, 3, 7, 8, 20, 39, 2], np.int32)
+    h = handle()
+    for bits in (8, 4):
+        q, e = h.aq_quantize_act(dev(x), bits, binding.AQ_SCALE_STATIC, -2, row_idx=dev(rows))
+        assert int(e.item()) == -2
+        assert np.array_equal(q.cpu().numpy(), oracle.quantize_act(x, bits, -2, rows))
+        q, e = h.aq_quantize_act(dev(x), bits, binding.AQ_SCALE_DYNAMIC, 0, row_idx=dev(rows))
+        e_ref = oracle.layer_exponent(x, bits, rows)
+        assert int(e.item()) == e_ref == (10 if bits == 8 else 14)      # +Inf counts as 65504
+        assert np.array_equal(q.cpu().numpy(), oracle.quantize_act(x, bits, e_ref, rows))
+    fin = np.array([2, 20, 39], np.int32)
+    q, e = h.aq_quantize_act(dev(x), 8, binding.AQ_SCALE_DYNAMIC, 0, row_idx=dev(fin))
+    assert int(e.item()) == oracle.layer_exponent(x, 8, fin)
+    z = np.zeros((4, 128), np.float16)
+    q, e = h.aq_quantize_act(dev(z), 8)
+    assert int(e.item()) == 0 and not q.any().item()
+
+
+def test_quantize_act_all_fp16_magnitudes_exponent():
+    # one value at a time through the absmax -> exponent path: every binade and mantissa edge
+    h = handle()
+    vals = [6e-8, 1e-4, 0.0078125, 0.99, 0.9921875, 1.0, 7.0, 7.5, 127.0, 127.06, 128.0, 254.0, 255.0,
+            1000.0, 32512.0, 65024.0, 65504.0]
+    for v in vals:
+        x = np.zeros((2, 128), np.float16)
+        x[1, 77] = -v
+        for bits in (8, 4):
+            _, e = h.aq_quantize_act(dev(x), bits)
+            assert int(e.item()) == oracle.layer_exponent(x, bits), (v, bits)
+
+
+# ---------------------------------------------------------------------------- the layer
+SHAPES = [
+    # M, K, N, group
+    (16, 768, 768, 0),         # OPT-125M-like single layer
+    (1, 256, 128, 0),
+    (3, 384, 200, 128),        # ragged N
+    (17, 512, 136, 0),
+    (129, 384, 200, 128),      # spans token tiles with a ragged tail
+    (300, 1024, 384, 0),
+    (260, 1152, 520, 128),
+]
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("M,K,N,group", SHAPES)
+def test_linear_w4a8_matches_checker(kernel, M, K, N, group):
+    x = inputs.activations(M, K, seed=M + N, outlier_frac=0.01, outlier_mult=20.0)
+    w = inputs.weights(N, K, seed=K + N)
+    gpu, ref = run_layer_both(x, w, 8, group, kernel)
+    assert gpu["e"] == ref["e"]
+    assert np.array_equal(gpu["q"], ref["q"])
+    assert np.array_equal(gpu["acc"], ref["acc"])
+    assert_y_close(gpu["y"], ref["y"])
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("M,K,N,group", [(16, 768, 768, 0), (129, 384, 200, 128), (260, 1152, 520, 128)])
+def test_linear_w4a4_matches_checker(kernel, M, K, N, group):
+    x = inputs.activations(M, K, seed=M + N + 1, outlier_frac=0.005, outlier_mult=30.0)
+    w = inputs.weights(N, K, seed=K + N + 1)
+    gpu, ref = run_layer_both(x, w, 4, group, kernel, clip=4)
+    assert gpu["e"] == ref["e"]
+    assert gpu["q"].min() == -8 and gpu["q"].max() == 7
+    assert np.array_equal(gpu["q"], ref["q"])
+    assert np.array_equal(gpu["acc"], ref["acc"])
+    assert_y_close(gpu["y"], ref["y"])
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_linear_extreme_codes_and_patterns(kernel):
+    """Largest-magnitude sums and an identity-like weight matrix: catches layout slips
+    (a swapped nibble, a transposed tile, a wrong swizzle) that random data could blur."""
+    h = handle()
+    M, K, N = 130, 512, 256
+    x = np.full((M, K), -128.0, np.float16)
+    w = np.full((N, K), -1.0, np.float16)                  # codes -7 after a/7 scaling... all equal -> -7
+    gpu, ref = run_layer_both(x, w, 8, 0, kernel, scale_mode=1, clip=0)
+    assert np.array_equal(gpu["acc"], ref["acc"]) and ref["acc"].max() == 128 * 7 * K
+    assert_y_close(gpu["y"], ref["y"])
+    # x[m,k] = small integers depending on (m,k); w picks single k per channel
+    xm = ((np.arange(M)[:, None] * 7 + np.arange(K)[None, :] * 3) % 255 - 127).astype(np.float16)
+    wm = np.zeros((N, K), np.float16)
+    wm[np.arange(N), (np.arange(N) * 5 + 3) % K] = 1.0
+    wm[np.arange(N), (np.arange(N) * 11 + 130) % K] = -0.5
+    for group in (0, 128):
+        gpu, ref = run_layer_both(xm, wm, 8, group, kernel, scale_mode=1, clip=0)
+        assert np.array_equal(gpu["q"], ref["q"])
+        assert np.array_equal(gpu["acc"], ref["acc"])
+        assert_y_close(gpu["y"], ref["y"])
+
+
+@pytest.mark.parametrize("kernel", KERNELS)
+def test_linear_with_row_idx_equals_compacted_input(kernel):
+    M_in, K, N = 200, 512, 256
+    x = inputs.activations(M_in, K, seed=77, outlier_frac=0.01, outlier_mult=25.0)
+    w = inputs.weights(N, K, seed=78)
+    scores = inputs.token_scores(M_in, 77)
+    n_keep = int(math.ceil(0.6 * M_in))
+    idx = oracle.token_select(scores, n_keep)
+    gpu, ref = run_layer_both(x, w, 8, 0, kernel, row_idx=idx)
+    assert gpu["e"] == ref["e"] and np.array_equal(gpu["q"], ref["q"])
+    assert np.array_equal(gpu["acc"], ref["acc"])
+    assert_y_close(gpu["y"], ref["y"])
+
+
+def test_results_are_deterministic_run_to_run():
+    M, K, N = 260, 1152, 520
+    x = inputs.activations(M, K, seed=9, outlier_frac=0.01, outlier_mult=20.0)
+    w = inputs.weights(N, K, seed=10)
+    h = handle()
+    packed, scales = h.aq_pack_w4(dev(w), 128)
+    xd = dev(x)
+    ws = h.alloc_workspace(M, K, N, 128)
+    first = None
+    for _ in range(10):
+        y = h.aq_linear_w4a8(xd, packed, scales, N, 128, workspace=ws).cpu().numpy().view(np.uint16)
+        first = y if first is None else first
+        assert np.array_equal(y, first)
+
+
+# ------------------------------------------------------------------------ token pruning
+@pytest.mark.parametrize("M,ratio", [(1, 1.0), (7, 0.5), (257, 0.6), (4096, 0.6), (1000, 0.0)])
+def test_token_select_and_compact(M, ratio):
+    h = handle()
+    scores = inputs.token_scores(M, seed=M)
+    if M > 100:
+        scores[::3] = scores[1]           # many equal scores around the cut
+    n_keep = int(math.ceil(ratio * M))
+    idx = h.aq_token_select(dev(scores), n_keep).cpu().numpy()
+    ref = oracle.token_select(scores, n_keep)
+    assert np.array_equal(idx, ref)
+    if n_keep:
+        x = inputs.activations(M, 128, seed=M + 1)
+        xp = h.aq_token_compact(dev(x), dev(ref)).cpu().numpy()
+        assert np.array_equal(xp.view(np.uint16), oracle.token_compact(x, ref).view(np.uint16))
+
+
+# --------------------------------------------------------------------- argument checking
+def test_bad_arguments_are_refused():
+    h = handle()
+    x = torch.zeros((4, 256), dtype=torch.float16, device="cuda")
+    w = torch.zeros((128, 256), dtype=torch.float16, device="cuda")
+    packed, scales = h.aq_pack_w4(w, 0)
+    with pytest.raises(binding.AgileqError) as ei:
+        h.aq_linear_w4a8(x, packed, scales, 128, 64)
+    assert ei.value.status == binding.AQ_ERR_SHAPE
+    small = torch.empty(256, dtype=torch.uint8, device="cuda")
+    with pytest.raises(binding.AgileqError) as ei:
+        h.aq_linear_w4a8(x, packed, scales, 128, 0, workspace=small)
+    assert ei.value.status == binding.AQ_ERR_WORKSPACE
+    ws = h.alloc_workspace(4, 256, 128, 0)
+    with pytest.raises(binding.AgileqError) as ei:
+        h.aq_linear_w4a8(x, packed, scales, 128, 0, workspace=ws[1:])
+    assert ei.value.status == binding.AQ_ERR_ALIGNMENT
+    with pytest.raises(binding.AgileqError) as ei:
+        h.aq_quantize_act(x, 5)
+    assert ei.value.status == binding.AQ_ERR_INVALID_ARG
+    with pytest.raises(binding.AgileqError) as ei:
+        h.aq_token_select(torch.zeros(8, device="cuda"), 9)
+    assert ei.value.status == binding.AQ_ERR_SHAPE
