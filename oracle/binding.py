@@ -10,7 +10,24 @@ import numpy as np
 
 _DIR = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_DIR, "aq_oracle.cpp")
-_LIB = os.path.join(_DIR, "libaq_oracle.so")
+
+
+def _cpu_tag() -> str:
+    """-march=native code only runs on a like CPU: key the library by the CPU's feature flags."""
+    import hashlib
+    flags = ""
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.startswith("flags"):
+                    flags = line
+                    break
+    except OSError:
+        pass
+    return hashlib.sha1(flags.encode()).hexdigest()[:10]
+
+
+_LIB = os.path.join(_DIR, f"libaq_oracle.{_cpu_tag()}.so")
 _lib = None
 
 
