@@ -1,0 +1,385 @@
+#!/usr/bin/env python
+"""Benchmark of the quantized linear layer (Agile-Quant, Sec. 4.4) on B200.
+
+One step = one pass of the whole path (layer absmax, activation quantization, integer
+product on packed 4-bit weights, fp16 output) over the three LLaMA-7B projection shapes at
+M = 2048 tokens with group-128 weight scales and int8 activations. Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+N > 1 is launched with torch.distributed.run, one rank per GPU; ranks run independent
+copies of the workload (no collective on the data path: the layer shards by batch), a
+barrier brackets the timed region and the slowest rank's time is used.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2312_05693_b200 import inputs  # noqa: E402
+
+WORKLOAD = "llama7b_prefill_w4a8"
+METRIC = "w4a8_linear_tops"
+UNIT = "TOPS"
+
+
+def layer_ops(M, shapes):
+    return sum(2.0 * M * s.K * s.N for s in shapes)
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 7:
+                self.rows.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, pw = [], [], []
+        reasons = set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+                pw.append(float(r[2]))
+            except ValueError:
+                continue
+            for name, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        busy = [c for c, p in zip(sm, pw) if p > 300.0] or sm
+        return {"sm_mhz": statistics.median(busy) if busy else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(pw) if pw else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def make_inputs(wl, M):
+    xs, ws = [], []
+    for i, s in enumerate(wl.shapes):
+        xs.append(inputs.activations(M, s.K, wl.seed, wl.outlier_frac, wl.outlier_mult, sub=i))
+        ws.append(inputs.weights(s.N, s.K, wl.seed, sub=i))
+    return xs, ws
+
+
+# ----------------------------------------------------------------------------------------
+# CPU baseline: the checker as it stands, on a bounded sample of the same workload
+# ----------------------------------------------------------------------------------------
+def cpu_sample_step(oracle, wl, xs, wq, rows):
+    t0 = time.perf_counter()
+    for i, s in enumerate(wl.shapes):
+        codes, sc = wq[i]
+        oracle.linear(xs[i][:rows], codes, sc, wl.act_bits, wl.group_size, 0, wl.clip_shift)
+    dt = time.perf_counter() - t0
+    return layer_ops(rows, wl.shapes) / dt / 1e12, dt
+
+
+def cpu_quantize_weights(oracle, wl, ws):
+    return [oracle.quantize_weights(w, wl.group_size) for w in ws]
+
+
+def cpu_baseline(wl, xs, ws, M, target_s=12.0):
+    import oracle
+    wq = cpu_quantize_weights(oracle, wl, ws)
+    _, dt = cpu_sample_step(oracle, wl, xs, wq, 32)
+    rows = int(min(M, max(32, 32 * target_s / max(dt, 1e-6))))
+    tops, dt = cpu_sample_step(oracle, wl, xs, wq, rows)
+    return {"value": tops, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"first {rows} of {M} token rows of all {len(wl.shapes)} layer shapes, "
+                      f"whole path, {dt:.1f} s"}
+
+
+def run_reference(args):
+    """--impl reference: the CPU checker timed on the same config, metric and unit."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    wl = inputs.WORKLOADS[WORKLOAD]
+    M = wl.Ms[0]
+    xs, ws = make_inputs(wl, M)
+    wq = cpu_quantize_weights(oracle, wl, ws)
+    _, dt = cpu_sample_step(oracle, wl, xs, wq, 16)
+    budget = 120.0 / max(args.steps + args.warmup, 1)
+    rows = int(min(M, max(16, 16 * min(budget, 8.0) / max(dt, 1e-6))))
+    for _ in range(args.warmup):
+        cpu_sample_step(oracle, wl, xs, wq, rows)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        cpu_sample_step(oracle, wl, xs, wq, rows)
+    dt = (time.perf_counter() - t0) / args.steps
+    tops = layer_ops(rows, wl.shapes) / dt / 1e12
+    sample = f"each step: first {rows} of {M} token rows of all {len(wl.shapes)} layer shapes, whole path"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": tops, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8xint4->int32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "M": M, "shapes_KN": [[s.K, s.N] for s in wl.shapes],
+                   "group_size": wl.group_size, "act_bits": wl.act_bits},
+        "cpu_baseline": {"value": tops, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": tops, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+# ----------------------------------------------------------------------------------------
+# decode measurement (extra keys): weight streaming at M <= 16
+# ----------------------------------------------------------------------------------------
+def bench_decode(h, peaks, iters=40):
+    from paper_2312_05693_b200 import binding
+    wl = inputs.WORKLOADS["llama13b_decode_w4a8"]
+    out = []
+    for s in wl.shapes:
+        wbytes = s.N * s.K // 2
+        copies = max(2, int(320e6 // wbytes) + 1)          # rotate through > 2x L2 of weights
+        w = torch.from_numpy(inputs.weights(s.N, s.K, wl.seed)).cuda()
+        packs = []
+        for c in range(copies):
+            p, sc = h.aq_pack_w4(w, 0)
+            packs.append((p, sc))
+        for M in wl.Ms:
+            x = torch.from_numpy(inputs.activations(M, s.K, wl.seed, wl.outlier_frac, wl.outlier_mult)).cuda()
+            q, e = h.aq_quantize_act(x, 8)
+            ws = h.alloc_workspace(M, s.K, s.N, 0)
+            y = torch.empty((M, s.N), dtype=torch.float16, device="cuda")
+            for i in range(copies):
+                h.aq_gemm_w4(q, packs[i][0], packs[i][1], s.N, 0, e, y=y, workspace=ws)
+            evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+                   for _ in range(iters)]
+            torch.cuda.synchronize()
+            for i in range(iters):
+                p, sc = packs[i % copies]
+                evs[i][0].record()
+                h.aq_gemm_w4(q, p, sc, s.N, 0, e, y=y, workspace=ws)
+                evs[i][1].record()
+            torch.cuda.synchronize()
+            ms = statistics.median(a.elapsed_time(b) for a, b in evs)
+            algo = wbytes + 2 * s.N + M * s.K + 2 * M * s.N
+            gbs = algo / (ms * 1e-3) / 1e9
+            out.append({"K": s.K, "N": s.N, "M": M, "us": ms * 1e3, "GBps": gbs,
+                        "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]})
+        del packs
+    return out
+
+
+# ----------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-decode", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    from paper_2312_05693_b200 import binding
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path)")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    peaks = load_peaks()
+    wl = inputs.WORKLOADS[WORKLOAD]
+    M = wl.Ms[0]
+    h = binding.Handle(local_rank)
+    xs_np, ws_np = make_inputs(wl, M)
+    fn = h.aq_linear_w4a8 if wl.act_bits == 8 else h.aq_linear_w4a4
+
+    layers = []
+    for i, s in enumerate(wl.shapes):
+        wd = torch.from_numpy(ws_np[i]).cuda()
+        packed, scales = h.aq_pack_w4(wd, wl.group_size)
+        del wd
+        layers.append({
+            "K": s.K, "N": s.N, "x": torch.from_numpy(xs_np[i]).cuda(), "packed": packed, "scales": scales,
+            "y": torch.empty((M, s.N), dtype=torch.float16, device="cuda"),
+            "ws": h.alloc_workspace(M, s.K, s.N, wl.group_size),
+            "x_host": torch.from_numpy(xs_np[i]).pin_memory(),
+            "y_host": torch.empty((M, s.N), dtype=torch.float16).pin_memory(),
+            "scratch": torch.empty(binding.aq_linear_host_scratch_bytes(M, s.K, s.N, wl.group_size),
+                                   dtype=torch.uint8, device="cuda"),
+        })
+    torch.cuda.synchronize()
+
+    def step():
+        for L in layers:
+            fn(L["x"], L["packed"], L["scales"], L["N"], wl.group_size, binding.AQ_SCALE_DYNAMIC,
+               wl.clip_shift, y=L["y"], workspace=L["ws"])
+
+    ops_per_step = layer_ops(M, wl.shapes)
+    # ---- main timed region: the public layer call, device-resident inputs
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    barrier()
+    ms_total = ev0.elapsed_time(ev1)
+
+    # ---- second pass, same kernels launched as two calls so the product kernel can be
+    #      bracketed by events on the launching stream (its duration feeds the roofline)
+    gemm_ev = []
+    for _ in range(args.steps):
+        for L in layers:
+            q, e = h.aq_quantize_act(L["x"], wl.act_bits, binding.AQ_SCALE_DYNAMIC, wl.clip_shift,
+                                     workspace=L["ws"][:256])
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            h.aq_gemm_w4(q, L["packed"], L["scales"], L["N"], wl.group_size, e, y=L["y"], workspace=L["ws"])
+            b.record()
+            gemm_ev.append((a, b, 2.0 * M * L["K"] * L["N"]))
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    gemm_ms = sum(a.elapsed_time(b) for a, b, _ in gemm_ev)
+    gemm_ops = sum(o for _, _, o in gemm_ev)
+    for L in layers:
+        st = h.aq_check_workspace(L["ws"])
+        if st != binding.AQ_OK:
+            raise SystemExit(f"kernel reported {binding.status_string(st)}")
+
+    # ---- end to end through the host-buffer entry point (H2D of x and D2H of y inside)
+    def step_host():
+        for L in layers:
+            h.aq_linear_host(wl.act_bits, L["x_host"], L["packed"], L["scales"], L["N"], wl.group_size,
+                             L["y_host"], L["scratch"], binding.AQ_SCALE_DYNAMIC, wl.clip_shift)
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(3):
+        step_host()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(e2e_steps):
+        step_host()
+    e1.record()
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / e2e_steps
+
+    times = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms = float(times[0]), float(times[1])
+    ms_per_step = ms_total / args.steps
+    value = world * ops_per_step / (ms_per_step * 1e-3) / 1e12
+    e2e_value = world * ops_per_step / (e2e_ms * 1e-3) / 1e12
+
+    int8_peak = 2.0 * peaks["bf16_tflops_sustained"]     # dense int8 = 2x dense bf16 (nominal ratio)
+    achieved = gemm_ops / (gemm_ms * 1e-3) / 1e12
+    roofline = {
+        "kernel": "gemm_tensor_kernel<128, grouped>", "bound": "tensor", "achieved": achieved,
+        "peak": int8_peak, "unit": "TFLOP/s", "frac": achieved / int8_peak, "traffic": None,
+        "peak_source": f"2 x bf16_tflops_sustained of {peaks['source']} peaks (int8:bf16 nominal 2:1)",
+        "frac_of_nominal_4500": achieved / 4500.0,
+        "timing": "CUDA events around each aq_gemm_w4 launch in a second pass of the same steps",
+        "avg_launch_us": gemm_ms * 1e3 / len(gemm_ev),
+    }
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8xint4->int32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "M": M, "shapes_KN": [[s.K, s.N] for s in wl.shapes],
+                   "group_size": wl.group_size, "act_bits": wl.act_bits, "parallelism": f"replicas x{world}",
+                   "l2": "per-step footprint (x, packed w, y of 3 layers) ~210 MB exceeds the 126 MB L2"},
+        "tokens_per_s": world * M * len(wl.shapes) / (ms_per_step * 1e-3),
+        "e2e": {"value": e2e_value, "unit": UNIT,
+                "h2d_bytes_per_step": int(sum(M * s.K * 2 for s in wl.shapes)),
+                "d2h_bytes_per_step": int(sum(M * s.N * 2 for s in wl.shapes)),
+                "ms_per_step": e2e_ms, "api": "aq_linear_host"},
+        "gpu_launches": args.steps * len(layers) * 3,
+        "clocks": clocks,
+        "roofline": roofline,
+    }
+    if rank == 0 and world == 1 and not args.no_decode:
+        try:
+            line["decode"] = bench_decode(h, peaks)
+        except Exception as ex:  # report, do not hide
+            line["decode"] = {"error": repr(ex)}
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(wl, xs_np, ws_np, M)
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

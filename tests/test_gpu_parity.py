@@ -132,7 +132,7 @@ def test_linear_extreme_codes_and_patterns(kernel):
     h = handle()
     M, K, N = 130, 512, 256
     x = np.full((M, K), -128.0, np.float16)
-    w = np.full((N, K), -1.0, np.float16)                  # codes -7 after a/7 scaling... all equal -> -7
+    w = np.full((N, K), -0.01, np.float16)                 # every code is -7
     gpu, ref = run_layer_both(x, w, 8, 0, kernel, scale_mode=1, clip=0)
     assert np.array_equal(gpu["acc"], ref["acc"]) and ref["acc"].max() == 128 * 7 * K
     assert_y_close(gpu["y"], ref["y"])
