@@ -218,6 +218,46 @@ def bench_decode(h, peaks, iters=40):
 
 
 # ----------------------------------------------------------------------------------------
+# single-shape case (for profiling one kernel on a small or a full-size shape)
+# ----------------------------------------------------------------------------------------
+def run_case(args):
+    """--case M,K,N,group[,bits[,kernel]]: quantize once, then time the product kernel alone."""
+    from paper_2312_05693_b200 import binding
+    parts = [int(v) for v in args.case.split(",")]
+    M, K, N, group = parts[:4]
+    bits = parts[4] if len(parts) > 4 else 8
+    kernel = parts[5] if len(parts) > 5 else binding.AQ_KERNEL_AUTO
+    torch.cuda.set_device(0)
+    h = binding.Handle(0)
+    h.aq_set_kernel(kernel)
+    x = torch.from_numpy(inputs.activations(M, K, 1, 0.005, 30.0)).cuda()
+    w = torch.from_numpy(inputs.weights(N, K, 1)).cuda()
+    wbytes = N * K // 2
+    copies = max(1, min(64, int(args.rotate_mb * 1e6 // wbytes)))
+    packs = [h.aq_pack_w4(w, group) for _ in range(copies)]
+    q, e = h.aq_quantize_act(x, bits)
+    ws = h.alloc_workspace(M, K, N, group)
+    y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+    for i in range(args.warmup):
+        h.aq_gemm_w4(q, packs[i % copies][0], packs[i % copies][1], N, group, e, y=y, workspace=ws)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+           for _ in range(args.steps)]
+    torch.cuda.synchronize()
+    for i in range(args.steps):
+        pk, sc = packs[i % copies]
+        evs[i][0].record()
+        h.aq_gemm_w4(q, pk, sc, N, group, e, y=y, workspace=ws)
+        evs[i][1].record()
+    torch.cuda.synchronize()
+    st = h.aq_check_workspace(ws)
+    ts = sorted(a.elapsed_time(b) for a, b in evs)
+    med = ts[len(ts) // 2]
+    algo = wbytes + M * K + 2 * M * N
+    print(json.dumps({"case": args.case, "status": st, "us_median": med * 1e3, "us_min": ts[0] * 1e3,
+                      "TOPS": 2.0 * M * K * N / (med * 1e-3) / 1e12, "GBps": algo / (med * 1e-3) / 1e9,
+                      "weight_copies": copies}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -226,7 +266,13 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--case", default=None, help="M,K,N,group[,bits[,kernel]]: time one product kernel")
+    ap.add_argument("--rotate-mb", type=float, default=0.0,
+                    help="with --case: rotate through this many MB of weight copies (defeats L2)")
     args = ap.parse_args()
+    if args.case:
+        run_case(args)
+        return
     if args.warmup < 3:
         args.warmup = 3
     if args.impl == "reference":

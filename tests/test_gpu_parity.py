@@ -207,7 +207,7 @@ def test_bad_arguments_are_refused():
     with pytest.raises(binding.AgileqError) as ei:
         h.aq_linear_w4a8(x, packed, scales, 128, 0, workspace=small)
     assert ei.value.status == binding.AQ_ERR_WORKSPACE
-    ws = h.alloc_workspace(4, 256, 128, 0)
+    ws = torch.empty(h.alloc_workspace(4, 256, 128, 0).numel() + 256, dtype=torch.uint8, device="cuda")
     with pytest.raises(binding.AgileqError) as ei:
         h.aq_linear_w4a8(x, packed, scales, 128, 0, workspace=ws[1:])
     assert ei.value.status == binding.AQ_ERR_ALIGNMENT
