@@ -3,19 +3,21 @@
 //
 // Operand roles are swapped with respect to y = x w^T: the 128 output channels of a tile
 // are the MMA's M dimension and the tokens its N dimension, so that
-//   * the 4-bit weights never touch shared memory: four warps read the packed layout from
-//     global memory (512 contiguous bytes per warp load), widen each nibble to the int8
-//     value 16*code with two logic ops per word, and store the result straight into
-//     tensor memory, where the MMA reads it as its A operand;
+//   * the 4-bit weights stay packed in shared memory (one contiguous 8 KB bulk copy per
+//     128 x 128 block): four warps widen each nibble to the int8 value 16*code with two
+//     logic ops per word and store the result straight into tensor memory, where the MMA
+//     reads it as its A operand, so the widened weights never take shared-memory bandwidth;
 //   * every epilogue thread owns one output channel, so its weight scale(s) sit in a
 //     register and the per-128-k group rescaling costs one FMA per element;
 //   * the int8 activation tile (tokens x 128 k) is the only shared-memory operand, staged
 //     by TMA with the 128-byte swizzle and read through an MMA shared-memory descriptor.
 //
 // One persistent CTA per SM walks a static list of (channel tile, token tile) pairs.
-// Warp roles: 0 = TMA producer, 1 = MMA issue + TMEM allocation, 2-5 = weight unpack,
-// 6-9 = epilogue. Two accumulator stages in TMEM let the epilogue of one accumulation
-// overlap the MMAs of the next. Every wait is bounded; on expiry the CTA records a status
+// Warp roles: 0 = TMA producer, 1 = MMA issue + TMEM allocation (2-3 idle), 4-11 = weight
+// unpack (two groups of four taking alternate k blocks), 12-19 = epilogue; registers are
+// moved from the first two roles to the epilogue with setmaxnreg. Two (one scale per channel)
+// or three (per-group scales) accumulator stages in TMEM let the epilogue of one
+// accumulation overlap the MMAs of the next ones. Every wait is bounded; on expiry the CTA records a status
 // word, stops issuing work and leaves through the common exit that frees TMEM.
 #include <cuda.h>
 
@@ -25,9 +27,19 @@ namespace aq {
 
 namespace {
 
-constexpr int kNumStages = 6;                 // ring depth: activation tiles (smem) and weight slices (TMEM)
-constexpr int kUnpackPrefetch = 4;            // packed 128-k blocks held in registers per unpack thread
-constexpr int kThreads = 320;
+constexpr int kNumStages = 6;                 // shared-memory ring: activation tile + packed weight block (+ scales)
+constexpr int kUnpackGroups = 2;              // groups of four unpack warps; group g takes k blocks g, g+2, ...
+constexpr int kFirstUnpackWarp = 4;           // warps 0-3: TMA producer, MMA issuer, two idle (one warpgroup)
+constexpr int kFirstEpiWarp = kFirstUnpackWarp + 4 * kUnpackGroups;
+// Registers per thread after the roles split (setmaxnreg works on aligned groups of four warps):
+constexpr int kRegsControl = 40, kRegsUnpack = 48, kRegsEpilogue = 168;
+constexpr int kEpiWarps = 8;                  // two warps per TMEM lane quarter, half of the token columns each
+constexpr int kThreads = (kFirstEpiWarp + kEpiWarps) * 32;
+// Grouped mode keeps every accumulator biased by this integer: the bit pattern of the float
+// 1.5 * 2^23. An int32 sum v with |v| < 2^22 then reads back from tensor memory as the float
+// 12582912 + v, so the epilogue needs no int->float conversion (one FADD removes the bias).
+constexpr uint32_t kMagicBits = 0x4B400000u;
+constexpr float kMagicFloat = 12582912.0f;
 constexpr int kAColsPerStage = 32;            // 128 k of int8 = 32 TMEM columns per lane
 constexpr unsigned long long kWaitCycles = 4000000000ull;   // ~2 s
 
@@ -82,6 +94,13 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, i
         ::"r"(smem_u32(dst)), "l"(map), "r"(x), "r"(y), "r"(smem_u32(bar))
         : "memory");
 }
+// Contiguous global -> shared copy through the TMA unit (both addresses 16-byte aligned, size % 16 == 0).
+__device__ __forceinline__ void tma_load_1d(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
+        : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
@@ -110,6 +129,15 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
         : "r"(taddr)
         : "memory");
 }
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&v)[32]) {
     asm volatile(
@@ -121,6 +149,41 @@ __device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&v)[32])
           "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
           "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
         : "memory");
+}
+__device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t (&v)[8]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+        : "memory");
+}
+__device__ __forceinline__ void tc_st32_fill(uint32_t taddr, uint32_t c) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, "
+        "%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};"
+        ::"r"(taddr), "r"(c) : "memory");
+}
+// Packed pairs of fp32 (one instruction, two lanes of data).
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(__float_as_uint(lo)), "r"(__float_as_uint(hi)));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    uint32_t a, b;
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
+    lo = __uint_as_float(a);
+    hi = __uint_as_float(b);
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t r;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
 }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -147,10 +210,14 @@ __host__ __device__ constexpr uint32_t idesc_i8(int m, int n) {
 template <int BM>
 struct SharedStorage {
     alignas(1024) uint8_t x[kNumStages][BM * 128];   // activation tiles, 128-byte swizzled rows
-    alignas(8) uint64_t full[kNumStages];            // TMA bytes + 4 unpack warps -> MMA
-    uint64_t empty[kNumStages];                      // MMA done with the stage -> producers
-    uint64_t acc_full[2];                            // MMA -> epilogue
-    uint64_t acc_empty[2];                           // epilogue (4 warps) -> MMA
+    alignas(128) uint8_t w[kNumStages][kBlockBytes]; // packed weight blocks (128 channels x 128 k)
+    alignas(16) __half sc[kNumStages][kTileN];       // weight scales of the block's group (grouped mode)
+    alignas(8) uint64_t tma_full[kNumStages];        // TMA bytes landed -> unpack warps, MMA
+    uint64_t smem_empty[kNumStages];                 // MMA done (+ epilogue took the scales) -> TMA producer
+    uint64_t a_full[8];                              // unpack warps stored the slice -> MMA
+    uint64_t a_empty[8];                             // MMA done with the slice -> unpack warps
+    uint64_t acc_full[3];                            // MMA -> epilogue
+    uint64_t acc_empty[3];                           // epilogue -> MMA
     uint32_t tmem_base;
     volatile uint32_t abort_flag;
 };
@@ -173,26 +240,36 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
     using Smem = SharedStorage<BM>;
     Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
 
-    constexpr int kAccCols = 2 * BM;
-    constexpr int kTmemColsUsed = kAccCols + kNumStages * kAColsPerStage;
+    constexpr int kNumAcc = GROUPED ? 3 : 2;          // accumulator stages in tensor memory
+    constexpr int kAccCols = kNumAcc * BM;
+    // the rest of tensor memory (up to 8 slices) is the ring of unpacked weight slices (A operand)
+    constexpr int kNumASlices = (512 - kAccCols) / kAColsPerStage >= 8 ? 8 : (512 - kAccCols) / kAColsPerStage;
+    static_assert(kNumASlices >= 4 && kNumASlices % kUnpackGroups == 0, "weight-slice ring");
+    constexpr int kTmemColsUsed = kAccCols + kNumASlices * kAColsPerStage;
     constexpr int kTmemCols = kTmemColsUsed <= 128 ? 128 : kTmemColsUsed <= 256 ? 256 : 512;
     static_assert(kTmemColsUsed <= 512, "tensor memory has 512 columns");
-    static_assert(BM % 32 == 0 && BM >= 32 && BM <= 256, "token tile");
+    static_assert(BM % 64 == 0 && BM >= 64 && BM <= 256, "token tile");
+    constexpr int kColsPerEpiWarp = BM / 2;           // each quarter's columns are split between two warps
+    static_assert(kColsPerEpiWarp % 16 == 0 && (!GROUPED || kColsPerEpiWarp % 32 == 0), "epilogue chunking");
+    constexpr uint32_t kStageBytes = BM * 128 + kBlockBytes + (GROUPED ? kTileN * 2 : 0);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KB = p.K / kTileK;
     const int my_tiles = p.n_tiles > (int)blockIdx.x
                              ? (p.n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
-    const long long total_iters = (long long)my_tiles * KB;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kNumStages; ++s) {
-            mbar_init(&sm.full[s], 1 + 4);
-            mbar_init(&sm.empty[s], 1);
+            mbar_init(&sm.tma_full[s], 1);
+            mbar_init(&sm.smem_empty[s], GROUPED ? 1 + kEpiWarps : 1);
         }
-        for (int a = 0; a < 2; ++a) {
+        for (int i = 0; i < kNumASlices; ++i) {
+            mbar_init(&sm.a_full[i], 4);
+            mbar_init(&sm.a_empty[i], 1);
+        }
+        for (int a = 0; a < kNumAcc; ++a) {
             mbar_init(&sm.acc_full[a], 1);
-            mbar_init(&sm.acc_empty[a], 4);
+            mbar_init(&sm.acc_empty[a], kEpiWarps);
         }
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -206,55 +283,64 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
-    const uint32_t tmem_acc = tmem;                 // columns [0, 2*BM)
-    const uint32_t tmem_a = tmem + kAccCols;        // columns [2*BM, 2*BM + stages*32)
+    const uint32_t tmem_acc = tmem;                 // columns [0, kNumAcc*BM)
+    const uint32_t tmem_a = tmem + kAccCols;        // then kNumASlices slices of 32 columns
     volatile uint32_t* abort_flag = &sm.abort_flag;
 
-    if (warp == 0) {
+    if (warp < kFirstUnpackWarp) {
+      asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsControl));
+      if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer
         if (lane == 0) {
-            long long it = 0;
+            uint32_t it = 0;
             for (int tl = 0; tl < my_tiles; ++tl) {
                 const int tile = blockIdx.x + tl * gridDim.x;
-                const int mt = tile % p.n_tiles_m;
+                const int mt = tile % p.n_tiles_m, nt = tile / p.n_tiles_m;
+                const uint8_t* wsrc = p.w_packed + (size_t)nt * KB * kBlockBytes;
                 for (int kb = 0; kb < KB; ++kb, ++it) {
                     const int s = (int)(it % kNumStages);
-                    const uint32_t ph = (uint32_t)(it / kNumStages) & 1u;
-                    if (!mbar_wait(&sm.empty[s], ph ^ 1u, abort_flag)) goto role_done;
-                    mbar_arrive_expect_tx(&sm.full[s], BM * 128);
-                    tma_load_2d(sm.x[s], &x_map, kb * kTileK, mt * BM, &sm.full[s]);
+                    const uint32_t ph = (it / kNumStages) & 1u;
+                    if (!mbar_wait(&sm.smem_empty[s], ph ^ 1u, abort_flag)) goto role_done;
+                    mbar_arrive_expect_tx(&sm.tma_full[s], kStageBytes);
+                    tma_load_2d(sm.x[s], &x_map, kb * kTileK, mt * BM, &sm.tma_full[s]);
+                    tma_load_1d(sm.w[s], wsrc + (size_t)kb * kBlockBytes, kBlockBytes, &sm.tma_full[s]);
+                    if (GROUPED)
+                        tma_load_1d(sm.sc[s], p.w_scales + (size_t)kb * p.Npad + nt * kTileN, kTileN * 2,
+                                    &sm.tma_full[s]);
                 }
             }
         }
-    } else if (warp == 1) {
+      } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             constexpr uint32_t idesc = idesc_i8(128, BM);
-            long long it = 0;
-            long long unit = 0;      // accumulations handed to the epilogue so far
+            uint32_t it = 0;
+            uint32_t unit = 0;      // accumulations handed to the epilogue so far
             for (int tl = 0; tl < my_tiles; ++tl) {
                 for (int kb = 0; kb < KB; ++kb, ++it) {
                     const bool first = GROUPED || kb == 0;
-                    const int a = (int)(unit & 1);
+                    const int a = (int)(unit % kNumAcc);
                     if (first) {
-                        const uint32_t aph = (uint32_t)(unit >> 1) & 1u;
-                        if (!mbar_wait(&sm.acc_empty[a], aph ^ 1u, abort_flag)) goto role_done;
-                        tc_fence_after();
+                        const uint32_t aph = (unit / kNumAcc) & 1u;
+                        // grouped: the epilogue's initial bias store counts as the first release
+                        if (!mbar_wait(&sm.acc_empty[a], GROUPED ? aph : (aph ^ 1u), abort_flag)) goto role_done;
                     }
                     const int s = (int)(it % kNumStages);
-                    const uint32_t ph = (uint32_t)(it / kNumStages) & 1u;
-                    if (!mbar_wait(&sm.full[s], ph, abort_flag)) goto role_done;
+                    const int ai = (int)(it % kNumASlices);
+                    if (!mbar_wait(&sm.tma_full[s], (it / kNumStages) & 1u, abort_flag)) goto role_done;
+                    if (!mbar_wait(&sm.a_full[ai], (it / kNumASlices) & 1u, abort_flag)) goto role_done;
                     tc_fence_after();
                     const uint32_t d_addr = tmem_acc + (uint32_t)(a * BM);
-                    const uint32_t a_addr = tmem_a + (uint32_t)(s * kAColsPerStage);
+                    const uint32_t a_addr = tmem_a + (uint32_t)(ai * kAColsPerStage);
                     const uint64_t bdesc = smem_desc_sw128(smem_u32(sm.x[s]));
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         // 32 k per instruction: 8 TMEM columns of A, 32 bytes along the swizzled row of B
                         tc_mma_i8_ts(d_addr, a_addr + 8 * j, bdesc + (uint64_t)(2 * j), idesc,
-                                     (first && j == 0) ? 0u : 1u);
+                                     (!GROUPED && first && j == 0) ? 0u : 1u);
                     }
-                    tc_commit(&sm.empty[s]);
+                    tc_commit(&sm.a_empty[ai]);
+                    tc_commit(&sm.smem_empty[s]);
                     const bool last = GROUPED || kb == KB - 1;
                     if (last) {
                         tc_commit(&sm.acc_full[a]);
@@ -263,84 +349,93 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
                 }
             }
         }
-    } else if (warp < 6) {
+      }
+    } else if (warp < kFirstEpiWarp) {
         // --------------------------------------------------- weight unpack -> tensor memory
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsUnpack));
         const int quarter = warp & 3;
+        const int group = (warp - kFirstUnpackWarp) >> 2;
         const int r = quarter * 32 + lane;            // row inside the 128-channel tile = TMEM lane
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
-        uint4 buf[kUnpackPrefetch][4];
-        auto block_ptr = [&](long long it) -> const uint4* {
-            const int tl = (int)(it / KB), kb = (int)(it % KB);
-            const int tile = blockIdx.x + tl * gridDim.x;
-            const int nt = tile / p.n_tiles_m;
-            return reinterpret_cast<const uint4*>(p.w_packed + ((size_t)nt * KB + kb) * kBlockBytes) + r;
-        };
+        const uint32_t total_iters = (uint32_t)my_tiles * (uint32_t)KB;
+        int pending = -1;                             // slice whose store has been issued but not published
+        for (uint32_t it = group; it < total_iters; it += kUnpackGroups) {
+            const int s = (int)(it % kNumStages);
+            const int ai = (int)(it % kNumASlices);
+            if (!mbar_wait_warp(&sm.tma_full[s], (it / kNumStages) & 1u, abort_flag)) goto role_done;
+            const uint4* src = reinterpret_cast<const uint4*>(sm.w[s]) + r;
+            uint4 d[4];
 #pragma unroll
-        for (int d = 0; d < kUnpackPrefetch; ++d) {
-            if (d < total_iters) {
-                const uint4* src = block_ptr(d);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) buf[d][j] = __ldg(src + j * kTileN);
-            }
-        }
-        for (long long it0 = 0; it0 < total_iters; it0 += kUnpackPrefetch) {
-#pragma unroll
-            for (int d = 0; d < kUnpackPrefetch; ++d) {
-                const long long it = it0 + d;
-                if (it >= total_iters) break;
-                uint32_t v[32];
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint32_t w[4] = {buf[d][j].x, buf[d][j].y, buf[d][j].z, buf[d][j].w};
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        v[8 * j + 2 * i] = (w[i] << 4) & 0xF0F0F0F0u;
-                        v[8 * j + 2 * i + 1] = w[i] & 0xF0F0F0F0u;
-                    }
-                }
-                if (it + kUnpackPrefetch < total_iters) {
-                    const uint4* src = block_ptr(it + kUnpackPrefetch);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) buf[d][j] = __ldg(src + j * kTileN);
-                }
-                const int s = (int)(it % kNumStages);
-                const uint32_t ph = (uint32_t)(it / kNumStages) & 1u;
-                if (!mbar_wait_warp(&sm.empty[s], ph ^ 1u, abort_flag)) goto role_done;
-                tc_fence_after();
-                tc_st32(tmem_a + lane_addr + (uint32_t)(s * kAColsPerStage), v);
+            for (int j = 0; j < 4; ++j) d[j] = src[j * kTileN];
+            if (pending >= 0) {                       // the previous stores had the loads above to finish
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.full[s]);
+                if (lane == 0) mbar_arrive(&sm.a_full[pending]);
             }
+            if (!mbar_wait_warp(&sm.a_empty[ai], ((it / kNumASlices) & 1u) ^ 1u, abort_flag)) goto role_done;
+            tc_fence_after();
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t w[4] = {d[j].x, d[j].y, d[j].z, d[j].w};
+                uint32_t v[8];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    v[2 * i] = (w[i] << 4) & 0xF0F0F0F0u;           // 16*code for k0..k0+3
+                    v[2 * i + 1] = w[i] & 0xF0F0F0F0u;              // 16*code for k0+4..k0+7
+                }
+                tc_st8(tmem_a + lane_addr + (uint32_t)(ai * kAColsPerStage + 8 * j), v);
+            }
+            pending = ai;
+        }
+        if (pending >= 0) {
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.a_full[pending]);
         }
     } else {
         // ----------------------------------------------------------------------- epilogue
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsEpilogue));
         const int quarter = warp & 3;
+        const int half = (warp - kFirstEpiWarp) >> 2;                                // which half of the token columns
         const int r = quarter * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+        const int col0 = half * kColsPerEpiWarp;
         const float pe = __int_as_float((127 + *p.scale_exp) << 23);     // 2^e
         const int G = GROUPED ? KB : 1;
-        long long unit = 0;
+        uint32_t unit = 0, it = 0;
+        if (GROUPED) {
+            // arm every accumulator stage with the bias; this is the first release of each stage
+            for (int a = 0; a < kNumAcc; ++a) {
+#pragma unroll
+                for (int c0 = 0; c0 < kColsPerEpiWarp; c0 += 32)
+                    tc_st32_fill(tmem_acc + lane_addr + (uint32_t)(a * BM + col0 + c0), kMagicBits);
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.acc_empty[a]);
+            }
+        }
         for (int tl = 0; tl < my_tiles; ++tl) {
             const int tile = blockIdx.x + tl * gridDim.x;
             const int mt = tile % p.n_tiles_m, nt = tile / p.n_tiles_m;
             const int n = nt * kTileN + r;
-            const int m_base = mt * BM;
+            const int m_base = mt * BM + col0;
             const bool n_ok = n < p.N;
             if (!GROUPED) {
-                const int a = (int)(unit & 1);
-                const uint32_t aph = (uint32_t)(unit >> 1) & 1u;
+                const int a = (int)(unit % kNumAcc);
+                const uint32_t aph = (unit / kNumAcc) & 1u;
                 const float sc = __half2float(p.w_scales[n]) * 0.0625f * pe;   // sums carry a factor 16
                 if (!mbar_wait_warp(&sm.acc_full[a], aph, abort_flag)) goto role_done;
                 tc_fence_after();
 #pragma unroll 1
-                for (int c0 = 0; c0 < BM; c0 += 32) {
-                    uint32_t v[32];
-                    tc_ld32(tmem_acc + lane_addr + (uint32_t)(a * BM + c0), v);
+                for (int c0 = 0; c0 < kColsPerEpiWarp; c0 += 16) {
+                    uint32_t v[16];
+                    tc_ld16(tmem_acc + lane_addr + (uint32_t)(a * BM + col0 + c0), v);
                     tc_wait_ld();
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
+                    for (int c = 0; c < 16; ++c) {
                         const int m = m_base + c0 + c;
                         if (n_ok && m < p.M) {
                             const int acc16 = (int)v[c];
@@ -354,40 +449,59 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
                 if (lane == 0) mbar_arrive(&sm.acc_empty[a]);
                 ++unit;
             } else {
-                float fsum[BM];
+                uint64_t fsum2[kColsPerEpiWarp / 2];                     // pairs of fp32 partial outputs
 #pragma unroll
-                for (int c = 0; c < BM; ++c) fsum[c] = 0.0f;
-                float s_next = __half2float(p.w_scales[n]) * 0.0625f;
-                for (int kb = 0; kb < KB; ++kb, ++unit) {
-                    const int a = (int)(unit & 1);
-                    const uint32_t aph = (uint32_t)(unit >> 1) & 1u;
-                    const float s = s_next;
-                    if (kb + 1 < KB) s_next = __half2float(p.w_scales[(size_t)(kb + 1) * p.Npad + n]) * 0.0625f;
+                for (int c = 0; c < kColsPerEpiWarp / 2; ++c) fsum2[c] = 0ull;
+                const uint64_t neg_magic2 = pack2(-kMagicFloat, -kMagicFloat);
+                for (int kb = 0; kb < KB; ++kb, ++unit, ++it) {
+                    const int a = (int)(unit % kNumAcc);
+                    const uint32_t aph = (unit / kNumAcc) & 1u;
+                    const int s = (int)(it % kNumStages);
                     if (!mbar_wait_warp(&sm.acc_full[a], aph, abort_flag)) goto role_done;
                     tc_fence_after();
+                    // the block's scales landed with its operands (the wait below passes at once and
+                    // orders the read after the copy); take ours, then let the stage go
+                    if (!mbar_wait_warp(&sm.tma_full[s], (it / kNumStages) & 1u, abort_flag)) goto role_done;
+                    const float sg = __half2float(sm.sc[s][r]) * 0.0625f;
+                    const uint64_t sg2 = pack2(sg, sg);
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm.smem_empty[s]);
 #pragma unroll
-                    for (int c0 = 0; c0 < BM; c0 += 32) {
+                    for (int c0 = 0; c0 < kColsPerEpiWarp; c0 += 32) {
+                        const uint32_t taddr = tmem_acc + lane_addr + (uint32_t)(a * BM + col0 + c0);
                         uint32_t v[32];
-                        tc_ld32(tmem_acc + lane_addr + (uint32_t)(a * BM + c0), v);
+                        tc_ld32(taddr, v);
                         tc_wait_ld();
+                        tc_st32_fill(taddr, kMagicBits);                 // re-arm the bias for the next use
 #pragma unroll
-                        for (int c = 0; c < 32; ++c) {
-                            fsum[c0 + c] = fmaf((float)(int)v[c], s, fsum[c0 + c]);
-                            if (p.acc_dump) {
+                        for (int c = 0; c < 32; c += 2) {
+                            // v holds the bits of the floats (magic + 16*sum): remove the bias, scale, add
+                            uint64_t t;
+                            asm("mov.b64 %0, {%1, %2};" : "=l"(t) : "r"(v[c]), "r"(v[c + 1]));
+                            t = add2(t, neg_magic2);
+                            fsum2[(c0 + c) / 2] = fma2(t, sg2, fsum2[(c0 + c) / 2]);
+                        }
+                        if (p.acc_dump) {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c) {
                                 const int m = m_base + c0 + c;
                                 if (n_ok && m < p.M)
-                                    p.acc_dump[((size_t)m * p.N + n) * G + kb] = (int)v[c] >> 4;
+                                    p.acc_dump[((size_t)m * p.N + n) * G + kb] = (int)(v[c] - kMagicBits) >> 4;
                             }
                         }
                     }
+                    tc_wait_st();
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&sm.acc_empty[a]);
                 }
 #pragma unroll
-                for (int c = 0; c < BM; ++c) {
+                for (int c = 0; c < kColsPerEpiWarp; c += 2) {
+                    float lo, hi;
+                    unpack2(fsum2[c / 2], lo, hi);
                     const int m = m_base + c;
-                    if (n_ok && m < p.M) p.y[(size_t)m * p.N + n] = __float2half_rn(fsum[c] * pe);
+                    if (n_ok && m < p.M) p.y[(size_t)m * p.N + n] = __float2half_rn(lo * pe);
+                    if (n_ok && m + 1 < p.M) p.y[(size_t)(m + 1) * p.N + n] = __float2half_rn(hi * pe);
                 }
             }
         }
@@ -450,7 +564,6 @@ cudaError_t launch_bm(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t str
 }  // namespace
 
 cudaError_t launch_gemm_tensor(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
-    if (a.M <= 32) return a.group ? launch_bm<32, true>(a, dev, stream) : launch_bm<32, false>(a, dev, stream);
     if (a.M <= 64) return a.group ? launch_bm<64, true>(a, dev, stream) : launch_bm<64, false>(a, dev, stream);
     return a.group ? launch_bm<128, true>(a, dev, stream) : launch_bm<128, false>(a, dev, stream);
 }
