@@ -13,9 +13,12 @@
 //     by TMA with the 128-byte swizzle and read through an MMA shared-memory descriptor.
 //
 // One persistent CTA per SM walks a static list of (channel tile, token tile) pairs.
-// Warp roles: 0 = TMA producer, 1 = MMA issue + TMEM allocation (2-3 idle), 4-11 = weight
-// unpack (two groups of four taking alternate k blocks), 12-19 = epilogue; registers are
-// moved from the first two roles to the epilogue with setmaxnreg. Two (one scale per channel)
+// Warp roles: 0 and 2 = TMA producers (activations / weights), 1 and 3 = MMA issuers (warp 1
+// also owns the TMEM allocation; warp 3 only works in per-group mode), 4-11 = weight unpack
+// (two groups of four taking alternate k blocks), 12-19 = epilogue; registers are moved from
+// the first two roles to the epilogue with setmaxnreg. One thread spends about 55 cycles per
+// MMA instruction and about 100 per TMA instruction, which is why issue is spread over
+// threads and why the tile is 256 tokens wide where tensor memory allows it. Two (one scale per channel)
 // or three (per-group scales) accumulator stages in TMEM let the epilogue of one
 // accumulation overlap the MMAs of the next ones. Every wait is bounded; on expiry the CTA records a status
 // word, stops issuing work and leaves through the common exit that frees TMEM.
@@ -27,9 +30,8 @@ namespace aq {
 
 namespace {
 
-constexpr int kNumStages = 6;                 // shared-memory ring: activation tile + packed weight block (+ scales)
 constexpr int kUnpackGroups = 2;              // groups of four unpack warps; group g takes k blocks g, g+2, ...
-constexpr int kFirstUnpackWarp = 4;           // warps 0-3: TMA producer, MMA issuer, two idle (one warpgroup)
+constexpr int kFirstUnpackWarp = 4;           // warps 0-3 (one warpgroup): two TMA producers, two MMA issuers
 constexpr int kFirstEpiWarp = kFirstUnpackWarp + 4 * kUnpackGroups;
 // Registers per thread after the roles split (setmaxnreg works on aligned groups of four warps):
 constexpr int kRegsControl = 40, kRegsUnpack = 48, kRegsEpilogue = 168;
@@ -208,12 +210,19 @@ __host__ __device__ constexpr uint32_t idesc_i8(int m, int n) {
 }
 
 template <int BM>
+struct TileConfig {
+    // shared-memory ring depth: activation tile + packed weight block (+ scales) per stage
+    static constexpr int kNumStages = BM >= 256 ? 5 : 6;
+};
+
+template <int BM>
 struct SharedStorage {
+    static constexpr int kNumStages = TileConfig<BM>::kNumStages;
     alignas(1024) uint8_t x[kNumStages][BM * 128];   // activation tiles, 128-byte swizzled rows
     alignas(128) uint8_t w[kNumStages][kBlockBytes]; // packed weight blocks (128 channels x 128 k)
     alignas(16) __half sc[kNumStages][kTileN];       // weight scales of the block's group (grouped mode)
-    alignas(8) uint64_t tma_full[kNumStages];        // TMA bytes landed -> unpack warps, MMA
-    uint64_t smem_empty[kNumStages];                 // MMA done (+ epilogue took the scales) -> TMA producer
+    alignas(8) uint64_t tma_full[kNumStages];        // both producers' bytes landed -> unpack warps
+    uint64_t smem_empty[kNumStages];                 // MMA done (+ epilogue took the scales) -> TMA producers
     uint64_t a_full[8];                              // unpack warps stored the slice -> MMA
     uint64_t a_empty[8];                             // MMA done with the slice -> unpack warps
     uint64_t acc_full[3];                            // MMA -> epilogue
@@ -240,7 +249,11 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
     using Smem = SharedStorage<BM>;
     Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
 
-    constexpr int kNumAcc = GROUPED ? 3 : 2;          // accumulator stages in tensor memory
+    constexpr int kNumStages = TileConfig<BM>::kNumStages;
+    // accumulator stages in tensor memory: three for per-group rescaling, otherwise as many
+    // 2 (or 1 for the 256-token tile) as leave room for the weight-slice ring
+    constexpr int kNumAcc = GROUPED ? 3 : (BM >= 256 ? 1 : 2);
+    constexpr int kNumMmaThreads = GROUPED ? 2 : 1;   // issuers alternate k blocks when every block has its own accumulator
     constexpr int kAccCols = kNumAcc * BM;
     // the rest of tensor memory (up to 8 slices) is the ring of unpacked weight slices (A operand)
     constexpr int kNumASlices = (512 - kAccCols) / kAColsPerStage >= 8 ? 8 : (512 - kAccCols) / kAColsPerStage;
@@ -260,7 +273,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kNumStages; ++s) {
-            mbar_init(&sm.tma_full[s], 1);
+            mbar_init(&sm.tma_full[s], 2);
             mbar_init(&sm.smem_empty[s], GROUPED ? 1 + kEpiWarps : 1);
         }
         for (int i = 0; i < kNumASlices; ++i) {
@@ -289,8 +302,8 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
 
     if (warp < kFirstUnpackWarp) {
       asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kRegsControl));
-      if (warp == 0) {
-        // ---------------------------------------------------------------- TMA producer
+      if (warp == 0 || warp == 2) {
+        // ------------- TMA producers: warp 0 streams activation tiles, warp 2 weight blocks (+ scales)
         if (lane == 0) {
             uint32_t it = 0;
             for (int tl = 0; tl < my_tiles; ++tl) {
@@ -301,51 +314,70 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
                     const int s = (int)(it % kNumStages);
                     const uint32_t ph = (it / kNumStages) & 1u;
                     if (!mbar_wait(&sm.smem_empty[s], ph ^ 1u, abort_flag)) goto role_done;
-                    mbar_arrive_expect_tx(&sm.tma_full[s], kStageBytes);
-                    tma_load_2d(sm.x[s], &x_map, kb * kTileK, mt * BM, &sm.tma_full[s]);
-                    tma_load_1d(sm.w[s], wsrc + (size_t)kb * kBlockBytes, kBlockBytes, &sm.tma_full[s]);
-                    if (GROUPED)
-                        tma_load_1d(sm.sc[s], p.w_scales + (size_t)kb * p.Npad + nt * kTileN, kTileN * 2,
-                                    &sm.tma_full[s]);
+                    if (warp == 0) {
+                        mbar_arrive_expect_tx(&sm.tma_full[s], BM * 128);
+                        tma_load_2d(sm.x[s], &x_map, kb * kTileK, mt * BM, &sm.tma_full[s]);
+                    } else {
+                        mbar_arrive_expect_tx(&sm.tma_full[s], kBlockBytes + (GROUPED ? kTileN * 2 : 0));
+                        tma_load_1d(sm.w[s], wsrc + (size_t)kb * kBlockBytes, kBlockBytes, &sm.tma_full[s]);
+                        if (GROUPED)
+                            tma_load_1d(sm.sc[s], p.w_scales + (size_t)kb * p.Npad + nt * kTileN, kTileN * 2,
+                                        &sm.tma_full[s]);
+                    }
                 }
             }
         }
-      } else if (warp == 1) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
+      } else {
+        // ------------- MMA issuers: warp 1 (and warp 3 in grouped mode, taking the odd k blocks)
+        const int mma_id = warp >> 1;                  // 0 or 1
+        if (lane == 0 && mma_id < kNumMmaThreads) {
             constexpr uint32_t idesc = idesc_i8(128, BM);
-            uint32_t it = 0;
-            uint32_t unit = 0;      // accumulations handed to the epilogue so far
-            for (int tl = 0; tl < my_tiles; ++tl) {
-                for (int kb = 0; kb < KB; ++kb, ++it) {
-                    const bool first = GROUPED || kb == 0;
-                    const int a = (int)(unit % kNumAcc);
-                    if (first) {
-                        const uint32_t aph = (unit / kNumAcc) & 1u;
-                        // grouped: the epilogue's initial bias store counts as the first release
-                        if (!mbar_wait(&sm.acc_empty[a], GROUPED ? aph : (aph ^ 1u), abort_flag)) goto role_done;
-                    }
+            const uint32_t total_iters = (uint32_t)my_tiles * (uint32_t)KB;
+            if (GROUPED) {
+                // every k block is one accumulation into its own (pre-biased) accumulator stage
+                for (uint32_t it = mma_id; it < total_iters; it += kNumMmaThreads) {
+                    const int a = (int)(it % kNumAcc);
                     const int s = (int)(it % kNumStages);
                     const int ai = (int)(it % kNumASlices);
-                    if (!mbar_wait(&sm.tma_full[s], (it / kNumStages) & 1u, abort_flag)) goto role_done;
+                    if (!mbar_wait(&sm.acc_empty[a], (it / kNumAcc) & 1u, abort_flag)) goto role_done;
                     if (!mbar_wait(&sm.a_full[ai], (it / kNumASlices) & 1u, abort_flag)) goto role_done;
                     tc_fence_after();
                     const uint32_t d_addr = tmem_acc + (uint32_t)(a * BM);
                     const uint32_t a_addr = tmem_a + (uint32_t)(ai * kAColsPerStage);
                     const uint64_t bdesc = smem_desc_sw128(smem_u32(sm.x[s]));
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        // 32 k per instruction: 8 TMEM columns of A, 32 bytes along the swizzled row of B
-                        tc_mma_i8_ts(d_addr, a_addr + 8 * j, bdesc + (uint64_t)(2 * j), idesc,
-                                     (!GROUPED && first && j == 0) ? 0u : 1u);
-                    }
+                    for (int j = 0; j < 4; ++j)
+                        tc_mma_i8_ts(d_addr, a_addr + 8 * j, bdesc + (uint64_t)(2 * j), idesc, 1u);
                     tc_commit(&sm.a_empty[ai]);
                     tc_commit(&sm.smem_empty[s]);
-                    const bool last = GROUPED || kb == KB - 1;
-                    if (last) {
-                        tc_commit(&sm.acc_full[a]);
-                        ++unit;
+                    tc_commit(&sm.acc_full[a]);
+                }
+            } else {
+                uint32_t it = 0;
+                for (int tl = 0; tl < my_tiles; ++tl) {
+                    const int a = (int)((uint32_t)tl % kNumAcc);
+                    const uint32_t aph = ((uint32_t)tl / kNumAcc) & 1u;
+                    if (!mbar_wait(&sm.acc_empty[a], aph ^ 1u, abort_flag)) goto role_done;
+                    for (int kb = 0; kb < KB; ++kb, ++it) {
+                        const int s = (int)(it % kNumStages);
+                        const int ai = (int)(it % kNumASlices);
+                        // the unpack warps publish a slice only after the stage's TMA bytes (activation
+                        // tile included) have landed, so this one wait covers both operands
+                        if (!mbar_wait(&sm.a_full[ai], (it / kNumASlices) & 1u, abort_flag)) goto role_done;
+                        tc_fence_after();
+                        const uint32_t d_addr = tmem_acc + (uint32_t)(a * BM);
+                        const uint32_t a_addr = tmem_a + (uint32_t)(ai * kAColsPerStage);
+                        const uint64_t bdesc = smem_desc_sw128(smem_u32(sm.x[s]));
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            // 32 k per instruction: 8 TMEM columns of A, 32 bytes along the swizzled row of B
+                            tc_mma_i8_ts(d_addr, a_addr + 8 * j, bdesc + (uint64_t)(2 * j), idesc,
+                                         (kb == 0 && j == 0) ? 0u : 1u);
+                        }
+                        tc_commit(&sm.a_empty[ai]);
+                        tc_commit(&sm.smem_empty[s]);
                     }
+                    tc_commit(&sm.acc_full[a]);
                 }
             }
         }
@@ -565,7 +597,10 @@ cudaError_t launch_bm(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t str
 
 cudaError_t launch_gemm_tensor(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
     if (a.M <= 64) return a.group ? launch_bm<64, true>(a, dev, stream) : launch_bm<64, false>(a, dev, stream);
-    return a.group ? launch_bm<128, true>(a, dev, stream) : launch_bm<128, false>(a, dev, stream);
+    if (a.group) return launch_bm<128, true>(a, dev, stream);
+    // one scale per channel: the 256-token tile halves the MMA instructions per unit of work
+    if (a.M <= 128) return launch_bm<128, false>(a, dev, stream);
+    return launch_bm<256, false>(a, dev, stream);
 }
 
 }  // namespace aq
