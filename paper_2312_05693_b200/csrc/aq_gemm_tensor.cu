@@ -59,8 +59,29 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t by
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
                  : "memory");
 }
+#ifndef AQ_SPIN_SLEEP_NS
+#define AQ_SPIN_SLEEP_NS 0
+#endif
+#ifndef AQ_EPI_PACKED
+#define AQ_EPI_PACKED 0
+#endif
+#ifndef AQ_WAIT_HINT_NS
+#define AQ_WAIT_HINT_NS 0
+#endif
+#ifndef AQ_WAIT_LANE0
+#define AQ_WAIT_LANE0 0
+#endif
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
+#if AQ_WAIT_HINT_NS > 0
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(AQ_WAIT_HINT_NS)
+        : "memory");
+#else
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
@@ -68,6 +89,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "=r"(ok)
         : "r"(smem_u32(bar)), "r"(parity)
         : "memory");
+#endif
     return ok != 0;
 }
 // Bounded wait. Returns false when the limit ran out or another role already gave up.
@@ -76,6 +98,9 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     const long long t0 = clock64();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
+#if AQ_SPIN_SLEEP_NS > 0
+        __nanosleep(AQ_SPIN_SLEEP_NS);
+#endif
         if ((++spins & 0x3FFu) == 0) {
             if (*abort_flag) return false;
             if ((unsigned long long)(clock64() - t0) > kWaitCycles) {
@@ -88,7 +113,13 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
 }
 // The same for a whole warp: all lanes agree on the outcome before any warp-wide instruction.
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+#if AQ_WAIT_LANE0
+    uint32_t ok = 0;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1u : 0u;
+    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+#else
     return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag) ? 1 : 0) != 0;
+#endif
 }
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
     asm volatile(
@@ -141,17 +172,6 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
         : "memory");
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&v)[32]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
-        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
-        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
-          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
-          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
-          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
-        : "memory");
-}
 __device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t (&v)[8]) {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
@@ -220,7 +240,12 @@ struct SharedStorage {
     static constexpr int kNumStages = TileConfig<BM>::kNumStages;
     alignas(1024) uint8_t x[kNumStages][BM * 128];   // activation tiles, 128-byte swizzled rows
     alignas(128) uint8_t w[kNumStages][kBlockBytes]; // packed weight blocks (128 channels x 128 k)
-    alignas(16) __half sc[kNumStages][kTileN];       // weight scales of the block's group (grouped mode)
+    // Weight scales of each block's group (grouped mode), in a ring three slots deeper than the
+    // stage ring. A slot is rewritten for block i only after the MMAs of block i - kNumStages
+    // completed, which (three accumulator stages) needs the epilogue of every block up to
+    // i - kNumStages - 3 to have finished: all reads of the slot's previous content are done.
+    static constexpr int kNumScaleSlots = kNumStages + 3;
+    alignas(16) __half sc[kNumScaleSlots][kTileN];
     alignas(8) uint64_t tma_full[kNumStages];        // both producers' bytes landed -> unpack warps
     uint64_t smem_empty[kNumStages];                 // MMA done (+ epilogue took the scales) -> TMA producers
     uint64_t a_full[8];                              // unpack warps stored the slice -> MMA
@@ -258,13 +283,13 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
     // the rest of tensor memory (up to 8 slices) is the ring of unpacked weight slices (A operand)
     constexpr int kNumASlices = (512 - kAccCols) / kAColsPerStage >= 8 ? 8 : (512 - kAccCols) / kAColsPerStage;
     static_assert(kNumASlices >= 4 && kNumASlices % kUnpackGroups == 0, "weight-slice ring");
+    static_assert(!GROUPED || kNumAcc == 3, "the scale ring's depth assumes three accumulator stages");
     constexpr int kTmemColsUsed = kAccCols + kNumASlices * kAColsPerStage;
     constexpr int kTmemCols = kTmemColsUsed <= 128 ? 128 : kTmemColsUsed <= 256 ? 256 : 512;
     static_assert(kTmemColsUsed <= 512, "tensor memory has 512 columns");
     static_assert(BM % 64 == 0 && BM >= 64 && BM <= 256, "token tile");
     constexpr int kColsPerEpiWarp = BM / 2;           // each quarter's columns are split between two warps
     static_assert(kColsPerEpiWarp % 16 == 0 && (!GROUPED || kColsPerEpiWarp % 32 == 0), "epilogue chunking");
-    constexpr uint32_t kStageBytes = BM * 128 + kBlockBytes + (GROUPED ? kTileN * 2 : 0);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KB = p.K / kTileK;
@@ -274,7 +299,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
     if (threadIdx.x == 0) {
         for (int s = 0; s < kNumStages; ++s) {
             mbar_init(&sm.tma_full[s], 2);
-            mbar_init(&sm.smem_empty[s], GROUPED ? 1 + kEpiWarps : 1);
+            mbar_init(&sm.smem_empty[s], 1);
         }
         for (int i = 0; i < kNumASlices; ++i) {
             mbar_init(&sm.a_full[i], 4);
@@ -321,8 +346,8 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
                         mbar_arrive_expect_tx(&sm.tma_full[s], kBlockBytes + (GROUPED ? kTileN * 2 : 0));
                         tma_load_1d(sm.w[s], wsrc + (size_t)kb * kBlockBytes, kBlockBytes, &sm.tma_full[s]);
                         if (GROUPED)
-                            tma_load_1d(sm.sc[s], p.w_scales + (size_t)kb * p.Npad + nt * kTileN, kTileN * 2,
-                                        &sm.tma_full[s]);
+                            tma_load_1d(sm.sc[it % Smem::kNumScaleSlots],
+                                        p.w_scales + (size_t)kb * p.Npad + nt * kTileN, kTileN * 2, &sm.tma_full[s]);
                     }
                 }
             }
@@ -435,7 +460,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         const int col0 = half * kColsPerEpiWarp;
         const float pe = __int_as_float((127 + *p.scale_exp) << 23);     // 2^e
-        const int G = GROUPED ? KB : 1;
+        [[maybe_unused]] const int G = GROUPED ? KB : 1;
         uint32_t unit = 0, it = 0;
         if (GROUPED) {
             // arm every accumulator stage with the bias; this is the first release of each stage
@@ -455,7 +480,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
             const int n = nt * kTileN + r;
             const int m_base = mt * BM + col0;
             const bool n_ok = n < p.N;
-            if (!GROUPED) {
+            if constexpr (!GROUPED) {
                 const int a = (int)(unit % kNumAcc);
                 const uint32_t aph = (unit / kNumAcc) & 1u;
                 const float sc = __half2float(p.w_scales[n]) * 0.0625f * pe;   // sums carry a factor 16
@@ -481,45 +506,57 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
                 if (lane == 0) mbar_arrive(&sm.acc_empty[a]);
                 ++unit;
             } else {
+#if AQ_EPI_PACKED
                 uint64_t fsum2[kColsPerEpiWarp / 2];                     // pairs of fp32 partial outputs
 #pragma unroll
                 for (int c = 0; c < kColsPerEpiWarp / 2; ++c) fsum2[c] = 0ull;
                 const uint64_t neg_magic2 = pack2(-kMagicFloat, -kMagicFloat);
+#else
+                float fsum[kColsPerEpiWarp];                             // fp32 partial outputs
+#pragma unroll
+                for (int c = 0; c < kColsPerEpiWarp; ++c) fsum[c] = 0.0f;
+#endif
                 for (int kb = 0; kb < KB; ++kb, ++unit, ++it) {
                     const int a = (int)(unit % kNumAcc);
                     const uint32_t aph = (unit / kNumAcc) & 1u;
-                    const int s = (int)(it % kNumStages);
                     if (!mbar_wait_warp(&sm.acc_full[a], aph, abort_flag)) goto role_done;
                     tc_fence_after();
-                    // the block's scales landed with its operands (the wait below passes at once and
-                    // orders the read after the copy); take ours, then let the stage go
-                    if (!mbar_wait_warp(&sm.tma_full[s], (it / kNumStages) & 1u, abort_flag)) goto role_done;
-                    const float sg = __half2float(sm.sc[s][r]) * 0.0625f;
+                    // This block's MMAs are complete, so its stage (scales included) had landed: the
+                    // issuer saw the unpack warps' signal, which they gave after seeing the TMA barrier.
+                    const float sg = __half2float(sm.sc[it % Smem::kNumScaleSlots][r]) * 0.0625f;
+#if AQ_EPI_PACKED
                     const uint64_t sg2 = pack2(sg, sg);
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&sm.smem_empty[s]);
+#endif
+                    static_assert(kColsPerEpiWarp == 32 || kColsPerEpiWarp == 64, "epilogue register plan");
+                    const uint32_t taddr = tmem_acc + lane_addr + (uint32_t)(a * BM + col0);
+                    uint32_t v[kColsPerEpiWarp];
+                    tc_ld32(taddr, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+                    if (kColsPerEpiWarp == 64) tc_ld32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32 % kColsPerEpiWarp]));
+                    tc_wait_ld();
+                    tc_st32_fill(taddr, kMagicBits);                     // re-arm the bias for the next use
+                    if (kColsPerEpiWarp == 64) tc_st32_fill(taddr + 32, kMagicBits);
+#if AQ_EPI_PACKED
 #pragma unroll
-                    for (int c0 = 0; c0 < kColsPerEpiWarp; c0 += 32) {
-                        const uint32_t taddr = tmem_acc + lane_addr + (uint32_t)(a * BM + col0 + c0);
-                        uint32_t v[32];
-                        tc_ld32(taddr, v);
-                        tc_wait_ld();
-                        tc_st32_fill(taddr, kMagicBits);                 // re-arm the bias for the next use
+                    for (int c = 0; c < kColsPerEpiWarp; c += 2) {
+                        // v holds the bits of the floats (magic + 16*sum): remove the bias, scale, add
+                        uint64_t t;
+                        asm("mov.b64 %0, {%1, %2};" : "=l"(t) : "r"(v[c]), "r"(v[c + 1]));
+                        t = add2(t, neg_magic2);
+                        fsum2[c / 2] = fma2(t, sg2, fsum2[c / 2]);
+                    }
+#else
 #pragma unroll
-                        for (int c = 0; c < 32; c += 2) {
-                            // v holds the bits of the floats (magic + 16*sum): remove the bias, scale, add
-                            uint64_t t;
-                            asm("mov.b64 %0, {%1, %2};" : "=l"(t) : "r"(v[c]), "r"(v[c + 1]));
-                            t = add2(t, neg_magic2);
-                            fsum2[(c0 + c) / 2] = fma2(t, sg2, fsum2[(c0 + c) / 2]);
-                        }
-                        if (p.acc_dump) {
+                    for (int c = 0; c < kColsPerEpiWarp; ++c) {
+                        // v holds the bits of the float (magic + 16*sum): remove the bias, scale, add
+                        fsum[c] = fmaf(__uint_as_float(v[c]) - kMagicFloat, sg, fsum[c]);
+                    }
+#endif
+                    if (p.acc_dump) {
 #pragma unroll
-                            for (int c = 0; c < 32; ++c) {
-                                const int m = m_base + c0 + c;
-                                if (n_ok && m < p.M)
-                                    p.acc_dump[((size_t)m * p.N + n) * G + kb] = (int)(v[c] - kMagicBits) >> 4;
-                            }
+                        for (int c = 0; c < kColsPerEpiWarp; ++c) {
+                            const int m = m_base + c;
+                            if (n_ok && m < p.M)
+                                p.acc_dump[((size_t)m * p.N + n) * G + kb] = (int)(v[c] - kMagicBits) >> 4;
                         }
                     }
                     tc_wait_st();
@@ -530,7 +567,12 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
 #pragma unroll
                 for (int c = 0; c < kColsPerEpiWarp; c += 2) {
                     float lo, hi;
+#if AQ_EPI_PACKED
                     unpack2(fsum2[c / 2], lo, hi);
+#else
+                    lo = fsum[c];
+                    hi = fsum[c + 1];
+#endif
                     const int m = m_base + c;
                     if (n_ok && m < p.M) p.y[(size_t)m * p.N + n] = __float2half_rn(lo * pe);
                     if (n_ok && m + 1 < p.M) p.y[(size_t)(m + 1) * p.N + n] = __float2half_rn(hi * pe);
