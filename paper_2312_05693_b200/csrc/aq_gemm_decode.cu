@@ -1,8 +1,24 @@
-// Integer product for few rows (M <= 16 per CTA pass): a weight-streaming reduction on
-// CUDA cores. Every packed weight byte is read from HBM exactly once per 16 activation
-// rows; products use dp4a (4 int8 x int8 per instruction) on weights widened to 16*code.
-// Computes the sums of Sec. 4.4 / Algorithm 1 and the floating-point output.
+// Integer product for few rows (M <= 16 per pass): weight-streaming reductions that read
+// every packed weight byte from HBM once per 16 activation rows. They compute the sums of
+// Sec. 4.4 / Algorithm 1 and the floating-point output.
+//
+// Two kernels:
+//  * a general one (per-group scales, or any M when forced): a CTA owns 32 output channels
+//    (one lane each), its 8 warps split K by 128-k block, products use dp4a on weights
+//    widened to 16*code, warps meet in shared memory;
+//  * a streaming one for one scale per channel and M <= 16: a thread-block cluster shares a
+//    128-channel tile and splits K; in each CTA a producer thread streams 8 KB packed blocks
+//    and their activation codes into a shared-memory ring with TMA, eight consumer warps
+//    multiply (dp4a up to 4 rows, the warp-level int8 MMA above), and the CTAs' partial sums
+//    are added into the leader CTA's shared memory over distributed shared memory (integer
+//    addition is exact in any order), which then writes the tile's outputs. No workspace, no
+//    global atomics.
+#include <cooperative_groups.h>
+#include <cuda.h>
+
 #include "aq_common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace aq {
 
@@ -131,6 +147,317 @@ gemm_decode_kernel(const int8_t* __restrict__ q, int M, int K, int N, int Npad,
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// Streaming kernel (one scale per channel, M <= 16)
+// ---------------------------------------------------------------------------------------
+constexpr int kStrStages = 8;
+constexpr int kStrConsumerWarps = 8;
+constexpr int kStrThreads = (1 + kStrConsumerWarps) * 32;
+constexpr unsigned long long kStrWaitCycles = 4000000000ull;
+
+__device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool str_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(s_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait; false when the limit ran out or another thread of the CTA already gave up.
+__device__ __forceinline__ bool str_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+    if (str_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t spins = 0;
+    while (!str_try_wait(bar, parity)) {
+        if ((++spins & 0x3FFu) == 0) {
+            if (*abort_flag) return false;
+            if ((unsigned long long)(clock64() - t0) > kStrWaitCycles) { *abort_flag = 1; return false; }
+        }
+    }
+    return true;
+}
+
+// Rows up to 4 use dp4a with one lane per channel; more rows use the warp-level int8 MMA
+// (m16n8k32) on 16 rows, with the activation tile stored 128-byte swizzled so that fragment
+// loads are free of bank conflicts.
+template <int MB> struct StreamCfg {
+    static constexpr bool kUseMma = MB > 4;
+    static constexpr int kRows = kUseMma ? 16 : MB;
+};
+
+template <int MB>
+struct StreamSmem {
+    static constexpr int kRows = StreamCfg<MB>::kRows;
+    alignas(1024) int8_t x[kStrStages][kRows * kTileK];    // activation codes of the unit's k block
+    alignas(128) uint8_t w[kStrStages][kBlockBytes];       // packed weight block of the unit
+    int part[4][kRows][32];                                // second k-half's partial sums
+    int sum[kRows][kTileN];                                // leader CTA: the tile's sums over all of K
+    alignas(8) uint64_t full[kStrStages];
+    uint64_t empty[kStrStages];
+    volatile uint32_t abort_flag;
+};
+
+struct StreamParams {
+    int M, K, N, Npad;
+    const uint8_t* w_packed;
+    const __half* w_scales;
+    const int32_t* scale_exp;
+    __half* y;
+    int32_t* acc_dump;
+    Control* ctl;
+};
+
+// grid = (split, channel tiles), cluster = (split, 1, 1): the CTAs of a cluster share a channel
+// tile and take consecutive k ranges; their sums meet in the leader's shared memory.
+template <int MB>
+__global__ void __launch_bounds__(kStrThreads, 2)
+gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const StreamParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    using Smem = StreamSmem<MB>;
+    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    constexpr bool kUseMma = StreamCfg<MB>::kUseMma;
+    constexpr int kRows = StreamCfg<MB>::kRows;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int KB = p.K / kTileK;
+    const int rank = blockIdx.x, split = gridDim.x;
+    const int tile = blockIdx.y;
+    const int kb0 = (int)((long long)KB * rank / split), kb1 = (int)((long long)KB * (rank + 1) / split);
+    constexpr uint32_t kUnitBytes = kBlockBytes + kRows * kTileK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStrStages; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(s_u32(&sm.full[s])) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s_u32(&sm.empty[s])), "r"(kStrConsumerWarps) : "memory");
+        }
+        sm.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int i = threadIdx.x; i < kRows * kTileN; i += kStrThreads) (&sm.sum[0][0])[i] = 0;
+    __syncthreads();
+    volatile uint32_t* abort_flag = &sm.abort_flag;
+    const uint8_t* wsrc = p.w_packed + (size_t)tile * KB * kBlockBytes;
+
+    auto issue = [&](int kb, int s) {
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                     ::"r"(s_u32(&sm.full[s])), "r"(kUnitBytes) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(s_u32(sm.w[s])), "l"(wsrc + (size_t)kb * kBlockBytes), "r"((uint32_t)kBlockBytes),
+                       "r"(s_u32(&sm.full[s])) : "memory");
+        asm volatile(
+            "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+            ::"r"(s_u32(sm.x[s])), "l"(&x_map), "r"(kb * kTileK), "r"(0), "r"(s_u32(&sm.full[s])) : "memory");
+    };
+    // the first ring-full of loads goes out before the cluster handshake below, so data is
+    // already streaming while the CTAs of the cluster meet
+    int issued = 0;
+    if (warp == 0 && lane == 0)
+        for (; issued < kStrStages && kb0 + issued < kb1; ++issued) issue(kb0 + issued, issued);
+    cluster.sync();                                   // every CTA's `sum` is zeroed before anyone adds to it
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int kb = kb0 + issued; kb < kb1; ++kb) {
+                const uint32_t i = (uint32_t)(kb - kb0);
+                const int s = (int)(i % kStrStages);
+                if (!str_wait(&sm.empty[s], ((i / kStrStages) & 1u) ^ 1u, abort_flag)) break;
+                issue(kb, s);
+            }
+        }
+    } else {
+        const int cw = warp - 1;
+        const int quarter = cw & 3, half = cw >> 2;
+        int* leader_sum = split > 1 ? cluster.map_shared_rank(&sm.sum[0][0], 0) : &sm.sum[0][0];
+        if constexpr (!kUseMma) {
+            const int r = quarter * 32 + lane;                       // channel inside the tile
+            int acc[MB];
+#pragma unroll
+            for (int m = 0; m < MB; ++m) acc[m] = 0;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                const uint32_t i = (uint32_t)(kb - kb0);
+                const int s = (int)(i % kStrStages);
+                if (!__all_sync(0xFFFFFFFFu, str_wait(&sm.full[s], (i / kStrStages) & 1u, abort_flag) ? 1 : 0)) break;
+#pragma unroll
+                for (int jj = 0; jj < 2; ++jj) {
+                    const int j = 2 * half + jj;
+                    const uint4 d = reinterpret_cast<const uint4*>(sm.w[s])[j * kTileN + r];
+                    const uint32_t w[4] = {d.x, d.y, d.z, d.w};
+                    uint32_t w8[8];
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        w8[2 * t] = (w[t] << 4) & 0xF0F0F0F0u;           // 16*code for k0..k0+3
+                        w8[2 * t + 1] = w[t] & 0xF0F0F0F0u;              // 16*code for k0+4..k0+7
+                    }
+#pragma unroll
+                    for (int m = 0; m < MB; ++m) {
+                        const uint4* xp = reinterpret_cast<const uint4*>(sm.x[s] + m * kTileK + 32 * j);
+                        const uint4 x0 = xp[0], x1 = xp[1];              // same address in every lane: broadcast
+                        int a = acc[m];
+                        a = __dp4a((int)w8[0], (int)x0.x, a);
+                        a = __dp4a((int)w8[1], (int)x0.y, a);
+                        a = __dp4a((int)w8[2], (int)x0.z, a);
+                        a = __dp4a((int)w8[3], (int)x0.w, a);
+                        a = __dp4a((int)w8[4], (int)x1.x, a);
+                        a = __dp4a((int)w8[5], (int)x1.y, a);
+                        a = __dp4a((int)w8[6], (int)x1.z, a);
+                        a = __dp4a((int)w8[7], (int)x1.w, a);
+                        acc[m] = a;
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s_u32(&sm.empty[s])) : "memory");
+            }
+            // the two k-halves of a channel meet in shared memory, then one integer add per
+            // (row, channel) into the leader CTA's sums (exact in any order)
+            if (half == 1) {
+#pragma unroll
+                for (int m = 0; m < MB; ++m) sm.part[quarter][m][lane] = acc[m];
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(kStrConsumerWarps * 32) : "memory");
+            if (half == 0) {
+#pragma unroll
+                for (int m = 0; m < MB; ++m)
+                    if (m < p.M) atomicAdd(&leader_sum[m * kTileN + r], acc[m] + sm.part[quarter][m][lane]);
+            }
+        } else {
+            // Warp-level int8 MMA, D[16 rows x 8 channels] += A[16 x 32 k] * B[32 k x 8 channels].
+            // Fragment owner: g = lane / 4 (row g and g+8 of A and D; channel g of B),
+            // t = lane % 4 (k bytes 4t..4t+3 and 16+4t..; D columns 2t, 2t+1).
+            const int g = lane >> 2, t = lane & 3;
+            int acc[4][4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int c = 0; c < 4; ++c) acc[i][c] = 0;
+            for (int kb = kb0; kb < kb1; ++kb) {
+                const uint32_t it = (uint32_t)(kb - kb0);
+                const int s = (int)(it % kStrStages);
+                if (!__all_sync(0xFFFFFFFFu, str_wait(&sm.full[s], (it / kStrStages) & 1u, abort_flag) ? 1 : 0)) break;
+#pragma unroll
+                for (int jj = 0; jj < 2; ++jj) {
+                    const int j = 2 * half + jj;
+                    // activation fragment: row-major 128-byte rows, 16-byte chunks XOR-swizzled by row % 8
+                    const int8_t* xr0 = sm.x[s] + g * kTileK;
+                    const int8_t* xr1 = sm.x[s] + (g + 8) * kTileK;
+                    const int c_lo = ((2 * j) ^ g) * 16 + 4 * t, c_hi = ((2 * j + 1) ^ g) * 16 + 4 * t;
+                    const uint32_t a0 = *reinterpret_cast<const uint32_t*>(xr0 + c_lo);
+                    const uint32_t a1 = *reinterpret_cast<const uint32_t*>(xr1 + c_lo);
+                    const uint32_t a2 = *reinterpret_cast<const uint32_t*>(xr0 + c_hi);
+                    const uint32_t a3 = *reinterpret_cast<const uint32_t*>(xr1 + c_hi);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        // weight fragment of channel 32*quarter + 8i + g: packed word t/2 holds k 4t..4t+3 in
+                        // its low (t even) or high (t odd) nibbles; word t/2 + 2 holds k 16+4t..
+                        const uint32_t* wp = reinterpret_cast<const uint32_t*>(
+                            sm.w[s] + (size_t)(j * kTileN + quarter * 32 + 8 * i + g) * 16) + (t >> 1);
+                        const uint32_t p0 = wp[0], p1 = wp[2];
+                        const uint32_t b0 = (t & 1) ? (p0 & 0xF0F0F0F0u) : ((p0 << 4) & 0xF0F0F0F0u);
+                        const uint32_t b1 = (t & 1) ? (p1 & 0xF0F0F0F0u) : ((p1 << 4) & 0xF0F0F0F0u);
+                        asm volatile(
+                            "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, "
+                            "{%8, %9}, {%0, %1, %2, %3};"
+                            : "+r"(acc[i][0]), "+r"(acc[i][1]), "+r"(acc[i][2]), "+r"(acc[i][3])
+                            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s_u32(&sm.empty[s])) : "memory");
+            }
+            // D fragment: acc[i][0..1] = row g, channels 8i+2t, +1; acc[i][2..3] = row g+8
+            if (half == 1) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) sm.part[quarter][g + 8 * (c >> 1)][8 * i + 2 * t + (c & 1)] = acc[i][c];
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(kStrConsumerWarps * 32) : "memory");
+            if (half == 0) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const int m = g + 8 * (c >> 1), ch = 8 * i + 2 * t + (c & 1);
+                        if (m < p.M)
+                            atomicAdd(&leader_sum[m * kTileN + quarter * 32 + ch], acc[i][c] + sm.part[quarter][m][ch]);
+                    }
+            }
+        }
+    }
+    // the output scale is fetched before the cluster meets so that its latency overlaps the wait
+    float sc = 0.0f;
+    const int out_r = (warp - 1) * 32 + lane;
+    const int out_n = tile * kTileN + out_r;
+    if (rank == 0 && warp >= 1 && warp <= 4 && out_n < p.N)
+        sc = __half2float(p.w_scales[out_n]) * __int_as_float((127 + *p.scale_exp) << 23);
+    cluster.sync();
+    if (rank == 0 && warp >= 1 && warp <= 4 && out_n < p.N) {
+#pragma unroll
+        for (int m = 0; m < MB; ++m) {
+            if (m < p.M) {
+                const int a = sm.sum[m][out_r] >> 4;                  // sums carry a factor 16
+                if (p.acc_dump) p.acc_dump[(size_t)m * p.N + out_n] = a;
+                p.y[(size_t)m * p.N + out_n] = __float2half_rn((float)a * sc);
+            }
+        }
+    }
+    if (sm.abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);          // let copies in flight land
+        if (threadIdx.x == 0) atomicOr(&p.ctl->status, 1u);
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+template <int MB>
+cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
+    using Smem = StreamSmem<MB>;
+    const size_t smem_bytes = sizeof(Smem) + 1024;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_decode_stream_kernel<MB>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    CUtensorMap map;
+    const cuuint64_t dims[2] = {(cuuint64_t)a.K, (cuuint64_t)a.M};
+    const cuuint64_t strides[1] = {(cuuint64_t)a.K};
+    const cuuint32_t box[2] = {128u, (cuuint32_t)StreamCfg<MB>::kRows};
+    const cuuint32_t estr[2] = {1u, 1u};
+    const CUresult r = reinterpret_cast<EncodeTiledFn>(dev.encode_tiled)(
+        &map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(a.q), dims, strides, box, estr,
+        CU_TENSOR_MAP_INTERLEAVE_NONE,
+        StreamCfg<MB>::kUseMma ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+        CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+    StreamParams p;
+    p.M = a.M; p.K = a.K; p.N = a.N; p.Npad = round_up(a.N, kTileN);
+    p.w_packed = a.w_packed; p.w_scales = a.w_scales; p.scale_exp = a.scale_exp;
+    p.y = a.y; p.acc_dump = a.acc_dump; p.ctl = a.ctl;
+    const int tiles = p.Npad / kTileN, KB = a.K / kTileK;
+    // as many k ranges per tile as keep all CTAs resident at once (two per SM), a power of two
+    // up to 4 so that clusters place easily, and at least two k blocks per CTA
+    int split = 1;
+    while (split < 4 && tiles * split * 2 <= 2 * dev.sm_count && KB / (split * 2) >= 2) split *= 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(split, tiles, 1);
+    cfg.blockDim = dim3(kStrThreads);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = split;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, gemm_decode_stream_kernel<MB>, map, p);
+}
+
 template <int MB>
 cudaError_t launch_mb(const GemmArgs& a, cudaStream_t stream) {
     const int Npad = round_up(a.N, kTileN);
@@ -147,7 +474,13 @@ cudaError_t launch_mb(const GemmArgs& a, cudaStream_t stream) {
 }  // namespace
 
 cudaError_t launch_gemm_decode(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
-    (void)dev;
+    if (!a.group && a.M <= 16) {
+        if (a.M <= 1) return launch_stream<1>(a, dev, stream);
+        if (a.M <= 2) return launch_stream<2>(a, dev, stream);
+        if (a.M <= 4) return launch_stream<4>(a, dev, stream);
+        if (a.M <= 8) return launch_stream<8>(a, dev, stream);
+        return launch_stream<16>(a, dev, stream);
+    }
     if (a.M <= 1) return launch_mb<1>(a, stream);
     if (a.M <= 2) return launch_mb<2>(a, stream);
     if (a.M <= 4) return launch_mb<4>(a, stream);

@@ -112,6 +112,26 @@ def test_linear_w4a8_matches_checker(kernel, M, K, N, group):
     assert_y_close(gpu["y"], ref["y"])
 
 
+@pytest.mark.parametrize("group", [0, 128])
+@pytest.mark.parametrize("M", [1, 2, 3, 4, 5, 8, 11, 16])
+def test_decode_rows_1_to_16(M, group):
+    """The M <= 16 path (dp4a up to 4 rows, warp MMA above) over several k splits and a ragged N."""
+    for K, N in [(1280, 392), (5120, 128)]:
+        x = inputs.activations(M, K, seed=M + K, outlier_frac=0.01, outlier_mult=20.0)
+        w = inputs.weights(N, K, seed=N + K)
+        gpu, ref = run_layer_both(x, w, 8, group, binding.AQ_KERNEL_AUTO)
+        assert gpu["e"] == ref["e"] and np.array_equal(gpu["q"], ref["q"])
+        assert np.array_equal(gpu["acc"], ref["acc"])
+        assert_y_close(gpu["y"], ref["y"])
+    # extreme codes: the largest sums the 16x-widened weights can produce
+    K, N = 13824, 128
+    x = np.full((M, K), -128.0, np.float16)
+    w = np.full((N, K), -0.01, np.float16)
+    gpu, ref = run_layer_both(x, w, 8, group, binding.AQ_KERNEL_AUTO, scale_mode=1, clip=0)
+    assert np.array_equal(gpu["acc"], ref["acc"])
+    assert_y_close(gpu["y"], ref["y"])
+
+
 @pytest.mark.parametrize("kernel", KERNELS)
 @pytest.mark.parametrize("M,K,N,group", [(16, 768, 768, 0), (129, 384, 200, 128), (260, 1152, 520, 128)])
 def test_linear_w4a4_matches_checker(kernel, M, K, N, group):
