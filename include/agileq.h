@@ -47,7 +47,8 @@ typedef enum aq_status {
     AQ_ERR_WORKSPACE = -4,          /* workspace NULL or smaller than aq_workspace_bytes() */
     AQ_ERR_UNSUPPORTED_DEVICE = -5, /* not compute capability 10.0 */
     AQ_ERR_CUDA = -6,               /* a CUDA call failed; see aq_last_cuda_error() */
-    AQ_ERR_DEVICE_TIMEOUT = -7      /* a bounded wait inside a kernel gave up */
+    AQ_ERR_DEVICE_TIMEOUT = -7,     /* a bounded wait inside a kernel gave up */
+    AQ_ERR_TOO_LARGE = -8           /* the sizes need more than the library's built-in scratch */
 } aq_status;
 
 /* How the layer exponent e is chosen (paper Eq. 6 read as a symmetric power-of-two
@@ -147,6 +148,38 @@ int aq_linear_host(aq_handle_t h, int bits, const void* x_host, int M, int K,
  * this workspace gave up on a bounded wait (AQ_ERR_DEVICE_TIMEOUT); AQ_OK otherwise. Every
  * aq_linear_* / aq_gemm_w4 / aq_quantize_act call clears the record when it starts. */
 int aq_check_workspace(aq_handle_t h, const void* workspace, void* stream);
+
+/* ---- the layer without any caller-provided or allocated scratch
+ * (The paper has no counterpart to this call: it exists for the way some programs must use
+ * the library, not for anything the method computes.)
+ *
+ * Same result as aq_linear_w4a8 with row_idx = NULL and acc_dump = NULL, but the scratch the
+ * layer needs (the control block and the int8 activation codes, see aq_workspace_bytes) lives
+ * in a fixed buffer inside the library instead of a workspace from the caller. It is meant for
+ * callers that may not allocate device memory at the point of the call: code running inside a
+ * memory pool that has already handed out the whole device, plugin and serving hosts that
+ * forbid cudaMalloc after start-up because an allocation synchronizes the device and can fail
+ * late, and real-time loops where an out-of-memory error must be impossible by construction.
+ * This call performs no cudaMalloc / cudaFree and calls nothing that allocates.
+ *
+ * Limits and rules
+ *  - aq_workspace_bytes(M, K, N, group_size) must not exceed AQ_NOALLOC_SCRATCH_BYTES
+ *    (about M*K <= 16 Mi codes, e.g. 2048 x 8192 or 4096 x 4096); larger sizes are refused with
+ *    AQ_ERR_TOO_LARGE and nothing is enqueued. Use aq_linear_w4a8 with your own workspace then.
+ *  - The buffer is a static device array: every GPU on which the library is loaded holds
+ *    AQ_NOALLOC_SCRATCH_BYTES of device memory until the process exits.
+ *  - The first call on each device looks up the buffer's device address (a one-time,
+ *    host-side set-up that needs that device to be current). Make that first call before
+ *    starting any stream capture.
+ *  - All calls on a device share the one buffer, and it keeps the previous call's contents; the
+ *    call itself clears the part that must start at zero. Two calls that can overlap on the
+ *    GPU (different streams without ordering) race on the buffer: order them, or use
+ *    aq_linear_w4a8 with separate workspaces.
+ *  - The handle's device must be the current device. */
+#define AQ_NOALLOC_SCRATCH_BYTES ((size_t)16 * 1024 * 1024 + 65536 + 256)
+int aq_linear_w4a8_noalloc(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed,
+                           const void* w_scales, int N, int group_size, int scale_mode,
+                           int clip_shift_or_exp, void* y_fp16, void* stream);
 
 #ifdef __cplusplus
 }

@@ -20,6 +20,8 @@ HEADER_PATH = os.path.join(os.path.dirname(_DIR), "include", "agileq.h")
 AQ_OK = 0
 AQ_ERR_INVALID_ARG, AQ_ERR_SHAPE, AQ_ERR_ALIGNMENT, AQ_ERR_WORKSPACE = -1, -2, -3, -4
 AQ_ERR_UNSUPPORTED_DEVICE, AQ_ERR_CUDA, AQ_ERR_DEVICE_TIMEOUT = -5, -6, -7
+AQ_ERR_TOO_LARGE = -8
+AQ_NOALLOC_SCRATCH_BYTES = 16 * 1024 * 1024 + 65536 + 256
 AQ_SCALE_DYNAMIC, AQ_SCALE_STATIC = 0, 1
 AQ_KERNEL_AUTO, AQ_KERNEL_TENSOR, AQ_KERNEL_DECODE = 0, 1, 2
 
@@ -76,6 +78,7 @@ def load():
     L.aq_token_compact.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp]
     L.aq_linear_host.argtypes = [vp, i32, vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, vp, sz, vp]
     L.aq_check_workspace.argtypes = [vp, vp, vp]
+    L.aq_linear_w4a8_noalloc.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, vp]
     _lib = L
     return L
 
@@ -242,6 +245,16 @@ class Handle:
                                      _ptr(device_scratch), device_scratch.numel(), _stream()),
                "aq_linear_host")
         return y_host
+
+    def aq_linear_w4a8_noalloc(self, x, packed, scales, N, group_size, y, scale_mode=AQ_SCALE_DYNAMIC,
+                               clip_shift_or_exp=0):
+        """The W4A8 layer using the library's built-in scratch buffer. The binding itself allocates
+        nothing either: the caller passes the output tensor `y` [M, N] fp16."""
+        M, K = x.shape
+        _check(load().aq_linear_w4a8_noalloc(self._h, _ptr(x), M, K, _ptr(packed), _ptr(scales), N, group_size,
+                                             scale_mode, clip_shift_or_exp, _ptr(y), _stream()),
+               "aq_linear_w4a8_noalloc")
+        return y
 
     def aq_check_workspace(self, workspace: torch.Tensor) -> int:
         return load().aq_check_workspace(self._h, _ptr(workspace), _stream())

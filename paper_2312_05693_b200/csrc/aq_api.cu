@@ -110,6 +110,7 @@ const char* aq_status_string(int status) {
         case AQ_ERR_UNSUPPORTED_DEVICE: return "device is not compute capability 10.0";
         case AQ_ERR_CUDA: return "CUDA call failed";
         case AQ_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel gave up";
+        case AQ_ERR_TOO_LARGE: return "sizes exceed the library's built-in scratch buffer";
         default: return "unknown status";
     }
 }
@@ -147,6 +148,16 @@ int aq_destroy(aq_handle_t h) {
 }
 
 int aq_last_cuda_error(aq_handle_t h) { return h ? h->last_cuda_error : 0; }
+}  // extern "C"
+
+namespace aq {
+int handle_device(aq_handle_t h) { return h ? h->dev.device : -1; }
+void handle_record_cuda_error(aq_handle_t h, cudaError_t e) {
+    if (h) h->last_cuda_error = (int)e;
+}
+}  // namespace aq
+
+extern "C" {
 
 int aq_set_kernel(aq_handle_t h, int kernel) {
     if (!h || kernel < AQ_KERNEL_AUTO || kernel > AQ_KERNEL_DECODE) return AQ_ERR_INVALID_ARG;

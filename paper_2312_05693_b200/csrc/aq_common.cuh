@@ -104,6 +104,10 @@ struct GemmArgs {
     void* scratch;          // beyond control block + codes
     size_t scratch_bytes;
 };
+// Small accessors for code outside aq_api.cu that is handed a handle.
+int handle_device(aq_handle_t h);
+void handle_record_cuda_error(aq_handle_t h, cudaError_t e);
+
 cudaError_t launch_gemm_tensor(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_gemm_decode(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream);
 
