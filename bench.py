@@ -129,6 +129,21 @@ def graph_replay_ms(launch, replays, warm=2):
     return a.elapsed_time(b) / replays
 
 
+def max_over_ranks(values, dist, device):
+    """Element-wise maximum over all ranks of a list of per-rank times (identity without a
+    process group). Every rank gets the same list back."""
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def aggregate_value(world, units_per_rank_step, ms_per_step):
+    """Whole-job throughput when every rank processes `units_per_rank_step` per step and the
+    slowest rank needs `ms_per_step` (replicas: work per GPU is fixed as N grows)."""
+    return world * units_per_rank_step / (ms_per_step * 1e-3)
+
+
 def make_inputs(wl, M):
     xs, ws = [], []
     for i, s in enumerate(wl.shapes):
@@ -387,13 +402,10 @@ def main():
     barrier()
     e2e_ms = e0.elapsed_time(e1) / e2e_steps
 
-    times = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms = float(times[0]), float(times[1])
+    ms_total, e2e_ms = max_over_ranks([ms_total, e2e_ms], dist, "cuda")
     ms_per_step = ms_total / args.steps
-    value = world * ops_per_step / (ms_per_step * 1e-3) / 1e12
-    e2e_value = world * ops_per_step / (e2e_ms * 1e-3) / 1e12
+    value = aggregate_value(world, ops_per_step, ms_per_step) / 1e12
+    e2e_value = aggregate_value(world, ops_per_step, e2e_ms) / 1e12
 
     int8_peak = 2.0 * peaks["bf16_tflops_sustained"]     # dense int8 = 2x dense bf16 (nominal ratio)
     achieved = gemm_ops / (gemm_ms * 1e-3) / 1e12
