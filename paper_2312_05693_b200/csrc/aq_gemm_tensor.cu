@@ -37,9 +37,9 @@ constexpr int kFirstEpiWarp = kFirstUnpackWarp + 4 * kUnpackGroups;
 constexpr int kRegsControl = 40, kRegsUnpack = 48, kRegsEpilogue = 168;
 constexpr int kEpiWarps = 8;                  // two warps per TMEM lane quarter, half of the token columns each
 constexpr int kThreads = (kFirstEpiWarp + kEpiWarps) * 32;
-// Grouped mode keeps every accumulator biased by this integer: the bit pattern of the float
-// 1.5 * 2^23. An int32 sum v with |v| < 2^22 then reads back from tensor memory as the float
-// 12582912 + v, so the epilogue needs no int->float conversion (one FADD removes the bias).
+// The bit pattern of the float 1.5 * 2^23: an integer add of it turns an int32 sum v, |v| < 2^22,
+// into the bits of the float 12582912 + v, so the per-group epilogue needs no int->float
+// conversion instruction (those saturated their pipe); one FADD removes the bias.
 constexpr uint32_t kMagicBits = 0x4B400000u;
 constexpr float kMagicFloat = 12582912.0f;
 constexpr int kAColsPerStage = 32;            // 128 k of int8 = 32 TMEM columns per lane
@@ -59,29 +59,8 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t by
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
                  : "memory");
 }
-#ifndef AQ_SPIN_SLEEP_NS
-#define AQ_SPIN_SLEEP_NS 0
-#endif
-#ifndef AQ_EPI_PACKED
-#define AQ_EPI_PACKED 0
-#endif
-#ifndef AQ_WAIT_HINT_NS
-#define AQ_WAIT_HINT_NS 0
-#endif
-#ifndef AQ_WAIT_LANE0
-#define AQ_WAIT_LANE0 0
-#endif
 __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
     uint32_t ok;
-#if AQ_WAIT_HINT_NS > 0
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity), "r"(AQ_WAIT_HINT_NS)
-        : "memory");
-#else
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
@@ -89,22 +68,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "=r"(ok)
         : "r"(smem_u32(bar)), "r"(parity)
         : "memory");
-#endif
     return ok != 0;
 }
 // Bounded wait. Returns false when the limit ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+// `code` (non-zero) names the wait; the first wait that gives up leaves its code in the flag.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          uint32_t code) {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
-#if AQ_SPIN_SLEEP_NS > 0
-        __nanosleep(AQ_SPIN_SLEEP_NS);
-#endif
         if ((++spins & 0x3FFu) == 0) {
             if (*abort_flag) return false;
             if ((unsigned long long)(clock64() - t0) > kWaitCycles) {
-                *abort_flag = 1;
+                if (*abort_flag == 0) *abort_flag = code;
                 return false;
             }
         }
@@ -112,14 +89,9 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     return true;
 }
 // The same for a whole warp: all lanes agree on the outcome before any warp-wide instruction.
-__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
-#if AQ_WAIT_LANE0
-    uint32_t ok = 0;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag) ? 1u : 0u;
-    return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
-#else
-    return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag) ? 1 : 0) != 0;
-#endif
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                               uint32_t code) {
+    return __all_sync(0xFFFFFFFFu, mbar_wait(bar, parity, abort_flag, code) ? 1 : 0) != 0;
 }
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
     asm volatile(
@@ -177,35 +149,6 @@ __device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t (&v)[8]) {
         "tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
         ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
         : "memory");
-}
-__device__ __forceinline__ void tc_st32_fill(uint32_t taddr, uint32_t c) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-        "{%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, "
-        "%1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1, %1};"
-        ::"r"(taddr), "r"(c) : "memory");
-}
-// Packed pairs of fp32 (one instruction, two lanes of data).
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(__float_as_uint(lo)), "r"(__float_as_uint(hi)));
-    return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
-    uint32_t a, b;
-    asm("mov.b64 {%0, %1}, %2;" : "=r"(a), "=r"(b) : "l"(v));
-    lo = __uint_as_float(a);
-    hi = __uint_as_float(b);
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-    uint64_t r;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-    return r;
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-    uint64_t r;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-    return r;
 }
 __device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
@@ -338,7 +281,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
                 for (int kb = 0; kb < KB; ++kb, ++it) {
                     const int s = (int)(it % kNumStages);
                     const uint32_t ph = (it / kNumStages) & 1u;
-                    if (!mbar_wait(&sm.smem_empty[s], ph ^ 1u, abort_flag)) goto role_done;
+                    if (!mbar_wait(&sm.smem_empty[s], ph ^ 1u, abort_flag, 1u)) goto role_done;
                     if (warp == 0) {
                         mbar_arrive_expect_tx(&sm.tma_full[s], BM * 128);
                         tma_load_2d(sm.x[s], &x_map, kb * kTileK, mt * BM, &sm.tma_full[s]);
@@ -359,20 +302,20 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
             constexpr uint32_t idesc = idesc_i8(128, BM);
             const uint32_t total_iters = (uint32_t)my_tiles * (uint32_t)KB;
             if (GROUPED) {
-                // every k block is one accumulation into its own (pre-biased) accumulator stage
+                // every k block is one accumulation into its own accumulator stage
                 for (uint32_t it = mma_id; it < total_iters; it += kNumMmaThreads) {
                     const int a = (int)(it % kNumAcc);
                     const int s = (int)(it % kNumStages);
                     const int ai = (int)(it % kNumASlices);
-                    if (!mbar_wait(&sm.acc_empty[a], (it / kNumAcc) & 1u, abort_flag)) goto role_done;
-                    if (!mbar_wait(&sm.a_full[ai], (it / kNumASlices) & 1u, abort_flag)) goto role_done;
+                    if (!mbar_wait(&sm.acc_empty[a], ((it / kNumAcc) & 1u) ^ 1u, abort_flag, 2u)) goto role_done;
+                    if (!mbar_wait(&sm.a_full[ai], (it / kNumASlices) & 1u, abort_flag, 3u)) goto role_done;
                     tc_fence_after();
                     const uint32_t d_addr = tmem_acc + (uint32_t)(a * BM);
                     const uint32_t a_addr = tmem_a + (uint32_t)(ai * kAColsPerStage);
                     const uint64_t bdesc = smem_desc_sw128(smem_u32(sm.x[s]));
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
-                        tc_mma_i8_ts(d_addr, a_addr + 8 * j, bdesc + (uint64_t)(2 * j), idesc, 1u);
+                        tc_mma_i8_ts(d_addr, a_addr + 8 * j, bdesc + (uint64_t)(2 * j), idesc, j > 0 ? 1u : 0u);
                     tc_commit(&sm.a_empty[ai]);
                     tc_commit(&sm.smem_empty[s]);
                     tc_commit(&sm.acc_full[a]);
@@ -382,13 +325,13 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
                 for (int tl = 0; tl < my_tiles; ++tl) {
                     const int a = (int)((uint32_t)tl % kNumAcc);
                     const uint32_t aph = ((uint32_t)tl / kNumAcc) & 1u;
-                    if (!mbar_wait(&sm.acc_empty[a], aph ^ 1u, abort_flag)) goto role_done;
+                    if (!mbar_wait(&sm.acc_empty[a], aph ^ 1u, abort_flag, 4u)) goto role_done;
                     for (int kb = 0; kb < KB; ++kb, ++it) {
                         const int s = (int)(it % kNumStages);
                         const int ai = (int)(it % kNumASlices);
                         // the unpack warps publish a slice only after the stage's TMA bytes (activation
                         // tile included) have landed, so this one wait covers both operands
-                        if (!mbar_wait(&sm.a_full[ai], (it / kNumASlices) & 1u, abort_flag)) goto role_done;
+                        if (!mbar_wait(&sm.a_full[ai], (it / kNumASlices) & 1u, abort_flag, 5u)) goto role_done;
                         tc_fence_after();
                         const uint32_t d_addr = tmem_acc + (uint32_t)(a * BM);
                         const uint32_t a_addr = tmem_a + (uint32_t)(ai * kAColsPerStage);
@@ -419,7 +362,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
         for (uint32_t it = group; it < total_iters; it += kUnpackGroups) {
             const int s = (int)(it % kNumStages);
             const int ai = (int)(it % kNumASlices);
-            if (!mbar_wait_warp(&sm.tma_full[s], (it / kNumStages) & 1u, abort_flag)) goto role_done;
+            if (!mbar_wait_warp(&sm.tma_full[s], (it / kNumStages) & 1u, abort_flag, 6u)) goto role_done;
             const uint4* src = reinterpret_cast<const uint4*>(sm.w[s]) + r;
             uint4 d[4];
 #pragma unroll
@@ -430,7 +373,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sm.a_full[pending]);
             }
-            if (!mbar_wait_warp(&sm.a_empty[ai], ((it / kNumASlices) & 1u) ^ 1u, abort_flag)) goto role_done;
+            if (!mbar_wait_warp(&sm.a_empty[ai], ((it / kNumASlices) & 1u) ^ 1u, abort_flag, 7u)) goto role_done;
             tc_fence_after();
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
@@ -462,18 +405,6 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
         const float pe = __int_as_float((127 + *p.scale_exp) << 23);     // 2^e
         [[maybe_unused]] const int G = GROUPED ? KB : 1;
         uint32_t unit = 0, it = 0;
-        if (GROUPED) {
-            // arm every accumulator stage with the bias; this is the first release of each stage
-            for (int a = 0; a < kNumAcc; ++a) {
-#pragma unroll
-                for (int c0 = 0; c0 < kColsPerEpiWarp; c0 += 32)
-                    tc_st32_fill(tmem_acc + lane_addr + (uint32_t)(a * BM + col0 + c0), kMagicBits);
-                tc_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.acc_empty[a]);
-            }
-        }
         for (int tl = 0; tl < my_tiles; ++tl) {
             const int tile = blockIdx.x + tl * gridDim.x;
             const int mt = tile % p.n_tiles_m, nt = tile / p.n_tiles_m;
@@ -484,7 +415,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
                 const int a = (int)(unit % kNumAcc);
                 const uint32_t aph = (unit / kNumAcc) & 1u;
                 const float sc = __half2float(p.w_scales[n]) * 0.0625f * pe;   // sums carry a factor 16
-                if (!mbar_wait_warp(&sm.acc_full[a], aph, abort_flag)) goto role_done;
+                if (!mbar_wait_warp(&sm.acc_full[a], aph, abort_flag, 8u)) goto role_done;
                 tc_fence_after();
 #pragma unroll 1
                 for (int c0 = 0; c0 < kColsPerEpiWarp; c0 += 16) {
@@ -506,76 +437,45 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
                 if (lane == 0) mbar_arrive(&sm.acc_empty[a]);
                 ++unit;
             } else {
-#if AQ_EPI_PACKED
-                uint64_t fsum2[kColsPerEpiWarp / 2];                     // pairs of fp32 partial outputs
-#pragma unroll
-                for (int c = 0; c < kColsPerEpiWarp / 2; ++c) fsum2[c] = 0ull;
-                const uint64_t neg_magic2 = pack2(-kMagicFloat, -kMagicFloat);
-#else
                 float fsum[kColsPerEpiWarp];                             // fp32 partial outputs
 #pragma unroll
                 for (int c = 0; c < kColsPerEpiWarp; ++c) fsum[c] = 0.0f;
-#endif
                 for (int kb = 0; kb < KB; ++kb, ++unit, ++it) {
                     const int a = (int)(unit % kNumAcc);
                     const uint32_t aph = (unit / kNumAcc) & 1u;
-                    if (!mbar_wait_warp(&sm.acc_full[a], aph, abort_flag)) goto role_done;
+                    if (!mbar_wait_warp(&sm.acc_full[a], aph, abort_flag, 9u)) goto role_done;
                     tc_fence_after();
                     // This block's MMAs are complete, so its stage (scales included) had landed: the
                     // issuer saw the unpack warps' signal, which they gave after seeing the TMA barrier.
                     const float sg = __half2float(sm.sc[it % Smem::kNumScaleSlots][r]) * 0.0625f;
-#if AQ_EPI_PACKED
-                    const uint64_t sg2 = pack2(sg, sg);
-#endif
                     static_assert(kColsPerEpiWarp == 32 || kColsPerEpiWarp == 64, "epilogue register plan");
                     const uint32_t taddr = tmem_acc + lane_addr + (uint32_t)(a * BM + col0);
                     uint32_t v[kColsPerEpiWarp];
                     tc_ld32(taddr, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
                     if (kColsPerEpiWarp == 64) tc_ld32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32 % kColsPerEpiWarp]));
                     tc_wait_ld();
-                    tc_st32_fill(taddr, kMagicBits);                     // re-arm the bias for the next use
-                    if (kColsPerEpiWarp == 64) tc_st32_fill(taddr + 32, kMagicBits);
-#if AQ_EPI_PACKED
-#pragma unroll
-                    for (int c = 0; c < kColsPerEpiWarp; c += 2) {
-                        // v holds the bits of the floats (magic + 16*sum): remove the bias, scale, add
-                        uint64_t t;
-                        asm("mov.b64 %0, {%1, %2};" : "=l"(t) : "r"(v[c]), "r"(v[c + 1]));
-                        t = add2(t, neg_magic2);
-                        fsum2[c / 2] = fma2(t, sg2, fsum2[c / 2]);
-                    }
-#else
+                    // the sums are in registers: the accumulator stage goes back to the MMA at once
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&sm.acc_empty[a]);
 #pragma unroll
                     for (int c = 0; c < kColsPerEpiWarp; ++c) {
-                        // v holds the bits of the float (magic + 16*sum): remove the bias, scale, add
-                        fsum[c] = fmaf(__uint_as_float(v[c]) - kMagicFloat, sg, fsum[c]);
+                        // int -> float without the conversion unit: adding the bits of 1.5 * 2^23 to an
+                        // integer |v| < 2^22 gives the bits of the float 12582912 + v
+                        fsum[c] = fmaf(__uint_as_float(v[c] + kMagicBits) - kMagicFloat, sg, fsum[c]);
                     }
-#endif
                     if (p.acc_dump) {
 #pragma unroll
                         for (int c = 0; c < kColsPerEpiWarp; ++c) {
                             const int m = m_base + c;
-                            if (n_ok && m < p.M)
-                                p.acc_dump[((size_t)m * p.N + n) * G + kb] = (int)(v[c] - kMagicBits) >> 4;
+                            if (n_ok && m < p.M) p.acc_dump[((size_t)m * p.N + n) * G + kb] = (int)v[c] >> 4;
                         }
                     }
-                    tc_wait_st();
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&sm.acc_empty[a]);
                 }
 #pragma unroll
-                for (int c = 0; c < kColsPerEpiWarp; c += 2) {
-                    float lo, hi;
-#if AQ_EPI_PACKED
-                    unpack2(fsum2[c / 2], lo, hi);
-#else
-                    lo = fsum[c];
-                    hi = fsum[c + 1];
-#endif
+                for (int c = 0; c < kColsPerEpiWarp; ++c) {
                     const int m = m_base + c;
-                    if (n_ok && m < p.M) p.y[(size_t)m * p.N + n] = __float2half_rn(lo * pe);
-                    if (n_ok && m + 1 < p.M) p.y[(size_t)(m + 1) * p.N + n] = __float2half_rn(hi * pe);
+                    if (n_ok && m < p.M) p.y[(size_t)m * p.N + n] = __float2half_rn(fsum[c] * pe);
                 }
             }
         }
@@ -589,7 +489,7 @@ role_done:
     if (sm.abort_flag) {
         // Give copies that may still be in flight time to land before shared memory is released.
         for (int i = 0; i < 64; ++i) __nanosleep(1000);
-        if (threadIdx.x == 0) atomicOr(&p.ctl->status, 1u);
+        if (threadIdx.x == 0) atomicCAS(&p.ctl->status, 0u, sm.abort_flag);   // the first CTA to give up names its wait
     }
     __syncthreads();
     if (warp == 1) {

@@ -182,6 +182,19 @@ def test_linear_with_row_idx_equals_compacted_input(kernel):
     assert_y_close(gpu["y"], ref["y"])
 
 
+@pytest.mark.parametrize("group", [0, 128])
+def test_several_tiles_per_cta_and_deep_k(group):
+    """More tiles than SMs and more k blocks than any ring is deep: every ring and every
+    accumulator stage wraps many times inside one persistent CTA."""
+    M, K, N = 1100, 2048, 4992          # 39 channel tiles x 9 (or 5) token tiles, 16 k blocks
+    x = inputs.activations(M, K, seed=123, outlier_frac=0.005, outlier_mult=30.0)
+    w = inputs.weights(N, K, seed=124)
+    gpu, ref = run_layer_both(x, w, 8, group, TENSOR)
+    assert gpu["e"] == ref["e"] and np.array_equal(gpu["q"], ref["q"])
+    assert np.array_equal(gpu["acc"], ref["acc"])
+    assert_y_close(gpu["y"], ref["y"])
+
+
 def test_results_are_deterministic_run_to_run():
     M, K, N = 260, 1152, 520
     x = inputs.activations(M, K, seed=9, outlier_frac=0.01, outlier_mult=20.0)
