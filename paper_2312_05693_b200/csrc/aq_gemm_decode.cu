@@ -192,7 +192,7 @@ struct StreamSmem {
     static constexpr int kRows = StreamCfg<MB>::kRows;
     alignas(1024) int8_t x[kStrStages][kRows * kTileK];    // activation codes of the unit's k block
     alignas(128) uint8_t w[kStrStages][kBlockBytes];       // packed weight block of the unit
-    int part[4][kRows][32];                                // second k-half's partial sums
+    int part[4][kRows][32];                                // the odd-k-block warp's partial sums
     int sum[kRows][kTileN];                                // leader CTA: the tile's sums over all of K
     alignas(8) uint64_t full[kStrStages];
     uint64_t empty[kStrStages];
@@ -230,7 +230,7 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStrStages; ++s) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(s_u32(&sm.full[s])) : "memory");
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s_u32(&sm.empty[s])), "r"(kStrConsumerWarps) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s_u32(&sm.empty[s])), "r"(kStrConsumerWarps / 2) : "memory");
         }
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -275,13 +275,12 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
             int acc[MB];
 #pragma unroll
             for (int m = 0; m < MB; ++m) acc[m] = 0;
-            for (int kb = kb0; kb < kb1; ++kb) {
+            for (int kb = kb0 + half; kb < kb1; kb += 2) {       // the two warps of a quarter take alternate k blocks
                 const uint32_t i = (uint32_t)(kb - kb0);
                 const int s = (int)(i % kStrStages);
                 if (!__all_sync(0xFFFFFFFFu, str_wait(&sm.full[s], (i / kStrStages) & 1u, abort_flag) ? 1 : 0)) break;
 #pragma unroll
-                for (int jj = 0; jj < 2; ++jj) {
-                    const int j = 2 * half + jj;
+                for (int j = 0; j < 4; ++j) {
                     const uint4 d = reinterpret_cast<const uint4*>(sm.w[s])[j * kTileN + r];
                     const uint32_t w[4] = {d.x, d.y, d.z, d.w};
                     uint32_t w8[8];
@@ -331,13 +330,12 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
             for (int i = 0; i < 4; ++i)
 #pragma unroll
                 for (int c = 0; c < 4; ++c) acc[i][c] = 0;
-            for (int kb = kb0; kb < kb1; ++kb) {
+            for (int kb = kb0 + half; kb < kb1; kb += 2) {       // the two warps of a quarter take alternate k blocks
                 const uint32_t it = (uint32_t)(kb - kb0);
                 const int s = (int)(it % kStrStages);
                 if (!__all_sync(0xFFFFFFFFu, str_wait(&sm.full[s], (it / kStrStages) & 1u, abort_flag) ? 1 : 0)) break;
 #pragma unroll
-                for (int jj = 0; jj < 2; ++jj) {
-                    const int j = 2 * half + jj;
+                for (int j = 0; j < 4; ++j) {
                     // activation fragment: row-major 128-byte rows, 16-byte chunks XOR-swizzled by row % 8
                     const int8_t* xr0 = sm.x[s] + g * kTileK;
                     const int8_t* xr1 = sm.x[s] + (g + 8) * kTileK;
@@ -439,8 +437,8 @@ cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t
     p.w_packed = a.w_packed; p.w_scales = a.w_scales; p.scale_exp = a.scale_exp;
     p.y = a.y; p.acc_dump = a.acc_dump; p.ctl = a.ctl;
     const int tiles = p.Npad / kTileN, KB = a.K / kTileK;
-    // as many k ranges per tile as keep all CTAs resident at once (two per SM), a power of two
-    // up to 4 so that clusters place easily, and at least two k blocks per CTA
+    // as many k ranges per tile (cluster size 1, 2 or 4: clusters of 7-8 measured slower) as keep
+    // all CTAs resident at once (two per SM), and at least two k blocks per CTA
     int split = 1;
     while (split < 4 && tiles * split * 2 <= 2 * dev.sm_count && KB / (split * 2) >= 2) split *= 2;
     cudaLaunchConfig_t cfg = {};

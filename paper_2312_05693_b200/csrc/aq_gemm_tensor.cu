@@ -404,7 +404,8 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
         const int col0 = half * kColsPerEpiWarp;
         const float pe = __int_as_float((127 + *p.scale_exp) << 23);     // 2^e
         [[maybe_unused]] const int G = GROUPED ? KB : 1;
-        uint32_t unit = 0, it = 0;
+        uint32_t unit = 0;
+        [[maybe_unused]] uint32_t g_a = 0, g_ph = 0, g_slot = 0;   // per-group mode: accumulator stage, its parity, scale slot
         for (int tl = 0; tl < my_tiles; ++tl) {
             const int tile = blockIdx.x + tl * gridDim.x;
             const int mt = tile % p.n_tiles_m, nt = tile / p.n_tiles_m;
@@ -440,14 +441,16 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
                 float fsum[kColsPerEpiWarp];                             // fp32 partial outputs
 #pragma unroll
                 for (int c = 0; c < kColsPerEpiWarp; ++c) fsum[c] = 0.0f;
-                for (int kb = 0; kb < KB; ++kb, ++unit, ++it) {
-                    const int a = (int)(unit % kNumAcc);
-                    const uint32_t aph = (unit / kNumAcc) & 1u;
-                    if (!mbar_wait_warp(&sm.acc_full[a], aph, abort_flag, 9u)) goto role_done;
+                for (int kb = 0; kb < KB; ++kb) {
+                    // ring positions are carried in counters (g_a, g_ph, g_slot): no division per block
+                    const int a = (int)g_a;
+                    if (!mbar_wait_warp(&sm.acc_full[a], g_ph, abort_flag, 9u)) goto role_done;
                     tc_fence_after();
                     // This block's MMAs are complete, so its stage (scales included) had landed: the
                     // issuer saw the unpack warps' signal, which they gave after seeing the TMA barrier.
-                    const float sg = __half2float(sm.sc[it % Smem::kNumScaleSlots][r]) * 0.0625f;
+                    const float sg = __half2float(sm.sc[g_slot][r]) * 0.0625f;
+                    if (++g_a == (uint32_t)kNumAcc) { g_a = 0; g_ph ^= 1u; }
+                    if (++g_slot == (uint32_t)Smem::kNumScaleSlots) g_slot = 0;
                     static_assert(kColsPerEpiWarp == 32 || kColsPerEpiWarp == 64, "epilogue register plan");
                     const uint32_t taddr = tmem_acc + lane_addr + (uint32_t)(a * BM + col0);
                     uint32_t v[kColsPerEpiWarp];
