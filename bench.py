@@ -242,9 +242,13 @@ def bench_decode(h, peaks, iters=40):
                 for i in range(copies):                      # a different weight copy per launch: HBM, not L2
                     h.aq_gemm_w4(q, packs[i][0], packs[i][1], s.N, 0, e, y=y, workspace=ws)
             ms = graph_replay_ms(launch, max(2, iters // copies)) / copies
+            def launch_layer():                              # the whole layer call: quantize kernel + product kernel
+                for i in range(copies):
+                    h.aq_linear_w4a8(x, packs[i][0], packs[i][1], s.N, 0, y=y, workspace=ws)
+            layer_ms = graph_replay_ms(launch_layer, max(2, iters // copies)) / copies
             algo = wbytes + 2 * s.N + M * s.K + 2 * M * s.N
             gbs = algo / (ms * 1e-3) / 1e9
-            out.append({"K": s.K, "N": s.N, "M": M, "us": ms * 1e3, "GBps": gbs,
+            out.append({"K": s.K, "N": s.N, "M": M, "us": ms * 1e3, "layer_us": layer_ms * 1e3, "GBps": gbs,
                         "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]})
         del packs
     return out

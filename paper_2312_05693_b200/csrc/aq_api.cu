@@ -51,9 +51,13 @@ Workspace carve(void* ws, int M, int K) {
     return w;
 }
 
+int kernel_for(aq_handle_t h, int M) {
+    const int choice = h->kernel_choice;
+    return choice == AQ_KERNEL_AUTO ? (M <= 16 ? AQ_KERNEL_DECODE : AQ_KERNEL_TENSOR) : choice;
+}
+
 int run_gemm(aq_handle_t h, const GemmArgs& g, cudaStream_t stream) {
-    int choice = h->kernel_choice;
-    if (choice == AQ_KERNEL_AUTO) choice = g.M <= 16 ? AQ_KERNEL_DECODE : AQ_KERNEL_TENSOR;
+    const int choice = kernel_for(h, g.M);
     const cudaError_t e = choice == AQ_KERNEL_DECODE ? launch_gemm_decode(g, h->dev, stream)
                                                      : launch_gemm_tensor(g, h->dev, stream);
     return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
@@ -75,16 +79,25 @@ int linear_impl(aq_handle_t h, int bits, const void* x, int M, int K, const void
         return AQ_ERR_ALIGNMENT;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const Workspace w = carve(workspace, M, K);
-    cudaError_t e = cudaMemsetAsync(w.ctl, 0, sizeof(Control), stream);
-    if (e != cudaSuccess) return cuda_fail(h, e);
     const __half* xh = static_cast<const __half*>(x);
-    if (scale_mode == AQ_SCALE_DYNAMIC) {
-        e = launch_absmax(xh, M, K, row_idx, w.ctl, h->dev, stream);
+    cudaError_t e;
+    if (quantize_small_fits(M, K)) {
+        // small activations (decode): one kernel finds the scale, writes the codes and initialises
+        // the control block
+        e = launch_quantize_small(xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, w.ctl, w.codes, nullptr,
+                                  stream);
+        if (e != cudaSuccess) return cuda_fail(h, e);
+    } else {
+        e = cudaMemsetAsync(w.ctl, 0, sizeof(Control), stream);
+        if (e != cudaSuccess) return cuda_fail(h, e);
+        if (scale_mode == AQ_SCALE_DYNAMIC) {
+            e = launch_absmax(xh, M, K, row_idx, w.ctl, h->dev, stream);
+            if (e != cudaSuccess) return cuda_fail(h, e);
+        }
+        e = launch_quantize(xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, w.ctl, w.codes, nullptr,
+                            h->dev, stream);
         if (e != cudaSuccess) return cuda_fail(h, e);
     }
-    e = launch_quantize(xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, w.ctl, w.codes, nullptr,
-                        h->dev, stream);
-    if (e != cudaSuccess) return cuda_fail(h, e);
     GemmArgs g;
     g.q = w.codes; g.M = M; g.K = K; g.N = N; g.group = group;
     g.w_packed = static_cast<const uint8_t*>(w_packed);
@@ -218,9 +231,14 @@ int aq_quantize_act(aq_handle_t h, const void* x_fp16, int M, int K, int bits, i
         return AQ_ERR_ALIGNMENT;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     Control* ctl = static_cast<Control*>(workspace);
+    const __half* xh = static_cast<const __half*>(x_fp16);
+    if (quantize_small_fits(M, K)) {
+        const cudaError_t es = launch_quantize_small(xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, ctl, q,
+                                                     scale_exp_out, stream);
+        return es == cudaSuccess ? AQ_OK : cuda_fail(h, es);
+    }
     cudaError_t e = cudaMemsetAsync(ctl, 0, sizeof(Control), stream);
     if (e != cudaSuccess) return cuda_fail(h, e);
-    const __half* xh = static_cast<const __half*>(x_fp16);
     if (scale_mode == AQ_SCALE_DYNAMIC) {
         e = launch_absmax(xh, M, K, row_idx, ctl, h->dev, stream);
         if (e != cudaSuccess) return cuda_fail(h, e);
@@ -258,8 +276,10 @@ int aq_gemm_w4(aq_handle_t h, const int8_t* q, int M, int K, const void* w_packe
         return AQ_ERR_ALIGNMENT;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const Workspace w = carve(workspace, M, K);
-    const cudaError_t e = cudaMemsetAsync(w.ctl, 0, sizeof(Control), stream);
-    if (e != cudaSuccess) return cuda_fail(h, e);
+    if (kernel_for(h, M) == AQ_KERNEL_TENSOR) {       // the decode kernels clear the status word themselves
+        const cudaError_t e = cudaMemsetAsync(w.ctl, 0, sizeof(Control), stream);
+        if (e != cudaSuccess) return cuda_fail(h, e);
+    }
     GemmArgs g;
     g.q = q; g.M = M; g.K = K; g.N = N; g.group = group_size;
     g.w_packed = static_cast<const uint8_t*>(w_packed);

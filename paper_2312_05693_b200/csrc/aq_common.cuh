@@ -86,6 +86,12 @@ cudaError_t launch_quantize(const __half* x, int M, int K, const int32_t* row_id
                             int scale_mode, int clip_shift_or_exp, Control* ctl, int8_t* q,
                             int32_t* scale_exp_out, const DeviceInfo& dev, cudaStream_t stream);
 
+// Activations of at most 262144 elements: one kernel that also initialises the control block.
+bool quantize_small_fits(int M, int K);
+cudaError_t launch_quantize_small(const __half* x, int M, int K, const int32_t* row_idx, int bits, int scale_mode,
+                                  int clip_shift_or_exp, Control* ctl, int8_t* q, int32_t* scale_exp_out,
+                                  cudaStream_t stream);
+
 cudaError_t launch_token_select(const float* scores, int M, int n_keep, int32_t* idx, void* scratch,
                                 cudaStream_t stream);
 cudaError_t launch_token_compact(const __half* x, int K, const int32_t* idx, int n_keep, __half* out,

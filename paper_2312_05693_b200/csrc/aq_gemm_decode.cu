@@ -9,7 +9,7 @@
 //  * a streaming one for one scale per channel and M <= 16: a thread-block cluster shares a
 //    128-channel tile and splits K; in each CTA a producer thread streams 8 KB packed blocks
 //    and their activation codes into a shared-memory ring with TMA, eight consumer warps
-//    multiply (dp4a up to 4 rows, the warp-level int8 MMA above), and the CTAs' partial sums
+//    multiply (dp4a for one row, the warp-level int8 MMA above), and the CTAs' partial sums
 //    are added into the leader CTA's shared memory over distributed shared memory (integer
 //    addition is exact in any order), which then writes the tile's outputs. No workspace, no
 //    global atomics.
@@ -35,8 +35,9 @@ __global__ void __launch_bounds__(kDecThreads)
 gemm_decode_kernel(const int8_t* __restrict__ q, int M, int K, int N, int Npad,
                    const uint8_t* __restrict__ w_packed, const __half* __restrict__ w_scales,
                    const int32_t* __restrict__ scale_exp, __half* __restrict__ y,
-                   int32_t* __restrict__ acc_dump) {
+                   int32_t* __restrict__ acc_dump, Control* __restrict__ ctl) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) ctl->status = 0;   // this kernel has no bounded waits
     const int KB = K / kTileK;
     const int n0 = blockIdx.x * 32;
     const int nt = n0 / kTileN, r = (n0 % kTileN) + lane;
@@ -179,7 +180,7 @@ __device__ __forceinline__ bool str_wait(uint64_t* bar, uint32_t parity, volatil
     return true;
 }
 
-// Rows up to 4 use dp4a with one lane per channel; more rows use the warp-level int8 MMA
+// One row uses dp4a with one lane per channel; more rows use the warp-level int8 MMA
 // (m16n8k32) on 16 rows, with the activation tile stored 128-byte swizzled so that fragment
 // loads are free of bank conflicts.
 template <int MB> struct StreamCfg {
@@ -235,6 +236,7 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) p.ctl->status = 0;   // nothing has given up yet
     for (int i = threadIdx.x; i < kRows * kTileN; i += kStrThreads) (&sm.sum[0][0])[i] = 0;
     __syncthreads();
     volatile uint32_t* abort_flag = &sm.abort_flag;
@@ -462,10 +464,10 @@ cudaError_t launch_mb(const GemmArgs& a, cudaStream_t stream) {
     dim3 grid(Npad / 32, (a.M + MB - 1) / MB);
     if (a.group)
         gemm_decode_kernel<MB, true><<<grid, kDecThreads, 0, stream>>>(
-            a.q, a.M, a.K, a.N, Npad, a.w_packed, a.w_scales, a.scale_exp, a.y, a.acc_dump);
+            a.q, a.M, a.K, a.N, Npad, a.w_packed, a.w_scales, a.scale_exp, a.y, a.acc_dump, a.ctl);
     else
         gemm_decode_kernel<MB, false><<<grid, kDecThreads, 0, stream>>>(
-            a.q, a.M, a.K, a.N, Npad, a.w_packed, a.w_scales, a.scale_exp, a.y, a.acc_dump);
+            a.q, a.M, a.K, a.N, Npad, a.w_packed, a.w_scales, a.scale_exp, a.y, a.acc_dump, a.ctl);
     return cudaGetLastError();
 }
 
@@ -473,10 +475,9 @@ cudaError_t launch_mb(const GemmArgs& a, cudaStream_t stream) {
 
 cudaError_t launch_gemm_decode(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
     if (!a.group && a.M <= 16) {
+        // one row: dp4a; 2..16 rows: the warp MMA on a 16-row tile (fewer instructions per weight
+        // chunk than dp4a from two rows on; measured faster at M = 4)
         if (a.M <= 1) return launch_stream<1>(a, dev, stream);
-        if (a.M <= 2) return launch_stream<2>(a, dev, stream);
-        if (a.M <= 4) return launch_stream<4>(a, dev, stream);
-        if (a.M <= 8) return launch_stream<8>(a, dev, stream);
         return launch_stream<16>(a, dev, stream);
     }
     if (a.M <= 1) return launch_mb<1>(a, stream);

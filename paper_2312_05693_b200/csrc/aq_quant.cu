@@ -1,7 +1,11 @@
 // Activation side: layer-wise absolute maximum, power-of-two quantization to int8 / int4
 // codes (paper Eq. 1, Eq. 2 / Eq. 5 with zp = 0, layer-wise scale of Sec. 4.4), and the
 // token selection / gather of Eq. 4.
+#include <cooperative_groups.h>
+
 #include "aq_common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace aq {
 
@@ -9,7 +13,7 @@ namespace {
 
 constexpr int kQuantThreads = 256;
 
-// ---- layer absmax: 16-byte loads, warp-shuffle reduction, one atomic per warp ----------
+// ---- layer absmax: 16-byte loads, warp-shuffle reduction, one atomic per CTA -----------
 __global__ void __launch_bounds__(kQuantThreads)
 absmax_kernel(const uint4* __restrict__ x, int M, int vec_per_row, const int32_t* __restrict__ row_idx,
               Control* __restrict__ ctl) {
@@ -29,7 +33,16 @@ absmax_kernel(const uint4* __restrict__ x, int M, int vec_per_row, const int32_t
     if (bits > 0x7C00u) bits = 0;                                       // never publish NaN
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) bits = max(bits, __shfl_xor_sync(0xFFFFFFFFu, bits, o));
-    if ((threadIdx.x & 31) == 0 && bits != 0) atomicMax(&ctl->absmax_bits, bits);
+    // warps meet in shared memory: one atomic per CTA on the single global word
+    __shared__ unsigned int warp_max[kQuantThreads / 32];
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = bits;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        unsigned int b = threadIdx.x < kQuantThreads / 32 ? warp_max[threadIdx.x] : 0u;
+#pragma unroll
+        for (int o = 4; o > 0; o >>= 1) b = max(b, __shfl_xor_sync(0xFFFFFFFFu, b, o));
+        if (threadIdx.x == 0 && b != 0) atomicMax(&ctl->absmax_bits, b);
+    }
 }
 
 __device__ inline int quantize_one(float v, float inv, float lo, float hi) {
@@ -73,6 +86,79 @@ quantize_kernel(const uint4* __restrict__ x, int M, int vec_per_row /* 16-elemen
         out[w] = word;
     }
     q[v] = make_uint4(out[0], out[1], out[2], out[3]);
+}
+
+// ---- small activations (decode): maximum, exponent and codes in ONE kernel -------------
+// One cluster of 8 CTAs x 512 threads holds the whole activation in registers (up to 8 vectors of
+// 8 halves per thread), so x is read once; the CTAs' maxima are exchanged through distributed
+// shared memory. The kernel also initialises the control block, so no memset precedes it.
+constexpr int kSmallCtas = 8, kSmallThreads = 512, kSmallVecs = 8;
+constexpr size_t kSmallMaxElems = (size_t)kSmallCtas * kSmallThreads * kSmallVecs * 8;   // 262144
+
+__global__ void __cluster_dims__(kSmallCtas, 1, 1) __launch_bounds__(kSmallThreads)
+quantize_small_kernel(const uint4* __restrict__ x, int M, int vec_per_row, const int32_t* __restrict__ row_idx,
+                      int bits, int scale_mode, int clip_shift_or_exp, Control* __restrict__ ctl,
+                      uint2* __restrict__ q, int32_t* __restrict__ scale_exp_out) {
+    cg::cluster_group cluster = cg::this_cluster();
+    __shared__ unsigned int warp_max[kSmallThreads / 32];
+    __shared__ unsigned int slots[kSmallCtas];
+    const int rank = (int)cluster.block_rank();
+    const int total = M * vec_per_row;
+    uint4 buf[kSmallVecs];
+    __half2 m2 = __float2half2_rn(0.0f);
+#pragma unroll
+    for (int i = 0; i < kSmallVecs; ++i) {
+        const int v = (i * kSmallCtas + rank) * kSmallThreads + (int)threadIdx.x;
+        buf[i] = make_uint4(0, 0, 0, 0);
+        if (v < total) {
+            const int m = v / vec_per_row, c = v % vec_per_row;
+            buf[i] = __ldg(x + (size_t)(row_idx ? row_idx[m] : m) * vec_per_row + c);
+            const __half2* h = reinterpret_cast<const __half2*>(&buf[i]);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) m2 = __hmax2(m2, __habs2(h[k]));   // NaN operands are dropped
+        }
+    }
+    unsigned int bits_max = max((unsigned int)__half_as_ushort(__low2half(m2)),
+                                (unsigned int)__half_as_ushort(__high2half(m2)));
+    if (bits_max > 0x7C00u) bits_max = 0;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) bits_max = max(bits_max, __shfl_xor_sync(0xFFFFFFFFu, bits_max, o));
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = bits_max;
+    __syncthreads();
+    if (threadIdx.x < kSmallCtas) {
+        unsigned int b = 0;
+        for (int w = 0; w < kSmallThreads / 32; ++w) b = max(b, warp_max[w]);
+        *cluster.map_shared_rank(&slots[rank], (int)threadIdx.x) = b;   // my maximum into every CTA's table
+    }
+    cluster.sync();
+    unsigned int all = 0;
+#pragma unroll
+    for (int r = 0; r < kSmallCtas; ++r) all = max(all, slots[r]);
+    const int e = scale_mode == AQ_SCALE_DYNAMIC ? layer_exponent_from_bits(all, bits) - clip_shift_or_exp
+                                                 : clip_shift_or_exp;
+    if (rank == 0 && threadIdx.x == 0) {
+        ctl->absmax_bits = all;
+        ctl->scale_exp = e;
+        ctl->status = 0;
+        ctl->counter = 0;
+        if (scale_exp_out) *scale_exp_out = e;
+    }
+    const float inv = __int_as_float((127 - e) << 23);      // 2^-e
+    const float lo = -(float)(1 << (bits - 1)), hi = (float)((1 << (bits - 1)) - 1);
+#pragma unroll
+    for (int i = 0; i < kSmallVecs; ++i) {
+        const int v = (i * kSmallCtas + rank) * kSmallThreads + (int)threadIdx.x;
+        if (v < total) {
+            const __half* h = reinterpret_cast<const __half*>(&buf[i]);
+            uint32_t w0 = 0, w1 = 0;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                w0 |= ((uint32_t)quantize_one(__half2float(h[b]), inv, lo, hi) & 0xFFu) << (8 * b);
+                w1 |= ((uint32_t)quantize_one(__half2float(h[4 + b]), inv, lo, hi) & 0xFFu) << (8 * b);
+            }
+            q[v] = make_uint2(w0, w1);
+        }
+    }
 }
 
 // ---- token selection: rank every score, keep rank < n_keep, then compact the flags ------
@@ -170,6 +256,17 @@ cudaError_t launch_quantize(const __half* x, int M, int K, const int32_t* row_id
     quantize_kernel<<<(unsigned int)blocks, kQuantThreads, 0, stream>>>(
         reinterpret_cast<const uint4*>(x), M, vec_per_row, row_idx, bits, scale_mode, clip_shift_or_exp,
         ctl, reinterpret_cast<uint4*>(q), scale_exp_out);
+    return cudaGetLastError();
+}
+
+bool quantize_small_fits(int M, int K) { return (size_t)M * (size_t)K <= kSmallMaxElems; }
+
+cudaError_t launch_quantize_small(const __half* x, int M, int K, const int32_t* row_idx, int bits, int scale_mode,
+                                  int clip_shift_or_exp, Control* ctl, int8_t* q, int32_t* scale_exp_out,
+                                  cudaStream_t stream) {
+    quantize_small_kernel<<<kSmallCtas, kSmallThreads, 0, stream>>>(
+        reinterpret_cast<const uint4*>(x), M, K / 8, row_idx, bits, scale_mode, clip_shift_or_exp, ctl,
+        reinterpret_cast<uint2*>(q), scale_exp_out);
     return cudaGetLastError();
 }
 
