@@ -37,6 +37,10 @@ constexpr int kFirstEpiWarp = kFirstUnpackWarp + 4 * kUnpackGroups;
 constexpr int kRegsControl = 40, kRegsUnpack = 48, kRegsEpilogue = 168;
 constexpr int kEpiWarps = 8;                  // two warps per TMEM lane quarter, half of the token columns each
 constexpr int kThreads = (kFirstEpiWarp + kEpiWarps) * 32;
+// setmaxnreg can only hand out what the launch allocated (96 registers for each of the threads): a
+// larger request would wait forever.
+static_assert(128 * kRegsControl + 32 * 4 * kUnpackGroups * kRegsUnpack + 32 * kEpiWarps * kRegsEpilogue <= kThreads * 96,
+              "register plan exceeds the launch allocation");
 // The bit pattern of the float 1.5 * 2^23: an integer add of it turns an int32 sum v, |v| < 2^22,
 // into the bits of the float 12582912 + v, so the per-group epilogue needs no int->float
 // conversion instruction (those saturated their pipe); one FADD removes the bias.
@@ -106,6 +110,16 @@ __device__ __forceinline__ void tma_load_1d(void* dst, const void* src, uint32_t
         ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
         : "memory");
 }
+// Shared -> global tile store through the TMA unit (bulk async-group completion). Elements of the
+// box that fall outside the tensor are not written.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, const void* src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                 ::"l"(map), "r"(x), "r"(y), "r"(smem_u32(src)) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// Wait until the TMA unit has read the source of every store this thread committed.
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint64_t* bar) {
@@ -189,6 +203,10 @@ struct SharedStorage {
     // i - kNumStages - 3 to have finished: all reads of the slot's previous content are done.
     static constexpr int kNumScaleSlots = kNumStages + 3;
     alignas(16) __half sc[kNumScaleSlots][kTileN];
+    // Per-group mode: each epilogue warp stages its 32 channels x BM/2 tokens of fp16 outputs here
+    // (token-major rows of 64 bytes) and hands them to a TMA store.
+    static constexpr int kStageRows = BM <= 128 ? BM / 2 : 1;
+    alignas(128) __half ystage[kEpiWarps][kStageRows][32];
     alignas(8) uint64_t tma_full[kNumStages];        // both producers' bytes landed -> unpack warps
     uint64_t smem_empty[kNumStages];                 // MMA done (+ epilogue took the scales) -> TMA producers
     uint64_t a_full[8];                              // unpack warps stored the slice -> MMA
@@ -208,11 +226,13 @@ struct TensorParams {
     __half* y;
     int32_t* acc_dump;
     Control* ctl;
+    int y_tma;                     // outputs leave through y_map (needs N % 8 == 0 and a 16-byte aligned y)
 };
 
 template <int BM, bool GROUPED>
 __global__ void __launch_bounds__(kThreads, 1)
-gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams p) {
+gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap y_map,
+                   const TensorParams p) {
     extern __shared__ uint8_t smem_raw[];
     using Smem = SharedStorage<BM>;
     Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -475,16 +495,32 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const TensorParams
                         }
                     }
                 }
+                if (p.y_tma) {
+                    if constexpr (BM <= 128) {
+                        // the previous tile's store must have read the staging rows before they change
+                        __half* stage = &sm.ystage[warp - kFirstEpiWarp][0][0];
+                        if (lane == 0) tma_store_wait_read();
+                        __syncwarp();
 #pragma unroll
-                for (int c = 0; c < kColsPerEpiWarp; ++c) {
-                    const int m = m_base + c;
-                    if (n_ok && m < p.M) p.y[(size_t)m * p.N + n] = __float2half_rn(fsum[c] * pe);
+                        for (int c = 0; c < kColsPerEpiWarp; ++c) stage[c * 32 + lane] = __float2half_rn(fsum[c] * pe);
+                        fence_proxy_async();
+                        __syncwarp();
+                        const int n0 = nt * kTileN + quarter * 32;
+                        if (lane == 0 && n0 < p.N && m_base < p.M) tma_store_2d(&y_map, stage, n0, m_base);
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < kColsPerEpiWarp; ++c) {
+                        const int m = m_base + c;
+                        if (n_ok && m < p.M) p.y[(size_t)m * p.N + n] = __float2half_rn(fsum[c] * pe);
+                    }
                 }
             }
         }
     }
 
 role_done:
+    if (GROUPED && warp >= kFirstEpiWarp && lane == 0) tma_store_wait_read();   // staging rows live until read
     __syncwarp();
     tc_fence_before();
     __syncthreads();
@@ -527,14 +563,29 @@ cudaError_t launch_bm(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t str
         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
 
+    CUtensorMap ymap = map;   // placeholder when the store path is off
+    int y_tma = 0;
+    if (GROUPED && BM <= 128 && a.N % 8 == 0 && (reinterpret_cast<uintptr_t>(a.y) & 15u) == 0) {
+        const cuuint64_t ydims[2] = {(cuuint64_t)a.N, (cuuint64_t)a.M};
+        const cuuint64_t ystrides[1] = {(cuuint64_t)a.N * 2};
+        const cuuint32_t ybox[2] = {32u, (cuuint32_t)(BM / 2)};
+        const CUresult ry = reinterpret_cast<EncodeTiledFn>(dev.encode_tiled)(
+            &ymap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, a.y, ydims, ystrides, ybox, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (ry != CUDA_SUCCESS) return cudaErrorInvalidValue;
+        y_tma = 1;
+    }
+
     TensorParams p;
+    p.y_tma = y_tma;
     p.M = a.M; p.K = a.K; p.N = a.N; p.Npad = round_up(a.N, kTileN);
     p.n_tiles_m = (a.M + BM - 1) / BM;
     p.n_tiles = p.n_tiles_m * (p.Npad / kTileN);
     p.w_packed = a.w_packed; p.w_scales = a.w_scales; p.scale_exp = a.scale_exp;
     p.y = a.y; p.acc_dump = a.acc_dump; p.ctl = a.ctl;
     const int grid = p.n_tiles < dev.sm_count ? p.n_tiles : dev.sm_count;
-    gemm_tensor_kernel<BM, GROUPED><<<grid, kThreads, smem_bytes, stream>>>(map, p);
+    gemm_tensor_kernel<BM, GROUPED><<<grid, kThreads, smem_bytes, stream>>>(map, ymap, p);
     return cudaGetLastError();
 }
 
