@@ -203,9 +203,9 @@ struct SharedStorage {
     // i - kNumStages - 3 to have finished: all reads of the slot's previous content are done.
     static constexpr int kNumScaleSlots = kNumStages + 3;
     alignas(16) __half sc[kNumScaleSlots][kTileN];
-    // Per-group mode: each epilogue warp stages its 32 channels x BM/2 tokens of fp16 outputs here
-    // (token-major rows of 64 bytes) and hands them to a TMA store.
-    static constexpr int kStageRows = BM <= 128 ? BM / 2 : 1;
+    // Each epilogue warp stages fp16 outputs of its 32 channels here, kStageRows tokens at a time
+    // (token-major rows of 64 bytes), and hands them to a TMA store.
+    static constexpr int kStageRows = BM <= 128 ? BM / 2 : 32;
     alignas(128) __half ystage[kEpiWarps][kStageRows][32];
     alignas(8) uint64_t tma_full[kNumStages];        // both producers' bytes landed -> unpack warps
     uint64_t smem_empty[kNumStages];                 // MMA done (+ epilogue took the scales) -> TMA producers
@@ -438,24 +438,44 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
                 const float sc = __half2float(p.w_scales[n]) * 0.0625f * pe;   // sums carry a factor 16
                 if (!mbar_wait_warp(&sm.acc_full[a], aph, abort_flag, 8u)) goto role_done;
                 tc_fence_after();
-#pragma unroll 1
-                for (int c0 = 0; c0 < kColsPerEpiWarp; c0 += 16) {
-                    uint32_t v[16];
-                    tc_ld16(tmem_acc + lane_addr + (uint32_t)(a * BM + col0 + c0), v);
-                    tc_wait_ld();
+                // all of this warp's sums go to registers and the accumulator returns to the MMA at once,
+                // so that the conversion and the stores below overlap the next tile's MMAs
+                uint32_t v[kColsPerEpiWarp];
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        const int m = m_base + c0 + c;
-                        if (n_ok && m < p.M) {
-                            const int acc16 = (int)v[c];
-                            p.y[(size_t)m * p.N + n] = __float2half_rn((float)acc16 * sc);
-                            if (p.acc_dump) p.acc_dump[(size_t)m * p.N + n] = acc16 >> 4;
-                        }
-                    }
-                }
+                for (int c0 = 0; c0 < kColsPerEpiWarp; c0 += 32)
+                    tc_ld32(tmem_acc + lane_addr + (uint32_t)(a * BM + col0 + c0), *reinterpret_cast<uint32_t(*)[32]>(&v[c0]));
+                tc_wait_ld();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&sm.acc_empty[a]);
+                if (p.y_tma) {
+                    __half* stage = &sm.ystage[warp - kFirstEpiWarp][0][0];
+                    const int n0 = nt * kTileN + quarter * 32;
+#pragma unroll
+                    for (int r0 = 0; r0 < kColsPerEpiWarp; r0 += Smem::kStageRows) {
+                        if (lane == 0) tma_store_wait_read();     // the previous store has read the staging rows
+                        __syncwarp();
+#pragma unroll
+                        for (int c = 0; c < Smem::kStageRows; ++c)
+                            stage[c * 32 + lane] = __float2half_rn((float)(int)v[r0 + c] * sc);
+                        fence_proxy_async();
+                        __syncwarp();
+                        if (lane == 0 && n0 < p.N && m_base + r0 < p.M) tma_store_2d(&y_map, stage, n0, m_base + r0);
+                    }
+                } else {
+#pragma unroll
+                    for (int c = 0; c < kColsPerEpiWarp; ++c) {
+                        const int m = m_base + c;
+                        if (n_ok && m < p.M) p.y[(size_t)m * p.N + n] = __float2half_rn((float)(int)v[c] * sc);
+                    }
+                }
+                if (p.acc_dump) {
+#pragma unroll
+                    for (int c = 0; c < kColsPerEpiWarp; ++c) {
+                        const int m = m_base + c;
+                        if (n_ok && m < p.M) p.acc_dump[(size_t)m * p.N + n] = (int)v[c] >> 4;
+                    }
+                }
                 ++unit;
             } else {
                 float fsum[kColsPerEpiWarp];                             // fp32 partial outputs
@@ -496,18 +516,17 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
                     }
                 }
                 if (p.y_tma) {
-                    if constexpr (BM <= 128) {
-                        // the previous tile's store must have read the staging rows before they change
-                        __half* stage = &sm.ystage[warp - kFirstEpiWarp][0][0];
-                        if (lane == 0) tma_store_wait_read();
-                        __syncwarp();
+                    static_assert(Smem::kStageRows == kColsPerEpiWarp, "per-group kernels stage a warp's whole tile");
+                    // the previous tile's store must have read the staging rows before they change
+                    __half* stage = &sm.ystage[warp - kFirstEpiWarp][0][0];
+                    if (lane == 0) tma_store_wait_read();
+                    __syncwarp();
 #pragma unroll
-                        for (int c = 0; c < kColsPerEpiWarp; ++c) stage[c * 32 + lane] = __float2half_rn(fsum[c] * pe);
-                        fence_proxy_async();
-                        __syncwarp();
-                        const int n0 = nt * kTileN + quarter * 32;
-                        if (lane == 0 && n0 < p.N && m_base < p.M) tma_store_2d(&y_map, stage, n0, m_base);
-                    }
+                    for (int c = 0; c < kColsPerEpiWarp; ++c) stage[c * 32 + lane] = __float2half_rn(fsum[c] * pe);
+                    fence_proxy_async();
+                    __syncwarp();
+                    const int n0 = nt * kTileN + quarter * 32;
+                    if (lane == 0 && n0 < p.N && m_base < p.M) tma_store_2d(&y_map, stage, n0, m_base);
                 } else {
 #pragma unroll
                     for (int c = 0; c < kColsPerEpiWarp; ++c) {
@@ -520,7 +539,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
     }
 
 role_done:
-    if (GROUPED && warp >= kFirstEpiWarp && lane == 0) tma_store_wait_read();   // staging rows live until read
+    if (warp >= kFirstEpiWarp && lane == 0) tma_store_wait_read();   // staging rows live until read
     __syncwarp();
     tc_fence_before();
     __syncthreads();
@@ -565,10 +584,10 @@ cudaError_t launch_bm(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t str
 
     CUtensorMap ymap = map;   // placeholder when the store path is off
     int y_tma = 0;
-    if (GROUPED && BM <= 128 && a.N % 8 == 0 && (reinterpret_cast<uintptr_t>(a.y) & 15u) == 0) {
+    if (a.N % 8 == 0 && (reinterpret_cast<uintptr_t>(a.y) & 15u) == 0) {
         const cuuint64_t ydims[2] = {(cuuint64_t)a.N, (cuuint64_t)a.M};
         const cuuint64_t ystrides[1] = {(cuuint64_t)a.N * 2};
-        const cuuint32_t ybox[2] = {32u, (cuuint32_t)(BM / 2)};
+        const cuuint32_t ybox[2] = {32u, (cuuint32_t)Smem::kStageRows};
         const CUresult ry = reinterpret_cast<EncodeTiledFn>(dev.encode_tiled)(
             &ymap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, a.y, ydims, ystrides, ybox, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
