@@ -91,11 +91,12 @@ int linear_impl(aq_handle_t h, int bits, const void* x, int M, int K, const void
         e = cudaMemsetAsync(w.ctl, 0, sizeof(Control), stream);
         if (e != cudaSuccess) return cuda_fail(h, e);
         if (scale_mode == AQ_SCALE_DYNAMIC) {
-            e = launch_absmax(xh, M, K, row_idx, w.ctl, h->dev, stream);
-            if (e != cudaSuccess) return cuda_fail(h, e);
+            e = launch_quantize_fused(xh, M, K, row_idx, bits, clip_shift_or_exp, w.ctl, w.codes, nullptr, h->dev,
+                                      stream);
+        } else {
+            e = launch_quantize(xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, w.ctl, w.codes, nullptr,
+                                h->dev, stream);
         }
-        e = launch_quantize(xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, w.ctl, w.codes, nullptr,
-                            h->dev, stream);
         if (e != cudaSuccess) return cuda_fail(h, e);
     }
     GemmArgs g;
@@ -240,11 +241,11 @@ int aq_quantize_act(aq_handle_t h, const void* x_fp16, int M, int K, int bits, i
     cudaError_t e = cudaMemsetAsync(ctl, 0, sizeof(Control), stream);
     if (e != cudaSuccess) return cuda_fail(h, e);
     if (scale_mode == AQ_SCALE_DYNAMIC) {
-        e = launch_absmax(xh, M, K, row_idx, ctl, h->dev, stream);
-        if (e != cudaSuccess) return cuda_fail(h, e);
+        e = launch_quantize_fused(xh, M, K, row_idx, bits, clip_shift_or_exp, ctl, q, scale_exp_out, h->dev, stream);
+    } else {
+        e = launch_quantize(xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, ctl, q, scale_exp_out, h->dev,
+                            stream);
     }
-    e = launch_quantize(xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, ctl, q, scale_exp_out, h->dev,
-                        stream);
     return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
 }
 

@@ -92,6 +92,12 @@ cudaError_t launch_quantize_small(const __half* x, int M, int K, const int32_t* 
                                   int clip_shift_or_exp, Control* ctl, int8_t* q, int32_t* scale_exp_out,
                                   cudaStream_t stream);
 
+// Dynamic scale, any size: one cooperative kernel (absmax, exponent, codes). The control block must
+// have been cleared (absmax_bits, counter) on the same stream before.
+cudaError_t launch_quantize_fused(const __half* x, int M, int K, const int32_t* row_idx, int bits, int clip_shift,
+                                  Control* ctl, int8_t* q, int32_t* scale_exp_out, const DeviceInfo& dev,
+                                  cudaStream_t stream);
+
 cudaError_t launch_token_select(const float* scores, int M, int n_keep, int32_t* idx, void* scratch,
                                 cudaStream_t stream);
 cudaError_t launch_token_compact(const __half* x, int K, const int32_t* idx, int n_keep, __half* out,

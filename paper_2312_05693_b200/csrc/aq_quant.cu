@@ -161,6 +161,115 @@ quantize_small_kernel(const uint4* __restrict__ x, int M, int vec_per_row, const
     }
 }
 
+// ---- larger activations, dynamic scale: maximum, exponent and codes in ONE cooperative kernel ----
+// One CTA per SM takes a contiguous share of X. First pass: 16-byte loads from HBM, running maximum,
+// and the loaded vectors are parked in shared memory (as much of the share as fits). The CTAs then
+// meet at a counter in the control block (all are resident: the launch is cooperative; the wait is
+// bounded all the same), every CTA derives the exponent from the global maximum, and the second
+// pass quantizes from shared memory (from L2 for what did not fit), so X crosses HBM once.
+constexpr int kFusedThreads = 1024;
+constexpr unsigned int kFusedWaitCode = 10;            // status value when the meeting point times out
+constexpr unsigned long long kFusedWaitCycles = 2000000000ull;   // ~1 s
+
+__device__ __forceinline__ unsigned int ld_acquire_u32(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+__global__ void __launch_bounds__(kFusedThreads, 1)
+quantize_fused_kernel(const uint4* __restrict__ x, int M, int units_per_row /* 16-element units */,
+                      const int32_t* __restrict__ row_idx, int bits, int clip_shift, Control* __restrict__ ctl,
+                      uint4* __restrict__ q, int32_t* __restrict__ scale_exp_out, unsigned int cache_units,
+                      unsigned int units_per_cta) {
+    extern __shared__ uint4 fused_cache[];             // [2][cache_units]: first and second vector of a unit
+    __shared__ unsigned int warp_max[kFusedThreads / 32];
+    __shared__ int e_shared;
+    __shared__ int gave_up;
+    const size_t total = (size_t)M * units_per_row;
+    const size_t u0 = (size_t)blockIdx.x * units_per_cta;
+    const size_t u1 = u0 + units_per_cta < total ? u0 + units_per_cta : total;
+
+    __half2 m2 = __float2half2_rn(0.0f);
+#pragma unroll 2
+    for (size_t u = u0 + threadIdx.x; u < u1; u += kFusedThreads) {
+        const int m = (int)(u / units_per_row), c = (int)(u % units_per_row);
+        const size_t src = ((size_t)(row_idx ? row_idx[m] : m) * units_per_row + c) * 2;
+        const uint4 d0 = __ldg(x + src), d1 = __ldg(x + src + 1);
+        const unsigned int local = (unsigned int)(u - u0);
+        if (local < cache_units) { fused_cache[local] = d0; fused_cache[cache_units + local] = d1; }
+        const __half2* h0 = reinterpret_cast<const __half2*>(&d0);
+        const __half2* h1 = reinterpret_cast<const __half2*>(&d1);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) m2 = __hmax2(m2, __hmax2(__habs2(h0[i]), __habs2(h1[i])));   // NaN operands are dropped
+    }
+    unsigned int bmax = max((unsigned int)__half_as_ushort(__low2half(m2)),
+                            (unsigned int)__half_as_ushort(__high2half(m2)));
+    if (bmax > 0x7C00u) bmax = 0;                                       // never publish NaN
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) bmax = max(bmax, __shfl_xor_sync(0xFFFFFFFFu, bmax, o));
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = bmax;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        unsigned int b = warp_max[threadIdx.x];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) b = max(b, __shfl_xor_sync(0xFFFFFFFFu, b, o));
+        if (threadIdx.x == 0) {
+            if (b != 0) atomicMax(&ctl->absmax_bits, b);
+            __threadfence();
+            atomicAdd(&ctl->counter, 1u);
+            // meeting point: every CTA has added its maximum once the counter reaches the grid size
+            const long long t0 = clock64();
+            int failed = 0;
+            while (ld_acquire_u32(&ctl->counter) < gridDim.x) {
+                if ((unsigned long long)(clock64() - t0) > kFusedWaitCycles) { failed = 1; break; }
+                __nanosleep(100);
+            }
+            gave_up = failed;
+            e_shared = layer_exponent_from_bits(ld_acquire_u32(&ctl->absmax_bits), bits) - clip_shift;
+        }
+    }
+    __syncthreads();
+    if (gave_up) {
+        if (threadIdx.x == 0) atomicCAS(&ctl->status, 0u, kFusedWaitCode);
+        return;
+    }
+    const int e = e_shared;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        ctl->scale_exp = e;
+        if (scale_exp_out) *scale_exp_out = e;
+    }
+    const float inv = __int_as_float((127 - e) << 23);      // 2^-e, |e| <= 40
+    const float lo = -(float)(1 << (bits - 1)), hi = (float)((1 << (bits - 1)) - 1);
+#pragma unroll 2
+    for (size_t u = u0 + threadIdx.x; u < u1; u += kFusedThreads) {
+        const unsigned int local = (unsigned int)(u - u0);
+        uint4 d0, d1;
+        if (local < cache_units) {
+            d0 = fused_cache[local]; d1 = fused_cache[cache_units + local];      // this thread's own stores
+        } else {
+            const int m = (int)(u / units_per_row), c = (int)(u % units_per_row);
+            const size_t src = ((size_t)(row_idx ? row_idx[m] : m) * units_per_row + c) * 2;
+            d0 = __ldg(x + src); d1 = __ldg(x + src + 1);
+        }
+        const __half* h0 = reinterpret_cast<const __half*>(&d0);
+        const __half* h1 = reinterpret_cast<const __half*>(&d1);
+        uint32_t out[4];
+#pragma unroll
+        for (int w = 0; w < 4; ++w) {
+            uint32_t word = 0;
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const int i = 4 * w + b;
+                const float f = __half2float(i < 8 ? h0[i] : h1[i - 8]);
+                word |= ((uint32_t)quantize_one(f, inv, lo, hi) & 0xFFu) << (8 * b);
+            }
+            out[w] = word;
+        }
+        q[u] = make_uint4(out[0], out[1], out[2], out[3]);
+    }
+}
+
 // ---- token selection: rank every score, keep rank < n_keep, then compact the flags ------
 // rank(i) = #{ j : s_j > s_i  or (s_j == s_i and j < i) }, so equal scores resolve toward
 // the lower index and exactly n_keep tokens have rank < n_keep.
@@ -257,6 +366,35 @@ cudaError_t launch_quantize(const __half* x, int M, int K, const int32_t* row_id
         reinterpret_cast<const uint4*>(x), M, vec_per_row, row_idx, bits, scale_mode, clip_shift_or_exp,
         ctl, reinterpret_cast<uint4*>(q), scale_exp_out);
     return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_fused(const __half* x, int M, int K, const int32_t* row_idx, int bits, int clip_shift,
+                                  Control* ctl, int8_t* q, int32_t* scale_exp_out, const DeviceInfo& dev,
+                                  cudaStream_t stream) {
+    int units_per_row = K / 16;
+    const size_t total = (size_t)M * units_per_row;
+    size_t grid = (total + kFusedThreads - 1) / kFusedThreads;
+    if (grid > (size_t)dev.sm_count) grid = (size_t)dev.sm_count;
+    unsigned int units_per_cta = (unsigned int)((total + grid - 1) / grid);
+    // shared-memory cache: the CTA's whole share when it fits, else as much as one CTA may hold
+    const size_t reserve = 8192;                       // static shared memory and alignment slack
+    const size_t max_cache = dev.smem_optin > reserve ? (dev.smem_optin - reserve) / 32 : 0;
+    unsigned int cache_units = units_per_cta < max_cache ? units_per_cta : (unsigned int)max_cache;
+    const size_t smem_bytes = (size_t)cache_units * 32;
+    static size_t attr_bytes = 0;
+    if (smem_bytes > attr_bytes) {
+        const cudaError_t e = cudaFuncSetAttribute(quantize_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)(dev.smem_optin - reserve));
+        if (e != cudaSuccess) return e;
+        attr_bytes = dev.smem_optin - reserve;
+    }
+    const uint4* xp = reinterpret_cast<const uint4*>(x);
+    uint4* qp = reinterpret_cast<uint4*>(q);
+    void* args[] = {&xp, &M, &units_per_row, &row_idx, &bits, &clip_shift, &ctl, &qp, &scale_exp_out, &cache_units,
+                    &units_per_cta};
+    // cooperative: the launch fails rather than start a grid whose CTAs could not all be resident
+    return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(quantize_fused_kernel), dim3((unsigned int)grid),
+                                       dim3(kFusedThreads), args, smem_bytes, stream);
 }
 
 bool quantize_small_fits(int M, int K) { return (size_t)M * (size_t)K <= kSmallMaxElems; }
