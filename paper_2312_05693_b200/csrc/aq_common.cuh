@@ -80,8 +80,6 @@ cudaError_t launch_pack_w4(const __half* w, int N, int K, int group, uint8_t* pa
                            cudaStream_t stream);
 cudaError_t launch_unpack_w4(const uint8_t* packed, int N, int K, int8_t* codes, cudaStream_t stream);
 
-cudaError_t launch_absmax(const __half* x, int M, int K, const int32_t* row_idx, Control* ctl,
-                          const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_quantize(const __half* x, int M, int K, const int32_t* row_idx, int bits,
                             int scale_mode, int clip_shift_or_exp, Control* ctl, int8_t* q,
                             int32_t* scale_exp_out, const DeviceInfo& dev, cudaStream_t stream);

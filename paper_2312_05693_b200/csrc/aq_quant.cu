@@ -13,42 +13,35 @@ namespace {
 
 constexpr int kQuantThreads = 256;
 
-// ---- layer absmax: 16-byte loads, warp-shuffle reduction, one atomic per CTA -----------
-__global__ void __launch_bounds__(kQuantThreads)
-absmax_kernel(const uint4* __restrict__ x, int M, int vec_per_row, const int32_t* __restrict__ row_idx,
-              Control* __restrict__ ctl) {
-    const size_t total = (size_t)M * vec_per_row;
-    __half2 m2 = __float2half2_rn(0.0f);
-    for (size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v < total;
-         v += (size_t)gridDim.x * blockDim.x) {
-        const int m = (int)(v / vec_per_row), c = (int)(v % vec_per_row);
-        const size_t src = (size_t)(row_idx ? row_idx[m] : m) * vec_per_row + c;
-        const uint4 d = __ldg(x + src);
-        const __half2* h = reinterpret_cast<const __half2*>(&d);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) m2 = __hmax2(m2, __habs2(h[i]));   // NaN operands are dropped
-    }
-    unsigned int bits = max((unsigned int)__half_as_ushort(__low2half(m2)),
-                            (unsigned int)__half_as_ushort(__high2half(m2)));
-    if (bits > 0x7C00u) bits = 0;                                       // never publish NaN
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) bits = max(bits, __shfl_xor_sync(0xFFFFFFFFu, bits, o));
-    // warps meet in shared memory: one atomic per CTA on the single global word
-    __shared__ unsigned int warp_max[kQuantThreads / 32];
-    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = bits;
-    __syncthreads();
-    if (threadIdx.x < 32) {
-        unsigned int b = threadIdx.x < kQuantThreads / 32 ? warp_max[threadIdx.x] : 0u;
-#pragma unroll
-        for (int o = 4; o > 0; o >>= 1) b = max(b, __shfl_xor_sync(0xFFFFFFFFu, b, o));
-        if (threadIdx.x == 0 && b != 0) atomicMax(&ctl->absmax_bits, b);
-    }
-}
-
 __device__ inline int quantize_one(float v, float inv, float lo, float hi) {
     const float t = v * inv;                 // exact: inv is a power of two
     if (t != t) return 0;                    // NaN
     return (int)fminf(fmaxf(rintf(t), lo), hi);
+}
+
+// Eight halves -> eight codes in two 32-bit words, in half2 arithmetic, for exponents whose 2^-e is a
+// normal half (|e| <= 14). Every step is exact or rounds exactly like the fp32 route: the product by
+// a power of two is exact unless it leaves the half range (overflow saturates to Inf and is clamped
+// like any large value; results below 2^-14 round to code 0 either way); NaN is cleared to 0 by a
+// lane mask; clamping to the integer bounds before rounding gives the same code as after; adding
+// 1536 (ulp 1 in [1024, 2048)) rounds to the nearest integer, ties to even, and leaves the code's
+// two's-complement byte in the low 8 bits of the half's bit pattern.
+__device__ __forceinline__ void quantize8_half2(const uint4& d, __half2 inv2, __half2 lo2, __half2 hi2, uint32_t& w0,
+                                                uint32_t& w1) {
+    const __half2* h = reinterpret_cast<const __half2*>(&d);
+    const __half2 bias = __floats2half2_rn(1536.0f, 1536.0f);
+    uint32_t r[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        __half2 t = __hmul2(h[i], inv2);
+        const uint32_t ok = __heq2_mask(t, t);                            // 0xFFFF per lane that is not NaN
+        uint32_t tb = *reinterpret_cast<uint32_t*>(&t) & ok;
+        t = *reinterpret_cast<__half2*>(&tb);
+        t = __hadd2(__hmin2(__hmax2(t, lo2), hi2), bias);
+        r[i] = *reinterpret_cast<uint32_t*>(&t);
+    }
+    w0 = __byte_perm(r[0], r[1], 0x6420);
+    w1 = __byte_perm(r[2], r[3], 0x6420);
 }
 
 // ---- quantize: 16 halves in (two 16-byte loads), 16 codes out (one 16-byte store) -----
@@ -241,6 +234,8 @@ quantize_fused_kernel(const uint4* __restrict__ x, int M, int units_per_row /* 1
     }
     const float inv = __int_as_float((127 - e) << 23);      // 2^-e, |e| <= 40
     const float lo = -(float)(1 << (bits - 1)), hi = (float)((1 << (bits - 1)) - 1);
+    const bool fast = e >= -14 && e <= 14;                   // 2^-e is a normal half
+    const __half2 inv2 = __float2half2_rn(fast ? inv : 1.0f), lo2 = __float2half2_rn(lo), hi2 = __float2half2_rn(hi);
 #pragma unroll 2
     for (size_t u = u0 + threadIdx.x; u < u1; u += kFusedThreads) {
         const unsigned int local = (unsigned int)(u - u0);
@@ -252,19 +247,24 @@ quantize_fused_kernel(const uint4* __restrict__ x, int M, int units_per_row /* 1
             const size_t src = ((size_t)(row_idx ? row_idx[m] : m) * units_per_row + c) * 2;
             d0 = __ldg(x + src); d1 = __ldg(x + src + 1);
         }
-        const __half* h0 = reinterpret_cast<const __half*>(&d0);
-        const __half* h1 = reinterpret_cast<const __half*>(&d1);
         uint32_t out[4];
+        if (fast) {
+            quantize8_half2(d0, inv2, lo2, hi2, out[0], out[1]);
+            quantize8_half2(d1, inv2, lo2, hi2, out[2], out[3]);
+        } else {
+            const __half* h0 = reinterpret_cast<const __half*>(&d0);
+            const __half* h1 = reinterpret_cast<const __half*>(&d1);
 #pragma unroll
-        for (int w = 0; w < 4; ++w) {
-            uint32_t word = 0;
+            for (int w = 0; w < 4; ++w) {
+                uint32_t word = 0;
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                const int i = 4 * w + b;
-                const float f = __half2float(i < 8 ? h0[i] : h1[i - 8]);
-                word |= ((uint32_t)quantize_one(f, inv, lo, hi) & 0xFFu) << (8 * b);
+                for (int b = 0; b < 4; ++b) {
+                    const int i = 4 * w + b;
+                    const float f = __half2float(i < 8 ? h0[i] : h1[i - 8]);
+                    word |= ((uint32_t)quantize_one(f, inv, lo, hi) & 0xFFu) << (8 * b);
+                }
+                out[w] = word;
             }
-            out[w] = word;
         }
         q[u] = make_uint4(out[0], out[1], out[2], out[3]);
     }
@@ -342,18 +342,6 @@ gather_rows_kernel(const uint4* __restrict__ x, int vec_per_row, const int32_t* 
 }
 
 }  // namespace
-
-cudaError_t launch_absmax(const __half* x, int M, int K, const int32_t* row_idx, Control* ctl,
-                          const DeviceInfo& dev, cudaStream_t stream) {
-    const int vec_per_row = K / 8;
-    const size_t total = (size_t)M * vec_per_row;
-    size_t blocks = (total + kQuantThreads - 1) / kQuantThreads;
-    const size_t cap = (size_t)dev.sm_count * 8;
-    if (blocks > cap) blocks = cap;
-    absmax_kernel<<<(unsigned int)blocks, kQuantThreads, 0, stream>>>(
-        reinterpret_cast<const uint4*>(x), M, vec_per_row, row_idx, ctl);
-    return cudaGetLastError();
-}
 
 cudaError_t launch_quantize(const __half* x, int M, int K, const int32_t* row_idx, int bits,
                             int scale_mode, int clip_shift_or_exp, Control* ctl, int8_t* q,
