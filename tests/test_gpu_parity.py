@@ -74,6 +74,43 @@ def test_quantize_act_static_rowidx_and_nonfinite():
     assert int(e.item()) == 0 and not q.any().item()
 
 
+@pytest.mark.parametrize("bits", [8, 4])
+def test_quantize_act_one_pass_kernel_edges(bits):
+    # sizes above the small-activation limit take the cooperative one-pass kernel: ragged split over
+    # the CTAs, exact ties, non-finite values, gathered (repeated, permuted) rows, and exponents on
+    # both sides of the half-precision fast path
+    M, K = 701, 1152
+    g = np.random.Generator(np.random.Philox(key=77 + bits))
+    h = handle()
+    # (a) multiples of 1/2 with max 127: e = 0 for 8 bits, every second value is an exact tie
+    x = (g.integers(-254, 255, size=(M, K)) * 0.5).astype(np.float16)
+    x[5, 7] = 127.0
+    for clip in (0, 2):
+        q, e = h.aq_quantize_act(dev(x), bits, binding.AQ_SCALE_DYNAMIC, clip)
+        e_ref = oracle.layer_exponent(x, bits) - clip
+        assert int(e.item()) == e_ref
+        assert np.array_equal(q.cpu().numpy(), oracle.quantize_act(x, bits, e_ref))
+    # (b) NaN / Inf inside, rows gathered with repeats and out of order
+    x2 = inputs.activations(M, K, seed=9, outlier_frac=0.01, outlier_mult=20.0)
+    x2[3, 5] = np.nan
+    x2[700, 1151] = np.nan
+    x2[17, 9] = np.inf
+    x2[18, 1] = -np.inf
+    rows = g.integers(0, M, size=650).astype(np.int32)
+    rows[:4] = [700, 3, 17, 18]
+    q, e = h.aq_quantize_act(dev(x2), bits, binding.AQ_SCALE_DYNAMIC, 0, row_idx=dev(rows))
+    e_ref = oracle.layer_exponent(x2, bits, rows)
+    assert int(e.item()) == e_ref == (10 if bits == 8 else 14)
+    assert np.array_equal(q.cpu().numpy(), oracle.quantize_act(x2, bits, e_ref, rows))
+    # (c) tiny and large magnitudes: exponents far below / near the top of what fp16 inputs can give
+    for scale in (2.0 ** -20, 2.0 ** -12, 300.0):
+        x3 = (inputs.activations(M, K, seed=11).astype(np.float32) * np.float32(scale)).astype(np.float16)
+        q, e = h.aq_quantize_act(dev(x3), bits)
+        e_ref = oracle.layer_exponent(x3, bits)
+        assert int(e.item()) == e_ref
+        assert np.array_equal(q.cpu().numpy(), oracle.quantize_act(x3, bits, e_ref))
+
+
 def test_quantize_act_all_fp16_magnitudes_exponent():
     # one value at a time through the absmax -> exponent path: every binade and mantissa edge
     h = handle()
