@@ -255,6 +255,72 @@ def bench_decode(h, peaks, iters=40):
 
 
 # ----------------------------------------------------------------------------------------
+# the other prefill workloads (extra keys): int4 activations, token-pruned prefill
+# ----------------------------------------------------------------------------------------
+def _event_ms(fn, reps):
+    """Mean device time of fn() over reps back-to-back calls (events on the current stream)."""
+    fn()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b) / reps
+
+
+def bench_w4a4(h, reps=30):
+    wl = inputs.WORKLOADS["llama7b_prefill_w4a4"]
+    M = wl.Ms[0]
+    layers = []
+    for s in wl.shapes:
+        x = torch.from_numpy(inputs.activations(M, s.K, wl.seed, wl.outlier_frac, wl.outlier_mult)).cuda()
+        p, sc = h.aq_pack_w4(torch.from_numpy(inputs.weights(s.N, s.K, wl.seed)).cuda(), wl.group_size)
+        layers.append((x, p, sc, s, h.alloc_workspace(M, s.K, s.N, wl.group_size),
+                       torch.empty((M, s.N), dtype=torch.float16, device="cuda")))
+    def step():
+        for x, p, sc, s, ws, y in layers:
+            h.aq_linear_w4a4(x, p, sc, s.N, wl.group_size, clip_shift_or_exp=wl.clip_shift, y=y, workspace=ws)
+    ms = _event_ms(step, reps)
+    ops = sum(2.0 * M * s.K * s.N for s in wl.shapes)
+    return {"workload": wl.name, "ms_per_step": ms, "TOPS": ops / (ms * 1e-3) / 1e12,
+            "note": "int4 codes travel in int8 containers: the tensor cores have no 4-bit integer kind"}
+
+
+def bench_pruned(h, reps=10):
+    wl = inputs.WORKLOADS["opt30b_pruned_prefill_w4a8"]
+    M = wl.Ms[0]
+    n_keep = wl.n_keep(M)
+    scores = torch.from_numpy(inputs.token_scores(M, wl.seed)).cuda()
+    out = []
+    for s in wl.shapes:
+        x = torch.from_numpy(inputs.activations(M, s.K, wl.seed, wl.outlier_frac, wl.outlier_mult)).cuda()
+        p, sc = h.aq_pack_w4(torch.from_numpy(inputs.weights(s.N, s.K, wl.seed)).cuda(), wl.group_size)
+        ws = h.alloc_workspace(n_keep, s.K, s.N, wl.group_size)
+        y = torch.empty((n_keep, s.N), dtype=torch.float16, device="cuda")
+        xc = torch.empty((n_keep, s.K), dtype=torch.float16, device="cuda")
+        def gathered():                      # select, copy the kept rows, then the layer
+            idx = h.aq_token_select(scores, n_keep)
+            h.aq_token_compact(x, idx, out=xc)
+            h.aq_linear_w4a8(xc, p, sc, s.N, wl.group_size, y=y, workspace=ws)
+        def fused():                         # select, then the layer reads the kept rows in place
+            idx = h.aq_token_select(scores, n_keep)
+            h.aq_linear_w4a8(x, p, sc, s.N, wl.group_size, row_idx=idx, y=y, workspace=ws)
+        q, e = h.aq_quantize_act(xc, 8)
+        def product():
+            h.aq_gemm_w4(q, p, sc, s.N, wl.group_size, e, y=y, workspace=ws)
+        ops = 2.0 * n_keep * s.K * s.N
+        r = {"K": s.K, "N": s.N, "M_in": M, "n_keep": n_keep}
+        for name, fn in (("select_gather_linear", gathered), ("select_rowidx_linear", fused), ("product_only", product)):
+            ms = _event_ms(fn, reps)
+            r[name] = {"us": ms * 1e3, "TOPS": ops / (ms * 1e-3) / 1e12}
+        out.append(r)
+        del x, p, sc, ws, y, xc, q
+    return out
+
+
+# ----------------------------------------------------------------------------------------
 # single-shape case (for profiling one kernel on a small or a full-size shape)
 # ----------------------------------------------------------------------------------------
 def run_case(args):
@@ -297,7 +363,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-decode", action="store_true")
+    ap.add_argument("--no-decode", action="store_true", help="skip the extra keys (decode, w4a4, pruned_prefill)")
     ap.add_argument("--case", default=None, help="M,K,N,group[,bits[,kernel]]: time one product kernel")
     ap.add_argument("--rotate-mb", type=float, default=0.0,
                     help="with --case: rotate through this many MB of weight copies (defeats L2)")
@@ -441,7 +507,7 @@ def main():
                 "h2d_bytes_per_step": int(sum(M * s.K * 2 for s in wl.shapes)),
                 "d2h_bytes_per_step": int(sum(M * s.N * 2 for s in wl.shapes)),
                 "ms_per_step": e2e_ms, "api": "aq_linear_host"},
-        "gpu_launches": args.steps * len(layers) * 3,
+        "gpu_launches": args.steps * len(layers) * 2,     # per layer: the fused quantize kernel and the product kernel
         "clocks": clocks,
         "roofline": roofline,
     }
@@ -450,6 +516,12 @@ def main():
             line["decode"] = bench_decode(h, peaks)
         except Exception as ex:  # report, do not hide
             line["decode"] = {"error": repr(ex)}
+    if rank == 0 and world == 1 and not args.no_decode:
+        for key, fn in (("w4a4", bench_w4a4), ("pruned_prefill", bench_pruned)):
+            try:
+                line[key] = fn(h)
+            except Exception as ex:  # report, do not hide
+                line[key] = {"error": repr(ex)}
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(wl, xs_np, ws_np, M)
     if rank == 0:

@@ -273,24 +273,28 @@ quantize_fused_kernel(const uint4* __restrict__ x, int M, int units_per_row /* 1
 // ---- token selection: rank every score, keep rank < n_keep, then compact the flags ------
 // rank(i) = #{ j : s_j > s_i  or (s_j == s_i and j < i) }, so equal scores resolve toward
 // the lower index and exactly n_keep tokens have rank < n_keep.
-__global__ void __launch_bounds__(256)
+// A CTA ranks 32 tokens: lane = token, and each of the 8 warps counts over one eighth of the scores
+// (a warp reads one score at a time, the same address in every lane).
+constexpr int kRankWarps = 8;
+__global__ void __launch_bounds__(32 * kRankWarps)
 token_rank_kernel(const float* __restrict__ scores, int M, int n_keep, uint8_t* __restrict__ keep) {
-    __shared__ float tile[1024];
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    __shared__ int ranks[32];
+    const int lane = threadIdx.x & 31, part = threadIdx.x >> 5;
+    const int i = blockIdx.x * 32 + lane;
+    if (part == 0) ranks[lane] = 0;
+    __syncthreads();
     const float si = i < M ? scores[i] : 0.0f;
+    const int per = (M + kRankWarps - 1) / kRankWarps;
+    const int j0 = part * per, j1 = min(M, j0 + per);
     int rank = 0;
-    for (int base = 0; base < M; base += 1024) {
-        for (int t = threadIdx.x; t < 1024; t += blockDim.x)
-            tile[t] = base + t < M ? scores[base + t] : -INFINITY;
-        __syncthreads();
-        const int lim = min(1024, M - base);
-        for (int t = 0; t < lim; ++t) {
-            const float sj = tile[t];
-            rank += (sj > si) || (sj == si && base + t < i);
-        }
-        __syncthreads();
+#pragma unroll 4
+    for (int j = j0; j < j1; ++j) {
+        const float sj = __ldg(scores + j);
+        rank += (sj > si) || (sj == si && j < i);
     }
-    if (i < M) keep[i] = rank < n_keep ? 1 : 0;
+    atomicAdd(&ranks[lane], rank);
+    __syncthreads();
+    if (part == 0 && i < M) keep[i] = ranks[lane] < n_keep ? 1 : 0;
 }
 
 // One CTA of 1024 threads: exclusive scan of the keep flags, ascending indices out.
@@ -399,7 +403,7 @@ cudaError_t launch_quantize_small(const __half* x, int M, int K, const int32_t* 
 cudaError_t launch_token_select(const float* scores, int M, int n_keep, int32_t* idx, void* scratch,
                                 cudaStream_t stream) {
     uint8_t* keep = static_cast<uint8_t*>(scratch);
-    token_rank_kernel<<<(M + 255) / 256, 256, 0, stream>>>(scores, M, n_keep, keep);
+    token_rank_kernel<<<(M + 31) / 32, 32 * kRankWarps, 0, stream>>>(scores, M, n_keep, keep);
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return err;
     token_compact_idx_kernel<<<1, 1024, 0, stream>>>(keep, M, idx);
