@@ -134,6 +134,8 @@ SHAPES = [
     (129, 384, 200, 128),      # spans token tiles with a ragged tail
     (300, 1024, 384, 0),
     (260, 1152, 520, 128),
+    (130, 256, 203, 128),      # N not a multiple of 8: outputs take direct stores instead of TMA stores
+    (70, 256, 77, 0),
 ]
 
 
