@@ -214,6 +214,62 @@ void orc_quantize_act(const uint16_t* x, int K, const int32_t* row_idx, int M,
 }
 
 // ---------------------------------------------------------------------------
+// TRIP factors (Eq. 5 with a per-channel alpha_k, zp = 0, s = 2^e): channel k is quantized with
+// the coarser step 2^(e + alpha_k),
+//     q = clip( round(x / 2^(e + alpha_k)), -2^(b-1), 2^(b-1)-1 ),
+// and enters the integer product as q * 2^alpha_k. Sec. 4.4 moves the factor onto the matching
+// weight column; q_k * (c_k * 2^alpha_k) and (q_k * 2^alpha_k) * c_k are the same integer, and
+// the second form is what is stored here (one int8 per value). Returns how many values did not
+// fit int8 (0 when bits = 4 and alpha <= 4).
+// ---------------------------------------------------------------------------
+long long orc_quantize_act_trip(const uint16_t* x, int K, const int32_t* row_idx, int M, int bits, int e,
+                                const uint8_t* alpha, int8_t* v) {
+    const float lo = (float)code_min(bits), hi = (float)code_max(bits);
+    long long misfit = 0;
+    for (int m = 0; m < M; ++m) {
+        const uint16_t* row = x + (size_t)(row_idx ? row_idx[m] : m) * K;
+        for (int k = 0; k < K; ++k) {
+            const int a = alpha[k];
+            const float t = std::ldexp(orc_half_to_float(row[k]), -(e + a));
+            int q = 0;
+            if (!std::isnan(t)) q = (int)std::min(std::max(round_half_even(t), lo), hi);
+            const int val = q * (1 << a);
+            if (val < -128 || val > 127) ++misfit;
+            v[(size_t)m * K + k] = (int8_t)val;
+        }
+    }
+    return misfit;
+}
+
+// Eq. 8, with the clipping of Eq. 5 inside the quantizer (without it the finest step would always
+// win): for every channel the alpha in {0..k_max} with the smallest squared reconstruction error
+// over the calibration tokens; the smallest alpha among equals. Errors are summed in binary64 over
+// tokens in ascending order, product and sum rounded separately (no fused multiply-add), so that
+// another implementation following the same order reaches the same decision. Non-finite values
+// are skipped.
+void orc_trip_calibrate(const uint16_t* x, int K, const int32_t* row_idx, int M, int bits, int e, int k_max,
+                        uint8_t* alpha_out) {
+    const double lo = (double)code_min(bits), hi = (double)code_max(bits);
+    for (int k = 0; k < K; ++k) {
+        int best = 0;
+        double best_err = 0.0;
+        for (int a = 0; a <= k_max; ++a) {
+            double err = 0.0;
+            for (int m = 0; m < M; ++m) {
+                const double xv = (double)orc_half_to_float(x[(size_t)(row_idx ? row_idx[m] : m) * K + k]);
+                if (!std::isfinite(xv)) continue;
+                const double q = std::min(std::max(std::nearbyint(std::ldexp(xv, -(e + a))), lo), hi);
+                const double d = xv - std::ldexp(q, e + a);
+                volatile double sq = d * d;            // rounded product, kept apart from the sum
+                err = err + sq;
+            }
+            if (a == 0 || err < best_err) { best = a; best_err = err; }
+        }
+        alpha_out[k] = (uint8_t)best;
+    }
+}
+
+// ---------------------------------------------------------------------------
 // Integer matrix product (Sec. 4.4; Algorithm 1 computes the same sums of 4-bit
 // products in SIMD lanes):  acc[m][n][g] = sum over k in group g of q[m][k]*c[n][k].
 // int32 result with an int64 shadow; the return value counts sums that did not fit

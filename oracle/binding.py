@@ -62,6 +62,7 @@ def lib():
         L.orc_progressive_ratio.restype = C.c_double
         L.orc_progressive_ratio.argtypes = [C.c_double, C.c_int]
         L.orc_num_threads.restype = C.c_int
+        L.orc_quantize_act_trip.restype = C.c_longlong
     return _lib
 
 
@@ -173,6 +174,35 @@ def quantize_act(x: np.ndarray, bits: int, e: int, row_idx: Optional[np.ndarray]
     q = np.empty((M, K), np.int8)
     lib().orc_quantize_act(_p(_half_bits(x)), K, _p(ri), M, bits, e, _p(q))
     return q
+
+
+def quantize_act_trip(x: np.ndarray, bits: int, e: int, alpha: np.ndarray,
+                      row_idx: Optional[np.ndarray] = None) -> np.ndarray:
+    """Eq. 5 with per-channel factors: int8 values q * 2^alpha_k at base exponent e."""
+    M_in, K = x.shape
+    ri = None if row_idx is None else _c(row_idx, np.int32)
+    M = M_in if ri is None else ri.shape[0]
+    al = _c(alpha, np.uint8)
+    assert al.shape == (K,)
+    v = np.empty((M, K), np.int8)
+    misfit = lib().orc_quantize_act_trip(_p(_half_bits(x)), K, _p(ri), M, bits, e, _p(al), _p(v))
+    assert misfit == 0, "a shifted code left the int8 range"
+    return v
+
+
+def trip_calibrate(x: np.ndarray, bits: int, e: int, k_max: int, row_idx: Optional[np.ndarray] = None) -> np.ndarray:
+    """Eq. 8: per-channel factor in {0..k_max} with the least squared error at base exponent e."""
+    M_in, K = x.shape
+    ri = None if row_idx is None else _c(row_idx, np.int32)
+    M = M_in if ri is None else ri.shape[0]
+    out = np.empty((K,), np.uint8)
+    lib().orc_trip_calibrate(_p(_half_bits(x)), K, _p(ri), M, bits, e, k_max, _p(out))
+    return out
+
+
+def trip_base_exponent(x: np.ndarray, bits: int, k_max: int, row_idx: Optional[np.ndarray] = None) -> int:
+    """Eq. 6 read as s = 2^(e0 - k_max): channels with the largest factor still reach the layer maximum."""
+    return layer_exponent(x, bits, row_idx) - k_max
 
 
 def int_gemm(q: np.ndarray, c: np.ndarray, group: int) -> np.ndarray:

@@ -404,3 +404,107 @@ def test_inputs_are_seeded_and_structured():
     assert 0.018 < w.astype(np.float32).std() < 0.022
     s = inputs.token_scores(100, 1)
     assert s.min() >= 0 and s.max() < 1 and s.dtype == np.float32
+
+
+# ------------------------------------------------------------------ TRIP factors (Eq. 5-8)
+def _trip_rows():
+    rows = []
+    for line in open(os.path.join(GOLDEN, "trip_hand_worked.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        e, a, x, v = line.split()
+        rows.append((int(e), int(a), float(x), int(v)))
+    return rows
+
+
+def test_trip_quantizer_hand_worked_table():
+    # Eq. 5 with a per-channel factor, values worked by hand
+    for e, a, x, v in _trip_rows():
+        xs = np.array([[x]], np.float16)
+        got = oracle.quantize_act_trip(xs, 4, e, np.array([a], np.uint8))
+        # the table's x are exactly representable in fp16 or far from a rounding boundary
+        assert int(got[0, 0]) == v, (e, a, x, v, int(got[0, 0]))
+
+
+def test_trip_quantizer_invariants_and_special_cases():
+    g = np.random.Generator(np.random.Philox(key=4242))
+    M, K = 64, 96
+    x = (g.standard_normal((M, K)) * 6).astype(np.float16)
+    x[:, 5] *= 20
+    alpha = g.integers(0, 5, size=K).astype(np.uint8)
+    for e in (-3, 0, 2):
+        v = oracle.quantize_act_trip(x, 4, e, alpha).astype(np.int64)
+        # alpha = 0 everywhere is the plain quantizer of Eq. 2 / Eq. 5
+        assert np.array_equal(oracle.quantize_act_trip(x, 4, e, np.zeros(K, np.uint8)), oracle.quantize_act(x, 4, e))
+        xf = x.astype(np.float64)
+        step = np.exp2(e + alpha.astype(np.float64))[None, :]
+        # every value is a multiple of 2^alpha with a 4-bit quotient, and fits int8
+        assert np.all(v % (1 << alpha.astype(np.int64))[None, :] == 0)
+        qq = v // (1 << alpha.astype(np.int64))[None, :]
+        assert qq.min() >= -8 and qq.max() <= 7 and v.min() >= -128 and v.max() <= 127
+        # inside the representable range the reconstruction is within half a (coarse) step; outside it saturates
+        inside = (xf >= -8 * step) & (xf <= 7 * step)
+        assert np.all(np.abs(xf - v * np.exp2(e))[inside] <= step.repeat(M, 0)[inside] / 2 + 1e-12)
+        assert np.all(qq[xf > 7 * step] == 7) and np.all(qq[xf < -8 * step] == -8)
+
+
+def test_trip_factor_on_weights_equals_factor_on_codes():
+    # Sec. 4.4: the factor is "transformed over the corresponding weights": shifting weight column k by
+    # alpha_k gives the same integer sums as shifting the activation codes of channel k
+    g = np.random.Generator(np.random.Philox(key=99))
+    M, K, N = 9, 256, 7
+    x = (g.standard_normal((M, K)) * 5).astype(np.float16)
+    alpha = g.integers(0, 5, size=K).astype(np.uint8)
+    c = g.integers(-8, 8, size=(N, K)).astype(np.int8)
+    e = -1
+    v = oracle.quantize_act_trip(x, 4, e, alpha)
+    acc_codes = oracle.int_gemm(v, c, 128)                                 # factor on the codes
+    q = v.astype(np.int64) // (1 << alpha.astype(np.int64))[None, :]
+    c_shift = c.astype(np.int64) * (1 << alpha.astype(np.int64))[None, :]   # factor on the weights (up to 8 bits)
+    ref = np.einsum("mgk,ngk->mng", q.reshape(M, 2, 128), c_shift.reshape(N, 2, 128))
+    assert np.array_equal(acc_codes.reshape(M, N, 2).astype(np.int64), ref)
+
+
+def test_trip_calibration_against_exact_rational_search():
+    # Eq. 8 (with the clipping of Eq. 5) by exhaustive search in exact rational arithmetic
+    from fractions import Fraction as F
+    import math
+    def rhe(t):
+        f = math.floor(t)
+        d = t - f
+        return f + 1 if d > F(1, 2) else f if d < F(1, 2) else (f if f % 2 == 0 else f + 1)
+    g = np.random.Generator(np.random.Philox(key=31))
+    M, K, k_max = 12, 10, 4
+    x = (g.standard_normal((M, K)) * 3).astype(np.float16)
+    x[:, 2] *= 30                      # an outlier channel
+    x[3, 7] = 90                       # a single outlier
+    x[:, 4] = 0                        # all zero: every alpha ties at error 0
+    x[:, 9] = (g.integers(-7, 8, size=M)).astype(np.float16)   # exactly representable at alpha 0
+    for e in (0, -1):
+        got = oracle.trip_calibrate(x, 4, e, k_max)
+        for k in range(K):
+            errs = []
+            for a in range(k_max + 1):
+                s = F(2) ** (e + a)
+                err = F(0)
+                for m in range(M):
+                    xv = F(float(x[m, k]))
+                    q = max(-8, min(7, rhe(xv / s)))
+                    err += (xv - q * s) ** 2
+                errs.append(err)
+            assert int(got[k]) == errs.index(min(errs)), (e, k, errs)
+        assert got[4] == 0
+        if e == 0:
+            assert got[9] == 0 and got[2] >= 3
+
+
+def test_trip_base_exponent_reaches_the_layer_maximum():
+    # Eq. 6 read as s = 2^(e0 - K): with the largest factor the step is the plain layer step again
+    x = np.zeros((2, 128), np.float16)
+    x[1, 3] = 100.0
+    for k_max in (0, 2, 4):
+        e = oracle.trip_base_exponent(x, 4, k_max)
+        assert e == oracle.layer_exponent(x, 4) - k_max
+        alpha = np.full(128, k_max, np.uint8)
+        v = oracle.quantize_act_trip(x, 4, e, alpha)
+        assert np.array_equal(v.astype(np.int64) >> k_max, oracle.quantize_act(x, 4, e + k_max).astype(np.int64))
