@@ -134,6 +134,35 @@ int aq_token_select(aq_handle_t h, const float* scores, int M, int n_keep, int32
 int aq_token_compact(aq_handle_t h, const void* x_fp16, int M, int K, const int32_t* idx,
                      int n_keep, void* x_out, void* stream);
 
+/* ---- per-channel TRIP factors (paper Eq. 5-8; Sec. 4.4 "Efficient TRIP Matrix Multiplication")
+ * alpha: K bytes on the device (16-byte aligned), one factor per input channel, each in
+ * 0..k_max, k_max <= 4. Channel k is quantized to a 4-bit code with the coarser step
+ * 2^(e + alpha_k) (Eq. 5), and the code enters the integer product shifted left by alpha_k,
+ * which is the factor "transformed over the corresponding weights" of Sec. 4.4 (a 4-bit code
+ * shifted by at most 4 still fits the int8 operand). The dynamic base exponent is
+ * e = e0 - k_max - clip_shift, e0 the plain 4-bit layer exponent (Eq. 6 read as
+ * s = 2^(e0 - K)), so channels with the largest factor still reach the layer maximum; in
+ * static mode e is given. Outputs are y = 2^e * sum_g s_w[n,g] * acc[m,n,g] as before.
+ * Factors above 4 are the caller's error (the shifted code would leave int8).
+ *
+ * aq_trip_calibrate: Eq. 8 with the clipping of Eq. 5: for every channel the factor in
+ * 0..k_max with the least squared reconstruction error over the M calibration rows (kept
+ * rows when row_idx is given), the smallest factor among equals; errors are summed in
+ * binary64 over rows in ascending order. Writes alpha_out[K] and the base exponent
+ * e = e0 - k_max of the calibration set. Non-finite values are skipped. */
+int aq_trip_calibrate(aq_handle_t h, const void* x_fp16, int M, int K, int k_max, const int32_t* row_idx,
+                      uint8_t* alpha_out, int32_t* scale_exp_out, void* workspace, size_t workspace_bytes,
+                      void* stream);
+/* As aq_quantize_act with bits = 4: q[m,k] = code * 2^alpha_k (int8). */
+int aq_quantize_act_trip(aq_handle_t h, const void* x_fp16, int M, int K, const uint8_t* alpha, int k_max,
+                         int scale_mode, int clip_shift_or_exp, const int32_t* row_idx, int8_t* q,
+                         int32_t* scale_exp_out, void* workspace, size_t workspace_bytes, void* stream);
+/* As aq_linear_w4a4 with the factors applied in the quantize step; the product kernels are unchanged. */
+int aq_linear_w4a4_trip(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed,
+                        const void* w_scales, int N, int group_size, const uint8_t* alpha, int k_max,
+                        int scale_mode, int clip_shift_or_exp, const int32_t* row_idx, void* y_fp16,
+                        int32_t* acc_dump, void* workspace, size_t workspace_bytes, void* stream);
+
 /* ---- host-buffer convenience (SYNCHRONIZES the stream before returning)
  * x_host fp16 [M,K] and y_host fp16 [M,N] are HOST pointers (pinned memory gives the best
  * rate). Copies x to the device scratch, runs the layer with `bits` (8 or 4), copies y

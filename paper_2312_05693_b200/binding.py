@@ -74,6 +74,9 @@ def load():
     L.aq_linear_w4a8.argtypes = lin
     L.aq_linear_w4a4.argtypes = lin
     L.aq_gemm_w4.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, vp, vp, vp, vp, sz, vp]
+    L.aq_trip_calibrate.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
+    L.aq_quantize_act_trip.argtypes = [vp, vp, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
+    L.aq_linear_w4a4_trip.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
     L.aq_token_select.argtypes = [vp, vp, i32, i32, vp, vp, sz, vp]
     L.aq_token_compact.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp]
     L.aq_linear_host.argtypes = [vp, i32, vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, vp, sz, vp]
@@ -205,6 +208,45 @@ class Handle:
                        clip_shift_or_exp=0, row_idx=None, y=None, acc_dump=None, workspace=None):
         return self._linear(load().aq_linear_w4a4, "aq_linear_w4a4", x, packed, scales, N, group_size,
                             scale_mode, clip_shift_or_exp, row_idx, y, acc_dump, workspace)
+
+    # ---- per-channel TRIP factors (Eq. 5-8)
+    def aq_trip_calibrate(self, x: torch.Tensor, k_max: int, row_idx: Optional[torch.Tensor] = None
+                          ) -> Tuple[torch.Tensor, torch.Tensor]:
+        M_in, K = x.shape
+        M = M_in if row_idx is None else row_idx.shape[0]
+        alpha = torch.empty(K, dtype=torch.uint8, device=x.device)
+        e = torch.empty(1, dtype=torch.int32, device=x.device)
+        ws = torch.empty(256, dtype=torch.uint8, device=x.device)
+        _check(load().aq_trip_calibrate(self._h, _ptr(x), M, K, k_max, _ptr(row_idx), _ptr(alpha), _ptr(e),
+                                        _ptr(ws), ws.numel(), _stream()), "aq_trip_calibrate")
+        return alpha, e
+
+    def aq_quantize_act_trip(self, x: torch.Tensor, alpha: torch.Tensor, k_max: int,
+                             scale_mode: int = AQ_SCALE_DYNAMIC, clip_shift_or_exp: int = 0,
+                             row_idx: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor]:
+        M_in, K = x.shape
+        M = M_in if row_idx is None else row_idx.shape[0]
+        q = torch.empty((M, K), dtype=torch.int8, device=x.device)
+        e = torch.empty(1, dtype=torch.int32, device=x.device)
+        ws = torch.empty(256, dtype=torch.uint8, device=x.device)
+        _check(load().aq_quantize_act_trip(self._h, _ptr(x), M, K, _ptr(alpha), k_max, scale_mode,
+                                           clip_shift_or_exp, _ptr(row_idx), _ptr(q), _ptr(e), _ptr(ws),
+                                           ws.numel(), _stream()), "aq_quantize_act_trip")
+        return q, e
+
+    def aq_linear_w4a4_trip(self, x, packed, scales, N, group_size, alpha, k_max, scale_mode=AQ_SCALE_DYNAMIC,
+                            clip_shift_or_exp=0, row_idx=None, y=None, acc_dump=None, workspace=None):
+        M_in, K = x.shape
+        M = M_in if row_idx is None else row_idx.shape[0]
+        if y is None:
+            y = torch.empty((M, N), dtype=torch.float16, device=x.device)
+        if workspace is None:
+            workspace = self.alloc_workspace(M, K, N, group_size)
+        _check(load().aq_linear_w4a4_trip(self._h, _ptr(x), M, K, _ptr(packed), _ptr(scales), N, group_size,
+                                          _ptr(alpha), k_max, scale_mode, clip_shift_or_exp, _ptr(row_idx),
+                                          _ptr(y), _ptr(acc_dump), _ptr(workspace), workspace.numel(), _stream()),
+               "aq_linear_w4a4_trip")
+        return y
 
     def aq_gemm_w4(self, q, packed, scales, N, group_size, scale_exp, y=None, acc_dump=None, workspace=None):
         M, K = q.shape

@@ -63,10 +63,31 @@ int run_gemm(aq_handle_t h, const GemmArgs& g, cudaStream_t stream) {
     return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
 }
 
+// Scale + codes with the kernel that fits the size and the scale mode. `alpha` / `k_max`: TRIP factors
+// or NULL / 0.
+cudaError_t quantize_dispatch(aq_handle_t h, const __half* xh, int M, int K, const int32_t* row_idx, int bits,
+                              int scale_mode, int clip_shift_or_exp, Control* ctl, int8_t* q, int32_t* scale_exp_out,
+                              const uint8_t* alpha, int k_max, cudaStream_t stream) {
+    if (quantize_small_fits(M, K))
+        // small activations (decode): one kernel finds the scale, writes the codes and initialises
+        // the control block
+        return launch_quantize_small(xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, ctl, q, scale_exp_out,
+                                     stream, alpha, k_max);
+    const cudaError_t e = cudaMemsetAsync(ctl, 0, sizeof(Control), stream);
+    if (e != cudaSuccess) return e;
+    if (scale_mode == AQ_SCALE_DYNAMIC)
+        return launch_quantize_fused(xh, M, K, row_idx, bits, clip_shift_or_exp, ctl, q, scale_exp_out, h->dev, stream,
+                                     alpha, k_max);
+    return launch_quantize(xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, ctl, q, scale_exp_out, h->dev,
+                           stream, alpha, k_max);
+}
+
+bool trip_args_ok(const uint8_t* alpha, int k_max) { return alpha && k_max >= 0 && k_max <= 4; }
+
 int linear_impl(aq_handle_t h, int bits, const void* x, int M, int K, const void* w_packed,
                 const void* w_scales, int N, int group, int scale_mode, int clip_shift_or_exp,
                 const int32_t* row_idx, void* y, int32_t* acc_dump, void* workspace, size_t workspace_bytes_,
-                void* stream_) {
+                void* stream_, const uint8_t* alpha = nullptr, int k_max = 0) {
     if (!h || !x || !w_packed || !w_scales || !y) return AQ_ERR_INVALID_ARG;
     if (scale_mode != AQ_SCALE_DYNAMIC && scale_mode != AQ_SCALE_STATIC) return AQ_ERR_INVALID_ARG;
     if (scale_mode == AQ_SCALE_DYNAMIC && (clip_shift_or_exp < 0 || clip_shift_or_exp > 16)) return AQ_ERR_INVALID_ARG;
@@ -80,25 +101,10 @@ int linear_impl(aq_handle_t h, int bits, const void* x, int M, int K, const void
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const Workspace w = carve(workspace, M, K);
     const __half* xh = static_cast<const __half*>(x);
-    cudaError_t e;
-    if (quantize_small_fits(M, K)) {
-        // small activations (decode): one kernel finds the scale, writes the codes and initialises
-        // the control block
-        e = launch_quantize_small(xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, w.ctl, w.codes, nullptr,
-                                  stream);
-        if (e != cudaSuccess) return cuda_fail(h, e);
-    } else {
-        e = cudaMemsetAsync(w.ctl, 0, sizeof(Control), stream);
-        if (e != cudaSuccess) return cuda_fail(h, e);
-        if (scale_mode == AQ_SCALE_DYNAMIC) {
-            e = launch_quantize_fused(xh, M, K, row_idx, bits, clip_shift_or_exp, w.ctl, w.codes, nullptr, h->dev,
-                                      stream);
-        } else {
-            e = launch_quantize(xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, w.ctl, w.codes, nullptr,
-                                h->dev, stream);
-        }
-        if (e != cudaSuccess) return cuda_fail(h, e);
-    }
+    if (alpha && !aligned(alpha, 16)) return AQ_ERR_ALIGNMENT;
+    const cudaError_t e = quantize_dispatch(h, xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, w.ctl, w.codes,
+                                            nullptr, alpha, k_max, stream);
+    if (e != cudaSuccess) return cuda_fail(h, e);
     GemmArgs g;
     g.q = w.codes; g.M = M; g.K = K; g.N = N; g.group = group;
     g.w_packed = static_cast<const uint8_t*>(w_packed);
@@ -216,9 +222,9 @@ int aq_unpack_w4(aq_handle_t h, const void* w_packed, int N, int K, int8_t* code
     return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
 }
 
-int aq_quantize_act(aq_handle_t h, const void* x_fp16, int M, int K, int bits, int scale_mode,
-                    int clip_shift_or_exp, const int32_t* row_idx, int8_t* q, int32_t* scale_exp_out,
-                    void* workspace, size_t workspace_bytes_, void* stream_) {
+static int quantize_impl(aq_handle_t h, const void* x_fp16, int M, int K, int bits, int scale_mode,
+                         int clip_shift_or_exp, const int32_t* row_idx, int8_t* q, int32_t* scale_exp_out,
+                         void* workspace, size_t workspace_bytes_, void* stream_, const uint8_t* alpha, int k_max) {
     if (!h || !x_fp16 || !q) return AQ_ERR_INVALID_ARG;
     if (bits != 8 && bits != 4) return AQ_ERR_INVALID_ARG;
     if (scale_mode != AQ_SCALE_DYNAMIC && scale_mode != AQ_SCALE_STATIC) return AQ_ERR_INVALID_ARG;
@@ -233,20 +239,53 @@ int aq_quantize_act(aq_handle_t h, const void* x_fp16, int M, int K, int bits, i
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     Control* ctl = static_cast<Control*>(workspace);
     const __half* xh = static_cast<const __half*>(x_fp16);
-    if (quantize_small_fits(M, K)) {
-        const cudaError_t es = launch_quantize_small(xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, ctl, q,
-                                                     scale_exp_out, stream);
-        return es == cudaSuccess ? AQ_OK : cuda_fail(h, es);
-    }
+    const cudaError_t e = quantize_dispatch(h, xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, ctl, q,
+                                            scale_exp_out, alpha, k_max, stream);
+    return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
+int aq_quantize_act(aq_handle_t h, const void* x_fp16, int M, int K, int bits, int scale_mode,
+                    int clip_shift_or_exp, const int32_t* row_idx, int8_t* q, int32_t* scale_exp_out,
+                    void* workspace, size_t workspace_bytes_, void* stream) {
+    return quantize_impl(h, x_fp16, M, K, bits, scale_mode, clip_shift_or_exp, row_idx, q, scale_exp_out, workspace,
+                         workspace_bytes_, stream, nullptr, 0);
+}
+
+int aq_quantize_act_trip(aq_handle_t h, const void* x_fp16, int M, int K, const uint8_t* alpha, int k_max,
+                         int scale_mode, int clip_shift_or_exp, const int32_t* row_idx, int8_t* q,
+                         int32_t* scale_exp_out, void* workspace, size_t workspace_bytes_, void* stream) {
+    if (!trip_args_ok(alpha, k_max)) return AQ_ERR_INVALID_ARG;
+    if (!aligned(alpha, 16)) return AQ_ERR_ALIGNMENT;
+    return quantize_impl(h, x_fp16, M, K, 4, scale_mode, clip_shift_or_exp, row_idx, q, scale_exp_out, workspace,
+                         workspace_bytes_, stream, alpha, k_max);
+}
+
+int aq_trip_calibrate(aq_handle_t h, const void* x_fp16, int M, int K, int k_max, const int32_t* row_idx,
+                      uint8_t* alpha_out, int32_t* scale_exp_out, void* workspace, size_t workspace_bytes_,
+                      void* stream_) {
+    if (!h || !x_fp16 || !alpha_out || k_max < 0 || k_max > 4) return AQ_ERR_INVALID_ARG;
+    const int s = check_shape(M, K, 1, 0);
+    if (s != AQ_OK) return s;
+    if (!workspace || workspace_bytes_ < sizeof(Control)) return AQ_ERR_WORKSPACE;
+    if (!aligned(x_fp16, 16) || !aligned(workspace, 256) || (scale_exp_out && !aligned(scale_exp_out, 4)) ||
+        (row_idx && !aligned(row_idx, 4)))
+        return AQ_ERR_ALIGNMENT;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    Control* ctl = static_cast<Control*>(workspace);
     cudaError_t e = cudaMemsetAsync(ctl, 0, sizeof(Control), stream);
     if (e != cudaSuccess) return cuda_fail(h, e);
-    if (scale_mode == AQ_SCALE_DYNAMIC) {
-        e = launch_quantize_fused(xh, M, K, row_idx, bits, clip_shift_or_exp, ctl, q, scale_exp_out, h->dev, stream);
-    } else {
-        e = launch_quantize(xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, ctl, q, scale_exp_out, h->dev,
-                            stream);
-    }
+    e = launch_trip_calibrate(static_cast<const __half*>(x_fp16), M, K, row_idx, 4, k_max, ctl, alpha_out,
+                              scale_exp_out, h->dev, stream);
     return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
+int aq_linear_w4a4_trip(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed,
+                        const void* w_scales, int N, int group_size, const uint8_t* alpha, int k_max,
+                        int scale_mode, int clip_shift_or_exp, const int32_t* row_idx, void* y_fp16,
+                        int32_t* acc_dump, void* workspace, size_t workspace_bytes_, void* stream) {
+    if (!trip_args_ok(alpha, k_max)) return AQ_ERR_INVALID_ARG;
+    return linear_impl(h, 4, x_fp16, M, K, w_packed, w_scales, N, group_size, scale_mode, clip_shift_or_exp,
+                       row_idx, y_fp16, acc_dump, workspace, workspace_bytes_, stream, alpha, k_max);
 }
 
 int aq_linear_w4a8(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed,

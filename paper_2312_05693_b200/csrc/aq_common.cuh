@@ -82,18 +82,25 @@ cudaError_t launch_unpack_w4(const uint8_t* packed, int N, int K, int8_t* codes,
 
 cudaError_t launch_quantize(const __half* x, int M, int K, const int32_t* row_idx, int bits,
                             int scale_mode, int clip_shift_or_exp, Control* ctl, int8_t* q,
-                            int32_t* scale_exp_out, const DeviceInfo& dev, cudaStream_t stream);
+                            int32_t* scale_exp_out, const DeviceInfo& dev, cudaStream_t stream,
+                            const uint8_t* alpha = nullptr, int k_max = 0);
 
 // Activations of at most 262144 elements: one kernel that also initialises the control block.
 bool quantize_small_fits(int M, int K);
 cudaError_t launch_quantize_small(const __half* x, int M, int K, const int32_t* row_idx, int bits, int scale_mode,
                                   int clip_shift_or_exp, Control* ctl, int8_t* q, int32_t* scale_exp_out,
-                                  cudaStream_t stream);
+                                  cudaStream_t stream, const uint8_t* alpha = nullptr, int k_max = 0);
 
 // Dynamic scale, any size: one cooperative kernel (absmax, exponent, codes). The control block must
 // have been cleared (absmax_bits, counter) on the same stream before.
 cudaError_t launch_quantize_fused(const __half* x, int M, int K, const int32_t* row_idx, int bits, int clip_shift,
                                   Control* ctl, int8_t* q, int32_t* scale_exp_out, const DeviceInfo& dev,
+                                  cudaStream_t stream, const uint8_t* alpha = nullptr, int k_max = 0);
+// TRIP factors (Eq. 5-8): `alpha` above is NULL or K bytes (16-byte aligned), one factor 0..k_max per
+// input channel: channel k is quantized with the step 2^(e + alpha_k), its code stored shifted left by
+// alpha_k, and the dynamic exponent is lowered by k_max (Eq. 6). The search of Eq. 8:
+cudaError_t launch_trip_calibrate(const __half* x, int M, int K, const int32_t* row_idx, int bits, int k_max,
+                                  Control* ctl, uint8_t* alpha_out, int32_t* scale_exp_out, const DeviceInfo& dev,
                                   cudaStream_t stream);
 
 cudaError_t launch_token_select(const float* scores, int M, int n_keep, int32_t* idx, void* scratch,

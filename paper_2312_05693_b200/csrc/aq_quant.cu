@@ -44,19 +44,49 @@ __device__ __forceinline__ void quantize8_half2(const uint4& d, __half2 inv2, __
     w1 = __byte_perm(r[2], r[3], 0x6420);
 }
 
+// 8 halves -> 8 values in fp32 arithmetic. With TRIP factors (Eq. 5 with a per-channel alpha,
+// `al` = the 8 factor bytes of these channels) channel k uses the step 2^(e + alpha_k) and its code
+// is stored shifted left by alpha_k, the form in which the factor enters the integer product.
+__device__ __forceinline__ uint2 quantize8_fp32(const uint4& d, int e, float lo, float hi, const uint2* al) {
+    const __half* h = reinterpret_cast<const __half*>(&d);
+    const uint8_t* ab = reinterpret_cast<const uint8_t*>(al);
+    uint32_t out[2];
+#pragma unroll
+    for (int w = 0; w < 2; ++w) {
+        uint32_t word = 0;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int i = 4 * w + b;
+            const int a = al ? (int)ab[i] : 0;
+            const float inv = __int_as_float((127 - e - a) << 23);           // 2^-(e + alpha)
+            word |= ((uint32_t)(quantize_one(__half2float(h[i]), inv, lo, hi) << a) & 0xFFu) << (8 * b);
+        }
+        out[w] = word;
+    }
+    return make_uint2(out[0], out[1]);
+}
+__device__ __forceinline__ uint4 quantize16_fp32(const uint4& d0, const uint4& d1, int e, float lo, float hi,
+                                                 const uint4* al) {
+    uint2 a0, a1;
+    if (al) { a0 = make_uint2(al->x, al->y); a1 = make_uint2(al->z, al->w); }
+    const uint2 r0 = quantize8_fp32(d0, e, lo, hi, al ? &a0 : nullptr);
+    const uint2 r1 = quantize8_fp32(d1, e, lo, hi, al ? &a1 : nullptr);
+    return make_uint4(r0.x, r0.y, r1.x, r1.y);
+}
+
 // ---- quantize: 16 halves in (two 16-byte loads), 16 codes out (one 16-byte store) -----
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_kernel(const uint4* __restrict__ x, int M, int vec_per_row /* 16-element units */,
                 const int32_t* __restrict__ row_idx, int bits, int scale_mode, int clip_shift_or_exp,
-                Control* __restrict__ ctl, uint4* __restrict__ q, int32_t* __restrict__ scale_exp_out) {
+                Control* __restrict__ ctl, uint4* __restrict__ q, int32_t* __restrict__ scale_exp_out,
+                const uint4* __restrict__ alpha, int k_max) {
     const int e = scale_mode == AQ_SCALE_DYNAMIC
-                      ? layer_exponent_from_bits(ctl->absmax_bits, bits) - clip_shift_or_exp
+                      ? layer_exponent_from_bits(ctl->absmax_bits, bits) - clip_shift_or_exp - k_max
                       : clip_shift_or_exp;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         ctl->scale_exp = e;
         if (scale_exp_out) *scale_exp_out = e;
     }
-    const float inv = __int_as_float((127 - e) << 23);      // 2^-e, |e| <= 40
     const float lo = -(float)(1 << (bits - 1)), hi = (float)((1 << (bits - 1)) - 1);
     const size_t total = (size_t)M * vec_per_row;
     const size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -64,21 +94,9 @@ quantize_kernel(const uint4* __restrict__ x, int M, int vec_per_row /* 16-elemen
     const int m = (int)(v / vec_per_row), c = (int)(v % vec_per_row);
     const size_t src = ((size_t)(row_idx ? row_idx[m] : m) * vec_per_row + c) * 2;
     const uint4 d0 = __ldg(x + src), d1 = __ldg(x + src + 1);
-    const __half* h0 = reinterpret_cast<const __half*>(&d0);
-    const __half* h1 = reinterpret_cast<const __half*>(&d1);
-    uint32_t out[4];
-#pragma unroll
-    for (int w = 0; w < 4; ++w) {
-        uint32_t word = 0;
-#pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            const int i = 4 * w + b;
-            const float f = __half2float(i < 8 ? h0[i] : h1[i - 8]);
-            word |= ((uint32_t)quantize_one(f, inv, lo, hi) & 0xFFu) << (8 * b);
-        }
-        out[w] = word;
-    }
-    q[v] = make_uint4(out[0], out[1], out[2], out[3]);
+    uint4 al;
+    if (alpha) al = __ldg(alpha + c);
+    q[v] = quantize16_fp32(d0, d1, e, lo, hi, alpha ? &al : nullptr);
 }
 
 // ---- small activations (decode): maximum, exponent and codes in ONE kernel -------------
@@ -91,7 +109,8 @@ constexpr size_t kSmallMaxElems = (size_t)kSmallCtas * kSmallThreads * kSmallVec
 __global__ void __cluster_dims__(kSmallCtas, 1, 1) __launch_bounds__(kSmallThreads)
 quantize_small_kernel(const uint4* __restrict__ x, int M, int vec_per_row, const int32_t* __restrict__ row_idx,
                       int bits, int scale_mode, int clip_shift_or_exp, Control* __restrict__ ctl,
-                      uint2* __restrict__ q, int32_t* __restrict__ scale_exp_out) {
+                      uint2* __restrict__ q, int32_t* __restrict__ scale_exp_out, const uint2* __restrict__ alpha,
+                      int k_max) {
     cg::cluster_group cluster = cg::this_cluster();
     __shared__ unsigned int warp_max[kSmallThreads / 32];
     __shared__ unsigned int slots[kSmallCtas];
@@ -127,7 +146,7 @@ quantize_small_kernel(const uint4* __restrict__ x, int M, int vec_per_row, const
     unsigned int all = 0;
 #pragma unroll
     for (int r = 0; r < kSmallCtas; ++r) all = max(all, slots[r]);
-    const int e = scale_mode == AQ_SCALE_DYNAMIC ? layer_exponent_from_bits(all, bits) - clip_shift_or_exp
+    const int e = scale_mode == AQ_SCALE_DYNAMIC ? layer_exponent_from_bits(all, bits) - clip_shift_or_exp - k_max
                                                  : clip_shift_or_exp;
     if (rank == 0 && threadIdx.x == 0) {
         ctl->absmax_bits = all;
@@ -136,20 +155,14 @@ quantize_small_kernel(const uint4* __restrict__ x, int M, int vec_per_row, const
         ctl->counter = 0;
         if (scale_exp_out) *scale_exp_out = e;
     }
-    const float inv = __int_as_float((127 - e) << 23);      // 2^-e
     const float lo = -(float)(1 << (bits - 1)), hi = (float)((1 << (bits - 1)) - 1);
 #pragma unroll
     for (int i = 0; i < kSmallVecs; ++i) {
         const int v = (i * kSmallCtas + rank) * kSmallThreads + (int)threadIdx.x;
         if (v < total) {
-            const __half* h = reinterpret_cast<const __half*>(&buf[i]);
-            uint32_t w0 = 0, w1 = 0;
-#pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                w0 |= ((uint32_t)quantize_one(__half2float(h[b]), inv, lo, hi) & 0xFFu) << (8 * b);
-                w1 |= ((uint32_t)quantize_one(__half2float(h[4 + b]), inv, lo, hi) & 0xFFu) << (8 * b);
-            }
-            q[v] = make_uint2(w0, w1);
+            uint2 al;
+            if (alpha) al = __ldg(alpha + v % vec_per_row);
+            q[v] = quantize8_fp32(buf[i], e, lo, hi, alpha ? &al : nullptr);
         }
     }
 }
@@ -174,7 +187,7 @@ __global__ void __launch_bounds__(kFusedThreads, 1)
 quantize_fused_kernel(const uint4* __restrict__ x, int M, int units_per_row /* 16-element units */,
                       const int32_t* __restrict__ row_idx, int bits, int clip_shift, Control* __restrict__ ctl,
                       uint4* __restrict__ q, int32_t* __restrict__ scale_exp_out, unsigned int cache_units,
-                      unsigned int units_per_cta) {
+                      unsigned int units_per_cta, const uint4* __restrict__ alpha, int k_max) {
     extern __shared__ uint4 fused_cache[];             // [2][cache_units]: first and second vector of a unit
     __shared__ unsigned int warp_max[kFusedThreads / 32];
     __shared__ int e_shared;
@@ -219,7 +232,7 @@ quantize_fused_kernel(const uint4* __restrict__ x, int M, int units_per_row /* 1
                 __nanosleep(100);
             }
             gave_up = failed;
-            e_shared = layer_exponent_from_bits(ld_acquire_u32(&ctl->absmax_bits), bits) - clip_shift;
+            e_shared = layer_exponent_from_bits(ld_acquire_u32(&ctl->absmax_bits), bits) - clip_shift - k_max;
         }
     }
     __syncthreads();
@@ -234,7 +247,7 @@ quantize_fused_kernel(const uint4* __restrict__ x, int M, int units_per_row /* 1
     }
     const float inv = __int_as_float((127 - e) << 23);      // 2^-e, |e| <= 40
     const float lo = -(float)(1 << (bits - 1)), hi = (float)((1 << (bits - 1)) - 1);
-    const bool fast = e >= -14 && e <= 14;                   // 2^-e is a normal half
+    const bool fast = alpha == nullptr && e >= -14 && e <= 14;   // 2^-e is a normal half
     const __half2 inv2 = __float2half2_rn(fast ? inv : 1.0f), lo2 = __float2half2_rn(lo), hi2 = __float2half2_rn(hi);
 #pragma unroll 2
     for (size_t u = u0 + threadIdx.x; u < u1; u += kFusedThreads) {
@@ -251,23 +264,68 @@ quantize_fused_kernel(const uint4* __restrict__ x, int M, int units_per_row /* 1
         if (fast) {
             quantize8_half2(d0, inv2, lo2, hi2, out[0], out[1]);
             quantize8_half2(d1, inv2, lo2, hi2, out[2], out[3]);
+            q[u] = make_uint4(out[0], out[1], out[2], out[3]);
         } else {
-            const __half* h0 = reinterpret_cast<const __half*>(&d0);
-            const __half* h1 = reinterpret_cast<const __half*>(&d1);
+            uint4 al;
+            if (alpha) al = __ldg(alpha + (size_t)(u % units_per_row));
+            q[u] = quantize16_fp32(d0, d1, e, lo, hi, alpha ? &al : nullptr);
+        }
+    }
+}
+
+// ---- TRIP calibration (Eq. 8 with the clipping of Eq. 5) ---------------------------------
+__global__ void __launch_bounds__(256)
+absmax_plain_kernel(const __half* __restrict__ x, int M, int K, const int32_t* __restrict__ row_idx,
+                    Control* __restrict__ ctl) {
+    const size_t total = (size_t)M * K;
+    unsigned int b = 0;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int m = (int)(i / K), k = (int)(i % K);
+        const unsigned int hb = __half_as_ushort(x[(size_t)(row_idx ? row_idx[m] : m) * K + k]) & 0x7FFFu;
+        if (hb <= 0x7C00u) b = max(b, hb);                                  // NaN is ignored
+    }
 #pragma unroll
-            for (int w = 0; w < 4; ++w) {
-                uint32_t word = 0;
+    for (int o = 16; o > 0; o >>= 1) b = max(b, __shfl_xor_sync(0xFFFFFFFFu, b, o));
+    if ((threadIdx.x & 31) == 0 && b != 0) atomicMax(&ctl->absmax_bits, b);
+}
+
+// One thread per channel walks the tokens in ascending order and keeps one binary64 error sum per
+// candidate factor (product and sum rounded separately), then takes the smallest factor among the
+// least errors. Consecutive threads read consecutive halves of a row.
+__global__ void __launch_bounds__(128)
+trip_calibrate_kernel(const __half* __restrict__ x, int M, int K, const int32_t* __restrict__ row_idx, int bits,
+                      int k_max, Control* __restrict__ ctl, uint8_t* __restrict__ alpha_out,
+                      int32_t* __restrict__ scale_exp_out) {
+    const int e = layer_exponent_from_bits(ctl->absmax_bits, bits) - k_max;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        ctl->scale_exp = e;
+        if (scale_exp_out) *scale_exp_out = e;
+    }
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= K) return;
+    const double lo = -(double)(1 << (bits - 1)), hi = (double)((1 << (bits - 1)) - 1);
+    double err[5] = {0.0, 0.0, 0.0, 0.0, 0.0};
+    for (int m = 0; m < M; ++m) {
+        const float xf = __half2float(x[(size_t)(row_idx ? row_idx[m] : m) * K + k]);
+        if (!isfinite(xf)) continue;
+        const double xv = (double)xf;
 #pragma unroll
-                for (int b = 0; b < 4; ++b) {
-                    const int i = 4 * w + b;
-                    const float f = __half2float(i < 8 ? h0[i] : h1[i - 8]);
-                    word |= ((uint32_t)quantize_one(f, inv, lo, hi) & 0xFFu) << (8 * b);
-                }
-                out[w] = word;
+        for (int a = 0; a < 5; ++a) {
+            if (a <= k_max) {
+                const double inv = __longlong_as_double((long long)(1023 - e - a) << 52);    // 2^-(e+a)
+                const double step = __longlong_as_double((long long)(1023 + e + a) << 52);   // 2^(e+a)
+                const double qv = fmin(fmax(rint(__dmul_rn(xv, inv)), lo), hi);
+                const double d = __dsub_rn(xv, __dmul_rn(qv, step));
+                err[a] = __dadd_rn(err[a], __dmul_rn(d, d));
             }
         }
-        q[u] = make_uint4(out[0], out[1], out[2], out[3]);
     }
+    int best = 0;
+    double best_err = err[0];
+#pragma unroll
+    for (int a = 1; a < 5; ++a)
+        if (a <= k_max && err[a] < best_err) { best = a; best_err = err[a]; }
+    alpha_out[k] = (uint8_t)best;
 }
 
 // ---- token selection: rank every score, keep rank < n_keep, then compact the flags ------
@@ -349,20 +407,21 @@ gather_rows_kernel(const uint4* __restrict__ x, int vec_per_row, const int32_t* 
 
 cudaError_t launch_quantize(const __half* x, int M, int K, const int32_t* row_idx, int bits,
                             int scale_mode, int clip_shift_or_exp, Control* ctl, int8_t* q,
-                            int32_t* scale_exp_out, const DeviceInfo& dev, cudaStream_t stream) {
+                            int32_t* scale_exp_out, const DeviceInfo& dev, cudaStream_t stream,
+                            const uint8_t* alpha, int k_max) {
     (void)dev;
     const int vec_per_row = K / 16;
     const size_t total = (size_t)M * vec_per_row;
     const size_t blocks = (total + kQuantThreads - 1) / kQuantThreads;
     quantize_kernel<<<(unsigned int)blocks, kQuantThreads, 0, stream>>>(
         reinterpret_cast<const uint4*>(x), M, vec_per_row, row_idx, bits, scale_mode, clip_shift_or_exp,
-        ctl, reinterpret_cast<uint4*>(q), scale_exp_out);
+        ctl, reinterpret_cast<uint4*>(q), scale_exp_out, reinterpret_cast<const uint4*>(alpha), k_max);
     return cudaGetLastError();
 }
 
 cudaError_t launch_quantize_fused(const __half* x, int M, int K, const int32_t* row_idx, int bits, int clip_shift,
                                   Control* ctl, int8_t* q, int32_t* scale_exp_out, const DeviceInfo& dev,
-                                  cudaStream_t stream) {
+                                  cudaStream_t stream, const uint8_t* alpha, int k_max) {
     int units_per_row = K / 16;
     const size_t total = (size_t)M * units_per_row;
     size_t grid = (total + kFusedThreads - 1) / kFusedThreads;
@@ -382,21 +441,37 @@ cudaError_t launch_quantize_fused(const __half* x, int M, int K, const int32_t* 
     }
     const uint4* xp = reinterpret_cast<const uint4*>(x);
     uint4* qp = reinterpret_cast<uint4*>(q);
+    const uint4* ap = reinterpret_cast<const uint4*>(alpha);
     void* args[] = {&xp, &M, &units_per_row, &row_idx, &bits, &clip_shift, &ctl, &qp, &scale_exp_out, &cache_units,
-                    &units_per_cta};
+                    &units_per_cta, &ap, &k_max};
     // cooperative: the launch fails rather than start a grid whose CTAs could not all be resident
     return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(quantize_fused_kernel), dim3((unsigned int)grid),
                                        dim3(kFusedThreads), args, smem_bytes, stream);
+}
+
+cudaError_t launch_trip_calibrate(const __half* x, int M, int K, const int32_t* row_idx, int bits, int k_max,
+                                  Control* ctl, uint8_t* alpha_out, int32_t* scale_exp_out, const DeviceInfo& dev,
+                                  cudaStream_t stream) {
+    const size_t total = (size_t)M * K;
+    size_t blocks = (total + 255) / 256;
+    const size_t cap = (size_t)dev.sm_count * 8;
+    if (blocks > cap) blocks = cap;
+    absmax_plain_kernel<<<(unsigned int)blocks, 256, 0, stream>>>(x, M, K, row_idx, ctl);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    trip_calibrate_kernel<<<(K + 127) / 128, 128, 0, stream>>>(x, M, K, row_idx, bits, k_max, ctl, alpha_out,
+                                                               scale_exp_out);
+    return cudaGetLastError();
 }
 
 bool quantize_small_fits(int M, int K) { return (size_t)M * (size_t)K <= kSmallMaxElems; }
 
 cudaError_t launch_quantize_small(const __half* x, int M, int K, const int32_t* row_idx, int bits, int scale_mode,
                                   int clip_shift_or_exp, Control* ctl, int8_t* q, int32_t* scale_exp_out,
-                                  cudaStream_t stream) {
+                                  cudaStream_t stream, const uint8_t* alpha, int k_max) {
     quantize_small_kernel<<<kSmallCtas, kSmallThreads, 0, stream>>>(
         reinterpret_cast<const uint4*>(x), M, K / 8, row_idx, bits, scale_mode, clip_shift_or_exp, ctl,
-        reinterpret_cast<uint2*>(q), scale_exp_out);
+        reinterpret_cast<uint2*>(q), scale_exp_out, reinterpret_cast<const uint2*>(alpha), k_max);
     return cudaGetLastError();
 }
 
