@@ -284,8 +284,30 @@ def bench_w4a4(h, reps=30):
             h.aq_linear_w4a4(x, p, sc, s.N, wl.group_size, clip_shift_or_exp=wl.clip_shift, y=y, workspace=ws)
     ms = _event_ms(step, reps)
     ops = sum(2.0 * M * s.K * s.N for s in wl.shapes)
-    return {"workload": wl.name, "ms_per_step": ms, "TOPS": ops / (ms * 1e-3) / 1e12,
-            "note": "int4 codes travel in int8 containers: the tensor cores have no 4-bit integer kind"}
+    out = {"workload": wl.name, "ms_per_step": ms, "TOPS": ops / (ms * 1e-3) / 1e12,
+           "note": "int4 codes travel in int8 containers: the tensor cores have no 4-bit integer kind"}
+    # the same step with per-channel TRIP factors (Eq. 5-8) found on these activations, k_max = 4
+    k_max = 4
+    alphas, cal_us, mse = [], [], []
+    for x, p, sc, s, ws, y in layers:
+        alphas.append(h.aq_trip_calibrate(x, k_max)[0])
+        cal_us.append(_event_ms(lambda: h.aq_trip_calibrate(x, k_max), 5) * 1e3)
+        # reconstruction error of the activations (measurement only): plain 4-bit codes at this
+        # workload's clip_shift against codes with factors
+        xf = x.float()
+        q0, e0 = h.aq_quantize_act(x, 4, clip_shift_or_exp=wl.clip_shift)
+        q1, e1 = h.aq_quantize_act_trip(x, alphas[-1], k_max)
+        err0 = (xf - q0.float() * 2.0 ** int(e0.item())).square().mean().item()
+        err1 = (xf - q1.float() * 2.0 ** int(e1.item())).square().mean().item()
+        mse.append({"plain": err0, "trip": err1})
+    def step_trip():
+        for (x, p, sc, s, ws, y), al in zip(layers, alphas):
+            h.aq_linear_w4a4_trip(x, p, sc, s.N, wl.group_size, al, k_max, y=y, workspace=ws)
+    ms_t = _event_ms(step_trip, reps)
+    out["trip"] = {"k_max": k_max, "ms_per_step": ms_t, "TOPS": ops / (ms_t * 1e-3) / 1e12,
+                   "calibrate_us": cal_us, "activation_mse": mse,
+                   "channels_with_factor": [int((a > 0).sum().item()) for a in alphas]}
+    return out
 
 
 def bench_pruned(h, reps=10):
