@@ -44,6 +44,35 @@ __device__ __forceinline__ void quantize8_half2(const uint4& d, __half2 inv2, __
     w1 = __byte_perm(r[2], r[3], 0x6420);
 }
 
+// The half2 route with TRIP factors (4-bit codes): lane k multiplies by 2^-(e + alpha_k), built from
+// the factor byte as a half bit pattern (exponent field 15 - e - alpha_k, which must be 1..30),
+// clamps to [-8, 7], rounds by adding and removing 1536, multiplies by 2^alpha_k (exact, |result|
+// <= 128) and adds 1536 again so that the value's two's-complement byte sits in the low 8 bits.
+__device__ __forceinline__ void quantize8_half2_trip(const uint4& d, int e, const uint2& al, uint32_t& w0, uint32_t& w1) {
+    const __half2* h = reinterpret_cast<const __half2*>(&d);
+    const __half2 bias = __floats2half2_rn(1536.0f, 1536.0f);
+    const __half2 lo2 = __floats2half2_rn(-8.0f, -8.0f), hi2 = __floats2half2_rn(7.0f, 7.0f);
+    const uint32_t inv_base = (uint32_t)(15 - e) * 0x04000400u;              // both lanes: (15 - e) << 10
+    const uint32_t one_base = 15u * 0x04000400u;                            // 1.0 in both lanes
+    uint32_t r[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t word = i < 2 ? al.x : al.y;
+        const uint32_t a0 = (word >> (16 * (i & 1))) & 0xFFu, a1 = (word >> (16 * (i & 1) + 8)) & 0xFFu;
+        const uint32_t apair = (a0 | (a1 << 16)) << 10;
+        uint32_t ib = inv_base - apair, sb = one_base + apair;
+        __half2 t = __hmul2(h[i], *reinterpret_cast<__half2*>(&ib));
+        const uint32_t ok = __heq2_mask(t, t);                              // clears NaN lanes
+        uint32_t tb = *reinterpret_cast<uint32_t*>(&t) & ok;
+        t = *reinterpret_cast<__half2*>(&tb);
+        t = __hsub2(__hadd2(__hmin2(__hmax2(t, lo2), hi2), bias), bias);    // the 4-bit code, rounded to nearest even
+        t = __hadd2(__hmul2(t, *reinterpret_cast<__half2*>(&sb)), bias);
+        r[i] = *reinterpret_cast<uint32_t*>(&t);
+    }
+    w0 = __byte_perm(r[0], r[1], 0x6420);
+    w1 = __byte_perm(r[2], r[3], 0x6420);
+}
+
 // 8 halves -> 8 values in fp32 arithmetic. With TRIP factors (Eq. 5 with a per-channel alpha,
 // `al` = the 8 factor bytes of these channels) channel k uses the step 2^(e + alpha_k) and its code
 // is stored shifted left by alpha_k, the form in which the factor enters the integer product.
@@ -248,6 +277,7 @@ quantize_fused_kernel(const uint4* __restrict__ x, int M, int units_per_row /* 1
     const float inv = __int_as_float((127 - e) << 23);      // 2^-e, |e| <= 40
     const float lo = -(float)(1 << (bits - 1)), hi = (float)((1 << (bits - 1)) - 1);
     const bool fast = alpha == nullptr && e >= -14 && e <= 14;   // 2^-e is a normal half
+    const bool fast_trip = alpha != nullptr && bits == 4 && e >= -14 && e <= 10;   // so is 2^-(e + alpha), alpha <= 4
     const __half2 inv2 = __float2half2_rn(fast ? inv : 1.0f), lo2 = __float2half2_rn(lo), hi2 = __float2half2_rn(hi);
 #pragma unroll 2
     for (size_t u = u0 + threadIdx.x; u < u1; u += kFusedThreads) {
@@ -264,6 +294,11 @@ quantize_fused_kernel(const uint4* __restrict__ x, int M, int units_per_row /* 1
         if (fast) {
             quantize8_half2(d0, inv2, lo2, hi2, out[0], out[1]);
             quantize8_half2(d1, inv2, lo2, hi2, out[2], out[3]);
+            q[u] = make_uint4(out[0], out[1], out[2], out[3]);
+        } else if (fast_trip) {
+            const uint4 al = __ldg(alpha + (size_t)(u % units_per_row));
+            quantize8_half2_trip(d0, e, make_uint2(al.x, al.y), out[0], out[1]);
+            quantize8_half2_trip(d1, e, make_uint2(al.z, al.w), out[2], out[3]);
             q[u] = make_uint4(out[0], out[1], out[2], out[3]);
         } else {
             uint4 al;

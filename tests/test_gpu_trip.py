@@ -51,6 +51,12 @@ def test_quantize_act_trip_matches_checker(M, K):
             e_ref = oracle.trip_base_exponent(x, 4, k_max) - clip
             assert int(e.item()) == e_ref
             assert np.array_equal(q.cpu().numpy(), oracle.quantize_act_trip(x, 4, e_ref, alpha))
+        # magnitudes whose exponent is outside the half-precision route
+        xs = (np.nan_to_num(x.astype(np.float32), nan=0.0, posinf=0.0, neginf=0.0) * np.float32(2.0 ** -21)).astype(np.float16)
+        q, e = h.aq_quantize_act_trip(dev(xs), dev(alpha), k_max)
+        e_ref = oracle.trip_base_exponent(xs, 4, k_max)
+        assert int(e.item()) == e_ref and e_ref < -14
+        assert np.array_equal(q.cpu().numpy(), oracle.quantize_act_trip(xs, 4, e_ref, alpha))
         rows = g.integers(0, M, size=max(1, M // 2)).astype(np.int32)
         q, e = h.aq_quantize_act_trip(dev(x), dev(alpha), k_max, binding.AQ_SCALE_STATIC, -1, row_idx=dev(rows))
         assert int(e.item()) == -1
