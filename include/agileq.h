@@ -163,6 +163,15 @@ int aq_linear_w4a4_trip(aq_handle_t h, const void* x_fp16, int M, int K, const v
                         int scale_mode, int clip_shift_or_exp, const int32_t* row_idx, void* y_fp16,
                         int32_t* acc_dump, void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---- progressive pruning schedule (paper Eq. 9; host only, no GPU work)
+ * With pruning at m layers and the ratio beta of tokens to be gone after the last of them, every
+ * pruning layer drops the fraction gamma = 1 - (1 - beta)^(1/m) of what reaches it. Writes
+ * n_keep_out[i], i = 0..m-1, the tokens kept after pruning layer i, starting from M tokens:
+ * n_keep_out[i] = ceil(n_keep_out[i-1] * (1 - gamma)) (at least 1), and *gamma_out (may be NULL).
+ * Each n_keep_out[i] is the n_keep argument of aq_token_select at that layer.
+ * Returns AQ_ERR_INVALID_ARG unless M >= 1, m >= 1, 0 <= beta < 1. */
+int aq_prune_schedule(int M, double beta, int m, int32_t* n_keep_out, double* gamma_out);
+
 /* ---- host-buffer convenience (SYNCHRONIZES the stream before returning)
  * x_host fp16 [M,K] and y_host fp16 [M,N] are HOST pointers (pinned memory gives the best
  * rate). Copies x to the device scratch, runs the layer with `bits` (8 or 4), copies y

@@ -74,6 +74,7 @@ def load():
     L.aq_linear_w4a8.argtypes = lin
     L.aq_linear_w4a4.argtypes = lin
     L.aq_gemm_w4.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, vp, vp, vp, vp, sz, vp]
+    L.aq_prune_schedule.argtypes = [i32, C.c_double, i32, vp, vp]
     L.aq_trip_calibrate.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
     L.aq_quantize_act_trip.argtypes = [vp, vp, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
     L.aq_linear_w4a4_trip.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
@@ -109,6 +110,15 @@ def aq_packed_w4_bytes(N: int, K: int) -> int:
 
 def aq_scales_bytes(N: int, K: int, group_size: int) -> int:
     return load().aq_scales_bytes(N, K, group_size)
+
+
+def aq_prune_schedule(M: int, beta: float, m: int):
+    """Eq. 9: (tokens kept after each of the m pruning layers, gamma). Host only."""
+    out = (C.c_int32 * m)()
+    gamma = C.c_double(0.0)
+    _check(load().aq_prune_schedule(M, beta, m, C.cast(out, C.c_void_p), C.cast(C.byref(gamma), C.c_void_p)),
+           "aq_prune_schedule")
+    return list(out), gamma.value
 
 
 def aq_workspace_bytes(M: int, K: int, N: int, group_size: int) -> int:

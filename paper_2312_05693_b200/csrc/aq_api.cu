@@ -2,6 +2,8 @@
 // step of the layer runs in the kernels of the sibling files; nothing here computes.
 #include <new>
 
+#include <math.h>
+
 #include "aq_common.cuh"
 
 struct aq_context {
@@ -352,6 +354,19 @@ int aq_token_compact(aq_handle_t h, const void* x_fp16, int M, int K, const int3
                                                static_cast<__half*>(x_out), h->dev,
                                                static_cast<cudaStream_t>(stream));
     return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
+int aq_prune_schedule(int M, double beta, int m, int32_t* n_keep_out, double* gamma_out) {
+    if (M < 1 || m < 1 || !(beta >= 0.0) || !(beta < 1.0) || !n_keep_out) return AQ_ERR_INVALID_ARG;
+    const double gamma = 1.0 - pow(1.0 - beta, 1.0 / (double)m);       // Eq. 9
+    if (gamma_out) *gamma_out = gamma;
+    int n = M;
+    for (int i = 0; i < m; ++i) {
+        const double kept = ceil((double)n * (1.0 - gamma) - 1e-9);       // the tolerance keeps exact products exact
+        n = kept < 1.0 ? 1 : (int)kept;
+        n_keep_out[i] = n;
+    }
+    return AQ_OK;
 }
 
 size_t aq_linear_host_scratch_bytes(int M, int K, int N, int group_size) {

@@ -2,6 +2,8 @@
 No kernel runs here (no GPU needed)."""
 import ctypes as C
 
+import pytest
+
 from paper_2312_05693_b200 import binding, build
 
 
@@ -38,3 +40,18 @@ def test_null_handle_is_rejected_without_touching_a_device():
     assert L.aq_set_kernel(None, 0) == binding.AQ_ERR_INVALID_ARG
     assert L.aq_pack_w4(None, None, 128, 128, 0, None, None, None) == binding.AQ_ERR_INVALID_ARG
     assert L.aq_create(None, 0) == binding.AQ_ERR_INVALID_ARG
+
+
+def test_prune_schedule_host_function():
+    # Eq. 9 (host only: runs without a GPU). After m layers about (1 - beta) of the tokens are left.
+    import oracle
+    keep, gamma = binding.aq_prune_schedule(4096, 0.4, 4)
+    assert abs(gamma - oracle.progressive_ratio(0.4, 4)) < 1e-15
+    assert len(keep) == 4 and all(a >= b for a, b in zip([4096] + keep, keep))
+    assert abs(keep[-1] - 4096 * 0.6) <= 4                     # ceil at every layer adds at most one token each
+    assert binding.aq_prune_schedule(4096, 0.75, 2)[0] == [2048, 1024]       # gamma = 1/2 exactly
+    assert binding.aq_prune_schedule(100, 0.0, 3)[0] == [100, 100, 100]
+    assert binding.aq_prune_schedule(3, 0.99, 5)[0][-1] >= 1
+    for bad in [(0, 0.5, 2), (10, 1.0, 2), (10, -0.1, 2), (10, 0.5, 0)]:
+        with pytest.raises(binding.AgileqError):
+            binding.aq_prune_schedule(*bad)
