@@ -365,6 +365,75 @@ long long orc_linear(const uint16_t* x, int K, const int32_t* row_idx, int M, in
     return ovf;
 }
 
+// ---------------------------------------------------------------------------
+// The unsigned quantizer with a zero point, exactly the form of Eq. 2 / Eq. 5-7 (alpha = 0):
+//     q = CLIP( round(x / s) + zp, 0, 2^b - 1 ),   zp = CLIP( round(-min / s), 0, 2^b - 1 ),
+// with the scale read as a power of two like everywhere else in this file: s = 2^e, e the smallest
+// integer with (2^b - 1) * 2^e >= max - min (Eq. 6 with alpha = 0). Readings: the range is widened to
+// contain 0 (min' = min(min, 0), max' = max(max, 0)), so that zp is a code; NaN is ignored by min and
+// max and maps to the code zp (value 0); +-Inf count as +-65504. Everything is exact in binary64.
+// ---------------------------------------------------------------------------
+void orc_asym_params(const uint16_t* x, int K, const int32_t* row_idx, int M, int bits, int* e_out, int* zp_out) {
+    double lo = 0.0, hi = 0.0;
+    for (int m = 0; m < M; ++m) {
+        const uint16_t* row = x + (size_t)(row_idx ? row_idx[m] : m) * K;
+        for (int k = 0; k < K; ++k) {
+            double v = (double)orc_half_to_float(row[k]);
+            if (std::isnan(v)) continue;
+            if (std::isinf(v)) v = v > 0 ? 65504.0 : -65504.0;
+            if (v < lo) lo = v;
+            if (v > hi) hi = v;
+        }
+    }
+    const double range = hi - lo, qr = (double)((1 << bits) - 1);
+    int e = 0;
+    if (range > 0.0) {
+        while (std::ldexp(qr, e) < range) ++e;
+        while (std::ldexp(qr, e - 1) >= range) --e;
+    }
+    const double zp = std::min(std::max(std::nearbyint(std::ldexp(-lo, -e)), 0.0), qr);
+    *e_out = e;
+    *zp_out = (int)zp;
+}
+
+// Unsigned codes of Eq. 2 for given e and zp, one per byte.
+void orc_quantize_act_asym(const uint16_t* x, int K, const int32_t* row_idx, int M, int bits, int e, int zp,
+                           uint8_t* q) {
+    const double qr = (double)((1 << bits) - 1);
+    for (int m = 0; m < M; ++m) {
+        const uint16_t* row = x + (size_t)(row_idx ? row_idx[m] : m) * K;
+        for (int k = 0; k < K; ++k) {
+            const double v = (double)orc_half_to_float(row[k]);
+            double r = (double)zp;
+            if (!std::isnan(v)) r = std::min(std::max(std::nearbyint(std::ldexp(v, -e)) + (double)zp, 0.0), qr);
+            q[(size_t)m * K + k] = (uint8_t)r;
+        }
+    }
+}
+
+// The layer with such codes: y[m][n] = fp16( 2^e * sum_g s_w[n][g] * sum_{k in g} (q[m][k] - zp) * c[n][k] ),
+// integer sums exact (int64), the rest in binary64 with one rounding to fp16. acc (may be NULL):
+// the integer sums [M][N][G].
+void orc_linear_asym(const uint8_t* q, int zp, const int8_t* c, const uint16_t* scales, int e, int M, int N, int K,
+                     int group, long long* acc /*[M][N][G] or NULL*/, uint16_t* y) {
+    const int gs = group > 0 ? group : K;
+    const int G = K / gs;
+#pragma omp parallel for schedule(static)
+    for (int m = 0; m < M; ++m) {
+        for (int n = 0; n < N; ++n) {
+            double s = 0.0;
+            for (int g = 0; g < G; ++g) {
+                long long a = 0;
+                for (int k = g * gs; k < (g + 1) * gs; ++k)
+                    a += (long long)((int)q[(size_t)m * K + k] - zp) * (long long)c[(size_t)n * K + k];
+                if (acc) acc[((size_t)m * N + n) * G + g] = a;
+                s += (double)a * (double)orc_half_to_float(scales[(size_t)n * G + g]);
+            }
+            y[(size_t)m * N + n] = orc_double_to_half(std::ldexp(s, e));
+        }
+    }
+}
+
 // Progressive pruning ratio, Eq. 9: gamma = 1 - (1 - beta)^(1/m).
 double orc_progressive_ratio(double beta, int m) { return 1.0 - std::pow(1.0 - beta, 1.0 / m); }
 

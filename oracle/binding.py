@@ -205,6 +205,42 @@ def trip_base_exponent(x: np.ndarray, bits: int, k_max: int, row_idx: Optional[n
     return layer_exponent(x, bits, row_idx) - k_max
 
 
+def asym_params(x: np.ndarray, bits: int, row_idx: Optional[np.ndarray] = None) -> Tuple[int, int]:
+    """(e, zp) of the unsigned quantizer of Eq. 2 / Eq. 5-7 with a power-of-two scale."""
+    M_in, K = x.shape
+    ri = None if row_idx is None else _c(row_idx, np.int32)
+    M = M_in if ri is None else ri.shape[0]
+    e, zp = C.c_int(0), C.c_int(0)
+    lib().orc_asym_params(_p(_half_bits(x)), K, _p(ri), M, bits, C.byref(e), C.byref(zp))
+    return e.value, zp.value
+
+
+def quantize_act_asym(x: np.ndarray, bits: int, e: int, zp: int, row_idx: Optional[np.ndarray] = None) -> np.ndarray:
+    """Unsigned codes CLIP(round(x / 2^e) + zp, 0, 2^b - 1)."""
+    M_in, K = x.shape
+    ri = None if row_idx is None else _c(row_idx, np.int32)
+    M = M_in if ri is None else ri.shape[0]
+    q = np.empty((M, K), np.uint8)
+    lib().orc_quantize_act_asym(_p(_half_bits(x)), K, _p(ri), M, bits, e, zp, _p(q))
+    return q
+
+
+def linear_asym(q: np.ndarray, zp: int, c: np.ndarray, scales: np.ndarray, e: int, group: int):
+    """(int64 sums [M,N,G] of (q - zp) * c, fp16 y [M,N])."""
+    q = _c(q, np.uint8)
+    c = _c(c, np.int8)
+    M, K = q.shape
+    N = c.shape[0]
+    G = num_groups(K, group)
+    scales = np.ascontiguousarray(scales)
+    assert scales.shape == (N, G) and scales.dtype == np.float16
+    acc = np.empty((M, N, G), np.int64)
+    y = np.empty((M, N), np.float16)
+    lib().orc_linear_asym(_p(q), zp, _p(c), _p(scales.view(np.uint16)), e, M, N, K, group, _p(acc),
+                          _p(y.view(np.uint16)))
+    return acc, y
+
+
 def int_gemm(q: np.ndarray, c: np.ndarray, group: int) -> np.ndarray:
     """int8 [M,K] x int8 [N,K] -> int32 [M,N,G]; raises if an int32 sum overflowed."""
     q = _c(q, np.int8)

@@ -508,3 +508,65 @@ def test_trip_base_exponent_reaches_the_layer_maximum():
         alpha = np.full(128, k_max, np.uint8)
         v = oracle.quantize_act_trip(x, 4, e, alpha)
         assert np.array_equal(v.astype(np.int64) >> k_max, oracle.quantize_act(x, 4, e + k_max).astype(np.int64))
+
+
+# ------------------------------------------- unsigned quantizer with a zero point (Eq. 2, Eq. 5-7)
+def test_asym_hand_worked_table():
+    for line in open(os.path.join(GOLDEN, "asym_hand_worked.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        f = line.split()
+        if f[0] == "P":
+            bits, lo, hi, e, zp = int(f[1]), float(f[2]), float(f[3]), int(f[4]), int(f[5])
+            x = np.array([[lo, hi, np.nan, 0.0]], np.float16)          # NaN is ignored
+            assert oracle.asym_params(x, bits) == (e, zp), line
+        else:
+            bits, e, zp, xv, code = int(f[1]), int(f[2]), int(f[3]), float(f[4]), int(f[5])
+            got = oracle.quantize_act_asym(np.array([[xv]], np.float16), bits, e, zp)
+            assert int(got[0, 0]) == code, line
+
+
+def test_asym_quantizer_invariants_and_reduction_to_the_signed_one():
+    g = np.random.Generator(np.random.Philox(key=808))
+    for bits in (8, 4):
+        x = (g.standard_normal((50, 64)) * 3 + 2.0).astype(np.float16)       # not centred: zp away from the middle
+        e, zp = oracle.asym_params(x, bits)
+        qr = (1 << bits) - 1
+        xf = x.astype(np.float64)
+        lo, hi = min(xf.min(), 0.0), max(xf.max(), 0.0)
+        assert qr * 2.0 ** e >= hi - lo > qr * 2.0 ** (e - 1)                # smallest power of two that covers the range
+        assert 0 <= zp <= qr and abs(zp - (-lo) / 2.0 ** e) <= 0.5
+        q = oracle.quantize_act_asym(x, bits, e, zp).astype(np.int64)
+        assert q.min() >= 0 and q.max() <= qr
+        deq = (q - zp) * 2.0 ** e
+        inside = (xf >= (0 - zp) * 2.0 ** e) & (xf <= (qr - zp) * 2.0 ** e)
+        assert np.all(np.abs(xf - deq)[inside] <= 2.0 ** e / 2 + 1e-12)
+        assert np.all(q[xf > (qr - zp) * 2.0 ** e] == qr)
+        # with zp in the middle of the code range this is the signed quantizer of Eq. 1 moved by 2^(b-1)
+        half = 1 << (bits - 1)
+        for ee in (e, e - 2):
+            assert np.array_equal(oracle.quantize_act_asym(x, bits, ee, half).astype(np.int64) - half,
+                                  oracle.quantize_act(x, bits, ee).astype(np.int64))
+
+
+def test_asym_layer_brute_force_and_zero_point_identity():
+    g = np.random.Generator(np.random.Philox(key=909))
+    M, K, N = 5, 256, 6
+    q = g.integers(0, 256, size=(M, K)).astype(np.uint8)
+    c = g.integers(-8, 8, size=(N, K)).astype(np.int8)
+    zp, e = 77, -3
+    for group in (0, 128):
+        G = 1 if group == 0 else K // 128
+        sc = (g.random((N, G)) * 0.01 + 0.001).astype(np.float16)
+        acc, y = oracle.linear_asym(q, zp, c, sc, e, group)
+        ref = np.einsum("mgk,ngk->mng", q.astype(np.int64).reshape(M, G, K // G) - zp,
+                        c.astype(np.int64).reshape(N, G, K // G))
+        assert np.array_equal(acc, ref)
+        # the form the integer product uses: signed codes q - 128 and one correction per (channel, group)
+        qs = (q.astype(np.int64) - 128).astype(np.int8)
+        raw = oracle.int_gemm(qs, c, group).reshape(M, N, G).astype(np.int64)
+        colsum = c.astype(np.int64).reshape(N, G, K // G).sum(axis=2)
+        assert np.array_equal(raw - (zp - 128) * colsum[None, :, :], ref)
+        # one rounding of the exact value
+        exact = (ref.astype(np.float64) * sc.astype(np.float64)[None, :, :]).sum(axis=2) * 2.0 ** e
+        assert np.array_equal(y, exact.astype(np.float16))
