@@ -163,6 +163,30 @@ int aq_linear_w4a4_trip(aq_handle_t h, const void* x_fp16, int M, int K, const v
                         int scale_mode, int clip_shift_or_exp, const int32_t* row_idx, void* y_fp16,
                         int32_t* acc_dump, void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---- activations with a zero point (paper Eq. 2, Eq. 5-7 with alpha = 0)
+ * Unsigned codes q = CLIP(round(x / s) + zp, 0, 2^b - 1), zp = CLIP(round(-min / s), 0, 2^b - 1), with
+ * the scale a power of two as everywhere here: s = 2^e, e the smallest integer with
+ * (2^b - 1) * 2^e >= max - min over the (kept) activations; the range is widened to contain 0. NaN
+ * is ignored by min / max and gets the code zp (value 0); +-Inf count as +-65504. The codes are
+ * stored as q - 2^(b-1) in int8, and the layer is
+ *   y[m,n] = fp16( 2^e * sum_g s_w[n,g] * sum_{k in g} (q[m,k] - zp) * c[n,k] ),
+ * computed as the signed integer product plus the per-channel term -(zp - 2^(b-1)) * r[n], with
+ * r[n] = sum_g s_w[n,g] * sum_{k in g} c[n,k] made once per weight matrix by aq_weight_offsets
+ * (float [N] on the device). acc_dump, when given, receives the signed product
+ * sum_{k in g} (q[m,k] - 2^(b-1)) * c[n,k] (the zero-point term is not in it). The scale is always
+ * dynamic. */
+int aq_weight_offsets(aq_handle_t h, const void* w_packed, const void* w_scales, int N, int K, int group_size,
+                      float* r_out, void* stream);
+int aq_quantize_act_asym(aq_handle_t h, const void* x_fp16, int M, int K, int bits, const int32_t* row_idx,
+                         int8_t* q, int32_t* scale_exp_out, int32_t* zero_point_out, void* workspace,
+                         size_t workspace_bytes, void* stream);
+int aq_linear_w4a8_asym(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed, const void* w_scales,
+                        const float* w_offsets, int N, int group_size, const int32_t* row_idx, void* y_fp16,
+                        int32_t* acc_dump, void* workspace, size_t workspace_bytes, void* stream);
+int aq_linear_w4a4_asym(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed, const void* w_scales,
+                        const float* w_offsets, int N, int group_size, const int32_t* row_idx, void* y_fp16,
+                        int32_t* acc_dump, void* workspace, size_t workspace_bytes, void* stream);
+
 /* ---- progressive pruning schedule (paper Eq. 9; host only, no GPU work)
  * With pruning at m layers and the ratio beta of tokens to be gone after the last of them, every
  * pruning layer drops the fraction gamma = 1 - (1 - beta)^(1/m) of what reaches it. Writes

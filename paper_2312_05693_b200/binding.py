@@ -74,6 +74,11 @@ def load():
     L.aq_linear_w4a8.argtypes = lin
     L.aq_linear_w4a4.argtypes = lin
     L.aq_gemm_w4.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, vp, vp, vp, vp, sz, vp]
+    L.aq_weight_offsets.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp]
+    L.aq_quantize_act_asym.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
+    lin_asym = [vp, vp, i32, i32, vp, vp, vp, i32, i32, vp, vp, vp, vp, sz, vp]
+    L.aq_linear_w4a8_asym.argtypes = lin_asym
+    L.aq_linear_w4a4_asym.argtypes = lin_asym
     L.aq_prune_schedule.argtypes = [i32, C.c_double, i32, vp, vp]
     L.aq_trip_calibrate.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
     L.aq_quantize_act_trip.argtypes = [vp, vp, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
@@ -218,6 +223,39 @@ class Handle:
                        clip_shift_or_exp=0, row_idx=None, y=None, acc_dump=None, workspace=None):
         return self._linear(load().aq_linear_w4a4, "aq_linear_w4a4", x, packed, scales, N, group_size,
                             scale_mode, clip_shift_or_exp, row_idx, y, acc_dump, workspace)
+
+    # ---- activations with a zero point (Eq. 2, Eq. 5-7)
+    def aq_weight_offsets(self, packed: torch.Tensor, scales: torch.Tensor, N: int, K: int, group_size: int
+                          ) -> torch.Tensor:
+        r = torch.empty(N, dtype=torch.float32, device=packed.device)
+        _check(load().aq_weight_offsets(self._h, _ptr(packed), _ptr(scales), N, K, group_size, _ptr(r), _stream()),
+               "aq_weight_offsets")
+        return r
+
+    def aq_quantize_act_asym(self, x: torch.Tensor, bits: int, row_idx: Optional[torch.Tensor] = None):
+        """(int8 codes q - 2^(b-1), e, zp)."""
+        M_in, K = x.shape
+        M = M_in if row_idx is None else row_idx.shape[0]
+        q = torch.empty((M, K), dtype=torch.int8, device=x.device)
+        e = torch.empty(1, dtype=torch.int32, device=x.device)
+        zp = torch.empty(1, dtype=torch.int32, device=x.device)
+        ws = torch.empty(256, dtype=torch.uint8, device=x.device)
+        _check(load().aq_quantize_act_asym(self._h, _ptr(x), M, K, bits, _ptr(row_idx), _ptr(q), _ptr(e), _ptr(zp),
+                                           _ptr(ws), ws.numel(), _stream()), "aq_quantize_act_asym")
+        return q, e, zp
+
+    def aq_linear_asym(self, bits, x, packed, scales, w_offsets, N, group_size, row_idx=None, y=None, acc_dump=None,
+                       workspace=None):
+        M_in, K = x.shape
+        M = M_in if row_idx is None else row_idx.shape[0]
+        if y is None:
+            y = torch.empty((M, N), dtype=torch.float16, device=x.device)
+        if workspace is None:
+            workspace = self.alloc_workspace(M, K, N, group_size)
+        fn = load().aq_linear_w4a8_asym if bits == 8 else load().aq_linear_w4a4_asym
+        _check(fn(self._h, _ptr(x), M, K, _ptr(packed), _ptr(scales), _ptr(w_offsets), N, group_size, _ptr(row_idx),
+                  _ptr(y), _ptr(acc_dump), _ptr(workspace), workspace.numel(), _stream()), "aq_linear_asym")
+        return y
 
     # ---- per-channel TRIP factors (Eq. 5-8)
     def aq_trip_calibrate(self, x: torch.Tensor, k_max: int, row_idx: Optional[torch.Tensor] = None

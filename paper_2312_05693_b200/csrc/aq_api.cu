@@ -37,10 +37,12 @@ struct Workspace {
     int8_t* codes;
     void* scratch;
     size_t scratch_bytes;
+    float* chan_offset;
 };
 
-size_t workspace_bytes(int M, int K) {
-    return sizeof(Control) + up256((size_t)M * K) + up256((size_t)M);
+// [control block][codes M*K][kernel scratch, M bytes][per-channel offsets of the zero-point variant, N floats]
+size_t workspace_bytes(int M, int K, int N) {
+    return sizeof(Control) + up256((size_t)M * K) + up256((size_t)M) + up256((size_t)N * sizeof(float));
 }
 
 Workspace carve(void* ws, int M, int K) {
@@ -50,6 +52,7 @@ Workspace carve(void* ws, int M, int K) {
     w.codes = reinterpret_cast<int8_t*>(b + sizeof(Control));
     w.scratch = b + sizeof(Control) + up256((size_t)M * K);
     w.scratch_bytes = up256((size_t)M);
+    w.chan_offset = reinterpret_cast<float*>(b + sizeof(Control) + up256((size_t)M * K) + up256((size_t)M));
     return w;
 }
 
@@ -89,14 +92,14 @@ bool trip_args_ok(const uint8_t* alpha, int k_max) { return alpha && k_max >= 0 
 int linear_impl(aq_handle_t h, int bits, const void* x, int M, int K, const void* w_packed,
                 const void* w_scales, int N, int group, int scale_mode, int clip_shift_or_exp,
                 const int32_t* row_idx, void* y, int32_t* acc_dump, void* workspace, size_t workspace_bytes_,
-                void* stream_, const uint8_t* alpha = nullptr, int k_max = 0) {
+                void* stream_, const uint8_t* alpha = nullptr, int k_max = 0, const float* w_offsets = nullptr) {
     if (!h || !x || !w_packed || !w_scales || !y) return AQ_ERR_INVALID_ARG;
     if (scale_mode != AQ_SCALE_DYNAMIC && scale_mode != AQ_SCALE_STATIC) return AQ_ERR_INVALID_ARG;
     if (scale_mode == AQ_SCALE_DYNAMIC && (clip_shift_or_exp < 0 || clip_shift_or_exp > 16)) return AQ_ERR_INVALID_ARG;
     if (scale_mode == AQ_SCALE_STATIC && (clip_shift_or_exp < -40 || clip_shift_or_exp > 40)) return AQ_ERR_INVALID_ARG;
     const int s = check_shape(M, K, N, group);
     if (s != AQ_OK) return s;
-    if (!workspace || workspace_bytes_ < workspace_bytes(M, K)) return AQ_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes_ < workspace_bytes(M, K, N)) return AQ_ERR_WORKSPACE;
     if (!aligned(x, 16) || !aligned(w_packed, 16) || !aligned(w_scales, 2) || !aligned(y, 2) ||
         !aligned(workspace, 256) || (acc_dump && !aligned(acc_dump, 4)) || (row_idx && !aligned(row_idx, 4)))
         return AQ_ERR_ALIGNMENT;
@@ -104,8 +107,18 @@ int linear_impl(aq_handle_t h, int bits, const void* x, int M, int K, const void
     const Workspace w = carve(workspace, M, K);
     const __half* xh = static_cast<const __half*>(x);
     if (alpha && !aligned(alpha, 16)) return AQ_ERR_ALIGNMENT;
-    const cudaError_t e = quantize_dispatch(h, xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, w.ctl, w.codes,
-                                            nullptr, alpha, k_max, stream);
+    cudaError_t e;
+    if (w_offsets) {
+        // zero-point variant: min / max, then e, zp and codes; then the per-channel term -(zp - 2^(b-1)) * r[n]
+        if (!aligned(w_offsets, 4)) return AQ_ERR_ALIGNMENT;
+        e = cudaMemsetAsync(w.ctl, 0, sizeof(Control), stream);
+        if (e == cudaSuccess)
+            e = launch_quantize_asym(xh, M, K, row_idx, bits, w.ctl, w.codes, nullptr, nullptr, h->dev, stream);
+        if (e == cudaSuccess) e = launch_chan_offsets(w_offsets, N, bits, w.ctl, w.chan_offset, stream);
+    } else {
+        e = quantize_dispatch(h, xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, w.ctl, w.codes, nullptr, alpha,
+                              k_max, stream);
+    }
     if (e != cudaSuccess) return cuda_fail(h, e);
     GemmArgs g;
     g.q = w.codes; g.M = M; g.K = K; g.N = N; g.group = group;
@@ -115,6 +128,7 @@ int linear_impl(aq_handle_t h, int bits, const void* x, int M, int K, const void
     g.y = static_cast<__half*>(y);
     g.acc_dump = acc_dump;
     g.ctl = w.ctl; g.scratch = w.scratch; g.scratch_bytes = w.scratch_bytes;
+    g.chan_offset = w_offsets ? w.chan_offset : nullptr;
     return run_gemm(h, g, stream);
 }
 
@@ -200,7 +214,7 @@ size_t aq_scales_bytes(int N, int K, int group_size) {
 
 size_t aq_workspace_bytes(int M, int K, int N, int group_size) {
     if (check_shape(M, K, N, group_size) != AQ_OK) return 0;
-    return workspace_bytes(M, K);
+    return workspace_bytes(M, K, N);
 }
 
 int aq_pack_w4(aq_handle_t h, const void* w_fp16, int N, int K, int group_size, void* w_packed,
@@ -312,7 +326,7 @@ int aq_gemm_w4(aq_handle_t h, const int8_t* q, int M, int K, const void* w_packe
     if (!h || !q || !w_packed || !w_scales || !scale_exp || !y_fp16) return AQ_ERR_INVALID_ARG;
     const int s = check_shape(M, K, N, group_size);
     if (s != AQ_OK) return s;
-    if (!workspace || workspace_bytes_ < workspace_bytes(M, K)) return AQ_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes_ < workspace_bytes(M, K, N)) return AQ_ERR_WORKSPACE;
     if (!aligned(q, 16) || !aligned(w_packed, 16) || !aligned(w_scales, 2) || !aligned(y_fp16, 2) ||
         !aligned(workspace, 256) || !aligned(scale_exp, 4) || (acc_dump && !aligned(acc_dump, 4)))
         return AQ_ERR_ALIGNMENT;
@@ -356,6 +370,53 @@ int aq_token_compact(aq_handle_t h, const void* x_fp16, int M, int K, const int3
     return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
 }
 
+int aq_weight_offsets(aq_handle_t h, const void* w_packed, const void* w_scales, int N, int K, int group_size,
+                      float* r_out, void* stream) {
+    if (!h || !w_packed || !w_scales || !r_out) return AQ_ERR_INVALID_ARG;
+    const int s = check_shape(1, K, N, group_size);
+    if (s != AQ_OK) return s;
+    if (!aligned(w_packed, 16) || !aligned(w_scales, 2) || !aligned(r_out, 4)) return AQ_ERR_ALIGNMENT;
+    const cudaError_t e = launch_weight_offsets(static_cast<const uint8_t*>(w_packed), static_cast<const __half*>(w_scales),
+                                                N, K, group_size, r_out, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
+int aq_quantize_act_asym(aq_handle_t h, const void* x_fp16, int M, int K, int bits, const int32_t* row_idx, int8_t* q,
+                         int32_t* scale_exp_out, int32_t* zero_point_out, void* workspace, size_t workspace_bytes_,
+                         void* stream_) {
+    if (!h || !x_fp16 || !q || (bits != 8 && bits != 4)) return AQ_ERR_INVALID_ARG;
+    const int s = check_shape(M, K, 1, 0);
+    if (s != AQ_OK) return s;
+    if (!workspace || workspace_bytes_ < sizeof(Control)) return AQ_ERR_WORKSPACE;
+    if (!aligned(x_fp16, 16) || !aligned(q, 16) || !aligned(workspace, 256) ||
+        (scale_exp_out && !aligned(scale_exp_out, 4)) || (zero_point_out && !aligned(zero_point_out, 4)) ||
+        (row_idx && !aligned(row_idx, 4)))
+        return AQ_ERR_ALIGNMENT;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    Control* ctl = static_cast<Control*>(workspace);
+    cudaError_t e = cudaMemsetAsync(ctl, 0, sizeof(Control), stream);
+    if (e == cudaSuccess)
+        e = launch_quantize_asym(static_cast<const __half*>(x_fp16), M, K, row_idx, bits, ctl, q, scale_exp_out,
+                                 zero_point_out, h->dev, stream);
+    return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
+int aq_linear_w4a8_asym(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed, const void* w_scales,
+                        const float* w_offsets, int N, int group_size, const int32_t* row_idx, void* y_fp16,
+                        int32_t* acc_dump, void* workspace, size_t workspace_bytes_, void* stream) {
+    if (!w_offsets) return AQ_ERR_INVALID_ARG;
+    return linear_impl(h, 8, x_fp16, M, K, w_packed, w_scales, N, group_size, AQ_SCALE_DYNAMIC, 0, row_idx, y_fp16,
+                       acc_dump, workspace, workspace_bytes_, stream, nullptr, 0, w_offsets);
+}
+
+int aq_linear_w4a4_asym(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed, const void* w_scales,
+                        const float* w_offsets, int N, int group_size, const int32_t* row_idx, void* y_fp16,
+                        int32_t* acc_dump, void* workspace, size_t workspace_bytes_, void* stream) {
+    if (!w_offsets) return AQ_ERR_INVALID_ARG;
+    return linear_impl(h, 4, x_fp16, M, K, w_packed, w_scales, N, group_size, AQ_SCALE_DYNAMIC, 0, row_idx, y_fp16,
+                       acc_dump, workspace, workspace_bytes_, stream, nullptr, 0, w_offsets);
+}
+
 int aq_prune_schedule(int M, double beta, int m, int32_t* n_keep_out, double* gamma_out) {
     if (M < 1 || m < 1 || !(beta >= 0.0) || !(beta < 1.0) || !n_keep_out) return AQ_ERR_INVALID_ARG;
     const double gamma = 1.0 - pow(1.0 - beta, 1.0 / (double)m);       // Eq. 9
@@ -371,7 +432,7 @@ int aq_prune_schedule(int M, double beta, int m, int32_t* n_keep_out, double* ga
 
 size_t aq_linear_host_scratch_bytes(int M, int K, int N, int group_size) {
     if (check_shape(M, K, N, group_size) != AQ_OK) return 0;
-    return up256((size_t)M * K * 2) + up256((size_t)M * N * 2) + workspace_bytes(M, K);
+    return up256((size_t)M * K * 2) + up256((size_t)M * N * 2) + workspace_bytes(M, K, N);
 }
 
 int aq_linear_host(aq_handle_t h, int bits, const void* x_host, int M, int K, const void* w_packed,
@@ -391,7 +452,7 @@ int aq_linear_host(aq_handle_t h, int bits, const void* x_host, int M, int K, co
     cudaError_t e = cudaMemcpyAsync(x_dev, x_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, stream);
     if (e != cudaSuccess) return cuda_fail(h, e);
     const int rc = linear_impl(h, bits, x_dev, M, K, w_packed, w_scales, N, group_size, scale_mode,
-                               clip_shift_or_exp, nullptr, y_dev, nullptr, ws, workspace_bytes(M, K), stream_);
+                               clip_shift_or_exp, nullptr, y_dev, nullptr, ws, workspace_bytes(M, K, N), stream_);
     if (rc != AQ_OK) return rc;
     e = cudaMemcpyAsync(y_host, y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, stream);
     if (e != cudaSuccess) return cuda_fail(h, e);

@@ -44,7 +44,9 @@ struct Control {
     int scale_exp;              // layer exponent e
     unsigned int status;        // non-zero: a bounded wait gave up
     unsigned int counter;       // scratch counter
-    unsigned int reserved[60];
+    unsigned int min_key, max_key;   // zero-point variant: order-preserving keys of min(x), max(x)
+    int zero_point;             // zero-point variant: zp of Eq. 7
+    unsigned int reserved[57];
 };
 static_assert(sizeof(Control) == 256, "control block is 256 bytes");
 
@@ -103,6 +105,17 @@ cudaError_t launch_trip_calibrate(const __half* x, int M, int K, const int32_t* 
                                   Control* ctl, uint8_t* alpha_out, int32_t* scale_exp_out, const DeviceInfo& dev,
                                   cudaStream_t stream);
 
+// Zero-point variant (Eq. 2, Eq. 5-7 with alpha = 0 and a power-of-two scale): minimum and maximum,
+// then e, zp and the codes, stored as q - 2^(b-1) in int8. The control block must have been cleared.
+cudaError_t launch_quantize_asym(const __half* x, int M, int K, const int32_t* row_idx, int bits, Control* ctl,
+                                 int8_t* q, int32_t* scale_exp_out, int32_t* zero_point_out, const DeviceInfo& dev,
+                                 cudaStream_t stream);
+// r[n] = sum_g s_w[n,g] * sum_{k in g} c[n,k], from the packed weights (float [N]).
+cudaError_t launch_weight_offsets(const uint8_t* packed, const __half* scales, int N, int K, int group, float* r,
+                                  cudaStream_t stream);
+// off[n] = -(zp - 2^(b-1)) * r[n] with zp from the control block.
+cudaError_t launch_chan_offsets(const float* r, int N, int bits, const Control* ctl, float* off, cudaStream_t stream);
+
 cudaError_t launch_token_select(const float* scores, int M, int n_keep, int32_t* idx, void* scratch,
                                 cudaStream_t stream);
 cudaError_t launch_token_compact(const __half* x, int K, const int32_t* idx, int n_keep, __half* out,
@@ -118,6 +131,7 @@ struct GemmArgs {
     __half* y;              // [M][N]
     int32_t* acc_dump;      // NULL or [M][N][G]
     Control* ctl;
+    const float* chan_offset = nullptr;   // NULL or [N]: added to sum_g s*acc before the 2^e factor (zero-point term)
     void* scratch;          // beyond control block + codes
     size_t scratch_bytes;
 };

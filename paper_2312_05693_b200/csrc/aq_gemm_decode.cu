@@ -35,7 +35,7 @@ __global__ void __launch_bounds__(kDecThreads)
 gemm_decode_kernel(const int8_t* __restrict__ q, int M, int K, int N, int Npad,
                    const uint8_t* __restrict__ w_packed, const __half* __restrict__ w_scales,
                    const int32_t* __restrict__ scale_exp, __half* __restrict__ y,
-                   int32_t* __restrict__ acc_dump, Control* __restrict__ ctl) {
+                   int32_t* __restrict__ acc_dump, Control* __restrict__ ctl, const float* __restrict__ chan_offset) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) ctl->status = 0;   // this kernel has no bounded waits
     const int KB = K / kTileK;
@@ -130,19 +130,20 @@ gemm_decode_kernel(const int8_t* __restrict__ q, int M, int K, int N, int Npad,
     const float pe = __int_as_float((127 + *scale_exp) << 23);   // 2^e
     for (int m = warp; m < MB; m += kDecWarps) {
         if (m0 + m >= M || n >= N) continue;
+        const float off = chan_offset ? chan_offset[n] : 0.0f;
         float out;
         if (GROUPED) {
             float s = 0.0f;
 #pragma unroll
             for (int w = 0; w < kDecWarps; ++w) s += __int_as_float(red[w][m][lane]);
-            out = s * pe;
+            out = (s + off) * pe;
         } else {
             int s = 0;
 #pragma unroll
             for (int w = 0; w < kDecWarps; ++w) s += red[w][m][lane];
             s >>= 4;
             if (acc_dump) acc_dump[(size_t)(m0 + m) * N + n] = s;
-            out = (float)s * __half2float(w_scales[n]) * pe;
+            out = fmaf((float)s, __half2float(w_scales[n]), off) * pe;
         }
         y[(size_t)(m0 + m) * N + n] = __float2half_rn(out);
     }
@@ -208,6 +209,7 @@ struct StreamParams {
     __half* y;
     int32_t* acc_dump;
     Control* ctl;
+    const float* chan_offset;
 };
 
 // grid = (split, channel tiles), cluster = (split, 1, 1): the CTAs of a cluster share a channel
@@ -386,11 +388,14 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
         }
     }
     // the output scale is fetched before the cluster meets so that its latency overlaps the wait
-    float sc = 0.0f;
+    float sc = 0.0f, off = 0.0f;
     const int out_r = (warp - 1) * 32 + lane;
     const int out_n = tile * kTileN + out_r;
-    if (rank == 0 && warp >= 1 && warp <= 4 && out_n < p.N)
-        sc = __half2float(p.w_scales[out_n]) * __int_as_float((127 + *p.scale_exp) << 23);
+    if (rank == 0 && warp >= 1 && warp <= 4 && out_n < p.N) {
+        const float pe = __int_as_float((127 + *p.scale_exp) << 23);
+        sc = __half2float(p.w_scales[out_n]) * pe;
+        if (p.chan_offset) off = p.chan_offset[out_n] * pe;
+    }
     cluster.sync();
     if (rank == 0 && warp >= 1 && warp <= 4 && out_n < p.N) {
 #pragma unroll
@@ -398,7 +403,7 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
             if (m < p.M) {
                 const int a = sm.sum[m][out_r] >> 4;                  // sums carry a factor 16
                 if (p.acc_dump) p.acc_dump[(size_t)m * p.N + out_n] = a;
-                p.y[(size_t)m * p.N + out_n] = __float2half_rn((float)a * sc);
+                p.y[(size_t)m * p.N + out_n] = __float2half_rn(fmaf((float)a, sc, off));
             }
         }
     }
@@ -437,7 +442,7 @@ cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t
     StreamParams p;
     p.M = a.M; p.K = a.K; p.N = a.N; p.Npad = round_up(a.N, kTileN);
     p.w_packed = a.w_packed; p.w_scales = a.w_scales; p.scale_exp = a.scale_exp;
-    p.y = a.y; p.acc_dump = a.acc_dump; p.ctl = a.ctl;
+    p.y = a.y; p.acc_dump = a.acc_dump; p.ctl = a.ctl; p.chan_offset = a.chan_offset;
     const int tiles = p.Npad / kTileN, KB = a.K / kTileK;
     // as many k ranges per tile (cluster size 1, 2 or 4: clusters of 7-8 measured slower) as keep
     // all CTAs resident at once (two per SM), and at least two k blocks per CTA
@@ -464,10 +469,10 @@ cudaError_t launch_mb(const GemmArgs& a, cudaStream_t stream) {
     dim3 grid(Npad / 32, (a.M + MB - 1) / MB);
     if (a.group)
         gemm_decode_kernel<MB, true><<<grid, kDecThreads, 0, stream>>>(
-            a.q, a.M, a.K, a.N, Npad, a.w_packed, a.w_scales, a.scale_exp, a.y, a.acc_dump, a.ctl);
+            a.q, a.M, a.K, a.N, Npad, a.w_packed, a.w_scales, a.scale_exp, a.y, a.acc_dump, a.ctl, a.chan_offset);
     else
         gemm_decode_kernel<MB, false><<<grid, kDecThreads, 0, stream>>>(
-            a.q, a.M, a.K, a.N, Npad, a.w_packed, a.w_scales, a.scale_exp, a.y, a.acc_dump, a.ctl);
+            a.q, a.M, a.K, a.N, Npad, a.w_packed, a.w_scales, a.scale_exp, a.y, a.acc_dump, a.ctl, a.chan_offset);
     return cudaGetLastError();
 }
 

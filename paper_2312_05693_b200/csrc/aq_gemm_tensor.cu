@@ -148,15 +148,6 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
         : "r"(taddr)
         : "memory");
 }
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-        : "r"(taddr)
-        : "memory");
-}
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_st8(uint32_t taddr, const uint32_t (&v)[8]) {
     asm volatile(
@@ -226,10 +217,13 @@ struct TensorParams {
     __half* y;
     int32_t* acc_dump;
     Control* ctl;
+    const float* chan_offset;      // NULL or [N]: per-channel term added before the 2^e factor
     int y_tma;                     // outputs leave through y_map (needs N % 8 == 0 and a 16-byte aligned y)
 };
 
-template <int BM, bool GROUPED>
+// OFFSET: add the per-channel term of the zero-point variant. A separate instantiation, so that the
+// code of the plain kernels does not change with it.
+template <int BM, bool GROUPED, bool OFFSET>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap y_map,
                    const TensorParams p) {
@@ -436,6 +430,8 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
                 const int a = (int)(unit % kNumAcc);
                 const uint32_t aph = (unit / kNumAcc) & 1u;
                 const float sc = __half2float(p.w_scales[n]) * 0.0625f * pe;   // sums carry a factor 16
+                [[maybe_unused]] float off_pe = 0.0f;
+                if constexpr (OFFSET) off_pe = (n_ok ? p.chan_offset[n] : 0.0f) * pe;
                 if (!mbar_wait_warp(&sm.acc_full[a], aph, abort_flag, 8u)) goto role_done;
                 tc_fence_after();
                 // all of this warp's sums go to registers and the accumulator returns to the MMA at once,
@@ -457,7 +453,8 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
                         __syncwarp();
 #pragma unroll
                         for (int c = 0; c < Smem::kStageRows; ++c)
-                            stage[c * 32 + lane] = __float2half_rn((float)(int)v[r0 + c] * sc);
+                            stage[c * 32 + lane] = __float2half_rn(OFFSET ? fmaf((float)(int)v[r0 + c], sc, off_pe)
+                                                                          : (float)(int)v[r0 + c] * sc);
                         fence_proxy_async();
                         __syncwarp();
                         if (lane == 0 && n0 < p.N && m_base + r0 < p.M) tma_store_2d(&y_map, stage, n0, m_base + r0);
@@ -466,7 +463,9 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
 #pragma unroll
                     for (int c = 0; c < kColsPerEpiWarp; ++c) {
                         const int m = m_base + c;
-                        if (n_ok && m < p.M) p.y[(size_t)m * p.N + n] = __float2half_rn((float)(int)v[c] * sc);
+                        if (n_ok && m < p.M)
+                            p.y[(size_t)m * p.N + n] =
+                                __float2half_rn(OFFSET ? fmaf((float)(int)v[c], sc, off_pe) : (float)(int)v[c] * sc);
                     }
                 }
                 if (p.acc_dump) {
@@ -515,6 +514,11 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
                         }
                     }
                 }
+                if constexpr (OFFSET) {                                  // read after the k loop
+                    const float off_n = n_ok ? p.chan_offset[n] : 0.0f;
+#pragma unroll
+                    for (int c = 0; c < kColsPerEpiWarp; ++c) fsum[c] += off_n;
+                }
                 if (p.y_tma) {
                     static_assert(Smem::kStageRows == kColsPerEpiWarp, "per-group kernels stage a warp's whole tile");
                     // the previous tile's store must have read the staging rows before they change
@@ -560,13 +564,13 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-template <int BM, bool GROUPED>
-cudaError_t launch_bm(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
+template <int BM, bool GROUPED, bool OFFSET>
+cudaError_t launch_off(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
     using Smem = SharedStorage<BM>;
     const size_t smem_bytes = sizeof(Smem) + 1024;
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tensor_kernel<BM, GROUPED>,
+        cudaError_t e = cudaFuncSetAttribute(gemm_tensor_kernel<BM, GROUPED, OFFSET>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
         if (e != cudaSuccess) return e;
         attr_done = true;
@@ -602,10 +606,15 @@ cudaError_t launch_bm(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t str
     p.n_tiles_m = (a.M + BM - 1) / BM;
     p.n_tiles = p.n_tiles_m * (p.Npad / kTileN);
     p.w_packed = a.w_packed; p.w_scales = a.w_scales; p.scale_exp = a.scale_exp;
-    p.y = a.y; p.acc_dump = a.acc_dump; p.ctl = a.ctl;
+    p.y = a.y; p.acc_dump = a.acc_dump; p.ctl = a.ctl; p.chan_offset = a.chan_offset;
     const int grid = p.n_tiles < dev.sm_count ? p.n_tiles : dev.sm_count;
-    gemm_tensor_kernel<BM, GROUPED><<<grid, kThreads, smem_bytes, stream>>>(map, ymap, p);
+    gemm_tensor_kernel<BM, GROUPED, OFFSET><<<grid, kThreads, smem_bytes, stream>>>(map, ymap, p);
     return cudaGetLastError();
+}
+
+template <int BM, bool GROUPED>
+cudaError_t launch_bm(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
+    return a.chan_offset ? launch_off<BM, GROUPED, true>(a, dev, stream) : launch_off<BM, GROUPED, false>(a, dev, stream);
 }
 
 }  // namespace

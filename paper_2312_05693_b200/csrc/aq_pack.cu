@@ -91,7 +91,42 @@ __global__ void unpack_w4_kernel(const uint8_t* __restrict__ packed, int N, int 
     codes[idx] = (int8_t)(nib >= 8 ? nib - 16 : nib);
 }
 
+// One thread per channel: the sum of its codes in every group, times the group's scale, in binary64.
+__global__ void weight_offsets_kernel(const uint8_t* __restrict__ packed, const __half* __restrict__ scales, int N,
+                                      int K, int group, float* __restrict__ r_out) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n >= N) return;
+    const int KB = K / kTileK, Npad = round_up(N, kTileN);
+    const int nt = n / kTileN, r = n % kTileN;
+    double total = 0.0;
+    long long run = 0;
+    for (int kb = 0; kb < KB; ++kb) {
+        int colsum = 0;
+        for (int j = 0; j < 4; ++j) {
+            const uint4 d = *reinterpret_cast<const uint4*>(packed + packed_unit_offset(KB, nt, kb, j, r));
+            const uint32_t w[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int b = 0; b < 8; ++b) {
+                    const int nib = (w[i] >> (4 * b)) & 0xF;
+                    colsum += nib >= 8 ? nib - 16 : nib;
+                }
+        }
+        if (group) total += (double)colsum * (double)__half2float(scales[(size_t)kb * Npad + n]);
+        else run += colsum;
+    }
+    if (!group) total = (double)run * (double)__half2float(scales[n]);
+    r_out[n] = (float)total;
+}
+
 }  // namespace
+
+cudaError_t launch_weight_offsets(const uint8_t* packed, const __half* scales, int N, int K, int group, float* r,
+                                  cudaStream_t stream) {
+    weight_offsets_kernel<<<(N + 127) / 128, 128, 0, stream>>>(packed, scales, N, K, group, r);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_pack_w4(const __half* w, int N, int K, int group, uint8_t* packed, __half* scales,
                            cudaStream_t stream) {

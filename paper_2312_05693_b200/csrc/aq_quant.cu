@@ -308,6 +308,102 @@ quantize_fused_kernel(const uint4* __restrict__ x, int M, int units_per_row /* 1
     }
 }
 
+// ---- zero-point variant (Eq. 2, Eq. 5-7 with alpha = 0, power-of-two scale) ---------------
+// Order-preserving map of a float's bits to an unsigned integer, so that atomicMin / atomicMax
+// on the keys give the minimum / maximum value.
+__device__ __forceinline__ unsigned int float_key(float f) {
+    const unsigned int b = __float_as_uint(f);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float key_float(unsigned int k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
+}
+constexpr unsigned int kZeroKey = 0x80000000u;         // key of +0.0: the range always contains 0
+
+__global__ void __launch_bounds__(256)
+minmax_kernel(const __half* __restrict__ x, int M, int K, const int32_t* __restrict__ row_idx,
+              Control* __restrict__ ctl) {
+    const size_t total = (size_t)M * K;
+    unsigned int kmin = kZeroKey, kmax = kZeroKey;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int m = (int)(i / K), k = (int)(i % K);
+        float v = __half2float(x[(size_t)(row_idx ? row_idx[m] : m) * K + k]);
+        if (v != v) continue;                                            // NaN is ignored
+        v = fminf(fmaxf(v, -65504.0f), 65504.0f);                        // +-Inf count as the largest half
+        const unsigned int key = float_key(v);
+        kmin = min(kmin, key);
+        kmax = max(kmax, key);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        kmin = min(kmin, __shfl_xor_sync(0xFFFFFFFFu, kmin, o));
+        kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, o));
+    }
+    if ((threadIdx.x & 31) == 0) {
+        // the control block is cleared to 0: keys are stored relative to the key of 0.0
+        if (kmax > kZeroKey) atomicMax(&ctl->max_key, kmax - kZeroKey);
+        if (kmin < kZeroKey) atomicMax(&ctl->min_key, kZeroKey - kmin);
+    }
+}
+
+// e = smallest integer with (2^b - 1) * 2^e >= max - min, zp = clip(round(-min / 2^e), 0, 2^b - 1), in
+// binary64 (exact for fp16 inputs), by every thread alike; then 16 codes per thread.
+__global__ void __launch_bounds__(kQuantThreads)
+quantize_asym_kernel(const uint4* __restrict__ x, int M, int vec_per_row /* 16-element units */,
+                     const int32_t* __restrict__ row_idx, int bits, Control* __restrict__ ctl, uint4* __restrict__ q,
+                     int32_t* __restrict__ scale_exp_out, int32_t* __restrict__ zero_point_out) {
+    const double hi = (double)key_float(kZeroKey + ctl->max_key), lo = (double)key_float(kZeroKey - ctl->min_key);
+    const double range = hi - lo, qr = (double)((1 << bits) - 1);
+    int e = 0;
+    if (range > 0.0) {
+        int ex;
+        frexp(range / qr, &ex);                      // a first guess within one of the answer
+        e = ex;
+        while (ldexp(qr, e) < range) ++e;
+        while (ldexp(qr, e - 1) >= range) --e;
+    }
+    const double zpd = fmin(fmax(rint(ldexp(-lo, -e)), 0.0), qr);
+    const int zp = (int)zpd;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        ctl->scale_exp = e;
+        ctl->zero_point = zp;
+        if (scale_exp_out) *scale_exp_out = e;
+        if (zero_point_out) *zero_point_out = zp;
+    }
+    const float inv = __int_as_float((127 - e) << 23);      // 2^-e
+    const float fzp = (float)zp, fqr = (float)qr;
+    const int half_range = 1 << (bits - 1);
+    const size_t total = (size_t)M * vec_per_row;
+    const size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (v >= total) return;
+    const int m = (int)(v / vec_per_row), c = (int)(v % vec_per_row);
+    const size_t src = ((size_t)(row_idx ? row_idx[m] : m) * vec_per_row + c) * 2;
+    const uint4 d0 = __ldg(x + src), d1 = __ldg(x + src + 1);
+    const __half* h0 = reinterpret_cast<const __half*>(&d0);
+    const __half* h1 = reinterpret_cast<const __half*>(&d1);
+    uint32_t out[4];
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+        uint32_t word = 0;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            const int i = 4 * w + b;
+            const float t = __half2float(i < 8 ? h0[i] : h1[i - 8]) * inv;    // exact
+            int code = zp;                                                    // NaN: value 0
+            if (t == t) code = (int)fminf(fmaxf(rintf(t) + fzp, 0.0f), fqr);
+            word |= ((uint32_t)(code - half_range) & 0xFFu) << (8 * b);
+        }
+        out[w] = word;
+    }
+    q[v] = make_uint4(out[0], out[1], out[2], out[3]);
+}
+
+__global__ void chan_offsets_kernel(const float* __restrict__ r, int N, int bits, const Control* __restrict__ ctl,
+                                    float* __restrict__ off) {
+    const int n = blockIdx.x * blockDim.x + threadIdx.x;
+    if (n < N) off[n] = -(float)(ctl->zero_point - (1 << (bits - 1))) * r[n];
+}
+
 // ---- TRIP calibration (Eq. 8 with the clipping of Eq. 5) ---------------------------------
 __global__ void __launch_bounds__(256)
 absmax_plain_kernel(const __half* __restrict__ x, int M, int K, const int32_t* __restrict__ row_idx,
@@ -496,6 +592,29 @@ cudaError_t launch_trip_calibrate(const __half* x, int M, int K, const int32_t* 
     if (e != cudaSuccess) return e;
     trip_calibrate_kernel<<<(K + 127) / 128, 128, 0, stream>>>(x, M, K, row_idx, bits, k_max, ctl, alpha_out,
                                                                scale_exp_out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quantize_asym(const __half* x, int M, int K, const int32_t* row_idx, int bits, Control* ctl,
+                                 int8_t* q, int32_t* scale_exp_out, int32_t* zero_point_out, const DeviceInfo& dev,
+                                 cudaStream_t stream) {
+    const size_t total = (size_t)M * K;
+    size_t blocks = (total + 255) / 256;
+    const size_t cap = (size_t)dev.sm_count * 8;
+    if (blocks > cap) blocks = cap;
+    minmax_kernel<<<(unsigned int)blocks, 256, 0, stream>>>(x, M, K, row_idx, ctl);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const int vec_per_row = K / 16;
+    const size_t units = (size_t)M * vec_per_row;
+    quantize_asym_kernel<<<(unsigned int)((units + kQuantThreads - 1) / kQuantThreads), kQuantThreads, 0, stream>>>(
+        reinterpret_cast<const uint4*>(x), M, vec_per_row, row_idx, bits, ctl, reinterpret_cast<uint4*>(q),
+        scale_exp_out, zero_point_out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_chan_offsets(const float* r, int N, int bits, const Control* ctl, float* off, cudaStream_t stream) {
+    chan_offsets_kernel<<<(N + 255) / 256, 256, 0, stream>>>(r, N, bits, ctl, off);
     return cudaGetLastError();
 }
 
