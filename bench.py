@@ -310,6 +310,26 @@ def bench_w4a4(h, reps=30):
     return out
 
 
+def bench_zero_point(h, reps=30):
+    """The benchmark step with the unsigned quantizer and a zero point (Eq. 2, Eq. 5-7), 8-bit codes."""
+    wl = inputs.WORKLOADS["llama7b_prefill_w4a8"]
+    M = wl.Ms[0]
+    layers = []
+    for s in wl.shapes:
+        x = torch.from_numpy(inputs.activations(M, s.K, wl.seed, wl.outlier_frac, wl.outlier_mult)).cuda()
+        p, sc = h.aq_pack_w4(torch.from_numpy(inputs.weights(s.N, s.K, wl.seed)).cuda(), wl.group_size)
+        r = h.aq_weight_offsets(p, sc, s.N, s.K, wl.group_size)          # once per weight matrix
+        layers.append((x, p, sc, r, s, h.alloc_workspace(M, s.K, s.N, wl.group_size),
+                       torch.empty((M, s.N), dtype=torch.float16, device="cuda")))
+    def step():
+        for x, p, sc, r, s, ws, y in layers:
+            h.aq_linear_asym(8, x, p, sc, r, s.N, wl.group_size, y=y, workspace=ws)
+    ms = _event_ms(step, reps)
+    ops = sum(2.0 * M * s.K * s.N for s in wl.shapes)
+    return {"workload": wl.name + " with zero point", "ms_per_step": ms, "TOPS": ops / (ms * 1e-3) / 1e12,
+            "note": "quantize is two plain kernels here (min/max, codes), not the fused one"}
+
+
 def bench_pruned(h, reps=10):
     wl = inputs.WORKLOADS["opt30b_pruned_prefill_w4a8"]
     M = wl.Ms[0]
@@ -539,7 +559,7 @@ def main():
         except Exception as ex:  # report, do not hide
             line["decode"] = {"error": repr(ex)}
     if rank == 0 and world == 1 and not args.no_decode:
-        for key, fn in (("w4a4", bench_w4a4), ("pruned_prefill", bench_pruned)):
+        for key, fn in (("w4a4", bench_w4a4), ("zero_point", bench_zero_point), ("pruned_prefill", bench_pruned)):
             try:
                 line[key] = fn(h)
             except Exception as ex:  # report, do not hide

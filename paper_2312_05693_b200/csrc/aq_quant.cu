@@ -321,19 +321,24 @@ __device__ __forceinline__ float key_float(unsigned int k) {
 constexpr unsigned int kZeroKey = 0x80000000u;         // key of +0.0: the range always contains 0
 
 __global__ void __launch_bounds__(256)
-minmax_kernel(const __half* __restrict__ x, int M, int K, const int32_t* __restrict__ row_idx,
-              Control* __restrict__ ctl) {
-    const size_t total = (size_t)M * K;
-    unsigned int kmin = kZeroKey, kmax = kZeroKey;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
-        const int m = (int)(i / K), k = (int)(i % K);
-        float v = __half2float(x[(size_t)(row_idx ? row_idx[m] : m) * K + k]);
-        if (v != v) continue;                                            // NaN is ignored
-        v = fminf(fmaxf(v, -65504.0f), 65504.0f);                        // +-Inf count as the largest half
-        const unsigned int key = float_key(v);
-        kmin = min(kmin, key);
-        kmax = max(kmax, key);
+minmax_kernel(const uint4* __restrict__ x, int M, int vec_per_row /* 8-element vectors */,
+              const int32_t* __restrict__ row_idx, Control* __restrict__ ctl) {
+    const size_t total = (size_t)M * vec_per_row;
+    __half2 lo2 = __float2half2_rn(0.0f), hi2 = __float2half2_rn(0.0f);      // the range always contains 0
+    for (size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v < total; v += (size_t)gridDim.x * blockDim.x) {
+        const int m = (int)(v / vec_per_row), c = (int)(v % vec_per_row);
+        const uint4 d = __ldg(x + (size_t)(row_idx ? row_idx[m] : m) * vec_per_row + c);
+        const __half2* h = reinterpret_cast<const __half2*>(&d);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {                                        // NaN operands are dropped
+            lo2 = __hmin2(lo2, h[i]);
+            hi2 = __hmax2(hi2, h[i]);
+        }
     }
+    // +-Inf count as the largest half
+    const float lo = fmaxf(fminf(__low2float(lo2), __high2float(lo2)), -65504.0f);
+    const float hi = fminf(fmaxf(__low2float(hi2), __high2float(hi2)), 65504.0f);
+    unsigned int kmin = float_key(lo), kmax = float_key(hi);
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         kmin = min(kmin, __shfl_xor_sync(0xFFFFFFFFu, kmin, o));
@@ -347,23 +352,29 @@ minmax_kernel(const __half* __restrict__ x, int M, int K, const int32_t* __restr
 }
 
 // e = smallest integer with (2^b - 1) * 2^e >= max - min, zp = clip(round(-min / 2^e), 0, 2^b - 1), in
-// binary64 (exact for fp16 inputs), by every thread alike; then 16 codes per thread.
+// binary64 (exact for fp16 inputs), by one thread of every CTA; then 16 codes per thread.
 __global__ void __launch_bounds__(kQuantThreads)
 quantize_asym_kernel(const uint4* __restrict__ x, int M, int vec_per_row /* 16-element units */,
                      const int32_t* __restrict__ row_idx, int bits, Control* __restrict__ ctl, uint4* __restrict__ q,
                      int32_t* __restrict__ scale_exp_out, int32_t* __restrict__ zero_point_out) {
-    const double hi = (double)key_float(kZeroKey + ctl->max_key), lo = (double)key_float(kZeroKey - ctl->min_key);
-    const double range = hi - lo, qr = (double)((1 << bits) - 1);
-    int e = 0;
-    if (range > 0.0) {
-        int ex;
-        frexp(range / qr, &ex);                      // a first guess within one of the answer
-        e = ex;
-        while (ldexp(qr, e) < range) ++e;
-        while (ldexp(qr, e - 1) >= range) --e;
+    __shared__ int params[2];
+    const double qr = (double)((1 << bits) - 1);
+    if (threadIdx.x == 0) {
+        const double hi = (double)key_float(kZeroKey + ctl->max_key), lo = (double)key_float(kZeroKey - ctl->min_key);
+        const double range = hi - lo;
+        int ee = 0;
+        if (range > 0.0) {
+            int ex;
+            frexp(range / qr, &ex);                  // a first guess within one of the answer
+            ee = ex;
+            while (ldexp(qr, ee) < range) ++ee;
+            while (ldexp(qr, ee - 1) >= range) --ee;
+        }
+        params[0] = ee;
+        params[1] = (int)fmin(fmax(rint(ldexp(-lo, -ee)), 0.0), qr);
     }
-    const double zpd = fmin(fmax(rint(ldexp(-lo, -e)), 0.0), qr);
-    const int zp = (int)zpd;
+    __syncthreads();
+    const int e = params[0], zp = params[1];
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         ctl->scale_exp = e;
         ctl->zero_point = zp;
@@ -598,11 +609,11 @@ cudaError_t launch_trip_calibrate(const __half* x, int M, int K, const int32_t* 
 cudaError_t launch_quantize_asym(const __half* x, int M, int K, const int32_t* row_idx, int bits, Control* ctl,
                                  int8_t* q, int32_t* scale_exp_out, int32_t* zero_point_out, const DeviceInfo& dev,
                                  cudaStream_t stream) {
-    const size_t total = (size_t)M * K;
+    const size_t total = (size_t)M * (K / 8);
     size_t blocks = (total + 255) / 256;
     const size_t cap = (size_t)dev.sm_count * 8;
     if (blocks > cap) blocks = cap;
-    minmax_kernel<<<(unsigned int)blocks, 256, 0, stream>>>(x, M, K, row_idx, ctl);
+    minmax_kernel<<<(unsigned int)blocks, 256, 0, stream>>>(reinterpret_cast<const uint4*>(x), M, K / 8, row_idx, ctl);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     const int vec_per_row = K / 16;
