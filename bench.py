@@ -330,6 +330,36 @@ def bench_zero_point(h, reps=30):
             "note": "quantize is two plain kernels here (min/max, codes), not the fused one"}
 
 
+def bench_chain(h, reps=30):
+    """Two layers back to back (the 4096 -> 11008 -> 4096 pair of the benchmark shapes): fp16 in between
+    against the chained call that hands the second layer its int8 codes directly (static exponent)."""
+    wl = inputs.WORKLOADS["llama7b_prefill_w4a8"]
+    M = wl.Ms[0]
+    s1, s2 = wl.shapes[1], wl.shapes[2]
+    x = torch.from_numpy(inputs.activations(M, s1.K, wl.seed, wl.outlier_frac, wl.outlier_mult)).cuda()
+    p1, sc1 = h.aq_pack_w4(torch.from_numpy(inputs.weights(s1.N, s1.K, wl.seed)).cuda(), wl.group_size)
+    p2, sc2 = h.aq_pack_w4(torch.from_numpy(inputs.weights(s2.N, s2.K, wl.seed + 1)).cuda(), wl.group_size)
+    ws1 = h.alloc_workspace(M, s1.K, s1.N, wl.group_size)
+    ws2 = h.alloc_workspace(M, s2.K, s2.N, wl.group_size)
+    y1 = torch.empty((M, s1.N), dtype=torch.float16, device="cuda")
+    y2 = torch.empty((M, s2.N), dtype=torch.float16, device="cuda")
+    q1 = torch.empty((M, s1.N), dtype=torch.int8, device="cuda")
+    h.aq_linear_w4a8(x, p1, sc1, s1.N, wl.group_size, y=y1, workspace=ws1)
+    _, e_mid = h.aq_quantize_act(y1, 8)                       # calibration: the exponent the middle activation needs
+    e_next = int(e_mid.item())
+    def plain():
+        h.aq_linear_w4a8(x, p1, sc1, s1.N, wl.group_size, y=y1, workspace=ws1)
+        h.aq_linear_w4a8(y1, p2, sc2, s2.N, wl.group_size, y=y2, workspace=ws2)
+    def chained():
+        h.aq_linear_chain(8, x, p1, sc1, s1.N, wl.group_size, 8, e_next, q_next=q1, workspace=ws1)
+        h.aq_gemm_w4(q1, p2, sc2, s2.N, wl.group_size, e_mid, y=y2, workspace=ws2)
+    ops = 2.0 * M * (s1.K * s1.N + s2.K * s2.N)
+    t_plain, t_chain = _event_ms(plain, reps), _event_ms(chained, reps)
+    return {"layers_KN": [[s1.K, s1.N], [s2.K, s2.N]], "M": M,
+            "fp16_between": {"us": t_plain * 1e3, "TOPS": ops / (t_plain * 1e-3) / 1e12},
+            "codes_between": {"us": t_chain * 1e3, "TOPS": ops / (t_chain * 1e-3) / 1e12}}
+
+
 def bench_pruned(h, reps=10):
     wl = inputs.WORKLOADS["opt30b_pruned_prefill_w4a8"]
     M = wl.Ms[0]
@@ -559,7 +589,8 @@ def main():
         except Exception as ex:  # report, do not hide
             line["decode"] = {"error": repr(ex)}
     if rank == 0 and world == 1 and not args.no_decode:
-        for key, fn in (("w4a4", bench_w4a4), ("zero_point", bench_zero_point), ("pruned_prefill", bench_pruned)):
+        for key, fn in (("w4a4", bench_w4a4), ("zero_point", bench_zero_point), ("chain", bench_chain),
+                        ("pruned_prefill", bench_pruned)):
             try:
                 line[key] = fn(h)
             except Exception as ex:  # report, do not hide

@@ -187,6 +187,24 @@ int aq_linear_w4a4_asym(aq_handle_t h, const void* x_fp16, int M, int K, const v
                         const float* w_offsets, int N, int group_size, const int32_t* row_idx, void* y_fp16,
                         int32_t* acc_dump, void* workspace, size_t workspace_bytes, void* stream);
 
+/* ---- chaining two layers (paper Sec. 4.4: the kernel's outputs are quantized back for the next
+ * operation instead of leaving as floating point)
+ * As aq_linear_w4a8 / aq_linear_w4a4, but instead of the fp16 outputs the call writes the NEXT layer's
+ * activation codes q_next [M,N] int8 row-major: q_next = clip(round(y16 / 2^next_exp), -2^(b-1),
+ * 2^(b-1)-1) with b = next_bits (8 or 4), where y16 is exactly the fp16 value the plain call would have
+ * written (so the codes equal aq_quantize_act of that output with the static exponent next_exp; NaN -> 0).
+ * The next layer then runs on the codes with aq_gemm_w4 (its scale_exp = next_exp on the device). The
+ * exponent has to be known beforehand (calibration), since a layer-wide maximum of y does not exist
+ * before the layer has finished. -40 <= next_exp <= 40. */
+int aq_linear_w4a8_chain(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed, const void* w_scales,
+                         int N, int group_size, int scale_mode, int clip_shift_or_exp, const int32_t* row_idx,
+                         int8_t* q_next, int next_bits, int next_exp, int32_t* acc_dump, void* workspace,
+                         size_t workspace_bytes, void* stream);
+int aq_linear_w4a4_chain(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed, const void* w_scales,
+                         int N, int group_size, int scale_mode, int clip_shift_or_exp, const int32_t* row_idx,
+                         int8_t* q_next, int next_bits, int next_exp, int32_t* acc_dump, void* workspace,
+                         size_t workspace_bytes, void* stream);
+
 /* ---- progressive pruning schedule (paper Eq. 9; host only, no GPU work)
  * With pruning at m layers and the ratio beta of tokens to be gone after the last of them, every
  * pruning layer drops the fraction gamma = 1 - (1 - beta)^(1/m) of what reaches it. Writes

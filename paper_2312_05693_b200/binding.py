@@ -79,6 +79,9 @@ def load():
     lin_asym = [vp, vp, i32, i32, vp, vp, vp, i32, i32, vp, vp, vp, vp, sz, vp]
     L.aq_linear_w4a8_asym.argtypes = lin_asym
     L.aq_linear_w4a4_asym.argtypes = lin_asym
+    lin_chain = [vp, vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, vp, i32, i32, vp, vp, sz, vp]
+    L.aq_linear_w4a8_chain.argtypes = lin_chain
+    L.aq_linear_w4a4_chain.argtypes = lin_chain
     L.aq_prune_schedule.argtypes = [i32, C.c_double, i32, vp, vp]
     L.aq_trip_calibrate.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
     L.aq_quantize_act_trip.argtypes = [vp, vp, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
@@ -223,6 +226,22 @@ class Handle:
                        clip_shift_or_exp=0, row_idx=None, y=None, acc_dump=None, workspace=None):
         return self._linear(load().aq_linear_w4a4, "aq_linear_w4a4", x, packed, scales, N, group_size,
                             scale_mode, clip_shift_or_exp, row_idx, y, acc_dump, workspace)
+
+    # ---- chaining: the next layer's codes instead of fp16 outputs (Sec. 4.4)
+    def aq_linear_chain(self, bits, x, packed, scales, N, group_size, next_bits, next_exp,
+                        scale_mode=AQ_SCALE_DYNAMIC, clip_shift_or_exp=0, row_idx=None, q_next=None, acc_dump=None,
+                        workspace=None):
+        M_in, K = x.shape
+        M = M_in if row_idx is None else row_idx.shape[0]
+        if q_next is None:
+            q_next = torch.empty((M, N), dtype=torch.int8, device=x.device)
+        if workspace is None:
+            workspace = self.alloc_workspace(M, K, N, group_size)
+        fn = load().aq_linear_w4a8_chain if bits == 8 else load().aq_linear_w4a4_chain
+        _check(fn(self._h, _ptr(x), M, K, _ptr(packed), _ptr(scales), N, group_size, scale_mode, clip_shift_or_exp,
+                  _ptr(row_idx), _ptr(q_next), next_bits, next_exp, _ptr(acc_dump), _ptr(workspace),
+                  workspace.numel(), _stream()), "aq_linear_chain")
+        return q_next
 
     # ---- activations with a zero point (Eq. 2, Eq. 5-7)
     def aq_weight_offsets(self, packed: torch.Tensor, scales: torch.Tensor, N: int, K: int, group_size: int

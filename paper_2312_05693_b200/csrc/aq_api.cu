@@ -92,15 +92,18 @@ bool trip_args_ok(const uint8_t* alpha, int k_max) { return alpha && k_max >= 0 
 int linear_impl(aq_handle_t h, int bits, const void* x, int M, int K, const void* w_packed,
                 const void* w_scales, int N, int group, int scale_mode, int clip_shift_or_exp,
                 const int32_t* row_idx, void* y, int32_t* acc_dump, void* workspace, size_t workspace_bytes_,
-                void* stream_, const uint8_t* alpha = nullptr, int k_max = 0, const float* w_offsets = nullptr) {
-    if (!h || !x || !w_packed || !w_scales || !y) return AQ_ERR_INVALID_ARG;
+                void* stream_, const uint8_t* alpha = nullptr, int k_max = 0, const float* w_offsets = nullptr,
+                int8_t* q_next = nullptr, int next_bits = 8, int next_exp = 0) {
+    if (!h || !x || !w_packed || !w_scales || (!y && !q_next)) return AQ_ERR_INVALID_ARG;
+    if (q_next && ((next_bits != 8 && next_bits != 4) || next_exp < -40 || next_exp > 40 || w_offsets))
+        return AQ_ERR_INVALID_ARG;
     if (scale_mode != AQ_SCALE_DYNAMIC && scale_mode != AQ_SCALE_STATIC) return AQ_ERR_INVALID_ARG;
     if (scale_mode == AQ_SCALE_DYNAMIC && (clip_shift_or_exp < 0 || clip_shift_or_exp > 16)) return AQ_ERR_INVALID_ARG;
     if (scale_mode == AQ_SCALE_STATIC && (clip_shift_or_exp < -40 || clip_shift_or_exp > 40)) return AQ_ERR_INVALID_ARG;
     const int s = check_shape(M, K, N, group);
     if (s != AQ_OK) return s;
     if (!workspace || workspace_bytes_ < workspace_bytes(M, K, N)) return AQ_ERR_WORKSPACE;
-    if (!aligned(x, 16) || !aligned(w_packed, 16) || !aligned(w_scales, 2) || !aligned(y, 2) ||
+    if (!aligned(x, 16) || !aligned(w_packed, 16) || !aligned(w_scales, 2) || (y && !aligned(y, 2)) ||
         !aligned(workspace, 256) || (acc_dump && !aligned(acc_dump, 4)) || (row_idx && !aligned(row_idx, 4)))
         return AQ_ERR_ALIGNMENT;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -129,6 +132,7 @@ int linear_impl(aq_handle_t h, int bits, const void* x, int M, int K, const void
     g.acc_dump = acc_dump;
     g.ctl = w.ctl; g.scratch = w.scratch; g.scratch_bytes = w.scratch_bytes;
     g.chan_offset = w_offsets ? w.chan_offset : nullptr;
+    g.q_next = q_next; g.next_bits = next_bits; g.next_exp = next_exp;
     return run_gemm(h, g, stream);
 }
 
@@ -415,6 +419,26 @@ int aq_linear_w4a4_asym(aq_handle_t h, const void* x_fp16, int M, int K, const v
     if (!w_offsets) return AQ_ERR_INVALID_ARG;
     return linear_impl(h, 4, x_fp16, M, K, w_packed, w_scales, N, group_size, AQ_SCALE_DYNAMIC, 0, row_idx, y_fp16,
                        acc_dump, workspace, workspace_bytes_, stream, nullptr, 0, w_offsets);
+}
+
+int aq_linear_w4a8_chain(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed, const void* w_scales,
+                         int N, int group_size, int scale_mode, int clip_shift_or_exp, const int32_t* row_idx,
+                         int8_t* q_next, int next_bits, int next_exp, int32_t* acc_dump, void* workspace,
+                         size_t workspace_bytes_, void* stream) {
+    if (!q_next) return AQ_ERR_INVALID_ARG;
+    return linear_impl(h, 8, x_fp16, M, K, w_packed, w_scales, N, group_size, scale_mode, clip_shift_or_exp, row_idx,
+                       nullptr, acc_dump, workspace, workspace_bytes_, stream, nullptr, 0, nullptr, q_next, next_bits,
+                       next_exp);
+}
+
+int aq_linear_w4a4_chain(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed, const void* w_scales,
+                         int N, int group_size, int scale_mode, int clip_shift_or_exp, const int32_t* row_idx,
+                         int8_t* q_next, int next_bits, int next_exp, int32_t* acc_dump, void* workspace,
+                         size_t workspace_bytes_, void* stream) {
+    if (!q_next) return AQ_ERR_INVALID_ARG;
+    return linear_impl(h, 4, x_fp16, M, K, w_packed, w_scales, N, group_size, scale_mode, clip_shift_or_exp, row_idx,
+                       nullptr, acc_dump, workspace, workspace_bytes_, stream, nullptr, 0, nullptr, q_next, next_bits,
+                       next_exp);
 }
 
 int aq_prune_schedule(int M, double beta, int m, int32_t* n_keep_out, double* gamma_out) {

@@ -132,6 +132,10 @@ struct GemmArgs {
     int32_t* acc_dump;      // NULL or [M][N][G]
     Control* ctl;
     const float* chan_offset = nullptr;   // NULL or [N]: added to sum_g s*acc before the 2^e factor (zero-point term)
+    // Chaining: when q_next is given the kernels write, instead of y, the next layer's activation codes
+    // [M][N] int8: clip(round(y16 / 2^next_exp), -2^(b-1), 2^(b-1)-1), y16 the fp16 value y would have held.
+    int8_t* q_next = nullptr;
+    int next_bits = 8, next_exp = 0;
     void* scratch;          // beyond control block + codes
     size_t scratch_bytes;
 };

@@ -28,6 +28,13 @@ constexpr int kDecWarps = 8;
 constexpr int kDecThreads = kDecWarps * 32;
 constexpr int kDecPrefetch = 4;      // 128-k blocks in flight per warp (4 x 16 B per lane each)
 
+// Chaining: the code the next layer's quantizer gives the fp16 output value (static exponent; NaN -> 0).
+__device__ __forceinline__ int next_code(__half hv, float inv, float lo, float hi) {
+    const float t = __half2float(hv) * inv;                 // exact: inv is a power of two
+    if (t != t) return 0;
+    return (int)fminf(fmaxf(rintf(t), lo), hi);
+}
+
 // CTA = 32 output channels (one lane each) x all of K, K split over the 8 warps by 128-k
 // block; grid.y walks the rows in chunks of MB.
 template <int MB, bool GROUPED>
@@ -35,7 +42,8 @@ __global__ void __launch_bounds__(kDecThreads)
 gemm_decode_kernel(const int8_t* __restrict__ q, int M, int K, int N, int Npad,
                    const uint8_t* __restrict__ w_packed, const __half* __restrict__ w_scales,
                    const int32_t* __restrict__ scale_exp, __half* __restrict__ y,
-                   int32_t* __restrict__ acc_dump, Control* __restrict__ ctl, const float* __restrict__ chan_offset) {
+                   int32_t* __restrict__ acc_dump, Control* __restrict__ ctl, const float* __restrict__ chan_offset,
+                   int8_t* __restrict__ q_next, float next_inv, float next_lo, float next_hi) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) ctl->status = 0;   // this kernel has no bounded waits
     const int KB = K / kTileK;
@@ -145,7 +153,9 @@ gemm_decode_kernel(const int8_t* __restrict__ q, int M, int K, int N, int Npad,
             if (acc_dump) acc_dump[(size_t)(m0 + m) * N + n] = s;
             out = fmaf((float)s, __half2float(w_scales[n]), off) * pe;
         }
-        y[(size_t)(m0 + m) * N + n] = __float2half_rn(out);
+        const __half hv = __float2half_rn(out);
+        if (q_next) q_next[(size_t)(m0 + m) * N + n] = (int8_t)next_code(hv, next_inv, next_lo, next_hi);
+        else y[(size_t)(m0 + m) * N + n] = hv;
     }
 }
 
@@ -210,6 +220,8 @@ struct StreamParams {
     int32_t* acc_dump;
     Control* ctl;
     const float* chan_offset;
+    int8_t* q_next;
+    float next_inv, next_lo, next_hi;
 };
 
 // grid = (split, channel tiles), cluster = (split, 1, 1): the CTAs of a cluster share a channel
@@ -403,7 +415,9 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
             if (m < p.M) {
                 const int a = sm.sum[m][out_r] >> 4;                  // sums carry a factor 16
                 if (p.acc_dump) p.acc_dump[(size_t)m * p.N + out_n] = a;
-                p.y[(size_t)m * p.N + out_n] = __float2half_rn(fmaf((float)a, sc, off));
+                const __half hv = __float2half_rn(fmaf((float)a, sc, off));
+                if (p.q_next) p.q_next[(size_t)m * p.N + out_n] = (int8_t)next_code(hv, p.next_inv, p.next_lo, p.next_hi);
+                else p.y[(size_t)m * p.N + out_n] = hv;
             }
         }
     }
@@ -443,6 +457,10 @@ cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t
     p.M = a.M; p.K = a.K; p.N = a.N; p.Npad = round_up(a.N, kTileN);
     p.w_packed = a.w_packed; p.w_scales = a.w_scales; p.scale_exp = a.scale_exp;
     p.y = a.y; p.acc_dump = a.acc_dump; p.ctl = a.ctl; p.chan_offset = a.chan_offset;
+    p.q_next = a.q_next;
+    p.next_inv = ldexpf(1.0f, -a.next_exp);
+    p.next_lo = -(float)(1 << (a.next_bits - 1));
+    p.next_hi = (float)((1 << (a.next_bits - 1)) - 1);
     const int tiles = p.Npad / kTileN, KB = a.K / kTileK;
     // as many k ranges per tile (cluster size 1, 2 or 4: clusters of 7-8 measured slower) as keep
     // all CTAs resident at once (two per SM), and at least two k blocks per CTA
@@ -469,10 +487,12 @@ cudaError_t launch_mb(const GemmArgs& a, cudaStream_t stream) {
     dim3 grid(Npad / 32, (a.M + MB - 1) / MB);
     if (a.group)
         gemm_decode_kernel<MB, true><<<grid, kDecThreads, 0, stream>>>(
-            a.q, a.M, a.K, a.N, Npad, a.w_packed, a.w_scales, a.scale_exp, a.y, a.acc_dump, a.ctl, a.chan_offset);
+            a.q, a.M, a.K, a.N, Npad, a.w_packed, a.w_scales, a.scale_exp, a.y, a.acc_dump, a.ctl, a.chan_offset,
+            a.q_next, ldexpf(1.0f, -a.next_exp), -(float)(1 << (a.next_bits - 1)), (float)((1 << (a.next_bits - 1)) - 1));
     else
         gemm_decode_kernel<MB, false><<<grid, kDecThreads, 0, stream>>>(
-            a.q, a.M, a.K, a.N, Npad, a.w_packed, a.w_scales, a.scale_exp, a.y, a.acc_dump, a.ctl, a.chan_offset);
+            a.q, a.M, a.K, a.N, Npad, a.w_packed, a.w_scales, a.scale_exp, a.y, a.acc_dump, a.ctl, a.chan_offset,
+            a.q_next, ldexpf(1.0f, -a.next_exp), -(float)(1 << (a.next_bits - 1)), (float)((1 << (a.next_bits - 1)) - 1));
     return cudaGetLastError();
 }
 

@@ -218,12 +218,22 @@ struct TensorParams {
     int32_t* acc_dump;
     Control* ctl;
     const float* chan_offset;      // NULL or [N]: per-channel term added before the 2^e factor
+    int8_t* q_next;                // chaining: the next layer's codes [M][N] are written instead of y
+    float next_inv, next_lo, next_hi;   // 2^-next_exp and the code range of the next layer
     int y_tma;                     // outputs leave through y_map (needs N % 8 == 0 and a 16-byte aligned y)
 };
 
-// OFFSET: add the per-channel term of the zero-point variant. A separate instantiation, so that the
-// code of the plain kernels does not change with it.
-template <int BM, bool GROUPED, bool OFFSET>
+// The code the next layer's quantizer gives the fp16 output value (static exponent; NaN -> 0).
+__device__ __forceinline__ int chain_code(__half hv, float inv, float lo, float hi) {
+    const float t = __half2float(hv) * inv;                 // exact: inv is a power of two
+    if (t != t) return 0;
+    return (int)fminf(fmaxf(rintf(t), lo), hi);
+}
+
+// OFFSET: add the per-channel term of the zero-point variant. CHAIN: write the next layer's codes
+// instead of fp16 outputs. Separate instantiations, so that the code of the plain kernels does not
+// change with them.
+template <int BM, bool GROUPED, bool OFFSET, bool CHAIN>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap y_map,
                    const TensorParams p) {
@@ -452,9 +462,15 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
                         if (lane == 0) tma_store_wait_read();     // the previous store has read the staging rows
                         __syncwarp();
 #pragma unroll
-                        for (int c = 0; c < Smem::kStageRows; ++c)
-                            stage[c * 32 + lane] = __float2half_rn(OFFSET ? fmaf((float)(int)v[r0 + c], sc, off_pe)
-                                                                          : (float)(int)v[r0 + c] * sc);
+                        for (int c = 0; c < Smem::kStageRows; ++c) {
+                            const __half hv = __float2half_rn(OFFSET ? fmaf((float)(int)v[r0 + c], sc, off_pe)
+                                                                     : (float)(int)v[r0 + c] * sc);
+                            if constexpr (CHAIN)
+                                reinterpret_cast<int8_t*>(stage)[c * 32 + lane] =
+                                    (int8_t)chain_code(hv, p.next_inv, p.next_lo, p.next_hi);
+                            else
+                                stage[c * 32 + lane] = hv;
+                        }
                         fence_proxy_async();
                         __syncwarp();
                         if (lane == 0 && n0 < p.N && m_base + r0 < p.M) tma_store_2d(&y_map, stage, n0, m_base + r0);
@@ -463,9 +479,14 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
 #pragma unroll
                     for (int c = 0; c < kColsPerEpiWarp; ++c) {
                         const int m = m_base + c;
-                        if (n_ok && m < p.M)
-                            p.y[(size_t)m * p.N + n] =
+                        if (n_ok && m < p.M) {
+                            const __half hv =
                                 __float2half_rn(OFFSET ? fmaf((float)(int)v[c], sc, off_pe) : (float)(int)v[c] * sc);
+                            if constexpr (CHAIN)
+                                p.q_next[(size_t)m * p.N + n] = (int8_t)chain_code(hv, p.next_inv, p.next_lo, p.next_hi);
+                            else
+                                p.y[(size_t)m * p.N + n] = hv;
+                        }
                     }
                 }
                 if (p.acc_dump) {
@@ -526,7 +547,14 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
                     if (lane == 0) tma_store_wait_read();
                     __syncwarp();
 #pragma unroll
-                    for (int c = 0; c < kColsPerEpiWarp; ++c) stage[c * 32 + lane] = __float2half_rn(fsum[c] * pe);
+                    for (int c = 0; c < kColsPerEpiWarp; ++c) {
+                        const __half hv = __float2half_rn(fsum[c] * pe);
+                        if constexpr (CHAIN)
+                            reinterpret_cast<int8_t*>(stage)[c * 32 + lane] =
+                                (int8_t)chain_code(hv, p.next_inv, p.next_lo, p.next_hi);
+                        else
+                            stage[c * 32 + lane] = hv;
+                    }
                     fence_proxy_async();
                     __syncwarp();
                     const int n0 = nt * kTileN + quarter * 32;
@@ -535,7 +563,13 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
 #pragma unroll
                     for (int c = 0; c < kColsPerEpiWarp; ++c) {
                         const int m = m_base + c;
-                        if (n_ok && m < p.M) p.y[(size_t)m * p.N + n] = __float2half_rn(fsum[c] * pe);
+                        if (n_ok && m < p.M) {
+                            const __half hv = __float2half_rn(fsum[c] * pe);
+                            if constexpr (CHAIN)
+                                p.q_next[(size_t)m * p.N + n] = (int8_t)chain_code(hv, p.next_inv, p.next_lo, p.next_hi);
+                            else
+                                p.y[(size_t)m * p.N + n] = hv;
+                        }
                     }
                 }
             }
@@ -564,13 +598,13 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-template <int BM, bool GROUPED, bool OFFSET>
+template <int BM, bool GROUPED, bool OFFSET, bool CHAIN>
 cudaError_t launch_off(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
     using Smem = SharedStorage<BM>;
     const size_t smem_bytes = sizeof(Smem) + 1024;
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tensor_kernel<BM, GROUPED, OFFSET>,
+        cudaError_t e = cudaFuncSetAttribute(gemm_tensor_kernel<BM, GROUPED, OFFSET, CHAIN>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
         if (e != cudaSuccess) return e;
         attr_done = true;
@@ -588,7 +622,20 @@ cudaError_t launch_off(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t st
 
     CUtensorMap ymap = map;   // placeholder when the store path is off
     int y_tma = 0;
-    if (a.N % 8 == 0 && (reinterpret_cast<uintptr_t>(a.y) & 15u) == 0) {
+    if (CHAIN) {
+        // the staged rows hold one byte per value: a map over the code matrix, 32-byte rows
+        if (a.N % 16 == 0 && (reinterpret_cast<uintptr_t>(a.q_next) & 15u) == 0) {
+            const cuuint64_t ydims[2] = {(cuuint64_t)a.N, (cuuint64_t)a.M};
+            const cuuint64_t ystrides[1] = {(cuuint64_t)a.N};
+            const cuuint32_t ybox[2] = {32u, (cuuint32_t)Smem::kStageRows};
+            const CUresult ry = reinterpret_cast<EncodeTiledFn>(dev.encode_tiled)(
+                &ymap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, a.q_next, ydims, ystrides, ybox, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (ry != CUDA_SUCCESS) return cudaErrorInvalidValue;
+            y_tma = 1;
+        }
+    } else if (a.N % 8 == 0 && (reinterpret_cast<uintptr_t>(a.y) & 15u) == 0) {
         const cuuint64_t ydims[2] = {(cuuint64_t)a.N, (cuuint64_t)a.M};
         const cuuint64_t ystrides[1] = {(cuuint64_t)a.N * 2};
         const cuuint32_t ybox[2] = {32u, (cuuint32_t)Smem::kStageRows};
@@ -607,14 +654,23 @@ cudaError_t launch_off(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t st
     p.n_tiles = p.n_tiles_m * (p.Npad / kTileN);
     p.w_packed = a.w_packed; p.w_scales = a.w_scales; p.scale_exp = a.scale_exp;
     p.y = a.y; p.acc_dump = a.acc_dump; p.ctl = a.ctl; p.chan_offset = a.chan_offset;
+    p.q_next = a.q_next;
+    p.next_inv = ldexpf(1.0f, -a.next_exp);
+    p.next_lo = -(float)(1 << (a.next_bits - 1));
+    p.next_hi = (float)((1 << (a.next_bits - 1)) - 1);
     const int grid = p.n_tiles < dev.sm_count ? p.n_tiles : dev.sm_count;
-    gemm_tensor_kernel<BM, GROUPED, OFFSET><<<grid, kThreads, smem_bytes, stream>>>(map, ymap, p);
+    gemm_tensor_kernel<BM, GROUPED, OFFSET, CHAIN><<<grid, kThreads, smem_bytes, stream>>>(map, ymap, p);
     return cudaGetLastError();
 }
 
 template <int BM, bool GROUPED>
 cudaError_t launch_bm(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
-    return a.chan_offset ? launch_off<BM, GROUPED, true>(a, dev, stream) : launch_off<BM, GROUPED, false>(a, dev, stream);
+    if (a.q_next) {
+        if (a.chan_offset) return cudaErrorInvalidValue;       // the two variants are not combined
+        return launch_off<BM, GROUPED, false, true>(a, dev, stream);
+    }
+    return a.chan_offset ? launch_off<BM, GROUPED, true, false>(a, dev, stream)
+                         : launch_off<BM, GROUPED, false, false>(a, dev, stream);
 }
 
 }  // namespace
