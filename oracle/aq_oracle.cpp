@@ -434,6 +434,62 @@ void orc_linear_asym(const uint8_t* q, int zp, const int8_t* c, const uint16_t* 
     }
 }
 
+// ---------------------------------------------------------------------------
+// Log2 quantizer, Eq. 3 (used for the softmax output, Sec. 5.1):
+//     Q(x|b) = Sign(x) * CLIP( round( -log2( |x| / max|X| ) ), 0, 2^(b-1) - 1 ),
+// i.e. x is represented by Sign(x) * max|X| * 2^-k. Readings: the maximum is taken over the whole
+// tensor (layer-wise, like every activation scale here); Sign(0) = 0 makes the value 0, which needs a
+// code of its own, so the stored int8 is Sign(x) * (k + 1) and 0 stands for an exact zero; NaN is
+// ignored by the maximum and stored as 0; +-Inf count as +-65504. The rounding is decided in binary64:
+// every boundary 2^-(k+1/2) is irrational, no ratio of two halves comes closer to one than about 2^-24
+// relative, far more than the error of log2 in binary64.
+// Returns the maximum (as a float; 0 for an all-zero tensor, in which case every code is 0).
+// ---------------------------------------------------------------------------
+float orc_log2_quantize(const uint16_t* x, long long count, int bits, int8_t* codes) {
+    double mx = 0.0;
+    for (long long i = 0; i < count; ++i) {
+        double v = std::fabs((double)orc_half_to_float(x[i]));
+        if (std::isnan(v)) continue;
+        if (std::isinf(v)) v = 65504.0;
+        if (v > mx) mx = v;
+    }
+    const double kmax = (double)((1 << (bits - 1)) - 1);
+    for (long long i = 0; i < count; ++i) {
+        double v = (double)orc_half_to_float(x[i]);
+        if (std::isnan(v) || v == 0.0 || mx == 0.0) { codes[i] = 0; continue; }
+        if (std::isinf(v)) v = v > 0 ? 65504.0 : -65504.0;
+        const double k = std::min(std::max(std::nearbyint(-std::log2(std::fabs(v) / mx)), 0.0), kmax);
+        codes[i] = (int8_t)((v > 0 ? 1 : -1) * ((int)k + 1));
+    }
+    return (float)mx;
+}
+
+// Attention-times-value with such codes (Sec. 5.1; "shift-only" products): P [H][M][J] as log2 codes
+// with maximum p_max, V [H][J][D] as int8 codes with the layer exponent e_v:
+//     acc[h][m][d] = sum_j Sign_j * ( Vq[h][j][d] * 2^(kmax - k_j) )            (exact integers)
+//     y[h][m][d]   = fp16( p_max * 2^(e_v - kmax) * acc[h][m][d] )               (one rounding)
+void orc_attn_v_log2(const int8_t* pcodes, float p_max, const int8_t* vq, int e_v, int H, int M, int J, int D,
+                     int bits, long long* acc_out /* or NULL */, uint16_t* y) {
+    const int kmax = (1 << (bits - 1)) - 1;
+#pragma omp parallel for schedule(static)
+    for (int hm = 0; hm < H * M; ++hm) {
+        const int h = hm / M;
+        const int8_t* prow = pcodes + (size_t)hm * J;
+        for (int d = 0; d < D; ++d) {
+            long long a = 0;
+            for (int j = 0; j < J; ++j) {
+                const int c = prow[j];
+                if (c == 0) continue;
+                const int k = (c > 0 ? c : -c) - 1;
+                const long long term = (long long)vq[((size_t)h * J + j) * D + d] * (1LL << (kmax - k));
+                a += c > 0 ? term : -term;
+            }
+            if (acc_out) acc_out[(size_t)hm * D + d] = a;
+            y[(size_t)hm * D + d] = orc_double_to_half(std::ldexp((double)p_max * (double)a, e_v - kmax));
+        }
+    }
+}
+
 // Progressive pruning ratio, Eq. 9: gamma = 1 - (1 - beta)^(1/m).
 double orc_progressive_ratio(double beta, int m) { return 1.0 - std::pow(1.0 - beta, 1.0 / m); }
 

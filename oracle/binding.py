@@ -63,6 +63,10 @@ def lib():
         L.orc_progressive_ratio.argtypes = [C.c_double, C.c_int]
         L.orc_num_threads.restype = C.c_int
         L.orc_quantize_act_trip.restype = C.c_longlong
+        L.orc_log2_quantize.restype = C.c_float
+        L.orc_log2_quantize.argtypes = [C.c_void_p, C.c_longlong, C.c_int, C.c_void_p]
+        L.orc_attn_v_log2.argtypes = [C.c_void_p, C.c_float, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                      C.c_int, C.c_void_p, C.c_void_p]
     return _lib
 
 
@@ -238,6 +242,27 @@ def linear_asym(q: np.ndarray, zp: int, c: np.ndarray, scales: np.ndarray, e: in
     y = np.empty((M, N), np.float16)
     lib().orc_linear_asym(_p(q), zp, _p(c), _p(scales.view(np.uint16)), e, M, N, K, group, _p(acc),
                           _p(y.view(np.uint16)))
+    return acc, y
+
+
+def log2_quantize(x: np.ndarray, bits: int) -> Tuple[np.ndarray, float]:
+    """Eq. 3: (int8 codes Sign * (k + 1), 0 = zero; the tensor's max|x|)."""
+    xb = _half_bits(x)
+    codes = np.empty(x.shape, np.int8)
+    mx = lib().orc_log2_quantize(_p(xb), xb.size, bits, _p(codes))
+    return codes, float(mx)
+
+
+def attn_v_log2(pcodes: np.ndarray, p_max: float, vq: np.ndarray, e_v: int, bits: int):
+    """(int64 sums [H,M,D], fp16 y [H,M,D]) of log2-coded P [H,M,J] times int8-coded V [H,J,D]."""
+    pcodes = _c(pcodes, np.int8)
+    vq = _c(vq, np.int8)
+    H, M, J = pcodes.shape
+    D = vq.shape[2]
+    assert vq.shape == (H, J, D)
+    acc = np.empty((H, M, D), np.int64)
+    y = np.empty((H, M, D), np.float16)
+    lib().orc_attn_v_log2(_p(pcodes), p_max, _p(vq), e_v, H, M, J, D, bits, _p(acc), _p(y.view(np.uint16)))
     return acc, y
 
 

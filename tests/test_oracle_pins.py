@@ -570,3 +570,71 @@ def test_asym_layer_brute_force_and_zero_point_identity():
         # one rounding of the exact value
         exact = (ref.astype(np.float64) * sc.astype(np.float64)[None, :, :]).sum(axis=2) * 2.0 ** e
         assert np.array_equal(y, exact.astype(np.float16))
+
+
+# ------------------------------------------------------- log2 quantizer and attention x value (Eq. 3)
+def test_log2_quantizer_hand_worked_table():
+    for line in open(os.path.join(GOLDEN, "log2_hand_worked.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        bits, mx, xv, stored = line.split()
+        x = np.array([float(mx), float(xv)], np.float16)
+        codes, got_max = oracle.log2_quantize(x, int(bits))
+        assert got_max == float(np.float16(float(mx)))
+        assert int(codes[1]) == int(stored), line
+        assert int(codes[0]) == 1                                  # the maximum itself has k = 0
+
+
+def test_log2_quantizer_against_exact_integer_rule_and_invariants():
+    # round(-log2 r) for r = (ma * 2^ea) / (mb * 2^eb) decided with integers only: the fractional part of
+    # log2 reaches one half exactly when the mantissa ratio reaches sqrt(2), i.e. when its square reaches 2
+    from fractions import Fraction as F
+    g = np.random.Generator(np.random.Philox(key=123))
+    x = (g.standard_normal(4000) * np.exp2(g.integers(-12, 3, size=4000))).astype(np.float16)
+    x[:5] = [0.0, -0.0, np.nan, 6.0, -6.0]
+    for bits in (4, 8):
+        codes, mx = oracle.log2_quantize(x, bits)
+        kmax = (1 << (bits - 1)) - 1
+        assert mx == float(np.nanmax(np.abs(x.astype(np.float64))))
+        for xv, c in zip(x.tolist(), codes.tolist()):
+            if xv != xv or xv == 0.0:
+                assert c == 0
+                continue
+            r = F(abs(xv)) / F(mx)                                 # exact ratio, 0 < r <= 1
+            k = 0
+            while r * 2 <= 1:                                      # bring r into (1/2, 1]
+                r *= 2
+                k += 1
+            if r * r < F(1, 2):                                    # below 2^-1/2: rounds up to the next k
+                k += 1
+            k = min(k, kmax)
+            assert c == (1 if xv > 0 else -1) * (k + 1), (xv, mx, c, k)
+            if k < kmax:                                           # the value lies within half a binade of 2^-k
+                assert 2.0 ** (-(k + 0.5)) < abs(xv) / mx <= 2.0 ** (-(k - 0.5))
+
+
+def test_attn_v_log2_brute_force_and_shift_form():
+    g = np.random.Generator(np.random.Philox(key=321))
+    H, M, J, D, bits = 2, 5, 40, 16, 4
+    kmax = 7
+    pc = g.integers(-8, 9, size=(H, M, J)).astype(np.int8)
+    vq = g.integers(-128, 128, size=(H, J, D)).astype(np.int8)
+    p_max, e_v = 0.8125, -3
+    acc, y = oracle.attn_v_log2(pc, p_max, vq, e_v, bits)
+    ref = np.zeros((H, M, D), dtype=object)
+    for h in range(H):
+        for m in range(M):
+            for j in range(J):
+                c = int(pc[h, m, j])
+                if c == 0:
+                    continue
+                sh = kmax - (abs(c) - 1)
+                for d in range(D):
+                    t = int(vq[h, j, d]) << sh                     # the product is a shift
+                    ref[h, m, d] += t if c > 0 else -t
+    assert np.array_equal(acc, ref.astype(np.int64))
+    exact = ref.astype(np.float64) * p_max * 2.0 ** (e_v - kmax)
+    assert np.array_equal(y, exact.astype(np.float16))
+    # the dequantized operands give the same number: p_hat = p_max * sign * 2^-k, v_hat = vq * 2^e_v
+    p_hat = np.where(pc == 0, 0.0, np.sign(pc) * p_max * np.exp2(-(np.abs(pc.astype(np.float64)) - 1)))
+    assert np.allclose(np.einsum("hmj,hjd->hmd", p_hat, vq.astype(np.float64) * 2.0 ** e_v), exact, rtol=1e-12)
