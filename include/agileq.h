@@ -205,6 +205,24 @@ int aq_linear_w4a4_chain(aq_handle_t h, const void* x_fp16, int M, int K, const 
                          int8_t* q_next, int next_bits, int next_exp, int32_t* acc_dump, void* workspace,
                          size_t workspace_bytes, void* stream);
 
+/* ---- log2 quantization of the softmax output and attention x value (paper Eq. 3, Sec. 5.1)
+ * aq_log2_quantize: x_fp16 holds `count` values (any shape); max|x| is taken over all of them.
+ *   k = CLIP(round(-log2(|x| / max|x|)), 0, 2^(b-1) - 1), so x ~ Sign(x) * max|x| * 2^-k. codes (int8, same
+ *   shape) hold Sign(x) * (k + 1), and 0 for an exact zero (Eq. 3's Sign(0) = 0) and for NaN; +-Inf count as
+ *   65504. max_bits_out (device, may be NULL) receives the fp16 bit pattern of max|x| in its low 16 bits.
+ *   bits 8 or 4. The rounding is exact (decided with integers).
+ * aq_attn_v_log2: P as such codes [H,M,J] (H heads, M query rows, J key rows) times V as int8 codes
+ *   [H,J,D] of aq_quantize_act (with its exponent on the device):
+ *     acc[h,m,d] = sum_j Sign_j * (v[h,j,d] << (kmax - k_j)),   y = fp16(max|P| * 2^(e_v - kmax) * acc).
+ *   Every product is a shift. bits must be 4 (kmax = 7: with 8-bit codes the shifts would reach 127 and
+ *   no integer accumulator holds them). D % 4 == 0, 256 % (D/4) == 0, D <= 1024, J <= 65536. acc_dump: NULL
+ *   or int32 [H,M,D]. */
+int aq_log2_quantize(aq_handle_t h, const void* x_fp16, long long count, int bits, int8_t* codes,
+                     uint32_t* max_bits_out, void* workspace, size_t workspace_bytes, void* stream);
+int aq_attn_v_log2(aq_handle_t h, const int8_t* p_codes, const uint32_t* p_max_bits, const int8_t* v_codes,
+                   const int32_t* v_scale_exp, int H, int M, int J, int D, int bits, void* y_fp16, int32_t* acc_dump,
+                   void* stream);
+
 /* ---- progressive pruning schedule (paper Eq. 9; host only, no GPU work)
  * With pruning at m layers and the ratio beta of tokens to be gone after the last of them, every
  * pruning layer drops the fraction gamma = 1 - (1 - beta)^(1/m) of what reaches it. Writes

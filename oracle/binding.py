@@ -255,6 +255,7 @@ def log2_quantize(x: np.ndarray, bits: int) -> Tuple[np.ndarray, float]:
 
 def attn_v_log2(pcodes: np.ndarray, p_max: float, vq: np.ndarray, e_v: int, bits: int):
     """(int64 sums [H,M,D], fp16 y [H,M,D]) of log2-coded P [H,M,J] times int8-coded V [H,J,D]."""
+    assert bits <= 5, "the shift form needs kmax <= 15"
     pcodes = _c(pcodes, np.int8)
     vq = _c(vq, np.int8)
     H, M, J = pcodes.shape

@@ -82,6 +82,8 @@ def load():
     lin_chain = [vp, vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, vp, i32, i32, vp, vp, sz, vp]
     L.aq_linear_w4a8_chain.argtypes = lin_chain
     L.aq_linear_w4a4_chain.argtypes = lin_chain
+    L.aq_log2_quantize.argtypes = [vp, vp, C.c_longlong, i32, vp, vp, vp, sz, vp]
+    L.aq_attn_v_log2.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp]
     L.aq_prune_schedule.argtypes = [i32, C.c_double, i32, vp, vp]
     L.aq_trip_calibrate.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
     L.aq_quantize_act_trip.argtypes = [vp, vp, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
@@ -226,6 +228,25 @@ class Handle:
                        clip_shift_or_exp=0, row_idx=None, y=None, acc_dump=None, workspace=None):
         return self._linear(load().aq_linear_w4a4, "aq_linear_w4a4", x, packed, scales, N, group_size,
                             scale_mode, clip_shift_or_exp, row_idx, y, acc_dump, workspace)
+
+    # ---- log2 codes of the softmax output and attention x value (Eq. 3)
+    def aq_log2_quantize(self, x: torch.Tensor, bits: int) -> Tuple[torch.Tensor, torch.Tensor]:
+        """(int8 codes of x's shape, uint32[1] holding the fp16 bits of max|x|)."""
+        codes = torch.empty(x.shape, dtype=torch.int8, device=x.device)
+        mx = torch.zeros(1, dtype=torch.int32, device=x.device)
+        ws = torch.empty(256, dtype=torch.uint8, device=x.device)
+        _check(load().aq_log2_quantize(self._h, _ptr(x), x.numel(), bits, _ptr(codes), _ptr(mx), _ptr(ws), ws.numel(),
+                                       _stream()), "aq_log2_quantize")
+        return codes, mx
+
+    def aq_attn_v_log2(self, p_codes, p_max_bits, v_codes, v_scale_exp, bits, y=None, acc_dump=None):
+        H, M, J = p_codes.shape
+        D = v_codes.shape[2]
+        if y is None:
+            y = torch.empty((H, M, D), dtype=torch.float16, device=p_codes.device)
+        _check(load().aq_attn_v_log2(self._h, _ptr(p_codes), _ptr(p_max_bits), _ptr(v_codes), _ptr(v_scale_exp), H, M, J,
+                                     D, bits, _ptr(y), _ptr(acc_dump), _stream()), "aq_attn_v_log2")
+        return y
 
     # ---- chaining: the next layer's codes instead of fp16 outputs (Sec. 4.4)
     def aq_linear_chain(self, bits, x, packed, scales, N, group_size, next_bits, next_exp,

@@ -441,6 +441,35 @@ int aq_linear_w4a4_chain(aq_handle_t h, const void* x_fp16, int M, int K, const 
                        next_exp);
 }
 
+int aq_log2_quantize(aq_handle_t h, const void* x_fp16, long long count, int bits, int8_t* codes,
+                     uint32_t* max_bits_out, void* workspace, size_t workspace_bytes_, void* stream_) {
+    if (!h || !x_fp16 || !codes || count < 1 || (bits != 8 && bits != 4)) return AQ_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes_ < sizeof(Control)) return AQ_ERR_WORKSPACE;
+    if (!aligned(x_fp16, 2) || !aligned(workspace, 256) || (max_bits_out && !aligned(max_bits_out, 4)))
+        return AQ_ERR_ALIGNMENT;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    Control* ctl = static_cast<Control*>(workspace);
+    cudaError_t e = cudaMemsetAsync(ctl, 0, sizeof(Control), stream);
+    if (e == cudaSuccess)
+        e = launch_log2_quantize(static_cast<const __half*>(x_fp16), count, bits, ctl, codes, max_bits_out, h->dev, stream);
+    return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
+int aq_attn_v_log2(aq_handle_t h, const int8_t* p_codes, const uint32_t* p_max_bits, const int8_t* v_codes,
+                   const int32_t* v_scale_exp, int H, int M, int J, int D, int bits, void* y_fp16, int32_t* acc_dump,
+                   void* stream) {
+    if (!h || !p_codes || !p_max_bits || !v_codes || !v_scale_exp || !y_fp16) return AQ_ERR_INVALID_ARG;
+    if (bits != 4) return AQ_ERR_INVALID_ARG;          // shifts up to kmax = 7; 8-bit codes would shift by up to 127
+    if (H < 1 || M < 1 || J < 1 || J > 65536 || D < 4 || D > 1024 || D % 4 != 0 || 256 % (D / 4) != 0 || H > 65535)
+        return AQ_ERR_SHAPE;
+    if (!aligned(v_codes, 4) || !aligned(y_fp16, 2) || !aligned(p_max_bits, 4) || !aligned(v_scale_exp, 4) ||
+        (acc_dump && !aligned(acc_dump, 4)))
+        return AQ_ERR_ALIGNMENT;
+    const cudaError_t e = launch_attn_v_log2(p_codes, p_max_bits, v_codes, v_scale_exp, H, M, J, D, bits,
+                                             static_cast<__half*>(y_fp16), acc_dump, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
 int aq_prune_schedule(int M, double beta, int m, int32_t* n_keep_out, double* gamma_out) {
     if (M < 1 || m < 1 || !(beta >= 0.0) || !(beta < 1.0) || !n_keep_out) return AQ_ERR_INVALID_ARG;
     const double gamma = 1.0 - pow(1.0 - beta, 1.0 / (double)m);       // Eq. 9

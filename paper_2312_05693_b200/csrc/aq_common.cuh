@@ -116,6 +116,12 @@ cudaError_t launch_weight_offsets(const uint8_t* packed, const __half* scales, i
 // off[n] = -(zp - 2^(b-1)) * r[n] with zp from the control block.
 cudaError_t launch_chan_offsets(const float* r, int N, int bits, const Control* ctl, float* off, cudaStream_t stream);
 
+// Log2 codes of Eq. 3 (two kernels: layer maximum, codes) and attention x value on them (aq_attn.cu).
+cudaError_t launch_log2_quantize(const __half* x, long long count, int bits, Control* ctl, int8_t* codes,
+                                 uint32_t* max_bits_out, const DeviceInfo& dev, cudaStream_t stream);
+cudaError_t launch_attn_v_log2(const int8_t* pcodes, const uint32_t* max_bits, const int8_t* vq, const int32_t* e_v,
+                               int H, int M, int J, int D, int bits, __half* y, int32_t* acc_dump, cudaStream_t stream);
+
 cudaError_t launch_token_select(const float* scores, int M, int n_keep, int32_t* idx, void* scratch,
                                 cudaStream_t stream);
 cudaError_t launch_token_compact(const __half* x, int K, const int32_t* idx, int n_keep, __half* out,

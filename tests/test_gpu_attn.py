@@ -1,0 +1,79 @@
+"""Log2 codes of the softmax output (paper Eq. 3) and attention x value on them, against the CPU checker."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2312_05693_b200 import binding, inputs
+from gpu_util import assert_y_close, dev, handle
+
+pytestmark = pytest.mark.gpu
+
+
+def _softmax_rows(H, M, J, seed):
+    g = np.random.Generator(np.random.Philox(key=seed))
+    s = g.standard_normal((H, M, J)).astype(np.float32) * 3.0
+    s -= s.max(axis=2, keepdims=True)
+    p = np.exp(s)
+    p /= p.sum(axis=2, keepdims=True)
+    return p.astype(np.float16)
+
+
+@pytest.mark.parametrize("bits", [4, 8])
+def test_log2_quantize_matches_checker(bits):
+    h = handle()
+    p = _softmax_rows(3, 37, 200, 51)
+    codes, mx = h.aq_log2_quantize(dev(p), bits)
+    ref, mref = oracle.log2_quantize(p, bits)
+    assert np.float16(mref).view(np.uint16) == (int(mx.item()) & 0xFFFF)
+    assert np.array_equal(codes.cpu().numpy(), ref)
+    # general values: both signs, zeros, subnormals, NaN, Inf, every binade
+    g = np.random.Generator(np.random.Philox(key=52))
+    x = (g.standard_normal(70000) * np.exp2(g.integers(-24, 8, size=70000))).astype(np.float16)
+    x[:6] = [0.0, -0.0, np.nan, 6e-8, -6e-8, 1.0]
+    for extra in (None, np.inf):
+        if extra is not None:
+            x[10] = extra
+        codes, mx = h.aq_log2_quantize(dev(x), bits)
+        ref, mref = oracle.log2_quantize(x, bits)
+        assert np.float16(mref).view(np.uint16) == (int(mx.item()) & 0xFFFF)
+        assert np.array_equal(codes.cpu().numpy(), ref)
+    z = np.zeros(64, np.float16)
+    codes, mx = h.aq_log2_quantize(dev(z), bits)
+    assert int(mx.item()) == 0 and not codes.any().item()
+
+
+@pytest.mark.parametrize("H,M,J,D", [(2, 33, 70, 128), (4, 128, 256, 128), (1, 5, 9, 256)])
+def test_attn_v_log2_matches_checker(H, M, J, D):
+    bits = 4
+    h = handle()
+    p = _softmax_rows(H, M, J, 53)
+    v = inputs.activations(H * J, D, seed=54, outlier_frac=0.01, outlier_mult=8.0)
+    pc, pmax = h.aq_log2_quantize(dev(p), bits)
+    vq, ev = h.aq_quantize_act(dev(v), 8)
+    acc = torch.full((H, M, D), -1, dtype=torch.int32, device="cuda")
+    y = h.aq_attn_v_log2(pc, pmax, vq.reshape(H, J, D), ev, bits, acc_dump=acc)
+    pc_ref, pmax_ref = oracle.log2_quantize(p, bits)
+    e_ref = oracle.layer_exponent(v, 8)
+    vq_ref = oracle.quantize_act(v, 8, e_ref).reshape(H, J, D)
+    assert np.array_equal(pc.cpu().numpy(), pc_ref) and int(ev.item()) == e_ref
+    acc_ref, y_ref = oracle.attn_v_log2(pc_ref, pmax_ref, vq_ref, e_ref, bits)
+    assert np.array_equal(acc.cpu().numpy().astype(np.int64), acc_ref)
+    assert_y_close(y.cpu().numpy().reshape(H * M, D), y_ref.reshape(H * M, D))
+    # and the codes carry the attention: against the unquantized product
+    exact = np.einsum("hmj,hjd->hmd", p.astype(np.float64), v.astype(np.float64).reshape(H, J, D))
+    err = np.abs(y.cpu().numpy().astype(np.float64) - exact).max()
+    assert err < 0.5 * np.abs(exact).max()
+
+
+def test_attn_bad_shapes_are_refused():
+    h = handle()
+    pc = torch.zeros((1, 4, 8), dtype=torch.int8, device="cuda")
+    mx = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for D in (6, 12, 2048):
+        vq = torch.zeros((1, 8, D), dtype=torch.int8, device="cuda")
+        with pytest.raises(binding.AgileqError):
+            h.aq_attn_v_log2(pc, mx, vq, ev, 4)
+    with pytest.raises(binding.AgileqError):
+        h.aq_attn_v_log2(pc, mx, torch.zeros((1, 8, 128), dtype=torch.int8, device="cuda"), ev, 8)   # 4-bit codes only
