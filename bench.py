@@ -360,6 +360,27 @@ def bench_chain(h, reps=30):
             "codes_between": {"us": t_chain * 1e3, "TOPS": ops / (t_chain * 1e-3) / 1e12}}
 
 
+def bench_attention(h, reps=5):
+    """Softmax output as 4-bit log2 codes times int8 value codes (Eq. 3), LLaMA-7B attention shape."""
+    H, M, J, D = 32, 2048, 2048, 128
+    g = torch.Generator(device="cuda").manual_seed(7)
+    scores = torch.randn((H, M, J), generator=g, device="cuda", dtype=torch.float32) * 3.0
+    p = torch.softmax(scores, dim=2).to(torch.float16)           # synthetic attention probabilities (input only)
+    del scores
+    v = torch.from_numpy(inputs.activations(H * J, D, 7, 0.01, 8.0)).cuda()
+    vq, ev = h.aq_quantize_act(v, 8)
+    vq = vq.reshape(H, J, D)
+    pc, pmax = h.aq_log2_quantize(p, 4)
+    y = torch.empty((H, M, D), dtype=torch.float16, device="cuda")
+    t_q = _event_ms(lambda: h.aq_log2_quantize(p, 4), reps)
+    t_av = _event_ms(lambda: h.aq_attn_v_log2(pc, pmax, vq, ev, 4, y=y), reps)
+    macs = float(H) * M * J * D
+    return {"H": H, "M": M, "J": J, "D": D,
+            "log2_quantize": {"us": t_q * 1e3, "GBps": 3.0 * H * M * J / (t_q * 1e-3) / 1e9},
+            "attn_v": {"us": t_av * 1e3, "Gshift_add_per_s": macs / (t_av * 1e-3) / 1e9,
+                       "note": "CUDA-core kernel: one shift and one add per product, no tensor cores"}}
+
+
 def bench_pruned(h, reps=10):
     wl = inputs.WORKLOADS["opt30b_pruned_prefill_w4a8"]
     M = wl.Ms[0]
@@ -590,7 +611,7 @@ def main():
             line["decode"] = {"error": repr(ex)}
     if rank == 0 and world == 1 and not args.no_decode:
         for key, fn in (("w4a4", bench_w4a4), ("zero_point", bench_zero_point), ("chain", bench_chain),
-                        ("pruned_prefill", bench_pruned)):
+                        ("attention_log2", bench_attention), ("pruned_prefill", bench_pruned)):
             try:
                 line[key] = fn(h)
             except Exception as ex:  # report, do not hide

@@ -222,6 +222,16 @@ int aq_log2_quantize(aq_handle_t h, const void* x_fp16, long long count, int bit
 int aq_attn_v_log2(aq_handle_t h, const int8_t* p_codes, const uint32_t* p_max_bits, const int8_t* v_codes,
                    const int32_t* v_scale_exp, int H, int M, int J, int D, int bits, void* y_fp16, int32_t* acc_dump,
                    void* stream);
+/* The same result on the tensor cores for a non-negative P (a softmax output), 4-bit codes: the factor
+ * 2^(kmax - k) is then an unsigned byte and the sums are a u8 x s8 -> s32 contraction over j
+ * (tcgen05.mma kind::i8, operands staged by TMA, accumulator in tensor memory). D is 64 or 128,
+ * J % 16 == 0; y must be 16-byte aligned. The workspace (aq_attn_workspace_bytes) holds a control block,
+ * the byte factors and the transposed value codes. A negative code in P is an error: it is counted as 0
+ * and aq_check_workspace on this workspace then returns AQ_ERR_INVALID_ARG. */
+size_t aq_attn_workspace_bytes(int H, int M, int J, int D);
+int aq_attn_v_log2_tc(aq_handle_t h, const int8_t* p_codes, const uint32_t* p_max_bits, const int8_t* v_codes,
+                      const int32_t* v_scale_exp, int H, int M, int J, int D, void* y_fp16, void* workspace,
+                      size_t workspace_bytes, void* stream);
 
 /* ---- progressive pruning schedule (paper Eq. 9; host only, no GPU work)
  * With pruning at m layers and the ratio beta of tokens to be gone after the last of them, every

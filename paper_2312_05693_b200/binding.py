@@ -84,6 +84,9 @@ def load():
     L.aq_linear_w4a4_chain.argtypes = lin_chain
     L.aq_log2_quantize.argtypes = [vp, vp, C.c_longlong, i32, vp, vp, vp, sz, vp]
     L.aq_attn_v_log2.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp]
+    L.aq_attn_workspace_bytes.restype = sz
+    L.aq_attn_workspace_bytes.argtypes = [i32, i32, i32, i32]
+    L.aq_attn_v_log2_tc.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, sz, vp]
     L.aq_prune_schedule.argtypes = [i32, C.c_double, i32, vp, vp]
     L.aq_trip_calibrate.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
     L.aq_quantize_act_trip.argtypes = [vp, vp, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
@@ -247,6 +250,18 @@ class Handle:
         _check(load().aq_attn_v_log2(self._h, _ptr(p_codes), _ptr(p_max_bits), _ptr(v_codes), _ptr(v_scale_exp), H, M, J,
                                      D, bits, _ptr(y), _ptr(acc_dump), _stream()), "aq_attn_v_log2")
         return y
+
+    def aq_attn_v_log2_tc(self, p_codes, p_max_bits, v_codes, v_scale_exp, y=None, workspace=None):
+        H, M, J = p_codes.shape
+        D = v_codes.shape[2]
+        if y is None:
+            y = torch.empty((H, M, D), dtype=torch.float16, device=p_codes.device)
+        if workspace is None:
+            workspace = torch.empty(load().aq_attn_workspace_bytes(H, M, J, D), dtype=torch.uint8, device=p_codes.device)
+        _check(load().aq_attn_v_log2_tc(self._h, _ptr(p_codes), _ptr(p_max_bits), _ptr(v_codes), _ptr(v_scale_exp), H, M,
+                                        J, D, _ptr(y), _ptr(workspace), workspace.numel(), _stream()),
+               "aq_attn_v_log2_tc")
+        return y, workspace
 
     # ---- chaining: the next layer's codes instead of fp16 outputs (Sec. 4.4)
     def aq_linear_chain(self, bits, x, packed, scales, N, group_size, next_bits, next_exp,

@@ -470,6 +470,30 @@ int aq_attn_v_log2(aq_handle_t h, const int8_t* p_codes, const uint32_t* p_max_b
     return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
 }
 
+size_t aq_attn_workspace_bytes(int H, int M, int J, int D) {
+    if (H < 1 || M < 1 || J < 1 || D < 1) return 0;
+    return sizeof(Control) + attn_tc_scratch_bytes(H, M, J, D);
+}
+
+int aq_attn_v_log2_tc(aq_handle_t h, const int8_t* p_codes, const uint32_t* p_max_bits, const int8_t* v_codes,
+                      const int32_t* v_scale_exp, int H, int M, int J, int D, void* y_fp16, void* workspace,
+                      size_t workspace_bytes_, void* stream_) {
+    if (!h || !p_codes || !p_max_bits || !v_codes || !v_scale_exp || !y_fp16) return AQ_ERR_INVALID_ARG;
+    if (H < 1 || H > 65535 || M < 1 || J < 16 || J > 65536 || J % 16 != 0 || (D != 64 && D != 128)) return AQ_ERR_SHAPE;
+    if ((long long)H * M > 0x7FFFFFFFll || (long long)H * D > 0x7FFFFFFFll) return AQ_ERR_SHAPE;
+    if (!workspace || workspace_bytes_ < aq_attn_workspace_bytes(H, M, J, D)) return AQ_ERR_WORKSPACE;
+    if (!aligned(p_codes, 4) || !aligned(v_codes, 1) || !aligned(y_fp16, 16) || !aligned(p_max_bits, 4) ||
+        !aligned(v_scale_exp, 4) || !aligned(workspace, 256))
+        return AQ_ERR_ALIGNMENT;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    Control* ctl = static_cast<Control*>(workspace);
+    cudaError_t e = cudaMemsetAsync(ctl, 0, sizeof(Control), stream);
+    if (e == cudaSuccess)
+        e = launch_attn_v_log2_tc(p_codes, p_max_bits, v_codes, v_scale_exp, H, M, J, D, static_cast<__half*>(y_fp16), ctl,
+                                  static_cast<uint8_t*>(workspace) + sizeof(Control), h->dev, stream);
+    return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
 int aq_prune_schedule(int M, double beta, int m, int32_t* n_keep_out, double* gamma_out) {
     if (M < 1 || m < 1 || !(beta >= 0.0) || !(beta < 1.0) || !n_keep_out) return AQ_ERR_INVALID_ARG;
     const double gamma = 1.0 - pow(1.0 - beta, 1.0 / (double)m);       // Eq. 9
@@ -521,6 +545,7 @@ int aq_check_workspace(aq_handle_t h, const void* workspace, void* stream_) {
     Control c;
     e = cudaMemcpy(&c, workspace, sizeof(Control), cudaMemcpyDeviceToHost);
     if (e != cudaSuccess) return cuda_fail(h, e);
+    if (c.status == 11u) return AQ_ERR_INVALID_ARG;     // aq_attn_v_log2_tc met a negative code
     return c.status ? AQ_ERR_DEVICE_TIMEOUT : AQ_OK;
 }
 

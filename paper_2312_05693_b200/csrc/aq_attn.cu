@@ -1,5 +1,7 @@
 // Log2 quantization of the softmax output (paper Eq. 3, Sec. 5.1) and the attention-times-value
 // product on its codes, where every product is a shift of the int8 value code.
+#include <cuda.h>
+
 #include "aq_common.cuh"
 
 namespace aq {
@@ -100,7 +102,291 @@ attn_v_log2_kernel(const int8_t* __restrict__ pcodes, const uint32_t* __restrict
     if (acc_dump) { acc_dump[o] = a0; acc_dump[o + 1] = a1; acc_dump[o + 2] = a2; acc_dump[o + 3] = a3; }
 }
 
+// ---- the same product on the tensor cores (non-negative P, i.e. a softmax output) --------------
+// With P >= 0 the factor 2^(kmax - k) is an unsigned byte (1..128), so the product is a plain
+// u8 x s8 -> s32 contraction over the key index j: acc[m][d] = sum_j w[m][j] * v[d][j], with both
+// operands stored j-major. tcgen05.mma kind::i8 reads both from shared memory (128-byte swizzle,
+// staged by TMA); the accumulator [128 query rows x D] lives in tensor memory.
+
+// codes -> weights: c > 0 -> 128 >> (c - 1); 0 -> 0; a negative code is not representable here:
+// it is recorded in the status word (11) and treated as 0.
+__global__ void __launch_bounds__(256)
+log2_weights_kernel(const int8_t* __restrict__ codes, long long count, uint8_t* __restrict__ w, Control* __restrict__ ctl) {
+    bool bad = false;
+    for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4; i < count; i += (long long)gridDim.x * blockDim.x * 4) {
+        if (i + 4 <= count) {
+            const char4 c = *reinterpret_cast<const char4*>(codes + i);
+            uchar4 o;
+            o.x = c.x > 0 ? (uint8_t)(128u >> (c.x - 1)) : 0; bad |= c.x < 0;
+            o.y = c.y > 0 ? (uint8_t)(128u >> (c.y - 1)) : 0; bad |= c.y < 0;
+            o.z = c.z > 0 ? (uint8_t)(128u >> (c.z - 1)) : 0; bad |= c.z < 0;
+            o.w = c.w > 0 ? (uint8_t)(128u >> (c.w - 1)) : 0; bad |= c.w < 0;
+            *reinterpret_cast<uchar4*>(w + i) = o;
+        } else {
+            for (long long t = i; t < count; ++t) {
+                const int c = codes[t];
+                w[t] = c > 0 ? (uint8_t)(128u >> (c - 1)) : 0;
+                bad |= c < 0;
+            }
+        }
+    }
+    if (bad) atomicCAS(&ctl->status, 0u, 11u);
+}
+
+// [H][J][D] int8 -> [H][D][J] int8 through a 32 x 32 shared-memory tile.
+__global__ void __launch_bounds__(256)
+transpose_i8_kernel(const int8_t* __restrict__ in, int J, int D, int8_t* __restrict__ out) {
+    __shared__ int8_t tile[32][33];
+    const int h = blockIdx.z, j0 = blockIdx.x * 32, d0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;          // 32 x 8
+    for (int r = ty; r < 32; r += 8) {
+        const int j = j0 + r, d = d0 + tx;
+        tile[r][tx] = (j < J && d < D) ? in[((size_t)h * J + j) * D + d] : (int8_t)0;
+    }
+    __syncthreads();
+    for (int r = ty; r < 32; r += 8) {
+        const int d = d0 + r, j = j0 + tx;
+        if (d < D && j < J) out[((size_t)h * D + d) * J + j] = tile[tx][r];
+    }
+}
+
+constexpr int kTcStages = 4;
+constexpr int kTcThreads = 192;                      // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+constexpr unsigned long long kTcWaitCycles = 4000000000ull;
+
+__device__ __forceinline__ uint32_t a_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool a_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(a_smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait; false when the limit ran out or another role gave up.
+__device__ __forceinline__ bool a_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+    if (a_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t spins = 0;
+    while (!a_try_wait(bar, parity)) {
+        if ((++spins & 0x3FFu) == 0) {
+            if (*abort_flag) return false;
+            if ((unsigned long long)(clock64() - t0) > kTcWaitCycles) { *abort_flag = 12u; return false; }
+        }
+    }
+    return true;
+}
+// K-major tile with 128-byte rows written by TMA with the 128-byte swizzle (see aq_gemm_tensor.cu).
+__device__ __forceinline__ uint64_t a_desc_sw128(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+template <int DN>
+struct AttnSmem {
+    alignas(1024) uint8_t a[kTcStages][128 * 128];   // weights tile: 128 query rows x 128 j
+    alignas(1024) uint8_t b[kTcStages][DN * 128];    // value tile: DN columns x 128 j
+    alignas(8) uint64_t full[kTcStages];
+    uint64_t empty[kTcStages];
+    uint64_t acc_full;
+    uint32_t tmem_base;
+    volatile uint32_t abort_flag;
+};
+
+// One CTA per (head, 128 query rows).
+template <int DN>
+__global__ void __launch_bounds__(kTcThreads, 1)
+attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__ CUtensorMap b_map,
+                 const uint32_t* __restrict__ max_bits, const int32_t* __restrict__ e_v, int M, int J,
+                 __half* __restrict__ y, Control* __restrict__ ctl) {
+    extern __shared__ uint8_t attn_smem_raw[];
+    using Smem = AttnSmem<DN>;
+    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(attn_smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int h = blockIdx.y, m0 = blockIdx.x * 128;
+    const int JB = (J + 127) / 128;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kTcStages; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(a_smem_u32(&sm.full[s])) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(a_smem_u32(&sm.empty[s])) : "memory");
+        }
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(a_smem_u32(&sm.acc_full)) : "memory");
+        sm.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(a_smem_u32(&sm.tmem_base)), "r"((uint32_t)DN) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = sm.tmem_base;
+    volatile uint32_t* abort_flag = &sm.abort_flag;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int jb = 0; jb < JB; ++jb) {
+                const int s = jb % kTcStages;
+                if (!a_wait(&sm.empty[s], ((jb / kTcStages) & 1) ^ 1, abort_flag)) break;
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
+                             ::"r"(a_smem_u32(&sm.full[s])), "r"((uint32_t)((128 + DN) * 128)) : "memory");
+                asm volatile(
+                    "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                    ::"r"(a_smem_u32(sm.a[s])), "l"(&a_map), "r"(jb * 128), "r"(h * M + m0), "r"(a_smem_u32(&sm.full[s]))
+                    : "memory");
+                asm volatile(
+                    "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                    ::"r"(a_smem_u32(sm.b[s])), "l"(&b_map), "r"(jb * 128), "r"(h * DN), "r"(a_smem_u32(&sm.full[s]))
+                    : "memory");
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // D = s32 (2 at bits 4-5), A unsigned 8-bit (0 at bits 7-9), B signed 8-bit (1 at bits 10-12),
+            // both K-major, N >> 3 at bits 17-22, M >> 4 at bits 24-28
+            constexpr uint32_t idesc = (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(DN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+            bool ok = true;
+            for (int jb = 0; jb < JB && ok; ++jb) {
+                const int s = jb % kTcStages;
+                ok = a_wait(&sm.full[s], (jb / kTcStages) & 1, abort_flag);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint64_t adesc = a_desc_sw128(a_smem_u32(sm.a[s]));
+                const uint64_t bdesc = a_desc_sw128(a_smem_u32(sm.b[s]));
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    const uint32_t accumulate = (jb == 0 && t == 0) ? 0u : 1u;
+                    asm volatile(
+                        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+                        ::"r"(tmem), "l"(adesc + (uint64_t)(2 * t)), "l"(bdesc + (uint64_t)(2 * t)), "r"(idesc), "r"(accumulate)
+                        : "memory");
+                }
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                             ::"r"(a_smem_u32(&sm.empty[s])) : "memory");
+            }
+            if (ok)
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                             ::"r"(a_smem_u32(&sm.acc_full)) : "memory");
+        }
+    } else {
+        const int quarter = warp & 3;                                     // TMEM lanes this warp may read
+        const int row = quarter * 32 + lane, m = m0 + row;
+        const bool ok = __all_sync(0xFFFFFFFFu, a_wait(&sm.acc_full, 0u, abort_flag) ? 1 : 0) != 0;
+        if (ok) {
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const float pmax = __half2float(__ushort_as_half((unsigned short)(*max_bits & 0xFFFFu)));
+            const float scale = pmax * __int_as_float((127 + *e_v - 7) << 23);
+            __half* yrow = y + ((size_t)h * M + m) * DN;
+#pragma unroll 1
+            for (int c0 = 0; c0 < DN; c0 += 32) {
+                uint32_t v[32];
+                asm volatile(
+                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                    "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                    "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                    : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                      "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                      "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                      "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                    : "r"(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0)
+                    : "memory");
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (m < M) {
+#pragma unroll
+                    for (int q8 = 0; q8 < 4; ++q8) {
+                        __half2 o[4];
+#pragma unroll
+                        for (int t = 0; t < 4; ++t)
+                            o[t] = __floats2half2_rn(scale * (float)(int)v[8 * q8 + 2 * t], scale * (float)(int)v[8 * q8 + 2 * t + 1]);
+                        *reinterpret_cast<uint4*>(yrow + c0 + 8 * q8) = *reinterpret_cast<uint4*>(o);
+                    }
+                }
+            }
+        }
+    }
+    __syncwarp();
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    if (sm.abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);                   // let copies in flight land
+        if (threadIdx.x == 0) atomicCAS(&ctl->status, 0u, sm.abort_flag);
+    }
+    __syncthreads();
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)DN) : "memory");
+}
+
+typedef CUresult (*AttnEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+template <int DN>
+cudaError_t launch_attn_tc(const uint8_t* w, const int8_t* vt, const uint32_t* max_bits, const int32_t* e_v, int H, int M,
+                           int J, __half* y, Control* ctl, const DeviceInfo& dev, cudaStream_t stream) {
+    using Smem = AttnSmem<DN>;
+    const size_t smem_bytes = sizeof(Smem) + 1024;
+    static bool attr_done = false;
+    if (!attr_done) {
+        const cudaError_t e = cudaFuncSetAttribute(attn_v_tc_kernel<DN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)smem_bytes);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    CUtensorMap amap, bmap;
+    const cuuint32_t estr[2] = {1u, 1u};
+    const cuuint64_t strides[1] = {(cuuint64_t)J};
+    const cuuint64_t adims[2] = {(cuuint64_t)J, (cuuint64_t)H * M};
+    const cuuint32_t abox[2] = {128u, 128u};
+    const cuuint64_t bdims[2] = {(cuuint64_t)J, (cuuint64_t)H * DN};
+    const cuuint32_t bbox[2] = {128u, (cuuint32_t)DN};
+    AttnEncodeFn enc = reinterpret_cast<AttnEncodeFn>(dev.encode_tiled);
+    if (enc(&amap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(w), adims, strides, abox, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
+    if (enc(&bmap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(vt), bdims, strides, bbox, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
+    dim3 grid((M + 127) / 128, H);
+    attn_v_tc_kernel<DN><<<grid, kTcThreads, smem_bytes, stream>>>(amap, bmap, max_bits, e_v, M, J, y, ctl);
+    return cudaGetLastError();
+}
+
 }  // namespace
+
+size_t attn_tc_scratch_bytes(int H, int M, int J, int D) {
+    const size_t a = ((size_t)H * M * J + 255) / 256 * 256, b = ((size_t)H * D * J + 255) / 256 * 256;
+    return a + b;
+}
+
+// scratch: [weights H*M*J, padded to 256][transposed value codes H*D*J]
+cudaError_t launch_attn_v_log2_tc(const int8_t* pcodes, const uint32_t* max_bits, const int8_t* vq, const int32_t* e_v,
+                                  int H, int M, int J, int D, __half* y, Control* ctl, void* scratch,
+                                  const DeviceInfo& dev, cudaStream_t stream) {
+    uint8_t* w = static_cast<uint8_t*>(scratch);
+    int8_t* vt = reinterpret_cast<int8_t*>(w + ((size_t)H * M * J + 255) / 256 * 256);
+    const long long count = (long long)H * M * J;
+    long long blocks = (count / 4 + 255) / 256;
+    const long long cap = (long long)dev.sm_count * 16;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    log2_weights_kernel<<<(unsigned int)blocks, 256, 0, stream>>>(pcodes, count, w, ctl);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    transpose_i8_kernel<<<dim3((J + 31) / 32, (D + 31) / 32, H), 256, 0, stream>>>(vq, J, D, vt);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    return D == 64 ? launch_attn_tc<64>(w, vt, max_bits, e_v, H, M, J, y, ctl, dev, stream)
+                   : launch_attn_tc<128>(w, vt, max_bits, e_v, H, M, J, y, ctl, dev, stream);
+}
 
 cudaError_t launch_log2_quantize(const __half* x, long long count, int bits, Control* ctl, int8_t* codes,
                                  uint32_t* max_bits_out, const DeviceInfo& dev, cudaStream_t stream) {

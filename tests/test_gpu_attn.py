@@ -77,3 +77,36 @@ def test_attn_bad_shapes_are_refused():
             h.aq_attn_v_log2(pc, mx, vq, ev, 4)
     with pytest.raises(binding.AgileqError):
         h.aq_attn_v_log2(pc, mx, torch.zeros((1, 8, 128), dtype=torch.int8, device="cuda"), ev, 8)   # 4-bit codes only
+
+
+@pytest.mark.parametrize("H,M,J,D", [(2, 33, 80, 128), (4, 128, 256, 128), (3, 300, 1040, 64), (1, 5, 16, 64)])
+def test_attn_v_log2_tensor_core_path_matches_checker(H, M, J, D):
+    h = handle()
+    p = _softmax_rows(H, M, J, 55)
+    v = inputs.activations(H * J, 128, seed=56, outlier_frac=0.01, outlier_mult=8.0)[:, :D].copy()
+    pc, pmax = h.aq_log2_quantize(dev(p), 4)
+    # value codes: the layer quantizer wants rows of 128 values, so quantize a [H*J*D/128, 128] view
+    vq, ev = h.aq_quantize_act(dev(v.reshape(-1, 128)), 8)
+    vq = vq.reshape(H, J, D)
+    y, ws = h.aq_attn_v_log2_tc(pc, pmax, vq, ev)
+    assert h.aq_check_workspace(ws) == binding.AQ_OK
+    pc_ref, pmax_ref = oracle.log2_quantize(p, 4)
+    e_ref = oracle.layer_exponent(v.reshape(-1, 128), 8)
+    vq_ref = oracle.quantize_act(v.reshape(-1, 128), 8, e_ref).reshape(H, J, D)
+    assert int(ev.item()) == e_ref
+    _, y_ref = oracle.attn_v_log2(pc_ref, pmax_ref, vq_ref, e_ref, 4)
+    assert_y_close(y.cpu().numpy().reshape(H * M, D), y_ref.reshape(H * M, D))
+    # bit for bit the same as the shift kernel (same integer sums, same scaling)
+    y_shift = h.aq_attn_v_log2(pc, pmax, vq, ev, 4)
+    assert torch.equal(y, y_shift)
+
+
+def test_attn_tensor_core_path_reports_negative_codes():
+    h = handle()
+    pc = torch.ones((1, 8, 16), dtype=torch.int8, device="cuda")
+    pc[0, 3, 5] = -2
+    mx = torch.full((1,), 0x3C00, dtype=torch.int32, device="cuda")
+    ev = torch.zeros(1, dtype=torch.int32, device="cuda")
+    vq = torch.ones((1, 16, 64), dtype=torch.int8, device="cuda")
+    y, ws = h.aq_attn_v_log2_tc(pc, mx, vq, ev)
+    assert h.aq_check_workspace(ws) == binding.AQ_ERR_INVALID_ARG
