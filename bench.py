@@ -374,11 +374,15 @@ def bench_attention(h, reps=5):
     y = torch.empty((H, M, D), dtype=torch.float16, device="cuda")
     t_q = _event_ms(lambda: h.aq_log2_quantize(p, 4), reps)
     t_av = _event_ms(lambda: h.aq_attn_v_log2(pc, pmax, vq, ev, 4, y=y), reps)
+    _, ws = h.aq_attn_v_log2_tc(pc, pmax, vq, ev, y=y)
+    t_tc = _event_ms(lambda: h.aq_attn_v_log2_tc(pc, pmax, vq, ev, y=y, workspace=ws), 4 * reps)
     macs = float(H) * M * J * D
     return {"H": H, "M": M, "J": J, "D": D,
             "log2_quantize": {"us": t_q * 1e3, "GBps": 3.0 * H * M * J / (t_q * 1e-3) / 1e9},
-            "attn_v": {"us": t_av * 1e3, "Gshift_add_per_s": macs / (t_av * 1e-3) / 1e9,
-                       "note": "CUDA-core kernel: one shift and one add per product, no tensor cores"}}
+            "attn_v_shift": {"us": t_av * 1e3, "Gproducts_per_s": macs / (t_av * 1e-3) / 1e9,
+                             "note": "CUDA-core kernel: one shift and one add per product"},
+            "attn_v_tensor": {"us": t_tc * 1e3, "TOPS": 2.0 * macs / (t_tc * 1e-3) / 1e12,
+                              "note": "factor conversion + value transpose + tcgen05 u8 x s8 kernel"}}
 
 
 def bench_pruned(h, reps=10):

@@ -9,15 +9,27 @@ namespace aq {
 namespace {
 
 // ---- layer-wide max |x| as an fp16 bit pattern (NaN ignored, Inf counts as 65504) -------------
+// 16-byte loads where the pointer allows; the first thread also takes the ragged tail.
 __global__ void __launch_bounds__(256)
 log2_absmax_kernel(const __half* __restrict__ x, long long count, Control* __restrict__ ctl) {
     unsigned int b = 0;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (long long)gridDim.x * blockDim.x) {
-        unsigned int hb = __half_as_ushort(x[i]) & 0x7FFFu;
-        if (hb > 0x7C00u) continue;
+    auto take = [&](unsigned int hb) {
+        hb &= 0x7FFFu;
+        if (hb > 0x7C00u) return;
         if (hb == 0x7C00u) hb = 0x7BFFu;
         b = max(b, hb);
+    };
+    const bool vec = (reinterpret_cast<uintptr_t>(x) & 15u) == 0;
+    const long long nvec = vec ? count / 8 : 0;
+    const uint4* xv = reinterpret_cast<const uint4*>(x);
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
+        const uint4 d = __ldg(xv + i);
+        const uint32_t w[4] = {d.x, d.y, d.z, d.w};
+#pragma unroll
+        for (int t = 0; t < 4; ++t) { take(w[t] & 0xFFFFu); take(w[t] >> 16); }
     }
+    if (blockIdx.x == 0 && threadIdx.x == 0)
+        for (long long i = nvec * 8; i < count; ++i) take(__half_as_ushort(x[i]));
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) b = max(b, __shfl_xor_sync(0xFFFFFFFFu, b, o));
     if ((threadIdx.x & 31) == 0 && b != 0) atomicMax(&ctl->absmax_bits, b);
@@ -37,6 +49,19 @@ __device__ __forceinline__ void half_parts(unsigned int hb, int& mant, int& expo
 // Eq. 3: k = clip(round(-log2(|x| / max)), 0, kmax), stored as Sign(x) * (k + 1), 0 for zero / NaN.
 // The rounding is decided with integers: -log2(r) = (Eb - Ea) + log2(mb / ma), and log2(mb / ma) passes
 // +-1/2 exactly when mb^2 passes 2 ma^2 or ma^2 / 2 (mantissas are 11-bit integers).
+__device__ __forceinline__ int log2_code(unsigned int raw, unsigned int mb_bits, int mb, int eb, int kmax) {
+    unsigned int hb = raw & 0x7FFFu;
+    if (hb == 0 || hb > 0x7C00u || mb_bits == 0) return 0;
+    if (hb == 0x7C00u) hb = 0x7BFFu;
+    int ma, ea;
+    half_parts(hb, ma, ea);
+    int k = eb - ea;
+    if (mb * mb >= 2 * ma * ma) k += 1;
+    else if (2 * mb * mb < ma * ma) k -= 1;
+    k = min(max(k, 0), kmax);
+    return (raw & 0x8000u) ? -(k + 1) : (k + 1);
+}
+
 __global__ void __launch_bounds__(256)
 log2_codes_kernel(const __half* __restrict__ x, long long count, int bits, const Control* __restrict__ ctl,
                   int8_t* __restrict__ codes, uint32_t* __restrict__ max_bits_out) {
@@ -45,22 +70,24 @@ log2_codes_kernel(const __half* __restrict__ x, long long count, int bits, const
     const int kmax = (1 << (bits - 1)) - 1;
     int mb = 1024, eb = 0;
     if (mb_bits) half_parts(mb_bits, mb, eb);
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < count; i += (long long)gridDim.x * blockDim.x) {
-        const unsigned int raw = __half_as_ushort(x[i]);
-        unsigned int hb = raw & 0x7FFFu;
-        int c = 0;
-        if (hb != 0 && hb <= 0x7C00u && mb_bits != 0) {
-            if (hb == 0x7C00u) hb = 0x7BFFu;
-            int ma, ea;
-            half_parts(hb, ma, ea);
-            int k = eb - ea;
-            if (mb * mb >= 2 * ma * ma) k += 1;
-            else if (2 * mb * mb < ma * ma) k -= 1;
-            k = min(max(k, 0), kmax);
-            c = (raw & 0x8000u) ? -(k + 1) : (k + 1);
+    const bool vec = (reinterpret_cast<uintptr_t>(x) & 15u) == 0 && (reinterpret_cast<uintptr_t>(codes) & 7u) == 0;
+    const long long nvec = vec ? count / 8 : 0;
+    const uint4* xv = reinterpret_cast<const uint4*>(x);
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
+        const uint4 d = __ldg(xv + i);
+        const uint32_t w[4] = {d.x, d.y, d.z, d.w};
+        uint32_t out[2] = {0u, 0u};
+#pragma unroll
+        for (int t = 0; t < 4; ++t) {
+            const uint32_t c0 = (uint32_t)log2_code(w[t] & 0xFFFFu, mb_bits, mb, eb, kmax) & 0xFFu;
+            const uint32_t c1 = (uint32_t)log2_code(w[t] >> 16, mb_bits, mb, eb, kmax) & 0xFFu;
+            out[t >> 1] |= (c0 | (c1 << 8)) << (16 * (t & 1));
         }
-        codes[i] = (int8_t)c;
+        *reinterpret_cast<uint2*>(codes + 8 * i) = make_uint2(out[0], out[1]);
     }
+    if (blockIdx.x == 0 && threadIdx.x == 0)
+        for (long long i = nvec * 8; i < count; ++i)
+            codes[i] = (int8_t)log2_code(__half_as_ushort(x[i]), mb_bits, mb, eb, kmax);
 }
 
 // ---- attention x value on the codes -----------------------------------------------------------
@@ -390,7 +417,7 @@ cudaError_t launch_attn_v_log2_tc(const int8_t* pcodes, const uint32_t* max_bits
 
 cudaError_t launch_log2_quantize(const __half* x, long long count, int bits, Control* ctl, int8_t* codes,
                                  uint32_t* max_bits_out, const DeviceInfo& dev, cudaStream_t stream) {
-    long long blocks = (count + 255) / 256;
+    long long blocks = (count / 8 + 255) / 256;
     const long long cap = (long long)dev.sm_count * 8;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
