@@ -453,6 +453,26 @@ def run_case(args):
                       "weight_copies": copies}))
 
 
+def run_attn_case(args):
+    """--attn-case H,M,J,D: time the tensor-core attention x value path on log2 codes."""
+    from paper_2312_05693_b200 import binding
+    H, M, J, D = [int(v) for v in args.attn_case.split(",")]
+    torch.cuda.set_device(0)
+    h = binding.Handle(0)
+    g = torch.Generator(device="cuda").manual_seed(7)
+    p = torch.softmax(torch.randn((H, M, J), generator=g, device="cuda") * 3.0, dim=2).to(torch.float16)
+    v = torch.from_numpy(inputs.activations(H * J * D // 128, 128, 7, 0.01, 8.0)).cuda()
+    vq, ev = h.aq_quantize_act(v, 8)
+    vq = vq.reshape(H, J, D)
+    pc, pmax = h.aq_log2_quantize(p, 4)
+    y, ws = h.aq_attn_v_log2_tc(pc, pmax, vq, ev)
+    for _ in range(args.warmup):
+        h.aq_attn_v_log2_tc(pc, pmax, vq, ev, y=y, workspace=ws)
+    ms = _event_ms(lambda: h.aq_attn_v_log2_tc(pc, pmax, vq, ev, y=y, workspace=ws), max(1, args.steps))
+    print(json.dumps({"attn_case": args.attn_case, "status": h.aq_check_workspace(ws), "us": ms * 1e3,
+                      "TOPS": 2.0 * H * M * J * D / (ms * 1e-3) / 1e12}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -464,9 +484,13 @@ def main():
     ap.add_argument("--case", default=None, help="M,K,N,group[,bits[,kernel]]: time one product kernel")
     ap.add_argument("--rotate-mb", type=float, default=0.0,
                     help="with --case: rotate through this many MB of weight copies (defeats L2)")
+    ap.add_argument("--attn-case", default=None, help="H,M,J,D: time the tensor-core attention x value path")
     args = ap.parse_args()
     if args.case:
         run_case(args)
+        return
+    if args.attn_case:
+        run_attn_case(args)
         return
     if args.warmup < 3:
         args.warmup = 3

@@ -137,26 +137,34 @@ attn_v_log2_kernel(const int8_t* __restrict__ pcodes, const uint32_t* __restrict
 
 // codes -> weights: c > 0 -> 128 >> (c - 1); 0 -> 0; a negative code is not representable here:
 // it is recorded in the status word (11) and treated as 0.
+__device__ __forceinline__ uint32_t log2_factors4(uint32_t c4, bool& bad) {
+    uint32_t o = 0;
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+        const int c = (int)(int8_t)((c4 >> (8 * t)) & 0xFFu);
+        bad |= c < 0;
+        o |= (c > 0 ? (128u >> (c - 1)) : 0u) << (8 * t);
+    }
+    return o;
+}
+
 __global__ void __launch_bounds__(256)
 log2_weights_kernel(const int8_t* __restrict__ codes, long long count, uint8_t* __restrict__ w, Control* __restrict__ ctl) {
     bool bad = false;
-    for (long long i = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 4; i < count; i += (long long)gridDim.x * blockDim.x * 4) {
-        if (i + 4 <= count) {
-            const char4 c = *reinterpret_cast<const char4*>(codes + i);
-            uchar4 o;
-            o.x = c.x > 0 ? (uint8_t)(128u >> (c.x - 1)) : 0; bad |= c.x < 0;
-            o.y = c.y > 0 ? (uint8_t)(128u >> (c.y - 1)) : 0; bad |= c.y < 0;
-            o.z = c.z > 0 ? (uint8_t)(128u >> (c.z - 1)) : 0; bad |= c.z < 0;
-            o.w = c.w > 0 ? (uint8_t)(128u >> (c.w - 1)) : 0; bad |= c.w < 0;
-            *reinterpret_cast<uchar4*>(w + i) = o;
-        } else {
-            for (long long t = i; t < count; ++t) {
-                const int c = codes[t];
-                w[t] = c > 0 ? (uint8_t)(128u >> (c - 1)) : 0;
-                bad |= c < 0;
-            }
-        }
+    const bool vec = (reinterpret_cast<uintptr_t>(codes) & 15u) == 0;       // w is 256-byte aligned scratch
+    const long long nvec = vec ? count / 16 : 0;
+    const uint4* cv = reinterpret_cast<const uint4*>(codes);
+    uint4* wv = reinterpret_cast<uint4*>(w);
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
+        const uint4 c = __ldg(cv + i);
+        wv[i] = make_uint4(log2_factors4(c.x, bad), log2_factors4(c.y, bad), log2_factors4(c.z, bad), log2_factors4(c.w, bad));
     }
+    if (blockIdx.x == 0 && threadIdx.x == 0)
+        for (long long t = nvec * 16; t < count; ++t) {
+            const int c = codes[t];
+            w[t] = c > 0 ? (uint8_t)(128u >> (c - 1)) : 0;
+            bad |= c < 0;
+        }
     if (bad) atomicCAS(&ctl->status, 0u, 11u);
 }
 
@@ -401,7 +409,7 @@ cudaError_t launch_attn_v_log2_tc(const int8_t* pcodes, const uint32_t* max_bits
     uint8_t* w = static_cast<uint8_t*>(scratch);
     int8_t* vt = reinterpret_cast<int8_t*>(w + ((size_t)H * M * J + 255) / 256 * 256);
     const long long count = (long long)H * M * J;
-    long long blocks = (count / 4 + 255) / 256;
+    long long blocks = (count / 16 + 255) / 256;
     const long long cap = (long long)dev.sm_count * 16;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
