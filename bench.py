@@ -377,7 +377,18 @@ def bench_attention(h, reps=5):
     _, ws = h.aq_attn_v_log2_tc(pc, pmax, vq, ev, y=y)
     t_tc = _event_ms(lambda: h.aq_attn_v_log2_tc(pc, pmax, vq, ev, y=y, workspace=ws), 4 * reps)
     macs = float(H) * M * J * D
-    return {"H": H, "M": M, "J": J, "D": D,
+    # query x key scores on int8 codes (reduction over the head dimension); the fp16 score matrix is the traffic
+    qa = torch.from_numpy(inputs.activations(H * M, D, 8, 0.01, 6.0)).cuda()
+    ka = torch.from_numpy(inputs.activations(H * J, D, 9, 0.01, 6.0)).cuda()
+    qc, eq = h.aq_quantize_act(qa, 8)
+    kc, ek = h.aq_quantize_act(ka, 8)
+    qc, kc = qc.reshape(H, M, D), kc.reshape(H, J, D)
+    s_out, ws_qk = h.aq_attn_qk_tc(qc, eq, kc, ek)
+    t_qk = _event_ms(lambda: h.aq_attn_qk_tc(qc, eq, kc, ek, s=s_out, workspace=ws_qk), 4 * reps)
+    qk = {"us": t_qk * 1e3, "TOPS": 2.0 * macs / (t_qk * 1e-3) / 1e12,
+          "GBps_scores_written": 2.0 * H * M * J / (t_qk * 1e-3) / 1e9}
+    del s_out, qa, ka
+    return {"H": H, "M": M, "J": J, "D": D, "qk_scores": qk,
             "log2_quantize": {"us": t_q * 1e3, "GBps": 3.0 * H * M * J / (t_q * 1e-3) / 1e9},
             "attn_v_shift": {"us": t_av * 1e3, "Gproducts_per_s": macs / (t_av * 1e-3) / 1e9,
                              "note": "CUDA-core kernel: one shift and one add per product"},

@@ -228,6 +228,12 @@ int aq_attn_v_log2(aq_handle_t h, const int8_t* p_codes, const uint32_t* p_max_b
  * J % 16 == 0; y must be 16-byte aligned. The workspace (aq_attn_workspace_bytes) holds a control block,
  * the byte factors and the transposed value codes. A negative code in P is an error: it is counted as 0
  * and aq_check_workspace on this workspace then returns AQ_ERR_INVALID_ARG. */
+/* Query x key scores on int8 (or 4-bit, stored in int8) codes of aq_quantize_act, reduction over the head
+ * dimension (Sec. 5.1): s[h,m,j] = fp16( 2^(e_q + e_k) * sum_d q[h,m,d] * k[h,j,d] ), q [H,M,D], k [H,J,D],
+ * s [H,M,J]. D must be 128, J % 8 == 0; all three 16-byte aligned. workspace: 256 bytes (control block). */
+int aq_attn_qk_tc(aq_handle_t h, const int8_t* q_codes, const int32_t* q_scale_exp, const int8_t* k_codes,
+                  const int32_t* k_scale_exp, int H, int M, int J, int D, void* s_fp16, void* workspace,
+                  size_t workspace_bytes, void* stream);
 size_t aq_attn_workspace_bytes(int H, int M, int J, int D);
 int aq_attn_v_log2_tc(aq_handle_t h, const int8_t* p_codes, const uint32_t* p_max_bits, const int8_t* v_codes,
                       const int32_t* v_scale_exp, int H, int M, int J, int D, void* y_fp16, void* workspace,

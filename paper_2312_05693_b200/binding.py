@@ -87,6 +87,7 @@ def load():
     L.aq_attn_workspace_bytes.restype = sz
     L.aq_attn_workspace_bytes.argtypes = [i32, i32, i32, i32]
     L.aq_attn_v_log2_tc.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, sz, vp]
+    L.aq_attn_qk_tc.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, sz, vp]
     L.aq_prune_schedule.argtypes = [i32, C.c_double, i32, vp, vp]
     L.aq_trip_calibrate.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
     L.aq_quantize_act_trip.argtypes = [vp, vp, i32, i32, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
@@ -262,6 +263,17 @@ class Handle:
                                         J, D, _ptr(y), _ptr(workspace), workspace.numel(), _stream()),
                "aq_attn_v_log2_tc")
         return y, workspace
+
+    def aq_attn_qk_tc(self, q_codes, q_exp, k_codes, k_exp, s=None, workspace=None):
+        H, M, D = q_codes.shape
+        J = k_codes.shape[1]
+        if s is None:
+            s = torch.empty((H, M, J), dtype=torch.float16, device=q_codes.device)
+        if workspace is None:
+            workspace = torch.empty(256, dtype=torch.uint8, device=q_codes.device)
+        _check(load().aq_attn_qk_tc(self._h, _ptr(q_codes), _ptr(q_exp), _ptr(k_codes), _ptr(k_exp), H, M, J, D, _ptr(s),
+                                    _ptr(workspace), workspace.numel(), _stream()), "aq_attn_qk_tc")
+        return s, workspace
 
     # ---- chaining: the next layer's codes instead of fp16 outputs (Sec. 4.4)
     def aq_linear_chain(self, bits, x, packed, scales, N, group_size, next_bits, next_exp,

@@ -494,6 +494,25 @@ int aq_attn_v_log2_tc(aq_handle_t h, const int8_t* p_codes, const uint32_t* p_ma
     return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
 }
 
+int aq_attn_qk_tc(aq_handle_t h, const int8_t* q_codes, const int32_t* q_scale_exp, const int8_t* k_codes,
+                  const int32_t* k_scale_exp, int H, int M, int J, int D, void* s_fp16, void* workspace,
+                  size_t workspace_bytes_, void* stream_) {
+    if (!h || !q_codes || !q_scale_exp || !k_codes || !k_scale_exp || !s_fp16) return AQ_ERR_INVALID_ARG;
+    if (H < 1 || H > 65535 || M < 1 || J < 8 || J % 8 != 0 || D != 128) return AQ_ERR_SHAPE;
+    if ((long long)H * M > 0x7FFFFFFFll || (long long)H * J > 0x7FFFFFFFll || (J + 127) / 128 > 65535) return AQ_ERR_SHAPE;
+    if (!workspace || workspace_bytes_ < sizeof(Control)) return AQ_ERR_WORKSPACE;
+    if (!aligned(q_codes, 16) || !aligned(k_codes, 16) || !aligned(s_fp16, 16) || !aligned(q_scale_exp, 4) ||
+        !aligned(k_scale_exp, 4) || !aligned(workspace, 256))
+        return AQ_ERR_ALIGNMENT;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    Control* ctl = static_cast<Control*>(workspace);
+    cudaError_t e = cudaMemsetAsync(ctl, 0, sizeof(Control), stream);
+    if (e == cudaSuccess)
+        e = launch_attn_qk_tc(q_codes, q_scale_exp, k_codes, k_scale_exp, H, M, J, D, static_cast<__half*>(s_fp16), ctl,
+                              h->dev, stream);
+    return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
 int aq_prune_schedule(int M, double beta, int m, int32_t* n_keep_out, double* gamma_out) {
     if (M < 1 || m < 1 || !(beta >= 0.0) || !(beta < 1.0) || !n_keep_out) return AQ_ERR_INVALID_ARG;
     const double gamma = 1.0 - pow(1.0 - beta, 1.0 / (double)m);       // Eq. 9

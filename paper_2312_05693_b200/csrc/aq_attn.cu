@@ -226,35 +226,46 @@ struct AttnSmem {
     alignas(1024) uint8_t b[kTcStages][DN * 128];    // value tile: DN columns x 128 j
     alignas(8) uint64_t full[kTcStages];
     uint64_t empty[kTcStages];
-    uint64_t acc_full;
+    uint64_t acc_full[2];                            // MMA -> epilogue, one per accumulator stage
+    uint64_t acc_empty[2];                           // epilogue (4 warps) -> MMA
     uint32_t tmem_base;
     volatile uint32_t abort_flag;
 };
 
-// One CTA per (head, 128 query rows).
-template <int DN>
+// Batched int8 contraction y[h][m][n] = scale * sum_k A[h*M + m][k] * B[h*NB + n][k] (both operands
+// k-major). One CTA per (128 rows of A, head) walks all tiles of DN rows of B, with two accumulator
+// stages in tensor memory so that the epilogue of one tile overlaps the MMAs of the next. A is unsigned
+// or signed bytes, B signed.
+// scale = (max_bits ? the half in its low 16 bits : 1) * 2^(*e1 + (e2 ? *e2 : 0) + e_off).
+// Used for attention x value (A = byte factors of the log2 codes, B = transposed value codes, k = key
+// index) and for the query x key product (A, B = int8 codes, k = head dimension).
+template <int DN, bool A_SIGNED>
 __global__ void __launch_bounds__(kTcThreads, 1)
 attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__ CUtensorMap b_map,
-                 const uint32_t* __restrict__ max_bits, const int32_t* __restrict__ e_v, int M, int J,
-                 __half* __restrict__ y, Control* __restrict__ ctl) {
+                 const uint32_t* __restrict__ max_bits, const int32_t* __restrict__ e1, const int32_t* __restrict__ e2,
+                 int e_off, int M, int J /* length of k */, int NB, __half* __restrict__ y, Control* __restrict__ ctl) {
     extern __shared__ uint8_t attn_smem_raw[];
     using Smem = AttnSmem<DN>;
     Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(attn_smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int h = blockIdx.y, m0 = blockIdx.x * 128;
     const int JB = (J + 127) / 128;
+    const int NT = (NB + DN - 1) / DN;                                    // tiles of B rows this CTA walks
     if (threadIdx.x == 0) {
         for (int s = 0; s < kTcStages; ++s) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(a_smem_u32(&sm.full[s])) : "memory");
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(a_smem_u32(&sm.empty[s])) : "memory");
         }
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(a_smem_u32(&sm.acc_full)) : "memory");
+        for (int a = 0; a < 2; ++a) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(a_smem_u32(&sm.acc_full[a])) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 4;" ::"r"(a_smem_u32(&sm.acc_empty[a])) : "memory");
+        }
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(a_smem_u32(&sm.tmem_base)), "r"((uint32_t)DN) : "memory");
+                     ::"r"(a_smem_u32(&sm.tmem_base)), "r"((uint32_t)(2 * DN)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -265,9 +276,11 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int jb = 0; jb < JB; ++jb) {
-                const int s = jb % kTcStages;
-                if (!a_wait(&sm.empty[s], ((jb / kTcStages) & 1) ^ 1, abort_flag)) break;
+            const int total = NT * JB;
+            for (int it = 0; it < total; ++it) {
+                const int nt = it / JB, jb = it % JB, n0 = nt * DN;
+                const int s = it % kTcStages;
+                if (!a_wait(&sm.empty[s], ((it / kTcStages) & 1) ^ 1, abort_flag)) break;
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
                              ::"r"(a_smem_u32(&sm.full[s])), "r"((uint32_t)((128 + DN) * 128)) : "memory");
                 asm volatile(
@@ -276,7 +289,7 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
                     : "memory");
                 asm volatile(
                     "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                    ::"r"(a_smem_u32(sm.b[s])), "l"(&b_map), "r"(jb * 128), "r"(h * DN), "r"(a_smem_u32(&sm.full[s]))
+                    ::"r"(a_smem_u32(sm.b[s])), "l"(&b_map), "r"(jb * 128), "r"(h * NB + n0), "r"(a_smem_u32(&sm.full[s]))
                     : "memory");
             }
         }
@@ -284,11 +297,17 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
         if (lane == 0) {
             // D = s32 (2 at bits 4-5), A unsigned 8-bit (0 at bits 7-9), B signed 8-bit (1 at bits 10-12),
             // both K-major, N >> 3 at bits 17-22, M >> 4 at bits 24-28
-            constexpr uint32_t idesc = (2u << 4) | (0u << 7) | (1u << 10) | ((uint32_t)(DN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+            constexpr uint32_t idesc = (2u << 4) | ((A_SIGNED ? 1u : 0u) << 7) | (1u << 10) | ((uint32_t)(DN >> 3) << 17) |
+                                       ((uint32_t)(128 >> 4) << 24);
             bool ok = true;
-            for (int jb = 0; jb < JB && ok; ++jb) {
-                const int s = jb % kTcStages;
-                ok = a_wait(&sm.full[s], (jb / kTcStages) & 1, abort_flag);
+            int it = 0;
+            for (int nt = 0; nt < NT && ok; ++nt) {
+              const int a = nt & 1;
+              ok = a_wait(&sm.acc_empty[a], ((nt >> 1) & 1) ^ 1, abort_flag);      // the epilogue has drained this stage
+              if (!ok) break;
+              for (int jb = 0; jb < JB && ok; ++jb, ++it) {
+                const int s = it % kTcStages;
+                ok = a_wait(&sm.full[s], (it / kTcStages) & 1, abort_flag);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint64_t adesc = a_desc_sw128(a_smem_u32(sm.a[s]));
@@ -299,25 +318,28 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
                     asm volatile(
                         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
                         "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-                        ::"r"(tmem), "l"(adesc + (uint64_t)(2 * t)), "l"(bdesc + (uint64_t)(2 * t)), "r"(idesc), "r"(accumulate)
+                        ::"r"(tmem + (uint32_t)(a * DN)), "l"(adesc + (uint64_t)(2 * t)), "l"(bdesc + (uint64_t)(2 * t)), "r"(idesc),
+                          "r"(accumulate)
                         : "memory");
                 }
                 asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
                              ::"r"(a_smem_u32(&sm.empty[s])) : "memory");
-            }
-            if (ok)
+              }
+              if (ok)
                 asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-                             ::"r"(a_smem_u32(&sm.acc_full)) : "memory");
+                             ::"r"(a_smem_u32(&sm.acc_full[a])) : "memory");
+            }
         }
     } else {
         const int quarter = warp & 3;                                     // TMEM lanes this warp may read
         const int row = quarter * 32 + lane, m = m0 + row;
-        const bool ok = __all_sync(0xFFFFFFFFu, a_wait(&sm.acc_full, 0u, abort_flag) ? 1 : 0) != 0;
-        if (ok) {
+        const float pmax = max_bits ? __half2float(__ushort_as_half((unsigned short)(*max_bits & 0xFFFFu))) : 1.0f;
+        const float scale = pmax * __int_as_float((127 + *e1 + (e2 ? *e2 : 0) + e_off) << 23);
+        for (int nt = 0; nt < NT; ++nt) {
+            const int a = nt & 1, n0 = nt * DN;
+            if (!(__all_sync(0xFFFFFFFFu, a_wait(&sm.acc_full[a], (nt >> 1) & 1, abort_flag) ? 1 : 0) != 0)) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const float pmax = __half2float(__ushort_as_half((unsigned short)(*max_bits & 0xFFFFu)));
-            const float scale = pmax * __int_as_float((127 + *e_v - 7) << 23);
-            __half* yrow = y + ((size_t)h * M + m) * DN;
+            __half* yrow = y + ((size_t)h * M + m) * NB + n0;
 #pragma unroll 1
             for (int c0 = 0; c0 < DN; c0 += 32) {
                 uint32_t v[32];
@@ -329,12 +351,13 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
                       "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
                       "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
                       "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-                    : "r"(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0)
+                    : "r"(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * DN + c0))
                     : "memory");
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 if (m < M) {
 #pragma unroll
                     for (int q8 = 0; q8 < 4; ++q8) {
+                        if (n0 + c0 + 8 * q8 >= NB) break;                   // NB is a multiple of 8
                         __half2 o[4];
 #pragma unroll
                         for (int t = 0; t < 4; ++t)
@@ -343,6 +366,10 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
                     }
                 }
             }
+            // this warp's part of the accumulator stage is in registers / written: hand the stage back
+            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(a_smem_u32(&sm.acc_empty[a])) : "memory");
         }
     }
     __syncwarp();
@@ -355,22 +382,23 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
     }
     __syncthreads();
     if (warp == 1)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)DN) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)(2 * DN)) : "memory");
 }
 
 typedef CUresult (*AttnEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-template <int DN>
-cudaError_t launch_attn_tc(const uint8_t* w, const int8_t* vt, const uint32_t* max_bits, const int32_t* e_v, int H, int M,
-                           int J, __half* y, Control* ctl, const DeviceInfo& dev, cudaStream_t stream) {
+template <int DN, bool A_SIGNED>
+cudaError_t launch_attn_tc(const void* w, const int8_t* vt, const uint32_t* max_bits, const int32_t* e1, const int32_t* e2,
+                           int e_off, int H, int M, int J, int NB, __half* y, Control* ctl, const DeviceInfo& dev,
+                           cudaStream_t stream) {
     using Smem = AttnSmem<DN>;
     const size_t smem_bytes = sizeof(Smem) + 1024;
     static bool attr_done = false;
     if (!attr_done) {
-        const cudaError_t e = cudaFuncSetAttribute(attn_v_tc_kernel<DN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   (int)smem_bytes);
+        const cudaError_t e = cudaFuncSetAttribute(attn_v_tc_kernel<DN, A_SIGNED>,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
@@ -379,10 +407,10 @@ cudaError_t launch_attn_tc(const uint8_t* w, const int8_t* vt, const uint32_t* m
     const cuuint64_t strides[1] = {(cuuint64_t)J};
     const cuuint64_t adims[2] = {(cuuint64_t)J, (cuuint64_t)H * M};
     const cuuint32_t abox[2] = {128u, 128u};
-    const cuuint64_t bdims[2] = {(cuuint64_t)J, (cuuint64_t)H * DN};
+    const cuuint64_t bdims[2] = {(cuuint64_t)J, (cuuint64_t)H * NB};
     const cuuint32_t bbox[2] = {128u, (cuuint32_t)DN};
     AttnEncodeFn enc = reinterpret_cast<AttnEncodeFn>(dev.encode_tiled);
-    if (enc(&amap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(w), adims, strides, abox, estr,
+    if (enc(&amap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(w), adims, strides, abox, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidValue;
@@ -391,7 +419,8 @@ cudaError_t launch_attn_tc(const uint8_t* w, const int8_t* vt, const uint32_t* m
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidValue;
     dim3 grid((M + 127) / 128, H);
-    attn_v_tc_kernel<DN><<<grid, kTcThreads, smem_bytes, stream>>>(amap, bmap, max_bits, e_v, M, J, y, ctl);
+    attn_v_tc_kernel<DN, A_SIGNED><<<grid, kTcThreads, smem_bytes, stream>>>(amap, bmap, max_bits, e1, e2, e_off, M, J,
+                                                                            NB, y, ctl);
     return cudaGetLastError();
 }
 
@@ -419,8 +448,14 @@ cudaError_t launch_attn_v_log2_tc(const int8_t* pcodes, const uint32_t* max_bits
     transpose_i8_kernel<<<dim3((J + 31) / 32, (D + 31) / 32, H), 256, 0, stream>>>(vq, J, D, vt);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    return D == 64 ? launch_attn_tc<64>(w, vt, max_bits, e_v, H, M, J, y, ctl, dev, stream)
-                   : launch_attn_tc<128>(w, vt, max_bits, e_v, H, M, J, y, ctl, dev, stream);
+    return D == 64 ? launch_attn_tc<64, false>(w, vt, max_bits, e_v, nullptr, -7, H, M, J, D, y, ctl, dev, stream)
+                   : launch_attn_tc<128, false>(w, vt, max_bits, e_v, nullptr, -7, H, M, J, D, y, ctl, dev, stream);
+}
+
+// Query x key: s[h][m][j] = 2^(e_q + e_k) * sum_d q[h][m][d] * k[h][j][d], int8 codes, D = 128.
+cudaError_t launch_attn_qk_tc(const int8_t* qc, const int32_t* e_q, const int8_t* kc, const int32_t* e_k, int H, int M,
+                              int J, int D, __half* s_out, Control* ctl, const DeviceInfo& dev, cudaStream_t stream) {
+    return launch_attn_tc<128, true>(qc, kc, nullptr, e_q, e_k, 0, H, M, D, J, s_out, ctl, dev, stream);
 }
 
 cudaError_t launch_log2_quantize(const __half* x, long long count, int bits, Control* ctl, int8_t* codes,

@@ -124,6 +124,9 @@ size_t attn_tc_scratch_bytes(int H, int M, int J, int D);
 cudaError_t launch_attn_v_log2_tc(const int8_t* pcodes, const uint32_t* max_bits, const int8_t* vq, const int32_t* e_v,
                                   int H, int M, int J, int D, __half* y, Control* ctl, void* scratch,
                                   const DeviceInfo& dev, cudaStream_t stream);
+// Query x key product on int8 codes (head dimension 128), same tensor-core kernel.
+cudaError_t launch_attn_qk_tc(const int8_t* qc, const int32_t* e_q, const int8_t* kc, const int32_t* e_k, int H, int M,
+                              int J, int D, __half* s_out, Control* ctl, const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_attn_v_log2(const int8_t* pcodes, const uint32_t* max_bits, const int8_t* vq, const int32_t* e_v,
                                int H, int M, int J, int D, int bits, __half* y, int32_t* acc_dump, cudaStream_t stream);
 

@@ -110,3 +110,26 @@ def test_attn_tensor_core_path_reports_negative_codes():
     vq = torch.ones((1, 16, 64), dtype=torch.int8, device="cuda")
     y, ws = h.aq_attn_v_log2_tc(pc, mx, vq, ev)
     assert h.aq_check_workspace(ws) == binding.AQ_ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("H,M,J", [(2, 33, 80), (3, 300, 1048), (1, 128, 128), (2, 5, 8)])
+def test_attn_qk_matches_checker(bits, H, M, J):
+    D = 128
+    h = handle()
+    q = inputs.activations(H * M, D, seed=57, outlier_frac=0.01, outlier_mult=6.0)
+    k = inputs.activations(H * J, D, seed=58, outlier_frac=0.01, outlier_mult=6.0)
+    qc, eq = h.aq_quantize_act(dev(q), bits)
+    kc, ek = h.aq_quantize_act(dev(k), bits)
+    s, ws = h.aq_attn_qk_tc(qc.reshape(H, M, D), eq, kc.reshape(H, J, D), ek)
+    assert h.aq_check_workspace(ws) == binding.AQ_OK
+    eq_ref, ek_ref = oracle.layer_exponent(q, bits), oracle.layer_exponent(k, bits)
+    assert (int(eq.item()), int(ek.item())) == (eq_ref, ek_ref)
+    qr = oracle.quantize_act(q, bits, eq_ref).reshape(H, M, D)
+    kr = oracle.quantize_act(k, bits, ek_ref).reshape(H, J, D)
+    ones = np.ones((J, 1), np.float16)
+    ref = np.stack([oracle.dequant(oracle.int_gemm(qr[i], kr[i], 0).reshape(M, J, 1), ones, eq_ref + ek_ref)
+                    for i in range(H)])
+    assert_y_close(s.cpu().numpy().reshape(H * M, J), ref.reshape(H * M, J))
+    # the integer sums are below 2^24 here, so the scaled fp16 values are the same bits
+    assert np.array_equal(s.cpu().numpy(), ref)
