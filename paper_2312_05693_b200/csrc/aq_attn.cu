@@ -224,6 +224,9 @@ template <int DN>
 struct AttnSmem {
     alignas(1024) uint8_t a[kTcStages][128 * 128];   // weights tile: 128 query rows x 128 j
     alignas(1024) uint8_t b[kTcStages][DN * 128];    // value tile: DN columns x 128 j
+    // Output staging: each epilogue warp owns two boxes of 32 rows x 64 halves (128-byte rows, written
+    // with the 128-byte swizzle of the store's tensor map), for alternate 64-column chunks.
+    alignas(1024) uint8_t ystage[4][2][32 * 128];
     alignas(8) uint64_t full[kTcStages];
     uint64_t empty[kTcStages];
     uint64_t acc_full[2];                            // MMA -> epilogue, one per accumulator stage
@@ -242,7 +245,7 @@ struct AttnSmem {
 template <int DN, bool A_SIGNED>
 __global__ void __launch_bounds__(kTcThreads, 1)
 attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__ CUtensorMap b_map,
-                 const uint32_t* __restrict__ max_bits, const int32_t* __restrict__ e1, const int32_t* __restrict__ e2,
+                 const __grid_constant__ CUtensorMap y_map, const uint32_t* __restrict__ max_bits, const int32_t* __restrict__ e1, const int32_t* __restrict__ e2,
                  int e_off, int M, int J /* length of k */, int NB, __half* __restrict__ y, Control* __restrict__ ctl) {
     extern __shared__ uint8_t attn_smem_raw[];
     using Smem = AttnSmem<DN>;
@@ -339,7 +342,7 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
             const int a = nt & 1, n0 = nt * DN;
             if (!(__all_sync(0xFFFFFFFFu, a_wait(&sm.acc_full[a], (nt >> 1) & 1, abort_flag) ? 1 : 0) != 0)) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            __half* yrow = y + ((size_t)h * M + m) * NB + n0;
+            const int ew = warp - 2;
 #pragma unroll 1
             for (int c0 = 0; c0 < DN; c0 += 32) {
                 uint32_t v[32];
@@ -354,15 +357,53 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
                     : "r"(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * DN + c0))
                     : "memory");
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (m < M) {
+                // 32 columns of this thread's row -> 64 bytes of its 128-byte staging row; 16-byte chunk j of
+                // row r sits at chunk position j ^ (r & 7), as the store's tensor map expects
+                const int row0 = m0 + quarter * 32;
+                if (row0 + 32 > M) {
+                    // a box of 32 rows would run into the next head's rows: this warp stores its rows itself
+                    if (m < M) {
+                        __half* yrow = y + ((size_t)h * M + m) * NB + n0;
 #pragma unroll
-                    for (int q8 = 0; q8 < 4; ++q8) {
-                        if (n0 + c0 + 8 * q8 >= NB) break;                   // NB is a multiple of 8
-                        __half2 o[4];
+                        for (int q8 = 0; q8 < 4; ++q8) {
+                            if (n0 + c0 + 8 * q8 >= NB) break;               // NB is a multiple of 8
+                            __half2 o[4];
 #pragma unroll
-                        for (int t = 0; t < 4; ++t)
-                            o[t] = __floats2half2_rn(scale * (float)(int)v[8 * q8 + 2 * t], scale * (float)(int)v[8 * q8 + 2 * t + 1]);
-                        *reinterpret_cast<uint4*>(yrow + c0 + 8 * q8) = *reinterpret_cast<uint4*>(o);
+                            for (int t = 0; t < 4; ++t)
+                                o[t] = __floats2half2_rn(scale * (float)(int)v[8 * q8 + 2 * t], scale * (float)(int)v[8 * q8 + 2 * t + 1]);
+                            *reinterpret_cast<uint4*>(yrow + c0 + 8 * q8) = *reinterpret_cast<uint4*>(o);
+                        }
+                    }
+                    continue;
+                }
+                const int box = (c0 >> 6) & 1, half_of_box = (c0 >> 5) & 1;
+                uint8_t* srow = sm.ystage[ew][box] + lane * 128;
+                if (half_of_box == 0) {
+                    // the box is about to be rewritten: the store that used it last must have read it (with two
+                    // boxes in rotation one younger store may still be pending)
+                    if (lane == 0) {
+                        if (DN > 64) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                        else asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    }
+                    __syncwarp();
+                }
+#pragma unroll
+                for (int q8 = 0; q8 < 4; ++q8) {
+                    __half2 o[4];
+#pragma unroll
+                    for (int t = 0; t < 4; ++t)
+                        o[t] = __floats2half2_rn(scale * (float)(int)v[8 * q8 + 2 * t], scale * (float)(int)v[8 * q8 + 2 * t + 1]);
+                    const int chunk = half_of_box * 4 + q8;
+                    *reinterpret_cast<uint4*>(srow + ((chunk ^ (lane & 7)) << 4)) = *reinterpret_cast<uint4*>(o);
+                }
+                if (half_of_box == 1 || c0 + 32 >= DN) {
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    const int col = n0 + (c0 & ~63);
+                    if (lane == 0 && col < NB) {
+                        asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+                                     ::"l"(&y_map), "r"(col), "r"(h * M + row0), "r"(a_smem_u32(sm.ystage[ew][box])) : "memory");
+                        asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                     }
                 }
             }
@@ -372,6 +413,7 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(a_smem_u32(&sm.acc_empty[a])) : "memory");
         }
     }
+    if (warp >= 2 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // staging rows live until read
     __syncwarp();
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -418,9 +460,17 @@ cudaError_t launch_attn_tc(const void* w, const int8_t* vt, const uint32_t* max_
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidValue;
+    // outputs: [H*M rows][NB] halves, stored in boxes of 64 columns x 32 rows with the 128-byte swizzle
+    CUtensorMap ymap;
+    const cuuint64_t ydims[2] = {(cuuint64_t)NB, (cuuint64_t)H * M};
+    const cuuint64_t ystrides[1] = {(cuuint64_t)NB * 2};
+    const cuuint32_t ybox[2] = {64u, 32u};
+    if (enc(&ymap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, y, ydims, ystrides, ybox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return cudaErrorInvalidValue;
     dim3 grid((M + 127) / 128, H);
-    attn_v_tc_kernel<DN, A_SIGNED><<<grid, kTcThreads, smem_bytes, stream>>>(amap, bmap, max_bits, e1, e2, e_off, M, J,
-                                                                            NB, y, ctl);
+    attn_v_tc_kernel<DN, A_SIGNED><<<grid, kTcThreads, smem_bytes, stream>>>(amap, bmap, ymap, max_bits, e1, e2, e_off, M,
+                                                                            J, NB, y, ctl);
     return cudaGetLastError();
 }
 
