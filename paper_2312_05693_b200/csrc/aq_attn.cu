@@ -22,6 +22,7 @@ log2_absmax_kernel(const __half* __restrict__ x, long long count, Control* __res
     const bool vec = (reinterpret_cast<uintptr_t>(x) & 15u) == 0;
     const long long nvec = vec ? count / 8 : 0;
     const uint4* xv = reinterpret_cast<const uint4*>(x);
+#pragma unroll 4
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
         const uint4 d = __ldg(xv + i);
         const uint32_t w[4] = {d.x, d.y, d.z, d.w};
@@ -49,15 +50,28 @@ __device__ __forceinline__ void half_parts(unsigned int hb, int& mant, int& expo
 // Eq. 3: k = clip(round(-log2(|x| / max)), 0, kmax), stored as Sign(x) * (k + 1), 0 for zero / NaN.
 // The rounding is decided with integers: -log2(r) = (Eb - Ea) + log2(mb / ma), and log2(mb / ma) passes
 // +-1/2 exactly when mb^2 passes 2 ma^2 or ma^2 / 2 (mantissas are 11-bit integers).
-__device__ __forceinline__ int log2_code(unsigned int raw, unsigned int mb_bits, int mb, int eb, int kmax) {
+// The two mantissa thresholds of the rounding rule for a given maximum mantissa mb (1024..2047):
+// t_up = largest ma with 2 ma^2 <= mb^2 (below or at it k rounds up), t_down = smallest ma with
+// ma^2 > 2 mb^2 (from it on k rounds down).
+__device__ __forceinline__ void log2_thresholds(int mb, int& t_up, int& t_down) {
+    int a = (int)(sqrtf(0.5f * (float)mb * (float)mb));
+    while (2 * (a + 1) * (a + 1) <= mb * mb) ++a;
+    while (2 * a * a > mb * mb) --a;
+    t_up = a;
+    int b = (int)(sqrtf(2.0f * (float)mb * (float)mb));
+    while (b * b > 2 * mb * mb) --b;
+    while ((b + 1) * (b + 1) <= 2 * mb * mb) ++b;
+    t_down = b + 1;
+}
+
+__device__ __forceinline__ int log2_code(unsigned int raw, unsigned int mb_bits, int eb, int t_up, int t_down, int kmax) {
     unsigned int hb = raw & 0x7FFFu;
     if (hb == 0 || hb > 0x7C00u || mb_bits == 0) return 0;
     if (hb == 0x7C00u) hb = 0x7BFFu;
     int ma, ea;
-    half_parts(hb, ma, ea);
-    int k = eb - ea;
-    if (mb * mb >= 2 * ma * ma) k += 1;
-    else if (2 * mb * mb < ma * ma) k -= 1;
+    if (hb >= 0x0400u) { ma = 1024 + (int)(hb & 0x3FFu); ea = (int)(hb >> 10) - 25; }   // normal: the common case
+    else half_parts(hb, ma, ea);
+    int k = eb - ea + (ma <= t_up ? 1 : 0) - (ma >= t_down ? 1 : 0);
     k = min(max(k, 0), kmax);
     return (raw & 0x8000u) ? -(k + 1) : (k + 1);
 }
@@ -68,26 +82,28 @@ log2_codes_kernel(const __half* __restrict__ x, long long count, int bits, const
     const unsigned int mb_bits = ctl->absmax_bits;
     if (blockIdx.x == 0 && threadIdx.x == 0 && max_bits_out) *max_bits_out = mb_bits;
     const int kmax = (1 << (bits - 1)) - 1;
-    int mb = 1024, eb = 0;
+    int mb = 1024, eb = 0, t_up = 0, t_down = 0;
     if (mb_bits) half_parts(mb_bits, mb, eb);
+    log2_thresholds(mb, t_up, t_down);
     const bool vec = (reinterpret_cast<uintptr_t>(x) & 15u) == 0 && (reinterpret_cast<uintptr_t>(codes) & 7u) == 0;
     const long long nvec = vec ? count / 8 : 0;
     const uint4* xv = reinterpret_cast<const uint4*>(x);
+#pragma unroll 4
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
         const uint4 d = __ldg(xv + i);
         const uint32_t w[4] = {d.x, d.y, d.z, d.w};
         uint32_t out[2] = {0u, 0u};
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
-            const uint32_t c0 = (uint32_t)log2_code(w[t] & 0xFFFFu, mb_bits, mb, eb, kmax) & 0xFFu;
-            const uint32_t c1 = (uint32_t)log2_code(w[t] >> 16, mb_bits, mb, eb, kmax) & 0xFFu;
+            const uint32_t c0 = (uint32_t)log2_code(w[t] & 0xFFFFu, mb_bits, eb, t_up, t_down, kmax) & 0xFFu;
+            const uint32_t c1 = (uint32_t)log2_code(w[t] >> 16, mb_bits, eb, t_up, t_down, kmax) & 0xFFu;
             out[t >> 1] |= (c0 | (c1 << 8)) << (16 * (t & 1));
         }
         *reinterpret_cast<uint2*>(codes + 8 * i) = make_uint2(out[0], out[1]);
     }
     if (blockIdx.x == 0 && threadIdx.x == 0)
         for (long long i = nvec * 8; i < count; ++i)
-            codes[i] = (int8_t)log2_code(__half_as_ushort(x[i]), mb_bits, mb, eb, kmax);
+            codes[i] = (int8_t)log2_code(__half_as_ushort(x[i]), mb_bits, eb, t_up, t_down, kmax);
 }
 
 // ---- attention x value on the codes -----------------------------------------------------------
