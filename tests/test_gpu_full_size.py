@@ -123,3 +123,64 @@ def test_opt30b_pruned_prefill_full_size():
     y_fused = h.aq_linear_w4a8(xd, packed, scales, s.N, 0, row_idx=idxd)
     y_plain = h.aq_linear_w4a8(xp, packed, scales, s.N, 0)
     assert torch.equal(y_fused, y_plain)
+
+
+def test_widened_entry_points_at_a_benchmark_shape():
+    """TRIP factors, the zero-point variant and the chained call on the LLaMA-7B (4096 -> 11008) layer at
+    M = 2048, through the tensor kernel as the benchmark runs them: codes and exponents in full, integer
+    sums and outputs on sampled positions."""
+    wl = inputs.WORKLOADS["llama7b_prefill_w4a4"]
+    h = handle()
+    M, shape, group = wl.Ms[0], wl.shapes[1], wl.group_size
+    K, N, G = shape.K, shape.N, shape.K // 128
+    x = inputs.activations(M, K, wl.seed, wl.outlier_frac, wl.outlier_mult, sub=1)
+    w = inputs.weights(N, K, wl.seed, sub=1)
+    xd = dev(x)
+    packed, scales = h.aq_pack_w4(dev(w), group)
+    codes, sc = oracle.quantize_weights(w, group)
+    rows, cols = inputs.sample_coords(M, N, N_SAMPLES, 77)
+    rt, ct = torch.from_numpy(rows.astype(np.int64)).cuda(), torch.from_numpy(cols.astype(np.int64)).cuda()
+    ws = h.alloc_workspace(M, K, N, group)
+    acc = torch.empty((M, N, G), dtype=torch.int32, device="cuda")
+
+    def close(y_s, y_ref):
+        scale = float(np.abs(y_ref.astype(np.float64)).max())
+        assert np.abs(y_s.astype(np.float64) - y_ref.astype(np.float64)).max() <= 1e-3 * scale
+
+    # ---- TRIP factors (Eq. 5-8), 4-bit codes, k_max = 4
+    k_max = 4
+    alpha_t, e_t = h.aq_trip_calibrate(xd, k_max)
+    e_ref = oracle.trip_base_exponent(x, 4, k_max)
+    alpha = oracle.trip_calibrate(x, 4, e_ref, k_max)
+    assert int(e_t.item()) == e_ref and np.array_equal(alpha_t.cpu().numpy(), alpha)
+    y = h.aq_linear_w4a4_trip(xd, packed, scales, N, group, alpha_t, k_max, acc_dump=acc, workspace=ws)
+    assert h.aq_check_workspace(ws) == binding.AQ_OK
+    v_ref = oracle.quantize_act_trip(x, 4, e_ref, alpha)
+    assert np.array_equal(ws[256:256 + M * K].view(torch.int8).reshape(M, K).cpu().numpy(), v_ref)
+    acc_ref, y_ref = oracle.linear_sampled(v_ref, codes, sc, e_ref, group, rows, cols)
+    assert np.array_equal(acc[rt, ct].cpu().numpy(), acc_ref)
+    close(y[rt, ct].cpu().numpy(), y_ref)
+
+    # ---- zero point (Eq. 2, Eq. 5-7), 8-bit codes, on shifted activations
+    xs = (x.astype(np.float32) + np.float32(2.0)).astype(np.float16)
+    r = h.aq_weight_offsets(packed, scales, N, K, group)
+    y = h.aq_linear_asym(8, dev(xs), packed, scales, r, N, group, acc_dump=acc, workspace=ws)
+    assert h.aq_check_workspace(ws) == binding.AQ_OK
+    e_a, zp = oracle.asym_params(xs, 8)
+    q_u = oracle.quantize_act_asym(xs, 8, e_a, zp)
+    q_s = (q_u.astype(np.int16) - 128).astype(np.int8)
+    assert np.array_equal(ws[256:256 + M * K].view(torch.int8).reshape(M, K).cpu().numpy(), q_s)
+    acc_raw, _ = oracle.linear_sampled(q_s, codes, sc, e_a, group, rows, cols)
+    assert np.array_equal(acc[rt, ct].cpu().numpy(), acc_raw)
+    colsum = codes.astype(np.int64).reshape(N, G, 128).sum(axis=2)
+    true_acc = acc_raw.astype(np.int64) - (zp - 128) * colsum[cols]
+    y_ref = ((true_acc.astype(np.float64) * sc.astype(np.float64)[cols]).sum(axis=1) * 2.0 ** e_a).astype(np.float16)
+    close(y[rt, ct].cpu().numpy(), y_ref)
+
+    # ---- chained call: the next layer's codes equal the quantizer applied to the plain call's fp16 output
+    y_plain = h.aq_linear_w4a8(xd, packed, scales, N, group, workspace=ws)
+    e_next = oracle.layer_exponent(y_plain[rt, ct].cpu().numpy().reshape(1, -1)[:, :N_SAMPLES // 128 * 128], 8)
+    q_next = h.aq_linear_chain(8, xd, packed, scales, N, group, 8, e_next, workspace=ws)
+    ref = oracle.quantize_act(y_plain.cpu().numpy(), 8, e_next)
+    assert np.array_equal(q_next.cpu().numpy(), ref)
+    del acc
