@@ -327,7 +327,7 @@ def bench_zero_point(h, reps=30):
     ms = _event_ms(step, reps)
     ops = sum(2.0 * M * s.K * s.N for s in wl.shapes)
     return {"workload": wl.name + " with zero point", "ms_per_step": ms, "TOPS": ops / (ms * 1e-3) / 1e12,
-            "note": "quantize is two plain kernels here (min/max, codes), not the fused one"}
+            "note": "one cooperative quantize kernel (min/max, e and zp, codes) plus the per-channel term"}
 
 
 def bench_chain(h, reps=30):

@@ -105,8 +105,9 @@ cudaError_t launch_trip_calibrate(const __half* x, int M, int K, const int32_t* 
                                   Control* ctl, uint8_t* alpha_out, int32_t* scale_exp_out, const DeviceInfo& dev,
                                   cudaStream_t stream);
 
-// Zero-point variant (Eq. 2, Eq. 5-7 with alpha = 0 and a power-of-two scale): minimum and maximum,
-// then e, zp and the codes, stored as q - 2^(b-1) in int8. The control block must have been cleared.
+// Zero-point variant (Eq. 2, Eq. 5-7 with alpha = 0 and a power-of-two scale): one cooperative kernel
+// finds minimum and maximum, then e, zp and the codes, stored as q - 2^(b-1) in int8. The control block
+// must have been cleared.
 cudaError_t launch_quantize_asym(const __half* x, int M, int K, const int32_t* row_idx, int bits, Control* ctl,
                                  int8_t* q, int32_t* scale_exp_out, int32_t* zero_point_out, const DeviceInfo& dev,
                                  cudaStream_t stream);

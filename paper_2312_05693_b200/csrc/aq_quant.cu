@@ -320,19 +320,59 @@ __device__ __forceinline__ float key_float(unsigned int k) {
 }
 constexpr unsigned int kZeroKey = 0x80000000u;         // key of +0.0: the range always contains 0
 
-__global__ void __launch_bounds__(256)
-minmax_kernel(const uint4* __restrict__ x, int M, int vec_per_row /* 8-element vectors */,
-              const int32_t* __restrict__ row_idx, Control* __restrict__ ctl) {
-    const size_t total = (size_t)M * vec_per_row;
+// 8 halves -> 8 stored codes (q - 2^(b-1)) of the zero-point quantizer in half2 arithmetic, for
+// exponents whose 2^-e is a normal half. The product by 2^-e is exact (or saturates and is clamped);
+// NaN lanes are cleared to 0, which becomes the code zp; clamping rint(t) + zp to [0, qr] equals
+// clamping t to [-zp, qr - zp] before rounding (integer bounds); adding 1536 rounds to nearest even;
+// adding the integer zp - 2^(b-1) keeps the sum inside [1024, 2048), so the code's byte is the low
+// 8 bits of the half's bit pattern.
+__device__ __forceinline__ void quantize8_half2_asym(const uint4& d, __half2 inv2, __half2 lo2, __half2 hi2,
+                                                     __half2 shift2, uint32_t& w0, uint32_t& w1) {
+    const __half2* h = reinterpret_cast<const __half2*>(&d);
+    const __half2 bias = __floats2half2_rn(1536.0f, 1536.0f);
+    uint32_t r[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        __half2 t = __hmul2(h[i], inv2);
+        const uint32_t ok = __heq2_mask(t, t);
+        uint32_t tb = *reinterpret_cast<uint32_t*>(&t) & ok;
+        t = *reinterpret_cast<__half2*>(&tb);
+        t = __hadd2(__hadd2(__hmin2(__hmax2(t, lo2), hi2), bias), shift2);
+        r[i] = *reinterpret_cast<uint32_t*>(&t);
+    }
+    w0 = __byte_perm(r[0], r[1], 0x6420);
+    w1 = __byte_perm(r[2], r[3], 0x6420);
+}
+
+// One cooperative kernel, as quantize_fused_kernel: first pass minimum and maximum (16-byte loads, the
+// share parked in shared memory), meeting point, e and zp in binary64 by one thread per CTA, second
+// pass codes from shared memory.
+__global__ void __launch_bounds__(kFusedThreads, 1)
+quantize_asym_fused_kernel(const uint4* __restrict__ x, int M, int units_per_row /* 16-element units */,
+                           const int32_t* __restrict__ row_idx, int bits, Control* __restrict__ ctl,
+                           uint4* __restrict__ q, int32_t* __restrict__ scale_exp_out,
+                           int32_t* __restrict__ zero_point_out, unsigned int cache_units, unsigned int units_per_cta) {
+    extern __shared__ uint4 fused_cache[];             // [2][cache_units]
+    __shared__ unsigned int warp_min[kFusedThreads / 32], warp_maxk[kFusedThreads / 32];
+    __shared__ int params[3];                          // e, zp, gave up
+    const size_t total = (size_t)M * units_per_row;
+    const size_t u0 = (size_t)blockIdx.x * units_per_cta;
+    const size_t u1 = u0 + units_per_cta < total ? u0 + units_per_cta : total;
+
     __half2 lo2 = __float2half2_rn(0.0f), hi2 = __float2half2_rn(0.0f);      // the range always contains 0
-    for (size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x; v < total; v += (size_t)gridDim.x * blockDim.x) {
-        const int m = (int)(v / vec_per_row), c = (int)(v % vec_per_row);
-        const uint4 d = __ldg(x + (size_t)(row_idx ? row_idx[m] : m) * vec_per_row + c);
-        const __half2* h = reinterpret_cast<const __half2*>(&d);
+#pragma unroll 2
+    for (size_t u = u0 + threadIdx.x; u < u1; u += kFusedThreads) {
+        const int m = (int)(u / units_per_row), c = (int)(u % units_per_row);
+        const size_t src = ((size_t)(row_idx ? row_idx[m] : m) * units_per_row + c) * 2;
+        const uint4 d0 = __ldg(x + src), d1 = __ldg(x + src + 1);
+        const unsigned int local = (unsigned int)(u - u0);
+        if (local < cache_units) { fused_cache[local] = d0; fused_cache[cache_units + local] = d1; }
+        const __half2* h0 = reinterpret_cast<const __half2*>(&d0);
+        const __half2* h1 = reinterpret_cast<const __half2*>(&d1);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {                                        // NaN operands are dropped
-            lo2 = __hmin2(lo2, h[i]);
-            hi2 = __hmax2(hi2, h[i]);
+            lo2 = __hmin2(lo2, __hmin2(h0[i], h1[i]));
+            hi2 = __hmax2(hi2, __hmax2(h0[i], h1[i]));
         }
     }
     // +-Inf count as the largest half
@@ -344,36 +384,50 @@ minmax_kernel(const uint4* __restrict__ x, int M, int vec_per_row /* 8-element v
         kmin = min(kmin, __shfl_xor_sync(0xFFFFFFFFu, kmin, o));
         kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, o));
     }
-    if ((threadIdx.x & 31) == 0) {
-        // the control block is cleared to 0: keys are stored relative to the key of 0.0
-        if (kmax > kZeroKey) atomicMax(&ctl->max_key, kmax - kZeroKey);
-        if (kmin < kZeroKey) atomicMax(&ctl->min_key, kZeroKey - kmin);
-    }
-}
-
-// e = smallest integer with (2^b - 1) * 2^e >= max - min, zp = clip(round(-min / 2^e), 0, 2^b - 1), in
-// binary64 (exact for fp16 inputs), by one thread of every CTA; then 16 codes per thread.
-__global__ void __launch_bounds__(kQuantThreads)
-quantize_asym_kernel(const uint4* __restrict__ x, int M, int vec_per_row /* 16-element units */,
-                     const int32_t* __restrict__ row_idx, int bits, Control* __restrict__ ctl, uint4* __restrict__ q,
-                     int32_t* __restrict__ scale_exp_out, int32_t* __restrict__ zero_point_out) {
-    __shared__ int params[2];
-    const double qr = (double)((1 << bits) - 1);
-    if (threadIdx.x == 0) {
-        const double hi = (double)key_float(kZeroKey + ctl->max_key), lo = (double)key_float(kZeroKey - ctl->min_key);
-        const double range = hi - lo;
-        int ee = 0;
-        if (range > 0.0) {
-            int ex;
-            frexp(range / qr, &ex);                  // a first guess within one of the answer
-            ee = ex;
-            while (ldexp(qr, ee) < range) ++ee;
-            while (ldexp(qr, ee - 1) >= range) --ee;
+    if ((threadIdx.x & 31) == 0) { warp_min[threadIdx.x >> 5] = kmin; warp_maxk[threadIdx.x >> 5] = kmax; }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        kmin = warp_min[threadIdx.x];
+        kmax = warp_maxk[threadIdx.x];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            kmin = min(kmin, __shfl_xor_sync(0xFFFFFFFFu, kmin, o));
+            kmax = max(kmax, __shfl_xor_sync(0xFFFFFFFFu, kmax, o));
         }
-        params[0] = ee;
-        params[1] = (int)fmin(fmax(rint(ldexp(-lo, -ee)), 0.0), qr);
+        if (threadIdx.x == 0) {
+            // the control block is cleared to 0: keys are stored relative to the key of 0.0
+            if (kmax > kZeroKey) atomicMax(&ctl->max_key, kmax - kZeroKey);
+            if (kmin < kZeroKey) atomicMax(&ctl->min_key, kZeroKey - kmin);
+            __threadfence();
+            atomicAdd(&ctl->counter, 1u);
+            const long long t0 = clock64();
+            int failed = 0;
+            while (ld_acquire_u32(&ctl->counter) < gridDim.x) {
+                if ((unsigned long long)(clock64() - t0) > kFusedWaitCycles) { failed = 1; break; }
+                __nanosleep(100);
+            }
+            const double qr = (double)((1 << bits) - 1);
+            const double dhi = (double)key_float(kZeroKey + ld_acquire_u32(&ctl->max_key));
+            const double dlo = (double)key_float(kZeroKey - ld_acquire_u32(&ctl->min_key));
+            const double range = dhi - dlo;
+            int ee = 0;
+            if (range > 0.0) {
+                int ex;
+                frexp(range / qr, &ex);              // a first guess within one of the answer
+                ee = ex;
+                while (ldexp(qr, ee) < range) ++ee;
+                while (ldexp(qr, ee - 1) >= range) --ee;
+            }
+            params[0] = ee;
+            params[1] = (int)fmin(fmax(rint(ldexp(-dlo, -ee)), 0.0), qr);
+            params[2] = failed;
+        }
     }
     __syncthreads();
+    if (params[2]) {
+        if (threadIdx.x == 0) atomicCAS(&ctl->status, 0u, kFusedWaitCode);
+        return;
+    }
     const int e = params[0], zp = params[1];
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         ctl->scale_exp = e;
@@ -381,32 +435,47 @@ quantize_asym_kernel(const uint4* __restrict__ x, int M, int vec_per_row /* 16-e
         if (scale_exp_out) *scale_exp_out = e;
         if (zero_point_out) *zero_point_out = zp;
     }
+    const int qr_i = (1 << bits) - 1, half_range = 1 << (bits - 1);
     const float inv = __int_as_float((127 - e) << 23);      // 2^-e
-    const float fzp = (float)zp, fqr = (float)qr;
-    const int half_range = 1 << (bits - 1);
-    const size_t total = (size_t)M * vec_per_row;
-    const size_t v = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (v >= total) return;
-    const int m = (int)(v / vec_per_row), c = (int)(v % vec_per_row);
-    const size_t src = ((size_t)(row_idx ? row_idx[m] : m) * vec_per_row + c) * 2;
-    const uint4 d0 = __ldg(x + src), d1 = __ldg(x + src + 1);
-    const __half* h0 = reinterpret_cast<const __half*>(&d0);
-    const __half* h1 = reinterpret_cast<const __half*>(&d1);
-    uint32_t out[4];
-#pragma unroll
-    for (int w = 0; w < 4; ++w) {
-        uint32_t word = 0;
-#pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            const int i = 4 * w + b;
-            const float t = __half2float(i < 8 ? h0[i] : h1[i - 8]) * inv;    // exact
-            int code = zp;                                                    // NaN: value 0
-            if (t == t) code = (int)fminf(fmaxf(rintf(t) + fzp, 0.0f), fqr);
-            word |= ((uint32_t)(code - half_range) & 0xFFu) << (8 * b);
+    const float fzp = (float)zp, fqr = (float)qr_i;
+    const bool fast = e >= -14 && e <= 14;                   // 2^-e is a normal half
+    const __half2 inv2 = __float2half2_rn(fast ? inv : 1.0f);
+    const __half2 clo2 = __float2half2_rn(-fzp), chi2 = __float2half2_rn(fqr - fzp);
+    const __half2 shift2 = __float2half2_rn((float)(zp - half_range));
+#pragma unroll 2
+    for (size_t u = u0 + threadIdx.x; u < u1; u += kFusedThreads) {
+        const unsigned int local = (unsigned int)(u - u0);
+        uint4 d0, d1;
+        if (local < cache_units) {
+            d0 = fused_cache[local]; d1 = fused_cache[cache_units + local];      // this thread's own stores
+        } else {
+            const int m = (int)(u / units_per_row), c = (int)(u % units_per_row);
+            const size_t src = ((size_t)(row_idx ? row_idx[m] : m) * units_per_row + c) * 2;
+            d0 = __ldg(x + src); d1 = __ldg(x + src + 1);
         }
-        out[w] = word;
+        uint32_t out[4];
+        if (fast) {
+            quantize8_half2_asym(d0, inv2, clo2, chi2, shift2, out[0], out[1]);
+            quantize8_half2_asym(d1, inv2, clo2, chi2, shift2, out[2], out[3]);
+        } else {
+            const __half* h0 = reinterpret_cast<const __half*>(&d0);
+            const __half* h1 = reinterpret_cast<const __half*>(&d1);
+#pragma unroll
+            for (int w = 0; w < 4; ++w) {
+                uint32_t word = 0;
+#pragma unroll
+                for (int b = 0; b < 4; ++b) {
+                    const int i = 4 * w + b;
+                    const float t = __half2float(i < 8 ? h0[i] : h1[i - 8]) * inv;    // exact
+                    int code = zp;                                                    // NaN: value 0
+                    if (t == t) code = (int)fminf(fmaxf(rintf(t) + fzp, 0.0f), fqr);
+                    word |= ((uint32_t)(code - half_range) & 0xFFu) << (8 * b);
+                }
+                out[w] = word;
+            }
+        }
+        q[u] = make_uint4(out[0], out[1], out[2], out[3]);
     }
-    q[v] = make_uint4(out[0], out[1], out[2], out[3]);
 }
 
 __global__ void chan_offsets_kernel(const float* __restrict__ r, int N, int bits, const Control* __restrict__ ctl,
@@ -609,19 +678,29 @@ cudaError_t launch_trip_calibrate(const __half* x, int M, int K, const int32_t* 
 cudaError_t launch_quantize_asym(const __half* x, int M, int K, const int32_t* row_idx, int bits, Control* ctl,
                                  int8_t* q, int32_t* scale_exp_out, int32_t* zero_point_out, const DeviceInfo& dev,
                                  cudaStream_t stream) {
-    const size_t total = (size_t)M * (K / 8);
-    size_t blocks = (total + 255) / 256;
-    const size_t cap = (size_t)dev.sm_count * 8;
-    if (blocks > cap) blocks = cap;
-    minmax_kernel<<<(unsigned int)blocks, 256, 0, stream>>>(reinterpret_cast<const uint4*>(x), M, K / 8, row_idx, ctl);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
-    const int vec_per_row = K / 16;
-    const size_t units = (size_t)M * vec_per_row;
-    quantize_asym_kernel<<<(unsigned int)((units + kQuantThreads - 1) / kQuantThreads), kQuantThreads, 0, stream>>>(
-        reinterpret_cast<const uint4*>(x), M, vec_per_row, row_idx, bits, ctl, reinterpret_cast<uint4*>(q),
-        scale_exp_out, zero_point_out);
-    return cudaGetLastError();
+    int units_per_row = K / 16;
+    const size_t total = (size_t)M * units_per_row;
+    size_t grid = (total + kFusedThreads - 1) / kFusedThreads;
+    if (grid > (size_t)dev.sm_count) grid = (size_t)dev.sm_count;
+    unsigned int units_per_cta = (unsigned int)((total + grid - 1) / grid);
+    const size_t reserve = 8192;
+    const size_t max_cache = dev.smem_optin > reserve ? (dev.smem_optin - reserve) / 32 : 0;
+    unsigned int cache_units = units_per_cta < max_cache ? units_per_cta : (unsigned int)max_cache;
+    const size_t smem_bytes = (size_t)cache_units * 32;
+    static bool attr_done = false;
+    if (!attr_done) {
+        const cudaError_t e = cudaFuncSetAttribute(quantize_asym_fused_kernel,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)(dev.smem_optin - reserve));
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    const uint4* xp = reinterpret_cast<const uint4*>(x);
+    uint4* qp = reinterpret_cast<uint4*>(q);
+    void* args[] = {&xp, &M, &units_per_row, &row_idx, &bits, &ctl, &qp, &scale_exp_out, &zero_point_out, &cache_units,
+                    &units_per_cta};
+    return cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(quantize_asym_fused_kernel),
+                                       dim3((unsigned int)grid), dim3(kFusedThreads), args, smem_bytes, stream);
 }
 
 cudaError_t launch_chan_offsets(const float* r, int N, int bits, const Control* ctl, float* off, cudaStream_t stream) {
