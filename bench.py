@@ -639,7 +639,10 @@ def main():
                 "h2d_bytes_per_step": int(sum(M * s.K * 2 for s in wl.shapes)),
                 "d2h_bytes_per_step": int(sum(M * s.N * 2 for s in wl.shapes)),
                 "ms_per_step": e2e_ms, "api": "aq_linear_host"},
-        "gpu_launches": args.steps * len(layers) * 2,     # per layer: the fused quantize kernel and the product kernel
+        # per layer: the fused quantize kernel and the product kernel, which is two launches where the tiles of a
+        # partial last round are shared between CTA pairs (the workspace then has room for their partial sums)
+        "gpu_launches": args.steps * sum(2 + (binding.aq_workspace_bytes(M, s.K, s.N, wl.group_size) >
+                                              binding.aq_workspace_bytes(M, s.K, s.N, 0)) for s in wl.shapes),
         "clocks": clocks,
         "roofline": roofline,
     }

@@ -38,14 +38,20 @@ struct Workspace {
     void* scratch;
     size_t scratch_bytes;
     float* chan_offset;
+    float* split_scratch;
+    size_t split_bytes;
 };
 
 // [control block][codes M*K][kernel scratch, M bytes][per-channel offsets of the zero-point variant, N floats]
-size_t workspace_bytes(int M, int K, int N) {
-    return sizeof(Control) + up256((size_t)M * K) + up256((size_t)M) + up256((size_t)N * sizeof(float));
+// [fp32 partial outputs of tiles that two CTAs share in the tensor kernel, sized for a 148-SM B200; a
+// device that would need more simply shares no tile]
+constexpr int kPlannedSmCount = 148;
+size_t workspace_bytes(int M, int K, int N, int group) {
+    return sizeof(Control) + up256((size_t)M * K) + up256((size_t)M) + up256((size_t)N * sizeof(float)) +
+           up256(tensor_split_scratch_bytes(M, K, N, group, kPlannedSmCount));
 }
 
-Workspace carve(void* ws, int M, int K) {
+Workspace carve(void* ws, int M, int K, int N, size_t total_bytes) {
     Workspace w;
     uint8_t* b = static_cast<uint8_t*>(ws);
     w.ctl = reinterpret_cast<Control*>(b);
@@ -53,6 +59,9 @@ Workspace carve(void* ws, int M, int K) {
     w.scratch = b + sizeof(Control) + up256((size_t)M * K);
     w.scratch_bytes = up256((size_t)M);
     w.chan_offset = reinterpret_cast<float*>(b + sizeof(Control) + up256((size_t)M * K) + up256((size_t)M));
+    const size_t used = sizeof(Control) + up256((size_t)M * K) + up256((size_t)M) + up256((size_t)N * sizeof(float));
+    w.split_scratch = reinterpret_cast<float*>(b + used);
+    w.split_bytes = total_bytes > used ? total_bytes - used : 0;
     return w;
 }
 
@@ -102,12 +111,12 @@ int linear_impl(aq_handle_t h, int bits, const void* x, int M, int K, const void
     if (scale_mode == AQ_SCALE_STATIC && (clip_shift_or_exp < -40 || clip_shift_or_exp > 40)) return AQ_ERR_INVALID_ARG;
     const int s = check_shape(M, K, N, group);
     if (s != AQ_OK) return s;
-    if (!workspace || workspace_bytes_ < workspace_bytes(M, K, N)) return AQ_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes_ < workspace_bytes(M, K, N, group)) return AQ_ERR_WORKSPACE;
     if (!aligned(x, 16) || !aligned(w_packed, 16) || !aligned(w_scales, 2) || (y && !aligned(y, 2)) ||
         !aligned(workspace, 256) || (acc_dump && !aligned(acc_dump, 4)) || (row_idx && !aligned(row_idx, 4)))
         return AQ_ERR_ALIGNMENT;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    const Workspace w = carve(workspace, M, K);
+    const Workspace w = carve(workspace, M, K, N, workspace_bytes_);
     const __half* xh = static_cast<const __half*>(x);
     if (alpha && !aligned(alpha, 16)) return AQ_ERR_ALIGNMENT;
     cudaError_t e;
@@ -131,6 +140,7 @@ int linear_impl(aq_handle_t h, int bits, const void* x, int M, int K, const void
     g.y = static_cast<__half*>(y);
     g.acc_dump = acc_dump;
     g.ctl = w.ctl; g.scratch = w.scratch; g.scratch_bytes = w.scratch_bytes;
+    g.split_scratch = w.split_scratch; g.split_bytes = w.split_bytes;
     g.chan_offset = w_offsets ? w.chan_offset : nullptr;
     g.q_next = q_next; g.next_bits = next_bits; g.next_exp = next_exp;
     return run_gemm(h, g, stream);
@@ -218,7 +228,7 @@ size_t aq_scales_bytes(int N, int K, int group_size) {
 
 size_t aq_workspace_bytes(int M, int K, int N, int group_size) {
     if (check_shape(M, K, N, group_size) != AQ_OK) return 0;
-    return workspace_bytes(M, K, N);
+    return workspace_bytes(M, K, N, group_size);
 }
 
 int aq_pack_w4(aq_handle_t h, const void* w_fp16, int N, int K, int group_size, void* w_packed,
@@ -330,12 +340,12 @@ int aq_gemm_w4(aq_handle_t h, const int8_t* q, int M, int K, const void* w_packe
     if (!h || !q || !w_packed || !w_scales || !scale_exp || !y_fp16) return AQ_ERR_INVALID_ARG;
     const int s = check_shape(M, K, N, group_size);
     if (s != AQ_OK) return s;
-    if (!workspace || workspace_bytes_ < workspace_bytes(M, K, N)) return AQ_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes_ < workspace_bytes(M, K, N, group_size)) return AQ_ERR_WORKSPACE;
     if (!aligned(q, 16) || !aligned(w_packed, 16) || !aligned(w_scales, 2) || !aligned(y_fp16, 2) ||
         !aligned(workspace, 256) || !aligned(scale_exp, 4) || (acc_dump && !aligned(acc_dump, 4)))
         return AQ_ERR_ALIGNMENT;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    const Workspace w = carve(workspace, M, K);
+    const Workspace w = carve(workspace, M, K, N, workspace_bytes_);
     if (kernel_for(h, M) == AQ_KERNEL_TENSOR) {       // the decode kernels clear the status word themselves
         const cudaError_t e = cudaMemsetAsync(w.ctl, 0, sizeof(Control), stream);
         if (e != cudaSuccess) return cuda_fail(h, e);
@@ -348,6 +358,7 @@ int aq_gemm_w4(aq_handle_t h, const int8_t* q, int M, int K, const void* w_packe
     g.y = static_cast<__half*>(y_fp16);
     g.acc_dump = acc_dump;
     g.ctl = w.ctl; g.scratch = w.scratch; g.scratch_bytes = w.scratch_bytes;
+    g.split_scratch = w.split_scratch; g.split_bytes = w.split_bytes;
     return run_gemm(h, g, stream);
 }
 
@@ -528,7 +539,7 @@ int aq_prune_schedule(int M, double beta, int m, int32_t* n_keep_out, double* ga
 
 size_t aq_linear_host_scratch_bytes(int M, int K, int N, int group_size) {
     if (check_shape(M, K, N, group_size) != AQ_OK) return 0;
-    return up256((size_t)M * K * 2) + up256((size_t)M * N * 2) + workspace_bytes(M, K, N);
+    return up256((size_t)M * K * 2) + up256((size_t)M * N * 2) + workspace_bytes(M, K, N, group_size);
 }
 
 int aq_linear_host(aq_handle_t h, int bits, const void* x_host, int M, int K, const void* w_packed,
@@ -548,7 +559,7 @@ int aq_linear_host(aq_handle_t h, int bits, const void* x_host, int M, int K, co
     cudaError_t e = cudaMemcpyAsync(x_dev, x_host, (size_t)M * K * 2, cudaMemcpyHostToDevice, stream);
     if (e != cudaSuccess) return cuda_fail(h, e);
     const int rc = linear_impl(h, bits, x_dev, M, K, w_packed, w_scales, N, group_size, scale_mode,
-                               clip_shift_or_exp, nullptr, y_dev, nullptr, ws, workspace_bytes(M, K, N), stream_);
+                               clip_shift_or_exp, nullptr, y_dev, nullptr, ws, workspace_bytes(M, K, N, group_size), stream_);
     if (rc != AQ_OK) return rc;
     e = cudaMemcpyAsync(y_host, y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, stream);
     if (e != cudaSuccess) return cuda_fail(h, e);

@@ -46,7 +46,8 @@ struct Control {
     unsigned int counter;       // scratch counter
     unsigned int min_key, max_key;   // zero-point variant: order-preserving keys of min(x), max(x)
     int zero_point;             // zero-point variant: zp of Eq. 7
-    unsigned int reserved[57];
+    unsigned int split_flags[57];   // tensor kernel: one bit per (shared tile, epilogue warp), "first half arrived"
+    static constexpr int kMaxSplitTiles = 57 * 32 / 8;
 };
 static_assert(sizeof(Control) == 256, "control block is 256 bytes");
 
@@ -151,6 +152,9 @@ struct GemmArgs {
     // [M][N] int8: clip(round(y16 / 2^next_exp), -2^(b-1), 2^(b-1)-1), y16 the fp16 value y would have held.
     int8_t* q_next = nullptr;
     int next_bits = 8, next_exp = 0;
+    // fp32 partial outputs of tiles whose k range two CTAs share (tensor kernel, per-group scales)
+    float* split_scratch = nullptr;
+    size_t split_bytes = 0;
     void* scratch;          // beyond control block + codes
     size_t scratch_bytes;
 };
@@ -159,6 +163,8 @@ int handle_device(aq_handle_t h);
 void handle_record_cuda_error(aq_handle_t h, cudaError_t e);
 
 cudaError_t launch_gemm_tensor(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream);
+// Bytes of split_scratch the tensor kernel can use for these sizes on a GPU with sm_count SMs (0: none).
+size_t tensor_split_scratch_bytes(int M, int K, int N, int group, int sm_count);
 cudaError_t launch_gemm_decode(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream);
 
 }  // namespace aq

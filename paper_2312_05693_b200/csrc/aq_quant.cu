@@ -184,6 +184,7 @@ quantize_small_kernel(const uint4* __restrict__ x, int M, int vec_per_row, const
         ctl->counter = 0;
         if (scale_exp_out) *scale_exp_out = e;
     }
+    if (rank == 0 && threadIdx.x < 57) ctl->split_flags[threadIdx.x] = 0;    // the product kernel's shared-tile bits
     const float lo = -(float)(1 << (bits - 1)), hi = (float)((1 << (bits - 1)) - 1);
 #pragma unroll
     for (int i = 0; i < kSmallVecs; ++i) {

@@ -234,6 +234,23 @@ def test_several_tiles_per_cta_and_deep_k(group):
     assert_y_close(gpu["y"], ref["y"])
 
 
+@pytest.mark.parametrize("M,N", [(200, 520), (1100, 2304)])
+def test_shared_tiles_of_a_partial_last_round(M, N):
+    """Deep reduction (64 k blocks) with a last round that fills less than half of the SMs: those tiles
+    are shared by two CTAs (half of K each, partial sums exchanged). 10 tiles: every tile is shared;
+    162 tiles: one whole round, then 14 shared tiles."""
+    K = 8192
+    x = inputs.activations(M, K, seed=125, outlier_frac=0.005, outlier_mult=30.0)
+    w = inputs.weights(N, K, seed=126)
+    assert binding.aq_workspace_bytes(M, K, N, 128) > binding.aq_workspace_bytes(M, K, N, 0)   # room for the partial sums
+    gpu, ref = run_layer_both(x, w, 8, 128, TENSOR)
+    assert gpu["e"] == ref["e"] and np.array_equal(gpu["q"], ref["q"])
+    assert np.array_equal(gpu["acc"], ref["acc"])
+    assert_y_close(gpu["y"], ref["y"])
+    gpu2, _ = run_layer_both(x, w, 8, 128, TENSOR, want_acc=False)
+    assert np.array_equal(gpu["y"].view(np.uint16), gpu2["y"].view(np.uint16))     # whichever half arrives second
+
+
 def test_results_are_deterministic_run_to_run():
     M, K, N = 260, 1152, 520
     x = inputs.activations(M, K, seed=9, outlier_frac=0.01, outlier_mult=20.0)
