@@ -698,8 +698,25 @@ cudaError_t launch_off(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t st
     p.split_base = split_base;
     p.split_scratch = a.split_scratch;
     const int grid = SPLIT ? 2 * split_tiles : (p.n_tiles < dev.sm_count ? p.n_tiles : dev.sm_count);
-    gemm_tensor_kernel<BM, GROUPED, OFFSET, CHAIN, SPLIT><<<grid, kThreads, smem_bytes, stream>>>(map, ymap, p);
-    return cudaGetLastError();
+    if constexpr (SPLIT) {
+        // This launch depends on nothing the preceding whole-round launch writes (other tiles of y; the
+        // partial sums and their flags are its own), so it may be set up while that one still runs: its
+        // CTAs start as SMs become free instead of after a launch gap.
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = smem_bytes;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = split_base > 0 ? 1 : 0;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        return cudaLaunchKernelEx(&cfg, gemm_tensor_kernel<BM, GROUPED, OFFSET, CHAIN, SPLIT>, map, ymap, p);
+    } else {
+        gemm_tensor_kernel<BM, GROUPED, OFFSET, CHAIN, SPLIT><<<grid, kThreads, smem_bytes, stream>>>(map, ymap, p);
+        return cudaGetLastError();
+    }
 }
 
 template <int BM, bool GROUPED>
