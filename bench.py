@@ -360,6 +360,25 @@ def bench_chain(h, reps=30):
             "codes_between": {"us": t_chain * 1e3, "TOPS": ops / (t_chain * 1e-3) / 1e12}}
 
 
+def bench_act4(h, reps=30):
+    """4-bit activation codes stored two per byte (Sec. 4.4): cost of the passes that pack them and
+    widen them again before the product, on the first int4 benchmark shape."""
+    wl = inputs.WORKLOADS["llama7b_prefill_w4a4"]
+    M, s = wl.Ms[0], wl.shapes[0]
+    x = torch.from_numpy(inputs.activations(M, s.K, wl.seed, wl.outlier_frac, wl.outlier_mult)).cuda()
+    p, sc = h.aq_pack_w4(torch.from_numpy(inputs.weights(s.N, s.K, wl.seed)).cuda(), wl.group_size)
+    ws = h.alloc_workspace(M, s.K, s.N, wl.group_size)
+    y = torch.empty((M, s.N), dtype=torch.float16, device="cuda")
+    q, e = h.aq_quantize_act(x, 4, clip_shift_or_exp=wl.clip_shift)
+    q4 = h.aq_act4_pack(q)
+    t_pack = graph_replay_ms(lambda: h.aq_act4_pack(q, q4), reps)
+    t_plain = _event_ms(lambda: h.aq_gemm_w4(q, p, sc, s.N, wl.group_size, e, y=y, workspace=ws), reps)
+    t_packed = _event_ms(lambda: h.aq_gemm_w4_act4(q4, p, sc, s.N, wl.group_size, e, y=y, workspace=ws), reps)
+    return {"M": M, "K": s.K, "N": s.N, "code_bytes": {"int8_containers": M * s.K, "packed": M * s.K // 2},
+            "pack_us": t_pack * 1e3, "product_us": t_plain * 1e3, "product_on_packed_us": t_packed * 1e3,
+            "note": "the product widens packed codes with one extra pass; the tensor cores take 8-bit integers"}
+
+
 def bench_attention(h, reps=5):
     """Softmax output as 4-bit log2 codes times int8 value codes (Eq. 3), LLaMA-7B attention shape."""
     H, M, J, D = 32, 2048, 2048, 128
@@ -652,7 +671,7 @@ def main():
         except Exception as ex:  # report, do not hide
             line["decode"] = {"error": repr(ex)}
     if rank == 0 and world == 1 and not args.no_decode:
-        for key, fn in (("w4a4", bench_w4a4), ("zero_point", bench_zero_point), ("chain", bench_chain),
+        for key, fn in (("w4a4", bench_w4a4), ("zero_point", bench_zero_point), ("chain", bench_chain), ("act4_storage", bench_act4),
                         ("attention_log2", bench_attention), ("pruned_prefill", bench_pruned)):
             try:
                 line[key] = fn(h)

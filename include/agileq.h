@@ -205,6 +205,29 @@ int aq_linear_w4a4_chain(aq_handle_t h, const void* x_fp16, int M, int K, const 
                          int8_t* q_next, int next_bits, int next_exp, int32_t* acc_dump, void* workspace,
                          size_t workspace_bytes, void* stream);
 
+/* ---- packed storage of 4-bit activation codes (paper Sec. 4.4: two adjacent 4-bit values share a
+ * byte, as the weights do)
+ * q4 [M, K/2] bytes, row-major, device: byte j of a row holds code 2j in bits 0-3 and code 2j+1 in
+ * bits 4-7, two's-complement nibbles. K % 32 == 0; q and q4 16-byte aligned; aq_act4_bytes = M*K/2
+ * (0 for sizes the calls reject).
+ * aq_act4_pack: q int8 [M,K] with values in [-8, 7] (only the low four bits of each are kept).
+ * aq_act4_unpack: the inverse, sign-extended int8 codes.
+ * aq_quantize_act4: aq_quantize_act with bits = 4 whose codes are written packed; K % 128 == 0; the
+ *   workspace must hold aq_workspace_bytes(M, K, 1, 0) (the codes pass through it in one-byte containers).
+ * aq_gemm_w4_act4: aq_gemm_w4 on packed codes. The tensor cores have no 4-bit integer operand, so the
+ *   codes are widened into the workspace's code area by one extra pass (M*K/2 bytes read, M*K written)
+ *   before the product; what the packed form halves is the storage and traffic between layers.
+ * Errors as for aq_quantize_act / aq_gemm_w4. */
+size_t aq_act4_bytes(int M, int K);
+int aq_act4_pack(aq_handle_t h, const int8_t* q, int M, int K, void* q4, void* stream);
+int aq_act4_unpack(aq_handle_t h, const void* q4, int M, int K, int8_t* q, void* stream);
+int aq_quantize_act4(aq_handle_t h, const void* x_fp16, int M, int K, int scale_mode, int clip_shift_or_exp,
+                     const int32_t* row_idx, void* q4, int32_t* scale_exp_out, void* workspace,
+                     size_t workspace_bytes, void* stream);
+int aq_gemm_w4_act4(aq_handle_t h, const void* q4, int M, int K, const void* w_packed, const void* w_scales,
+                    int N, int group_size, const int32_t* scale_exp, void* y_fp16, int32_t* acc_dump,
+                    void* workspace, size_t workspace_bytes, void* stream);
+
 /* ---- log2 quantization of the softmax output and attention x value (paper Eq. 3, Sec. 5.1)
  * aq_log2_quantize: x_fp16 holds `count` values (any shape); max|x| is taken over all of them.
  *   k = CLIP(round(-log2(|x| / max|x|)), 0, 2^(b-1) - 1), so x ~ Sign(x) * max|x| * 2^-k. codes (int8, same

@@ -140,6 +140,15 @@ def unpack_w4(packed: np.ndarray) -> np.ndarray:
     return out
 
 
+def pack_act4(codes: np.ndarray) -> np.ndarray:
+    """4-bit activation codes [M, K] -> [M, K/2] bytes; the nibble order is the one of pack_w4."""
+    return pack_w4(codes)
+
+
+def unpack_act4(packed: np.ndarray) -> np.ndarray:
+    return unpack_w4(packed)
+
+
 def token_select(scores: np.ndarray, n_keep: int) -> np.ndarray:
     scores = _c(scores, np.float32)
     idx = np.empty((n_keep,), np.int32)

@@ -74,6 +74,12 @@ def load():
     L.aq_linear_w4a8.argtypes = lin
     L.aq_linear_w4a4.argtypes = lin
     L.aq_gemm_w4.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, vp, vp, vp, vp, sz, vp]
+    L.aq_act4_bytes.restype = sz
+    L.aq_act4_bytes.argtypes = [i32, i32]
+    L.aq_act4_pack.argtypes = [vp, vp, i32, i32, vp, vp]
+    L.aq_act4_unpack.argtypes = [vp, vp, i32, i32, vp, vp]
+    L.aq_quantize_act4.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, sz, vp]
+    L.aq_gemm_w4_act4.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, vp, vp, vp, vp, sz, vp]
     L.aq_weight_offsets.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp]
     L.aq_quantize_act_asym.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
     lin_asym = [vp, vp, i32, i32, vp, vp, vp, i32, i32, vp, vp, vp, vp, sz, vp]
@@ -372,6 +378,44 @@ class Handle:
         _check(load().aq_gemm_w4(self._h, _ptr(q), M, K, _ptr(packed), _ptr(scales), N, group_size,
                                  _ptr(scale_exp), _ptr(y), _ptr(acc_dump), _ptr(workspace),
                                  workspace.numel(), _stream()), "aq_gemm_w4")
+        return y
+
+    def aq_act4_pack(self, q: torch.Tensor, q4: Optional[torch.Tensor] = None) -> torch.Tensor:
+        M, K = q.shape
+        if q4 is None:
+            q4 = torch.empty((M, K // 2), dtype=torch.uint8, device=q.device)
+        _check(load().aq_act4_pack(self._h, _ptr(q), M, K, _ptr(q4), _stream()), "aq_act4_pack")
+        return q4
+
+    def aq_act4_unpack(self, q4: torch.Tensor) -> torch.Tensor:
+        M, K2 = q4.shape
+        q = torch.empty((M, 2 * K2), dtype=torch.int8, device=q4.device)
+        _check(load().aq_act4_unpack(self._h, _ptr(q4), M, 2 * K2, _ptr(q), _stream()), "aq_act4_unpack")
+        return q
+
+    def aq_quantize_act4(self, x: torch.Tensor, scale_mode: int = AQ_SCALE_DYNAMIC, clip_shift_or_exp: int = 0,
+                         row_idx: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None):
+        M_in, K = x.shape
+        M = M_in if row_idx is None else row_idx.shape[0]
+        q4 = torch.empty((M, K // 2), dtype=torch.uint8, device=x.device)
+        e = torch.empty(1, dtype=torch.int32, device=x.device)
+        if workspace is None:
+            workspace = self.alloc_workspace(M, K, 1, 0)
+        _check(load().aq_quantize_act4(self._h, _ptr(x), M, K, scale_mode, clip_shift_or_exp, _ptr(row_idx),
+                                       _ptr(q4), _ptr(e), _ptr(workspace), workspace.numel(), _stream()),
+               "aq_quantize_act4")
+        return q4, e
+
+    def aq_gemm_w4_act4(self, q4, packed, scales, N, group_size, scale_exp, y=None, acc_dump=None, workspace=None):
+        M, K2 = q4.shape
+        K = 2 * K2
+        if y is None:
+            y = torch.empty((M, N), dtype=torch.float16, device=q4.device)
+        if workspace is None:
+            workspace = self.alloc_workspace(M, K, N, group_size)
+        _check(load().aq_gemm_w4_act4(self._h, _ptr(q4), M, K, _ptr(packed), _ptr(scales), N, group_size,
+                                      _ptr(scale_exp), _ptr(y), _ptr(acc_dump), _ptr(workspace),
+                                      workspace.numel(), _stream()), "aq_gemm_w4_act4")
         return y
 
     def aq_token_select(self, scores: torch.Tensor, n_keep: int, workspace=None) -> torch.Tensor:

@@ -362,6 +362,59 @@ int aq_gemm_w4(aq_handle_t h, const int8_t* q, int M, int K, const void* w_packe
     return run_gemm(h, g, stream);
 }
 
+size_t aq_act4_bytes(int M, int K) {
+    if (M < 1 || K < 32 || K % 32) return 0;
+    return (size_t)M * (size_t)K / 2;
+}
+
+int aq_act4_pack(aq_handle_t h, const int8_t* q, int M, int K, void* q4, void* stream) {
+    if (!h || !q || !q4) return AQ_ERR_INVALID_ARG;
+    if (M < 1 || K < 32 || K % 32) return AQ_ERR_SHAPE;
+    if (!aligned(q, 16) || !aligned(q4, 16)) return AQ_ERR_ALIGNMENT;
+    const cudaError_t e = launch_act4_pack(q, (size_t)M * K, static_cast<uint8_t*>(q4), static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
+int aq_act4_unpack(aq_handle_t h, const void* q4, int M, int K, int8_t* q, void* stream) {
+    if (!h || !q || !q4) return AQ_ERR_INVALID_ARG;
+    if (M < 1 || K < 32 || K % 32) return AQ_ERR_SHAPE;
+    if (!aligned(q, 16) || !aligned(q4, 16)) return AQ_ERR_ALIGNMENT;
+    const cudaError_t e = launch_act4_unpack(static_cast<const uint8_t*>(q4), (size_t)M * K, q, static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
+int aq_quantize_act4(aq_handle_t h, const void* x_fp16, int M, int K, int scale_mode, int clip_shift_or_exp,
+                     const int32_t* row_idx, void* q4, int32_t* scale_exp_out, void* workspace,
+                     size_t workspace_bytes_, void* stream) {
+    if (!q4) return AQ_ERR_INVALID_ARG;
+    if (!aligned(q4, 16)) return AQ_ERR_ALIGNMENT;
+    if (M < 1 || K < 128 || K % 128) return AQ_ERR_SHAPE;
+    // the codes pass through the workspace's code area in one-byte containers on their way to the nibbles
+    if (!workspace || workspace_bytes_ < sizeof(Control) + up256((size_t)M * K)) return AQ_ERR_WORKSPACE;
+    int8_t* codes = reinterpret_cast<int8_t*>(static_cast<uint8_t*>(workspace) + sizeof(Control));
+    const int s = quantize_impl(h, x_fp16, M, K, 4, scale_mode, clip_shift_or_exp, row_idx, codes, scale_exp_out,
+                                workspace, workspace_bytes_, stream, nullptr, 0);
+    if (s != AQ_OK) return s;
+    const cudaError_t e = launch_act4_pack(codes, (size_t)M * K, static_cast<uint8_t*>(q4), static_cast<cudaStream_t>(stream));
+    return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
+int aq_gemm_w4_act4(aq_handle_t h, const void* q4, int M, int K, const void* w_packed, const void* w_scales,
+                    int N, int group_size, const int32_t* scale_exp, void* y_fp16, int32_t* acc_dump,
+                    void* workspace, size_t workspace_bytes_, void* stream_) {
+    if (!h || !q4) return AQ_ERR_INVALID_ARG;
+    const int s = check_shape(M, K, N, group_size);
+    if (s != AQ_OK) return s;
+    if (!workspace || workspace_bytes_ < workspace_bytes(M, K, N, group_size)) return AQ_ERR_WORKSPACE;
+    if (!aligned(q4, 16) || !aligned(workspace, 256)) return AQ_ERR_ALIGNMENT;
+    const Workspace w = carve(workspace, M, K, N, workspace_bytes_);
+    const cudaError_t e = launch_act4_unpack(static_cast<const uint8_t*>(q4), (size_t)M * K, w.codes,
+                                             static_cast<cudaStream_t>(stream_));
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    return aq_gemm_w4(h, w.codes, M, K, w_packed, w_scales, N, group_size, scale_exp, y_fp16, acc_dump, workspace,
+                      workspace_bytes_, stream_);
+}
+
 int aq_token_select(aq_handle_t h, const float* scores, int M, int n_keep, int32_t* idx, void* workspace,
                     size_t workspace_bytes_, void* stream) {
     if (!h || !scores || (!idx && n_keep > 0)) return AQ_ERR_INVALID_ARG;

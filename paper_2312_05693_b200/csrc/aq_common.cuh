@@ -82,6 +82,10 @@ struct DeviceInfo {
 cudaError_t launch_pack_w4(const __half* w, int N, int K, int group, uint8_t* packed, __half* scales,
                            cudaStream_t stream);
 cudaError_t launch_unpack_w4(const uint8_t* packed, int N, int K, int8_t* codes, cudaStream_t stream);
+// 4-bit activation codes, two per byte (code 2j in the low nibble of byte j); count = number of codes, a
+// multiple of 16, both buffers 16-byte (codes) / 8-byte (packed) aligned.
+cudaError_t launch_act4_pack(const int8_t* q, size_t count, uint8_t* out, cudaStream_t stream);
+cudaError_t launch_act4_unpack(const uint8_t* packed, size_t count, int8_t* q, cudaStream_t stream);
 
 cudaError_t launch_quantize(const __half* x, int M, int K, const int32_t* row_idx, int bits,
                             int scale_mode, int clip_shift_or_exp, Control* ctl, int8_t* q,

@@ -120,7 +120,59 @@ __global__ void weight_offsets_kernel(const uint8_t* __restrict__ packed, const 
     r_out[n] = (float)total;
 }
 
+// Packed storage of 4-bit activation codes: byte j of a row holds code 2j in bits 0-3 and code 2j+1 in
+// bits 4-7 (two's-complement nibbles). One thread turns 16 codes into 8 bytes or back.
+__global__ void __launch_bounds__(256)
+act4_pack_kernel(const uint4* __restrict__ q, size_t n16, uint2* __restrict__ out) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n16) return;
+    const uint4 c = q[i];
+    const uint32_t w[4] = {c.x, c.y, c.z, c.w};
+    uint32_t r[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const uint32_t t = w[k] & 0x0F0F0F0Fu;       // low nibble of every code
+        r[k] = t | (t >> 4);                         // bytes 0 and 2 now hold the two pairs of this word
+    }
+    out[i] = make_uint2(__byte_perm(r[0], r[1], 0x6420), __byte_perm(r[2], r[3], 0x6420));
+}
+
+__global__ void __launch_bounds__(256)
+act4_unpack_kernel(const uint2* __restrict__ p, size_t n16, uint4* __restrict__ q) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n16) return;
+    const uint2 b = p[i];
+    const uint32_t w[2] = {b.x, b.y};
+    uint32_t o[4];
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        uint32_t lo = w[k] & 0x0F0F0F0Fu, hi = (w[k] >> 4) & 0x0F0F0F0Fu;
+        // sign extension inside each byte: bit 3 set -> bits 4-7 set (8 * 30 = 0xF0, no carry between bytes)
+        lo |= (lo & 0x08080808u) * 0x1Eu;
+        hi |= (hi & 0x08080808u) * 0x1Eu;
+        o[2 * k] = __byte_perm(lo, hi, 0x5140);      // codes 0..3 of this word's 8: lo0 hi0 lo1 hi1
+        o[2 * k + 1] = __byte_perm(lo, hi, 0x7362);  // codes 4..7: lo2 hi2 lo3 hi3
+    }
+    q[i] = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
 }  // namespace
+
+cudaError_t launch_act4_pack(const int8_t* q, size_t count, uint8_t* out, cudaStream_t stream) {
+    const size_t n16 = count / 16;
+    if (n16 == 0) return cudaSuccess;
+    act4_pack_kernel<<<(unsigned int)((n16 + 255) / 256), 256, 0, stream>>>(reinterpret_cast<const uint4*>(q), n16,
+                                                                          reinterpret_cast<uint2*>(out));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_act4_unpack(const uint8_t* packed, size_t count, int8_t* q, cudaStream_t stream) {
+    const size_t n16 = count / 16;
+    if (n16 == 0) return cudaSuccess;
+    act4_unpack_kernel<<<(unsigned int)((n16 + 255) / 256), 256, 0, stream>>>(reinterpret_cast<const uint2*>(packed), n16,
+                                                                            reinterpret_cast<uint4*>(q));
+    return cudaGetLastError();
+}
 
 cudaError_t launch_weight_offsets(const uint8_t* packed, const __half* scales, int N, int K, int group, float* r,
                                   cudaStream_t stream) {

@@ -28,6 +28,7 @@ def test_size_functions_and_status_strings():
     ws = binding.aq_workspace_bytes(16, 768, 768, 0)
     assert ws % 256 == 0 and ws >= 256 + 16 * 768
     assert binding.aq_workspace_bytes(0, 768, 768, 0) == 0
+    assert L.aq_act4_bytes(16, 768) == 16 * 768 // 2 and L.aq_act4_bytes(16, 48) == 0   # K % 32 == 0
     assert binding.aq_workspace_bytes(16, 768 + 64, 768, 0) == 0
     assert binding.aq_linear_host_scratch_bytes(16, 768, 768, 0) >= ws + 16 * 768 * 2 * 2
     seen = {binding.status_string(s) for s in range(0, -8, -1)}

@@ -195,6 +195,22 @@ def test_pack_unpack_identity_and_nibble_order():
     assert np.array_equal(oracle.unpack_w4(oracle.pack_w4(c)), c)
 
 
+def test_packed_activation_codes_by_hand_and_by_arithmetic():
+    # Two 4-bit codes per byte (Sec. 4.4), even k in the low nibble: [-8, 7, -1, 0] -> 0x78, 0x0F.
+    assert oracle.pack_act4(np.array([[-8, 7, -1, 0]], np.int8))[0].tolist() == [0x78, 0x0F]
+    assert oracle.unpack_act4(np.array([[0x78, 0x0F]], np.uint8))[0].tolist() == [-8, 7, -1, 0]
+    # against the arithmetic definition byte = (even mod 16) + 16 * (odd mod 16), written with numpy
+    rng = np.random.default_rng(11)
+    q = rng.integers(-8, 8, size=(7, 96)).astype(np.int8)
+    ref = (q[:, 0::2].astype(np.int32) % 16 + 16 * (q[:, 1::2].astype(np.int32) % 16)).astype(np.uint8)
+    assert np.array_equal(oracle.pack_act4(q), ref)
+    assert np.array_equal(oracle.unpack_act4(ref), q)
+    # the product does not care how the codes were stored
+    c = rng.integers(-8, 8, size=(5, 128)).astype(np.int8)
+    q2 = rng.integers(-8, 8, size=(3, 128)).astype(np.int8)
+    assert np.array_equal(oracle.int_gemm(oracle.unpack_act4(oracle.pack_act4(q2)), c, 0), oracle.int_gemm(q2, c, 0))
+
+
 # --------------------------------------------------------------------- integer product
 def _brute(q, c, group):
     M, K = q.shape
