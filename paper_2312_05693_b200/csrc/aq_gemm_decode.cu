@@ -251,7 +251,6 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) p.ctl->status = 0;   // nothing has given up yet
-    for (int i = threadIdx.x; i < kRows * kTileN; i += kStrThreads) (&sm.sum[0][0])[i] = 0;
     __syncthreads();
     volatile uint32_t* abort_flag = &sm.abort_flag;
     const uint8_t* wsrc = p.w_packed + (size_t)tile * KB * kBlockBytes;
@@ -266,16 +265,9 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
             "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
             ::"r"(s_u32(sm.x[s])), "l"(&x_map), "r"(kb * kTileK), "r"(0), "r"(s_u32(&sm.full[s])) : "memory");
     };
-    // the first ring-full of loads goes out before the cluster handshake below, so data is
-    // already streaming while the CTAs of the cluster meet
-    int issued = 0;
-    if (warp == 0 && lane == 0)
-        for (; issued < kStrStages && kb0 + issued < kb1; ++issued) issue(kb0 + issued, issued);
-    cluster.sync();                                   // every CTA's `sum` is zeroed before anyone adds to it
-
     if (warp == 0) {
         if (lane == 0) {
-            for (int kb = kb0 + issued; kb < kb1; ++kb) {
+            for (int kb = kb0; kb < kb1; ++kb) {
                 const uint32_t i = (uint32_t)(kb - kb0);
                 const int s = (int)(i % kStrStages);
                 if (!str_wait(&sm.empty[s], ((i / kStrStages) & 1u) ^ 1u, abort_flag)) break;
@@ -285,7 +277,6 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     } else {
         const int cw = warp - 1;
         const int quarter = cw & 3, half = cw >> 2;
-        int* leader_sum = split > 1 ? cluster.map_shared_rank(&sm.sum[0][0], 0) : &sm.sum[0][0];
         if constexpr (!kUseMma) {
             const int r = quarter * 32 + lane;                       // channel inside the tile
             int acc[MB];
@@ -324,8 +315,7 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
                 __syncwarp();
                 if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s_u32(&sm.empty[s])) : "memory");
             }
-            // the two k-halves of a channel meet in shared memory, then one integer add per
-            // (row, channel) into the leader CTA's sums (exact in any order)
+            // the two k-halves of a channel meet in shared memory: this CTA's sums over its k range
             if (half == 1) {
 #pragma unroll
                 for (int m = 0; m < MB; ++m) sm.part[quarter][m][lane] = acc[m];
@@ -333,8 +323,7 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
             asm volatile("bar.sync 1, %0;" ::"n"(kStrConsumerWarps * 32) : "memory");
             if (half == 0) {
 #pragma unroll
-                for (int m = 0; m < MB; ++m)
-                    if (m < p.M) atomicAdd(&leader_sum[m * kTileN + r], acc[m] + sm.part[quarter][m][lane]);
+                for (int m = 0; m < MB; ++m) sm.sum[m][r] = acc[m] + sm.part[quarter][m][lane];
             }
         } else {
             // Warp-level int8 MMA, D[16 rows x 8 channels] += A[16 x 32 k] * B[32 k x 8 channels].
@@ -352,23 +341,23 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
                 if (!__all_sync(0xFFFFFFFFu, str_wait(&sm.full[s], (it / kStrStages) & 1u, abort_flag) ? 1 : 0)) break;
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    // activation fragment: row-major 128-byte rows, 16-byte chunks XOR-swizzled by row % 8
-                    const int8_t* xr0 = sm.x[s] + g * kTileK;
-                    const int8_t* xr1 = sm.x[s] + (g + 8) * kTileK;
-                    const int c_lo = ((2 * j) ^ g) * 16 + 4 * t, c_hi = ((2 * j + 1) ^ g) * 16 + 4 * t;
-                    const uint32_t a0 = *reinterpret_cast<const uint32_t*>(xr0 + c_lo);
-                    const uint32_t a1 = *reinterpret_cast<const uint32_t*>(xr1 + c_lo);
-                    const uint32_t a2 = *reinterpret_cast<const uint32_t*>(xr0 + c_hi);
-                    const uint32_t a3 = *reinterpret_cast<const uint32_t*>(xr1 + c_hi);
+                    // The sum over k does not depend on which k sits in which slot of the instruction, as long
+                    // as both operands agree: lane t feeds its slots "k 4t.." and "k 16+4t.." with the k range
+                    // 8t..8t+3 and 8t+4..8t+7 of this 32-k chunk, i.e. with the two nibble planes of ONE packed
+                    // word and eight consecutive activation bytes (one 8-byte load per row).
+                    // activation rows: 128 bytes, 16-byte chunks XOR-swizzled by row % 8
+                    const int x_off = (((2 * j + (t >> 1)) ^ g) << 4) + 8 * (t & 1);
+                    const uint2 xa = *reinterpret_cast<const uint2*>(sm.x[s] + g * kTileK + x_off);
+                    const uint2 xb = *reinterpret_cast<const uint2*>(sm.x[s] + (g + 8) * kTileK + x_off);
+                    const uint32_t a0 = xa.x, a1 = xb.x, a2 = xa.y, a3 = xb.y;
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
-                        // weight fragment of channel 32*quarter + 8i + g: packed word t/2 holds k 4t..4t+3 in
-                        // its low (t even) or high (t odd) nibbles; word t/2 + 2 holds k 16+4t..
-                        const uint32_t* wp = reinterpret_cast<const uint32_t*>(
-                            sm.w[s] + (size_t)(j * kTileN + quarter * 32 + 8 * i + g) * 16) + (t >> 1);
-                        const uint32_t p0 = wp[0], p1 = wp[2];
-                        const uint32_t b0 = (t & 1) ? (p0 & 0xF0F0F0F0u) : ((p0 << 4) & 0xF0F0F0F0u);
-                        const uint32_t b1 = (t & 1) ? (p1 & 0xF0F0F0F0u) : ((p1 << 4) & 0xF0F0F0F0u);
+                        // weight fragment of channel 32*quarter + 8i + g: packed word t holds k 8t..8t+3 in its
+                        // low nibbles and k 8t+4..8t+7 in its high nibbles
+                        const uint32_t pw = reinterpret_cast<const uint32_t*>(
+                            sm.w[s] + (size_t)(j * kTileN + quarter * 32 + 8 * i + g) * 16)[t];
+                        const uint32_t b0 = (pw << 4) & 0xF0F0F0F0u;
+                        const uint32_t b1 = pw & 0xF0F0F0F0u;
                         asm volatile(
                             "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, "
                             "{%8, %9}, {%0, %1, %2, %3};"
@@ -393,34 +382,43 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         const int m = g + 8 * (c >> 1), ch = 8 * i + 2 * t + (c & 1);
-                        if (m < p.M)
-                            atomicAdd(&leader_sum[m * kTileN + quarter * 32 + ch], acc[i][c] + sm.part[quarter][m][ch]);
+                        sm.sum[m][quarter * 32 + ch] = acc[i][c] + sm.part[quarter][m][ch];
                     }
             }
         }
     }
-    // the output scale is fetched before the cluster meets so that its latency overlaps the wait
-    float sc = 0.0f, off = 0.0f;
-    const int out_r = (warp - 1) * 32 + lane;
+    // Every CTA of the cluster now holds the tile's sums over its own k range. After the cluster meets,
+    // CTA `rank` finishes a slice of 128 / split channels: it reads that slice of every CTA's sums over
+    // distributed shared memory (integer addition is exact in any order), scales and writes the outputs.
+    // The scale is fetched before the cluster meets so that its latency overlaps the wait.
+    const int cw = kTileN / split;                            // split is 1, 2 or 4
+    const int ft = (int)threadIdx.x - 32;                     // the 256 consumer threads finish; cw divides 256
+    const int out_r = rank * cw + (ft >= 0 ? ft % cw : 0);
     const int out_n = tile * kTileN + out_r;
-    if (rank == 0 && warp >= 1 && warp <= 4 && out_n < p.N) {
+    float sc = 0.0f, off = 0.0f;
+    if (ft >= 0 && out_n < p.N) {
         const float pe = __int_as_float((127 + *p.scale_exp) << 23);
         sc = __half2float(p.w_scales[out_n]) * pe;
         if (p.chan_offset) off = p.chan_offset[out_n] * pe;
     }
-    cluster.sync();
-    if (rank == 0 && warp >= 1 && warp <= 4 && out_n < p.N) {
+    if (split > 1) cluster.sync(); else __syncthreads();
+    if (ft >= 0 && out_n < p.N) {
+        const int* src[4];
 #pragma unroll
-        for (int m = 0; m < MB; ++m) {
-            if (m < p.M) {
-                const int a = sm.sum[m][out_r] >> 4;                  // sums carry a factor 16
-                if (p.acc_dump) p.acc_dump[(size_t)m * p.N + out_n] = a;
-                const __half hv = __float2half_rn(fmaf((float)a, sc, off));
-                if (p.q_next) p.q_next[(size_t)m * p.N + out_n] = (int8_t)next_code(hv, p.next_inv, p.next_lo, p.next_hi);
-                else p.y[(size_t)m * p.N + out_n] = hv;
-            }
+        for (int c = 0; c < 4; ++c)
+            src[c] = (split > 1 && c < split) ? cluster.map_shared_rank(&sm.sum[0][0], c) : &sm.sum[0][0];
+        for (int m = ft / cw; m < p.M && m < kRows; m += (kStrConsumerWarps * 32) / cw) {
+            int a = src[0][m * kTileN + out_r];
+            if (split > 1) a += src[1][m * kTileN + out_r];
+            if (split > 2) a += src[2][m * kTileN + out_r] + src[3][m * kTileN + out_r];
+            a >>= 4;                                              // sums carry a factor 16
+            if (p.acc_dump) p.acc_dump[(size_t)m * p.N + out_n] = a;
+            const __half hv = __float2half_rn(fmaf((float)a, sc, off));
+            if (p.q_next) p.q_next[(size_t)m * p.N + out_n] = (int8_t)next_code(hv, p.next_inv, p.next_lo, p.next_hi);
+            else p.y[(size_t)m * p.N + out_n] = hv;
         }
     }
+    if (split > 1) cluster.sync();                            // nobody leaves while its sums may still be read
     if (sm.abort_flag) {
         for (int i = 0; i < 64; ++i) __nanosleep(1000);          // let copies in flight land
         if (threadIdx.x == 0) atomicOr(&p.ctl->status, 1u);
