@@ -9,10 +9,10 @@
 //  * a streaming one for one scale per channel and M <= 16: a thread-block cluster shares a
 //    128-channel tile and splits K; in each CTA a producer thread streams 8 KB packed blocks
 //    and their activation codes into a shared-memory ring with TMA, eight consumer warps
-//    multiply (dp4a for one row, the warp-level int8 MMA above), and the CTAs' partial sums
-//    are added into the leader CTA's shared memory over distributed shared memory (integer
-//    addition is exact in any order), which then writes the tile's outputs. No workspace, no
-//    global atomics.
+//    multiply (dp4a for one row, the warp-level int8 MMA above). Every CTA keeps the sums over
+//    its k range in its own shared memory; the cluster meets once, and every CTA then finishes a
+//    slice of the tile's channels by reading the other CTAs' sums over distributed shared memory
+//    (integer addition is exact in any order). No workspace, no atomics.
 #include <cooperative_groups.h>
 #include <cuda.h>
 
@@ -205,7 +205,7 @@ struct StreamSmem {
     alignas(1024) int8_t x[kStrStages][kRows * kTileK];    // activation codes of the unit's k block
     alignas(128) uint8_t w[kStrStages][kBlockBytes];       // packed weight block of the unit
     int part[4][kRows][32];                                // the odd-k-block warp's partial sums
-    int sum[kRows][kTileN];                                // leader CTA: the tile's sums over all of K
+    int sum[kRows][kTileN];                                // this CTA's sums over its k range
     alignas(8) uint64_t full[kStrStages];
     uint64_t empty[kStrStages];
     volatile uint32_t abort_flag;
@@ -225,7 +225,7 @@ struct StreamParams {
 };
 
 // grid = (split, channel tiles), cluster = (split, 1, 1): the CTAs of a cluster share a channel
-// tile and take consecutive k ranges; their sums meet in the leader's shared memory.
+// tile and take consecutive k ranges; CTA r adds up and writes channels [r, r+1) * 128 / split.
 template <int MB>
 __global__ void __launch_bounds__(kStrThreads, 2)
 gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const StreamParams p) {
