@@ -143,6 +143,7 @@ int linear_impl(aq_handle_t h, int bits, const void* x, int M, int K, const void
     g.split_scratch = w.split_scratch; g.split_bytes = w.split_bytes;
     g.chan_offset = w_offsets ? w.chan_offset : nullptr;
     g.q_next = q_next; g.next_bits = next_bits; g.next_exp = next_exp;
+    g.after_quantize = true;
     return run_gemm(h, g, stream);
 }
 

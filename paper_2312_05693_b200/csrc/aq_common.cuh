@@ -156,6 +156,12 @@ struct GemmArgs {
     // [M][N] int8: clip(round(y16 / 2^next_exp), -2^(b-1), 2^(b-1)-1), y16 the fp16 value y would have held.
     int8_t* q_next = nullptr;
     int next_bits = 8, next_exp = 0;
+    // The launch directly before this one on the stream is this call's own quantize (or offset) kernel: the
+    // status word is already initialised, and the few-row streaming kernel may be set up and start
+    // streaming weights while that kernel still runs (programmatic dependent launch; it waits for
+    // that grid before it touches the codes). Weights cannot be in flight then: the preceding kernel
+    // was launched normally, after everything before it had completed.
+    bool after_quantize = false;
     // fp32 partial outputs of tiles whose k range two CTAs share (tensor kernel, per-group scales)
     float* split_scratch = nullptr;
     size_t split_bytes = 0;

@@ -43,9 +43,10 @@ gemm_decode_kernel(const int8_t* __restrict__ q, int M, int K, int N, int Npad,
                    const uint8_t* __restrict__ w_packed, const __half* __restrict__ w_scales,
                    const int32_t* __restrict__ scale_exp, __half* __restrict__ y,
                    int32_t* __restrict__ acc_dump, Control* __restrict__ ctl, const float* __restrict__ chan_offset,
-                   int8_t* __restrict__ q_next, float next_inv, float next_lo, float next_hi) {
+                   int8_t* __restrict__ q_next, float next_inv, float next_lo, float next_hi, int clear_status) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) ctl->status = 0;   // this kernel has no bounded waits
+    // this kernel has no bounded waits; after a quantize kernel of the same call the word is that kernel's
+    if (clear_status && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) ctl->status = 0;
     const int KB = K / kTileK;
     const int n0 = blockIdx.x * 32;
     const int nt = n0 / kTileN, r = (n0 % kTileN) + lane;
@@ -213,6 +214,7 @@ struct StreamSmem {
 
 struct StreamParams {
     int M, K, N, Npad;
+    const int8_t* q;
     const uint8_t* w_packed;
     const __half* w_scales;
     const int32_t* scale_exp;
@@ -222,6 +224,7 @@ struct StreamParams {
     const float* chan_offset;
     int8_t* q_next;
     float next_inv, next_lo, next_hi;
+    int clear_status;
 };
 
 // grid = (split, channel tiles), cluster = (split, 1, 1): the CTAs of a cluster share a channel
@@ -243,6 +246,8 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     constexpr uint32_t kUnitBytes = kBlockBytes + kRows * kTileK;
 
     if (threadIdx.x == 0) {
+        if constexpr (kRows > 1)     // start the descriptor's fetch now; the first tile load would wait for it
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&x_map) : "memory");
         for (int s = 0; s < kStrStages; ++s) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(s_u32(&sm.full[s])) : "memory");
             asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s_u32(&sm.empty[s])), "r"(kStrConsumerWarps / 2) : "memory");
@@ -250,28 +255,49 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) p.ctl->status = 0;   // nothing has given up yet
     __syncthreads();
     volatile uint32_t* abort_flag = &sm.abort_flag;
     const uint8_t* wsrc = p.w_packed + (size_t)tile * KB * kBlockBytes;
 
-    auto issue = [&](int kb, int s) {
+    // a stage's barrier expects the weight block and the activation codes; the two copies may be issued apart
+    auto issue_w = [&](int kb, int s) {
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
                      ::"r"(s_u32(&sm.full[s])), "r"(kUnitBytes) : "memory");
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                      ::"r"(s_u32(sm.w[s])), "l"(wsrc + (size_t)kb * kBlockBytes), "r"((uint32_t)kBlockBytes),
                        "r"(s_u32(&sm.full[s])) : "memory");
-        asm volatile(
-            "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-            ::"r"(s_u32(sm.x[s])), "l"(&x_map), "r"(kb * kTileK), "r"(0), "r"(s_u32(&sm.full[s])) : "memory");
     };
+    auto issue_x = [&](int kb, int s) {
+        if constexpr (kRows == 1) {
+            // one row: its 128 codes are contiguous, a plain bulk copy needs no tensor-map fetch
+            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                         ::"r"(s_u32(sm.x[s])), "l"(p.q + (size_t)kb * kTileK), "r"((uint32_t)kTileK),
+                           "r"(s_u32(&sm.full[s])) : "memory");
+        } else {
+            asm volatile(
+                "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                ::"r"(s_u32(sm.x[s])), "l"(&x_map), "r"(kb * kTileK), "r"(0), "r"(s_u32(&sm.full[s])) : "memory");
+        }
+    };
+    // The weights do not depend on the kernel before this one: the first ring of weight blocks is on its
+    // way before this grid waits for that kernel (a no-op unless the launch allowed the overlap), and only
+    // then are the status word, the codes, the exponent and the offsets touched.
+    int issued = 0;
+    if (!p.clear_status) {                            // launched behind this call's own quantize kernel
+        if (warp == 0 && lane == 0)
+            for (; issued < kStrStages && kb0 + issued < kb1; ++issued) issue_w(kb0 + issued, issued);
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+    }
+    if (p.clear_status && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) p.ctl->status = 0;   // nothing has given up yet
     if (warp == 0) {
         if (lane == 0) {
-            for (int kb = kb0; kb < kb1; ++kb) {
+            for (int i = 0; i < issued; ++i) issue_x(kb0 + i, i);
+            for (int kb = kb0 + issued; kb < kb1; ++kb) {
                 const uint32_t i = (uint32_t)(kb - kb0);
                 const int s = (int)(i % kStrStages);
                 if (!str_wait(&sm.empty[s], ((i / kStrStages) & 1u) ^ 1u, abort_flag)) break;
-                issue(kb, s);
+                issue_w(kb, s);
+                issue_x(kb, s);
             }
         }
     } else {
@@ -453,6 +479,8 @@ cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t
     if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
     StreamParams p;
     p.M = a.M; p.K = a.K; p.N = a.N; p.Npad = round_up(a.N, kTileN);
+    p.q = a.q;
+    p.clear_status = a.after_quantize ? 0 : 1;
     p.w_packed = a.w_packed; p.w_scales = a.w_scales; p.scale_exp = a.scale_exp;
     p.y = a.y; p.acc_dump = a.acc_dump; p.ctl = a.ctl; p.chan_offset = a.chan_offset;
     p.q_next = a.q_next;
@@ -469,13 +497,15 @@ cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t
     cfg.blockDim = dim3(kStrThreads);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = split;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = a.after_quantize ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, gemm_decode_stream_kernel<MB>, map, p);
 }
 
@@ -486,11 +516,13 @@ cudaError_t launch_mb(const GemmArgs& a, cudaStream_t stream) {
     if (a.group)
         gemm_decode_kernel<MB, true><<<grid, kDecThreads, 0, stream>>>(
             a.q, a.M, a.K, a.N, Npad, a.w_packed, a.w_scales, a.scale_exp, a.y, a.acc_dump, a.ctl, a.chan_offset,
-            a.q_next, ldexpf(1.0f, -a.next_exp), -(float)(1 << (a.next_bits - 1)), (float)((1 << (a.next_bits - 1)) - 1));
+            a.q_next, ldexpf(1.0f, -a.next_exp), -(float)(1 << (a.next_bits - 1)), (float)((1 << (a.next_bits - 1)) - 1),
+            a.after_quantize ? 0 : 1);
     else
         gemm_decode_kernel<MB, false><<<grid, kDecThreads, 0, stream>>>(
             a.q, a.M, a.K, a.N, Npad, a.w_packed, a.w_scales, a.scale_exp, a.y, a.acc_dump, a.ctl, a.chan_offset,
-            a.q_next, ldexpf(1.0f, -a.next_exp), -(float)(1 << (a.next_bits - 1)), (float)((1 << (a.next_bits - 1)) - 1));
+            a.q_next, ldexpf(1.0f, -a.next_exp), -(float)(1 << (a.next_bits - 1)), (float)((1 << (a.next_bits - 1)) - 1),
+            a.after_quantize ? 0 : 1);
     return cudaGetLastError();
 }
 

@@ -143,6 +143,9 @@ quantize_small_kernel(const uint4* __restrict__ x, int M, int vec_per_row, const
     cg::cluster_group cluster = cg::this_cluster();
     __shared__ unsigned int warp_max[kSmallThreads / 32];
     __shared__ unsigned int slots[kSmallCtas];
+    // A product kernel launched with programmatic stream serialization may be set up on the idle SMs
+    // while this one runs (it waits for this grid before it reads the codes); no effect otherwise.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int rank = (int)cluster.block_rank();
     const int total = M * vec_per_row;
     uint4 buf[kSmallVecs];
