@@ -157,9 +157,9 @@ struct GemmArgs {
     int8_t* q_next = nullptr;
     int next_bits = 8, next_exp = 0;
     // The launch directly before this one on the stream is this call's own quantize (or offset) kernel: the
-    // status word is already initialised, and the few-row streaming kernel may be set up and start
-    // streaming weights while that kernel still runs (programmatic dependent launch; it waits for
-    // that grid before it touches the codes). Weights cannot be in flight then: the preceding kernel
+    // status word is already initialised, and the product kernels may be set up (the few-row streaming
+    // kernel also starts streaming weights) while that kernel still runs (programmatic dependent launch;
+    // they wait for that grid before they touch the codes). Weights cannot be in flight then: the preceding kernel
     // was launched normally, after everything before it had completed.
     bool after_quantize = false;
     // fp32 partial outputs of tiles whose k range two CTAs share (tensor kernel, per-group scales)

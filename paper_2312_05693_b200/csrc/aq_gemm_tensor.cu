@@ -307,6 +307,11 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
       if (warp == 0 || warp == 2) {
         // ------------- TMA producers: warp 0 streams activation tiles, warp 2 weight blocks (+ scales)
         if (lane == 0) {
+            // Launched behind the call's own quantize kernel with programmatic stream serialization, this
+            // grid is set up while that one drains: the codes (and, in the epilogue, the exponent and the
+            // offsets) are touched only after it has completed; the weight producer does not wait. A no-op
+            // for a normal launch.
+            if (warp == 0) asm volatile("griddepcontrol.wait;" ::: "memory");
             uint32_t it = 0;
             for (int tl = 0; tl < my_tiles; ++tl) {
                 const int tile = SPLIT ? p.split_base + ((int)blockIdx.x >> 1) : (int)(blockIdx.x + tl * gridDim.x);
@@ -436,6 +441,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
         const int r = quarter * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         const int col0 = half * kColsPerEpiWarp;
+        asm volatile("griddepcontrol.wait;" ::: "memory");               // see the activation producer
         const float pe = __int_as_float((127 + *p.scale_exp) << 23);     // 2^e
         [[maybe_unused]] const int G = GROUPED ? KB : 1;
         uint32_t unit = 0;
@@ -714,8 +720,19 @@ cudaError_t launch_off(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t st
         cfg.numAttrs = 1;
         return cudaLaunchKernelEx(&cfg, gemm_tensor_kernel<BM, GROUPED, OFFSET, CHAIN, SPLIT>, map, ymap, p);
     } else {
-        gemm_tensor_kernel<BM, GROUPED, OFFSET, CHAIN, SPLIT><<<grid, kThreads, smem_bytes, stream>>>(map, ymap, p);
-        return cudaGetLastError();
+        // Behind the call's own quantize kernel the launch may overlap that kernel's drain (the kernel
+        // waits for it before it reads what it wrote).
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = smem_bytes;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = a.after_quantize ? 1 : 0;
+        return cudaLaunchKernelEx(&cfg, gemm_tensor_kernel<BM, GROUPED, OFFSET, CHAIN, SPLIT>, map, ymap, p);
     }
 }
 

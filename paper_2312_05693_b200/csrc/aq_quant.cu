@@ -228,6 +228,9 @@ quantize_fused_kernel(const uint4* __restrict__ x, int M, int units_per_row /* 1
     const size_t total = (size_t)M * units_per_row;
     const size_t u0 = (size_t)blockIdx.x * units_per_cta;
     const size_t u1 = u0 + units_per_cta < total ? u0 + units_per_cta : total;
+    // a product kernel launched with programmatic stream serialization may be scheduled as soon as this
+    // grid's CTAs leave their SMs (it waits for this grid before it reads the codes); no effect otherwise
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     __half2 m2 = __float2half2_rn(0.0f);
 #pragma unroll 2
