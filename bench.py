@@ -374,8 +374,17 @@ def bench_act4(h, reps=30):
     t_pack = graph_replay_ms(lambda: h.aq_act4_pack(q, q4), reps)
     t_plain = _event_ms(lambda: h.aq_gemm_w4(q, p, sc, s.N, wl.group_size, e, y=y, workspace=ws), reps)
     t_packed = _event_ms(lambda: h.aq_gemm_w4_act4(q4, p, sc, s.N, wl.group_size, e, y=y, workspace=ws), reps)
+    # the chained layer call whose epilogue writes the next layer's 4-bit codes: one byte each / packed
+    e_next = -2
+    qn = torch.empty((M, s.N), dtype=torch.int8, device="cuda")
+    qn4 = torch.empty((M, s.N // 2), dtype=torch.uint8, device="cuda")
+    t_chain = _event_ms(lambda: h.aq_linear_chain(4, x, p, sc, s.N, wl.group_size, 4, e_next,
+                                                  clip_shift_or_exp=wl.clip_shift, q_next=qn, workspace=ws), reps)
+    t_chain4 = _event_ms(lambda: h.aq_linear_chain_act4(4, x, p, sc, s.N, wl.group_size, e_next,
+                                                        clip_shift_or_exp=wl.clip_shift, q4_next=qn4, workspace=ws), reps)
     return {"M": M, "K": s.K, "N": s.N, "code_bytes": {"int8_containers": M * s.K, "packed": M * s.K // 2},
             "pack_us": t_pack * 1e3, "product_us": t_plain * 1e3, "product_on_packed_us": t_packed * 1e3,
+            "chained_layer_us": {"codes_one_byte_each": t_chain * 1e3, "codes_packed_by_the_epilogue": t_chain4 * 1e3},
             "note": "the product widens packed codes with one extra pass; the tensor cores take 8-bit integers"}
 
 

@@ -218,6 +218,9 @@ int aq_linear_w4a4_chain(aq_handle_t h, const void* x_fp16, int M, int K, const 
  *   codes are widened into the workspace's code area by one extra pass (M*K/2 bytes read, M*K written)
  *   before the product; what the packed form halves is the storage and traffic between layers.
  * Errors as for aq_quantize_act / aq_gemm_w4. */
+/* aq_linear_w4a8_chain_act4 / aq_linear_w4a4_chain_act4: the chained calls above with next_bits = 4 whose
+ *   codes leave the product kernels' epilogue already packed, q4_next [M, N/2] (N % 32 == 0, 16-byte
+ *   aligned): no one-byte containers are written between the two layers. */
 size_t aq_act4_bytes(int M, int K);
 int aq_act4_pack(aq_handle_t h, const int8_t* q, int M, int K, void* q4, void* stream);
 int aq_act4_unpack(aq_handle_t h, const void* q4, int M, int K, int8_t* q, void* stream);
@@ -227,6 +230,14 @@ int aq_quantize_act4(aq_handle_t h, const void* x_fp16, int M, int K, int scale_
 int aq_gemm_w4_act4(aq_handle_t h, const void* q4, int M, int K, const void* w_packed, const void* w_scales,
                     int N, int group_size, const int32_t* scale_exp, void* y_fp16, int32_t* acc_dump,
                     void* workspace, size_t workspace_bytes, void* stream);
+int aq_linear_w4a8_chain_act4(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed,
+                              const void* w_scales, int N, int group_size, int scale_mode, int clip_shift_or_exp,
+                              const int32_t* row_idx, void* q4_next, int next_exp, int32_t* acc_dump, void* workspace,
+                              size_t workspace_bytes, void* stream);
+int aq_linear_w4a4_chain_act4(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed,
+                              const void* w_scales, int N, int group_size, int scale_mode, int clip_shift_or_exp,
+                              const int32_t* row_idx, void* q4_next, int next_exp, int32_t* acc_dump, void* workspace,
+                              size_t workspace_bytes, void* stream);
 
 /* ---- log2 quantization of the softmax output and attention x value (paper Eq. 3, Sec. 5.1)
  * aq_log2_quantize: x_fp16 holds `count` values (any shape); max|x| is taken over all of them.

@@ -80,6 +80,8 @@ def load():
     L.aq_act4_unpack.argtypes = [vp, vp, i32, i32, vp, vp]
     L.aq_quantize_act4.argtypes = [vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, sz, vp]
     L.aq_gemm_w4_act4.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, vp, vp, vp, vp, sz, vp]
+    for f in ("aq_linear_w4a8_chain_act4", "aq_linear_w4a4_chain_act4"):
+        getattr(L, f).argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, vp, i32, vp, vp, sz, vp]
     L.aq_weight_offsets.argtypes = [vp, vp, vp, i32, i32, i32, vp, vp]
     L.aq_quantize_act_asym.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, sz, vp]
     lin_asym = [vp, vp, i32, i32, vp, vp, vp, i32, i32, vp, vp, vp, vp, sz, vp]
@@ -379,6 +381,20 @@ class Handle:
                                  _ptr(scale_exp), _ptr(y), _ptr(acc_dump), _ptr(workspace),
                                  workspace.numel(), _stream()), "aq_gemm_w4")
         return y
+
+    def aq_linear_chain_act4(self, bits, x, packed, scales, N, group_size, next_exp, scale_mode=AQ_SCALE_DYNAMIC,
+                             clip_shift_or_exp=0, row_idx=None, q4_next=None, acc_dump=None, workspace=None):
+        M_in, K = x.shape
+        M = M_in if row_idx is None else row_idx.shape[0]
+        if q4_next is None:
+            q4_next = torch.empty((M, N // 2), dtype=torch.uint8, device=x.device)
+        if workspace is None:
+            workspace = self.alloc_workspace(M, K, N, group_size)
+        fn = load().aq_linear_w4a8_chain_act4 if bits == 8 else load().aq_linear_w4a4_chain_act4
+        _check(fn(self._h, _ptr(x), M, K, _ptr(packed), _ptr(scales), N, group_size, scale_mode, clip_shift_or_exp,
+                  _ptr(row_idx), _ptr(q4_next), next_exp, _ptr(acc_dump), _ptr(workspace), workspace.numel(),
+                  _stream()), "aq_linear_chain_act4")
+        return q4_next
 
     def aq_act4_pack(self, q: torch.Tensor, q4: Optional[torch.Tensor] = None) -> torch.Tensor:
         M, K = q.shape

@@ -102,8 +102,11 @@ int linear_impl(aq_handle_t h, int bits, const void* x, int M, int K, const void
                 const void* w_scales, int N, int group, int scale_mode, int clip_shift_or_exp,
                 const int32_t* row_idx, void* y, int32_t* acc_dump, void* workspace, size_t workspace_bytes_,
                 void* stream_, const uint8_t* alpha = nullptr, int k_max = 0, const float* w_offsets = nullptr,
-                int8_t* q_next = nullptr, int next_bits = 8, int next_exp = 0) {
+                int8_t* q_next = nullptr, int next_bits = 8, int next_exp = 0, bool next_packed = false) {
     if (!h || !x || !w_packed || !w_scales || (!y && !q_next)) return AQ_ERR_INVALID_ARG;
+    if (next_packed && (!q_next || next_bits != 4)) return AQ_ERR_INVALID_ARG;
+    if (next_packed && N % 32 != 0) return AQ_ERR_SHAPE;
+    if (next_packed && !aligned(q_next, 16)) return AQ_ERR_ALIGNMENT;
     if (q_next && ((next_bits != 8 && next_bits != 4) || next_exp < -40 || next_exp > 40 || w_offsets))
         return AQ_ERR_INVALID_ARG;
     if (scale_mode != AQ_SCALE_DYNAMIC && scale_mode != AQ_SCALE_STATIC) return AQ_ERR_INVALID_ARG;
@@ -143,6 +146,7 @@ int linear_impl(aq_handle_t h, int bits, const void* x, int M, int K, const void
     g.split_scratch = w.split_scratch; g.split_bytes = w.split_bytes;
     g.chan_offset = w_offsets ? w.chan_offset : nullptr;
     g.q_next = q_next; g.next_bits = next_bits; g.next_exp = next_exp;
+    g.next_packed = next_packed;
     g.after_quantize = true;
     return run_gemm(h, g, stream);
 }
@@ -504,6 +508,26 @@ int aq_linear_w4a4_chain(aq_handle_t h, const void* x_fp16, int M, int K, const 
     return linear_impl(h, 4, x_fp16, M, K, w_packed, w_scales, N, group_size, scale_mode, clip_shift_or_exp, row_idx,
                        nullptr, acc_dump, workspace, workspace_bytes_, stream, nullptr, 0, nullptr, q_next, next_bits,
                        next_exp);
+}
+
+int aq_linear_w4a8_chain_act4(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed,
+                              const void* w_scales, int N, int group_size, int scale_mode, int clip_shift_or_exp,
+                              const int32_t* row_idx, void* q4_next, int next_exp, int32_t* acc_dump, void* workspace,
+                              size_t workspace_bytes_, void* stream) {
+    if (!q4_next) return AQ_ERR_INVALID_ARG;
+    return linear_impl(h, 8, x_fp16, M, K, w_packed, w_scales, N, group_size, scale_mode, clip_shift_or_exp, row_idx,
+                       nullptr, acc_dump, workspace, workspace_bytes_, stream, nullptr, 0, nullptr,
+                       static_cast<int8_t*>(q4_next), 4, next_exp, true);
+}
+
+int aq_linear_w4a4_chain_act4(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed,
+                              const void* w_scales, int N, int group_size, int scale_mode, int clip_shift_or_exp,
+                              const int32_t* row_idx, void* q4_next, int next_exp, int32_t* acc_dump, void* workspace,
+                              size_t workspace_bytes_, void* stream) {
+    if (!q4_next) return AQ_ERR_INVALID_ARG;
+    return linear_impl(h, 4, x_fp16, M, K, w_packed, w_scales, N, group_size, scale_mode, clip_shift_or_exp, row_idx,
+                       nullptr, acc_dump, workspace, workspace_bytes_, stream, nullptr, 0, nullptr,
+                       static_cast<int8_t*>(q4_next), 4, next_exp, true);
 }
 
 int aq_log2_quantize(aq_handle_t h, const void* x_fp16, long long count, int bits, int8_t* codes,

@@ -156,6 +156,9 @@ struct GemmArgs {
     // [M][N] int8: clip(round(y16 / 2^next_exp), -2^(b-1), 2^(b-1)-1), y16 the fp16 value y would have held.
     int8_t* q_next = nullptr;
     int next_bits = 8, next_exp = 0;
+    // the next layer's 4-bit codes leave packed, two per byte [M][N/2] (code 2j in the low nibble of byte j);
+    // needs next_bits == 4, N % 32 == 0 and a 16-byte aligned q_next
+    bool next_packed = false;
     // The launch directly before this one on the stream is this call's own quantize (or offset) kernel: the
     // status word is already initialised, and the product kernels may be set up (the few-row streaming
     // kernel also starts streaming weights) while that kernel still runs (programmatic dependent launch;

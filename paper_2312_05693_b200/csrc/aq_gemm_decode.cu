@@ -35,6 +35,18 @@ __device__ __forceinline__ int next_code(__half hv, float inv, float lo, float h
     return (int)fminf(fmaxf(rintf(t), lo), hi);
 }
 
+// Chaining: a warp's codes of one token (lane = consecutive channels) are stored one byte each or, packed,
+// the even lane stores its code and its neighbour's in one byte of q4 [M][N/2]. All 32 lanes call this
+// together; `valid` lanes (the same for a lane pair) store.
+__device__ __forceinline__ void store_next_code(int8_t* q_next, size_t index, int code, int packed, bool valid, int lane) {
+    if (packed) {
+        const int hi = __shfl_down_sync(0xFFFFFFFFu, code, 1);
+        if (valid && !(lane & 1)) reinterpret_cast<uint8_t*>(q_next)[index >> 1] = (uint8_t)((code & 0xF) | (hi << 4));
+    } else if (valid) {
+        q_next[index] = (int8_t)code;
+    }
+}
+
 // CTA = 32 output channels (one lane each) x all of K, K split over the 8 warps by 128-k
 // block; grid.y walks the rows in chunks of MB.
 template <int MB, bool GROUPED>
@@ -43,7 +55,8 @@ gemm_decode_kernel(const int8_t* __restrict__ q, int M, int K, int N, int Npad,
                    const uint8_t* __restrict__ w_packed, const __half* __restrict__ w_scales,
                    const int32_t* __restrict__ scale_exp, __half* __restrict__ y,
                    int32_t* __restrict__ acc_dump, Control* __restrict__ ctl, const float* __restrict__ chan_offset,
-                   int8_t* __restrict__ q_next, float next_inv, float next_lo, float next_hi, int clear_status) {
+                   int8_t* __restrict__ q_next, float next_inv, float next_lo, float next_hi, int clear_status,
+                   int next_packed) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // this kernel has no bounded waits; after a quantize kernel of the same call the word is that kernel's
     if (clear_status && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) ctl->status = 0;
@@ -138,8 +151,9 @@ gemm_decode_kernel(const int8_t* __restrict__ q, int M, int K, int N, int Npad,
     __syncthreads();
     const float pe = __int_as_float((127 + *scale_exp) << 23);   // 2^e
     for (int m = warp; m < MB; m += kDecWarps) {
-        if (m0 + m >= M || n >= N) continue;
-        const float off = chan_offset ? chan_offset[n] : 0.0f;
+        if (m0 + m >= M) continue;                               // the same for the whole warp
+        const bool n_ok = n < N;
+        const float off = chan_offset && n_ok ? chan_offset[n] : 0.0f;
         float out;
         if (GROUPED) {
             float s = 0.0f;
@@ -151,12 +165,14 @@ gemm_decode_kernel(const int8_t* __restrict__ q, int M, int K, int N, int Npad,
 #pragma unroll
             for (int w = 0; w < kDecWarps; ++w) s += red[w][m][lane];
             s >>= 4;
-            if (acc_dump) acc_dump[(size_t)(m0 + m) * N + n] = s;
-            out = fmaf((float)s, __half2float(w_scales[n]), off) * pe;
+            if (acc_dump && n_ok) acc_dump[(size_t)(m0 + m) * N + n] = s;
+            out = fmaf((float)s, n_ok ? __half2float(w_scales[n]) : 0.0f, off) * pe;
         }
         const __half hv = __float2half_rn(out);
-        if (q_next) q_next[(size_t)(m0 + m) * N + n] = (int8_t)next_code(hv, next_inv, next_lo, next_hi);
-        else y[(size_t)(m0 + m) * N + n] = hv;
+        if (q_next)
+            store_next_code(q_next, (size_t)(m0 + m) * N + n, next_code(hv, next_inv, next_lo, next_hi), next_packed, n_ok, lane);
+        else if (n_ok)
+            y[(size_t)(m0 + m) * N + n] = hv;
     }
 }
 
@@ -225,6 +241,7 @@ struct StreamParams {
     int8_t* q_next;
     float next_inv, next_lo, next_hi;
     int clear_status;
+    int next_packed;
 };
 
 // grid = (split, channel tiles), cluster = (split, 1, 1): the CTAs of a cluster share a channel
@@ -440,7 +457,10 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
             a >>= 4;                                              // sums carry a factor 16
             if (p.acc_dump) p.acc_dump[(size_t)m * p.N + out_n] = a;
             const __half hv = __float2half_rn(fmaf((float)a, sc, off));
-            if (p.q_next) p.q_next[(size_t)m * p.N + out_n] = (int8_t)next_code(hv, p.next_inv, p.next_lo, p.next_hi);
+            // (a warp's lanes hold consecutive channels and run this loop together: 128 / split >= 32)
+            if (p.q_next)
+                store_next_code(p.q_next, (size_t)m * p.N + out_n, next_code(hv, p.next_inv, p.next_lo, p.next_hi),
+                                p.next_packed, true, lane);
             else p.y[(size_t)m * p.N + out_n] = hv;
         }
     }
@@ -481,6 +501,7 @@ cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t
     p.M = a.M; p.K = a.K; p.N = a.N; p.Npad = round_up(a.N, kTileN);
     p.q = a.q;
     p.clear_status = a.after_quantize ? 0 : 1;
+    p.next_packed = a.next_packed ? 1 : 0;
     p.w_packed = a.w_packed; p.w_scales = a.w_scales; p.scale_exp = a.scale_exp;
     p.y = a.y; p.acc_dump = a.acc_dump; p.ctl = a.ctl; p.chan_offset = a.chan_offset;
     p.q_next = a.q_next;
@@ -517,12 +538,12 @@ cudaError_t launch_mb(const GemmArgs& a, cudaStream_t stream) {
         gemm_decode_kernel<MB, true><<<grid, kDecThreads, 0, stream>>>(
             a.q, a.M, a.K, a.N, Npad, a.w_packed, a.w_scales, a.scale_exp, a.y, a.acc_dump, a.ctl, a.chan_offset,
             a.q_next, ldexpf(1.0f, -a.next_exp), -(float)(1 << (a.next_bits - 1)), (float)((1 << (a.next_bits - 1)) - 1),
-            a.after_quantize ? 0 : 1);
+            a.after_quantize ? 0 : 1, a.next_packed ? 1 : 0);
     else
         gemm_decode_kernel<MB, false><<<grid, kDecThreads, 0, stream>>>(
             a.q, a.M, a.K, a.N, Npad, a.w_packed, a.w_scales, a.scale_exp, a.y, a.acc_dump, a.ctl, a.chan_offset,
             a.q_next, ldexpf(1.0f, -a.next_exp), -(float)(1 << (a.next_bits - 1)), (float)((1 << (a.next_bits - 1)) - 1),
-            a.after_quantize ? 0 : 1);
+            a.after_quantize ? 0 : 1, a.next_packed ? 1 : 0);
     return cudaGetLastError();
 }
 

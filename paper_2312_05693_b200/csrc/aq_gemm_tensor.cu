@@ -222,6 +222,7 @@ struct TensorParams {
     float* split_scratch;          // [shared tile][half][epilogue warp][column][lane] fp32 partial outputs
     int8_t* q_next;                // chaining: the next layer's codes [M][N] are written instead of y
     float next_inv, next_lo, next_hi;   // 2^-next_exp and the code range of the next layer
+    int next_packed;               // chaining: 4-bit codes leave two per byte (even channel in the low nibble)
     int y_tma;                     // outputs leave through y_map (needs N % 8 == 0 and a 16-byte aligned y)
 };
 
@@ -230,6 +231,18 @@ __device__ __forceinline__ int chain_code(__half hv, float inv, float lo, float 
     const float t = __half2float(hv) * inv;                 // exact: inv is a power of two
     if (t != t) return 0;
     return (int)fminf(fmaxf(rintf(t), lo), hi);
+}
+
+// Chaining: a warp's 32 codes of one token (lane = channel) go to the staging row: one byte each, or, for
+// packed 4-bit codes, the even lane stores its code and its neighbour's in one byte (rows of 16 bytes).
+// All 32 lanes call this together.
+__device__ __forceinline__ void stage_code(__half* stage, int c, int lane, int code, int packed) {
+    if (packed) {
+        const int hi = __shfl_down_sync(0xFFFFFFFFu, code, 1);
+        if (!(lane & 1)) reinterpret_cast<uint8_t*>(stage)[c * 16 + (lane >> 1)] = (uint8_t)((code & 0xF) | (hi << 4));
+    } else {
+        reinterpret_cast<int8_t*>(stage)[c * 32 + lane] = (int8_t)code;
+    }
 }
 
 // OFFSET: add the per-channel term of the zero-point variant. CHAIN: write the next layer's codes
@@ -482,14 +495,14 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
                             const __half hv = __float2half_rn(OFFSET ? fmaf((float)(int)v[r0 + c], sc, off_pe)
                                                                      : (float)(int)v[r0 + c] * sc);
                             if constexpr (CHAIN)
-                                reinterpret_cast<int8_t*>(stage)[c * 32 + lane] =
-                                    (int8_t)chain_code(hv, p.next_inv, p.next_lo, p.next_hi);
+                                stage_code(stage, c, lane, chain_code(hv, p.next_inv, p.next_lo, p.next_hi), p.next_packed);
                             else
                                 stage[c * 32 + lane] = hv;
                         }
                         fence_proxy_async();
                         __syncwarp();
-                        if (lane == 0 && n0 < p.N && m_base + r0 < p.M) tma_store_2d(&y_map, stage, n0, m_base + r0);
+                        if (lane == 0 && n0 < p.N && m_base + r0 < p.M)
+                            tma_store_2d(&y_map, stage, (CHAIN && p.next_packed) ? n0 >> 1 : n0, m_base + r0);
                     }
                 } else {
 #pragma unroll
@@ -588,15 +601,15 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
                     for (int c = 0; c < kColsPerEpiWarp; ++c) {
                         const __half hv = __float2half_rn(fsum[c] * pe);
                         if constexpr (CHAIN)
-                            reinterpret_cast<int8_t*>(stage)[c * 32 + lane] =
-                                (int8_t)chain_code(hv, p.next_inv, p.next_lo, p.next_hi);
+                            stage_code(stage, c, lane, chain_code(hv, p.next_inv, p.next_lo, p.next_hi), p.next_packed);
                         else
                             stage[c * 32 + lane] = hv;
                     }
                     fence_proxy_async();
                     __syncwarp();
                     const int n0 = nt * kTileN + quarter * 32;
-                    if (lane == 0 && n0 < p.N && m_base < p.M) tma_store_2d(&y_map, stage, n0, m_base);
+                    if (lane == 0 && n0 < p.N && m_base < p.M)
+                        tma_store_2d(&y_map, stage, (CHAIN && p.next_packed) ? n0 >> 1 : n0, m_base);
                 } else {
 #pragma unroll
                     for (int c = 0; c < kColsPerEpiWarp; ++c) {
@@ -665,11 +678,15 @@ cudaError_t launch_off(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t st
     CUtensorMap ymap = map;   // placeholder when the store path is off
     int y_tma = 0;
     if (CHAIN) {
-        // the staged rows hold one byte per value: a map over the code matrix, 32-byte rows
+        // the staged rows hold one byte per value (or per two values when packed): a map over the code
+        // matrix, 32-byte (16-byte) rows
+        if (a.next_packed && (a.N % 32 != 0 || (reinterpret_cast<uintptr_t>(a.q_next) & 15u) != 0))
+            return cudaErrorInvalidValue;                    // packed codes only leave through the TMA store
         if (a.N % 16 == 0 && (reinterpret_cast<uintptr_t>(a.q_next) & 15u) == 0) {
-            const cuuint64_t ydims[2] = {(cuuint64_t)a.N, (cuuint64_t)a.M};
-            const cuuint64_t ystrides[1] = {(cuuint64_t)a.N};
-            const cuuint32_t ybox[2] = {32u, (cuuint32_t)Smem::kStageRows};
+            const cuuint64_t row_bytes = a.next_packed ? (cuuint64_t)a.N / 2 : (cuuint64_t)a.N;
+            const cuuint64_t ydims[2] = {row_bytes, (cuuint64_t)a.M};
+            const cuuint64_t ystrides[1] = {row_bytes};
+            const cuuint32_t ybox[2] = {a.next_packed ? 16u : 32u, (cuuint32_t)Smem::kStageRows};
             const CUresult ry = reinterpret_cast<EncodeTiledFn>(dev.encode_tiled)(
                 &ymap, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, a.q_next, ydims, ystrides, ybox, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
@@ -700,6 +717,7 @@ cudaError_t launch_off(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t st
     p.next_inv = ldexpf(1.0f, -a.next_exp);
     p.next_lo = -(float)(1 << (a.next_bits - 1));
     p.next_hi = (float)((1 << (a.next_bits - 1)) - 1);
+    p.next_packed = a.next_packed ? 1 : 0;
     if (tile_limit >= 0) p.n_tiles = tile_limit;
     p.split_base = split_base;
     p.split_scratch = a.split_scratch;

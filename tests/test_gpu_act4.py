@@ -79,8 +79,9 @@ def test_chained_layers_with_packed_intermediate_codes():
     y1 = h.aq_linear_w4a4(dev(x), p1, s1, N1, group, clip_shift_or_exp=2).cpu().numpy()
     e_next = oracle.layer_exponent(y1, 4) - 1
     q1 = h.aq_linear_chain(4, dev(x), p1, s1, N1, group, 4, e_next, clip_shift_or_exp=2)   # int8 containers
-    q1_packed = h.aq_act4_pack(q1)                                                         # what is stored
+    q1_packed = h.aq_linear_chain_act4(4, dev(x), p1, s1, N1, group, e_next, clip_shift_or_exp=2)   # what is stored
     assert q1_packed.numel() * 2 == q1.numel()
+    assert torch.equal(q1_packed, h.aq_act4_pack(q1))
     e_dev = torch.tensor([e_next], dtype=torch.int32, device="cuda")
     y2_packed = h.aq_gemm_w4_act4(q1_packed, p2, s2, N2, group, e_dev)
     y2_plain = h.aq_gemm_w4(q1, p2, s2, N2, group, e_dev)
@@ -88,6 +89,38 @@ def test_chained_layers_with_packed_intermediate_codes():
     c2, sc2 = oracle.quantize_weights(inputs.weights(N2, N1, 64), group)
     acc = oracle.int_gemm(oracle.quantize_act(y1, 4, e_next), c2, group)
     assert_y_close(y2_packed.cpu().numpy(), oracle.dequant(acc.reshape(M, N2, N1 // 128), sc2, e_next))
+
+
+@pytest.mark.parametrize("kernel", [binding.AQ_KERNEL_DECODE, binding.AQ_KERNEL_TENSOR])
+@pytest.mark.parametrize("bits", [8, 4])
+@pytest.mark.parametrize("M,K,N,group", [(1, 256, 128, 0), (16, 768, 768, 0), (129, 384, 224, 128), (300, 1024, 384, 0),
+                                         (260, 1152, 544, 128)])
+def test_chained_epilogue_writes_packed_codes(kernel, bits, M, K, N, group):
+    x = inputs.activations(M, K, seed=65, outlier_frac=0.01, outlier_mult=20.0)
+    h = handle()
+    packed, scales = h.aq_pack_w4(dev(inputs.weights(N, K, 65)), group)
+    clip = 0 if bits == 8 else 2
+    lin = h.aq_linear_w4a8 if bits == 8 else h.aq_linear_w4a4
+    h.aq_set_kernel(kernel)
+    try:
+        y = lin(dev(x), packed, scales, N, group, clip_shift_or_exp=clip).cpu().numpy()
+        e_next = oracle.layer_exponent(y, 4) - 1
+        q4 = h.aq_linear_chain_act4(bits, dev(x), packed, scales, N, group, e_next, clip_shift_or_exp=clip)
+        torch.cuda.synchronize()
+    finally:
+        h.aq_set_kernel(binding.AQ_KERNEL_AUTO)
+    ref = oracle.quantize_act(y, 4, e_next)
+    assert q4.shape == (M, N // 2)
+    assert np.array_equal(q4.cpu().numpy(), oracle.pack_act4(ref))
+    assert ref.min() == -8 or ref.max() == 7                                  # it did clip
+
+
+def test_packed_chain_refuses_what_it_cannot_pack():
+    h = handle()
+    x = dev(inputs.activations(8, 128, seed=1))
+    p, s = h.aq_pack_w4(dev(inputs.weights(200, 128, 1)), 0)
+    with pytest.raises(binding.AgileqError):
+        h.aq_linear_chain_act4(8, x, p, s, 200, 0, 0)                          # N % 32 != 0
 
 
 def test_bad_arguments_are_refused():
