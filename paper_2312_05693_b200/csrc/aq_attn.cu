@@ -22,12 +22,23 @@ log2_absmax_kernel(const __half* __restrict__ x, long long count, Control* __res
     const bool vec = (reinterpret_cast<uintptr_t>(x) & 15u) == 0;
     const long long nvec = vec ? count / 8 : 0;
     const uint4* xv = reinterpret_cast<const uint4*>(x);
+    // two values per instruction: the half2 maximum returns the other operand when one is NaN, so NaN
+    // never enters; Inf does and is replaced by the largest finite value below
+    __half2 m2 = __float2half2_rn(0.0f);
 #pragma unroll 4
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
         const uint4 d = __ldg(xv + i);
         const uint32_t w[4] = {d.x, d.y, d.z, d.w};
 #pragma unroll
-        for (int t = 0; t < 4; ++t) { take(w[t] & 0xFFFFu); take(w[t] >> 16); }
+        for (int t = 0; t < 4; ++t) {
+            const uint32_t a = w[t] & 0x7FFF7FFFu;
+            m2 = __hmax2(m2, *reinterpret_cast<const __half2*>(&a));
+        }
+    }
+    {
+        const uint32_t mw = *reinterpret_cast<const uint32_t*>(&m2);
+        take(mw & 0xFFFFu);
+        take(mw >> 16);
     }
     if (blockIdx.x == 0 && threadIdx.x == 0)
         for (long long i = nvec * 8; i < count; ++i) take(__half_as_ushort(x[i]));
@@ -66,14 +77,16 @@ __device__ __forceinline__ void log2_thresholds(int mb, int& t_up, int& t_down) 
 
 __device__ __forceinline__ int log2_code(unsigned int raw, unsigned int mb_bits, int eb, int t_up, int t_down, int kmax) {
     unsigned int hb = raw & 0x7FFFu;
-    if (hb == 0 || hb > 0x7C00u || mb_bits == 0) return 0;
-    if (hb == 0x7C00u) hb = 0x7BFFu;
-    int ma, ea;
-    if (hb >= 0x0400u) { ma = 1024 + (int)(hb & 0x3FFu); ea = (int)(hb >> 10) - 25; }   // normal: the common case
-    else half_parts(hb, ma, ea);
+    const bool none = hb == 0 || hb > 0x7C00u || mb_bits == 0;      // zero, NaN, or an all-zero layer
+    hb = min(hb, 0x7BFFu);                                           // Inf counts as the largest finite value
+    // Without branches (softmax outputs mix normal and subnormal values inside every warp): the exact
+    // conversion to binary32 normalises subnormals, |x| = (1024 + top ten fraction bits) * 2^(E - 10).
+    const unsigned int fb = __float_as_uint(__half2float(__ushort_as_half((unsigned short)hb)));
+    const int ma = 1024 + (int)((fb >> 13) & 0x3FFu);
+    const int ea = (int)(fb >> 23) - 137;
     int k = eb - ea + (ma <= t_up ? 1 : 0) - (ma >= t_down ? 1 : 0);
-    k = min(max(k, 0), kmax);
-    return (raw & 0x8000u) ? -(k + 1) : (k + 1);
+    k = min(max(k, 0), kmax) + 1;
+    return none ? 0 : ((raw & 0x8000u) ? -k : k);
 }
 
 __global__ void __launch_bounds__(256)
