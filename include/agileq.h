@@ -217,10 +217,12 @@ int aq_linear_w4a4_chain(aq_handle_t h, const void* x_fp16, int M, int K, const 
  * aq_gemm_w4_act4: aq_gemm_w4 on packed codes. The tensor cores have no 4-bit integer operand, so the
  *   codes are widened into the workspace's code area by one extra pass (M*K/2 bytes read, M*K written)
  *   before the product; what the packed form halves is the storage and traffic between layers.
- * Errors as for aq_quantize_act / aq_gemm_w4. */
-/* aq_linear_w4a8_chain_act4 / aq_linear_w4a4_chain_act4: the chained calls above with next_bits = 4 whose
- *   codes leave the product kernels' epilogue already packed, q4_next [M, N/2] (N % 32 == 0, 16-byte
- *   aligned): no one-byte containers are written between the two layers. */
+ * aq_linear_w4a8_chain_act4 / aq_linear_w4a4_chain_act4: the chained calls above with next_bits = 4 whose
+ *   codes leave the product kernels' epilogue already packed, q4_next [M, N/2]: no one-byte containers
+ *   are written between the two layers. N % 32 == 0 (else AQ_ERR_SHAPE), q4_next 16-byte aligned (else
+ *   AQ_ERR_ALIGNMENT).
+ * All buffers are device memory owned by the caller; the calls enqueue on `stream` and return at once.
+ * Other errors as for aq_quantize_act / aq_gemm_w4 / the chained calls. */
 size_t aq_act4_bytes(int M, int K);
 int aq_act4_pack(aq_handle_t h, const int8_t* q, int M, int K, void* q4, void* stream);
 int aq_act4_unpack(aq_handle_t h, const void* q4, int M, int K, int8_t* q, void* stream);
