@@ -293,6 +293,15 @@ int aq_linear_host(aq_handle_t h, int bits, const void* x_host, int M, int K,
                    const void* w_packed, const void* w_scales, int N, int group_size,
                    int scale_mode, int clip_shift_or_exp, void* y_host, void* device_scratch,
                    size_t scratch_bytes, void* stream);
+/* The same without the final synchronisation: the two copies and the layer are enqueued on `stream`
+ * and the call returns. x_host, y_host (pinned, or the copies are not asynchronous) and device_scratch
+ * belong to the call until the stream has been synchronised; y_host is valid from then on. Calls on
+ * different streams, each with its own scratch, overlap their copies (one direction each) and their
+ * kernels. */
+int aq_linear_host_async(aq_handle_t h, int bits, const void* x_host, int M, int K,
+                         const void* w_packed, const void* w_scales, int N, int group_size,
+                         int scale_mode, int clip_shift_or_exp, void* y_host, void* device_scratch,
+                         size_t scratch_bytes, void* stream);
 
 /* SYNCHRONIZES the stream, then reports whether a kernel of the most recent call that used
  * this workspace gave up on a bounded wait (AQ_ERR_DEVICE_TIMEOUT); AQ_OK otherwise. Every

@@ -103,6 +103,7 @@ def load():
     L.aq_token_select.argtypes = [vp, vp, i32, i32, vp, vp, sz, vp]
     L.aq_token_compact.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp]
     L.aq_linear_host.argtypes = [vp, i32, vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, vp, sz, vp]
+    L.aq_linear_host_async.argtypes = L.aq_linear_host.argtypes
     L.aq_check_workspace.argtypes = [vp, vp, vp]
     L.aq_linear_w4a8_noalloc.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, vp]
     _lib = L
@@ -461,6 +462,18 @@ class Handle:
                                      group_size, scale_mode, clip_shift_or_exp, _ptr(y_host),
                                      _ptr(device_scratch), device_scratch.numel(), _stream()),
                "aq_linear_host")
+        return y_host
+
+    def aq_linear_host_async(self, bits: int, x_host: torch.Tensor, packed, scales, N, group_size,
+                             y_host: torch.Tensor, device_scratch: torch.Tensor,
+                             scale_mode=AQ_SCALE_DYNAMIC, clip_shift_or_exp=0):
+        """As aq_linear_host, but only enqueues on torch's current stream: y_host is valid once that
+        stream has been synchronised; the buffers belong to the call until then."""
+        M, K = x_host.shape
+        _check(load().aq_linear_host_async(self._h, bits, _ptr(x_host), M, K, _ptr(packed), _ptr(scales), N,
+                                           group_size, scale_mode, clip_shift_or_exp, _ptr(y_host),
+                                           _ptr(device_scratch), device_scratch.numel(), _stream()),
+               "aq_linear_host_async")
         return y_host
 
     def aq_linear_w4a8_noalloc(self, x, packed, scales, N, group_size, y, scale_mode=AQ_SCALE_DYNAMIC,

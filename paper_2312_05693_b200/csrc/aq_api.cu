@@ -620,9 +620,9 @@ size_t aq_linear_host_scratch_bytes(int M, int K, int N, int group_size) {
     return up256((size_t)M * K * 2) + up256((size_t)M * N * 2) + workspace_bytes(M, K, N, group_size);
 }
 
-int aq_linear_host(aq_handle_t h, int bits, const void* x_host, int M, int K, const void* w_packed,
-                   const void* w_scales, int N, int group_size, int scale_mode, int clip_shift_or_exp,
-                   void* y_host, void* device_scratch, size_t scratch_bytes, void* stream_) {
+static int linear_host_impl(aq_handle_t h, int bits, const void* x_host, int M, int K, const void* w_packed,
+                            const void* w_scales, int N, int group_size, int scale_mode, int clip_shift_or_exp,
+                            void* y_host, void* device_scratch, size_t scratch_bytes, void* stream_, bool wait) {
     if (!h || !x_host || !y_host) return AQ_ERR_INVALID_ARG;
     if (bits != 8 && bits != 4) return AQ_ERR_INVALID_ARG;
     const int s = check_shape(M, K, N, group_size);
@@ -641,8 +641,23 @@ int aq_linear_host(aq_handle_t h, int bits, const void* x_host, int M, int K, co
     if (rc != AQ_OK) return rc;
     e = cudaMemcpyAsync(y_host, y_dev, (size_t)M * N * 2, cudaMemcpyDeviceToHost, stream);
     if (e != cudaSuccess) return cuda_fail(h, e);
+    if (!wait) return AQ_OK;
     e = cudaStreamSynchronize(stream);
     return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
+int aq_linear_host(aq_handle_t h, int bits, const void* x_host, int M, int K, const void* w_packed,
+                   const void* w_scales, int N, int group_size, int scale_mode, int clip_shift_or_exp,
+                   void* y_host, void* device_scratch, size_t scratch_bytes, void* stream) {
+    return linear_host_impl(h, bits, x_host, M, K, w_packed, w_scales, N, group_size, scale_mode, clip_shift_or_exp,
+                            y_host, device_scratch, scratch_bytes, stream, true);
+}
+
+int aq_linear_host_async(aq_handle_t h, int bits, const void* x_host, int M, int K, const void* w_packed,
+                         const void* w_scales, int N, int group_size, int scale_mode, int clip_shift_or_exp,
+                         void* y_host, void* device_scratch, size_t scratch_bytes, void* stream) {
+    return linear_host_impl(h, bits, x_host, M, K, w_packed, w_scales, N, group_size, scale_mode, clip_shift_or_exp,
+                            y_host, device_scratch, scratch_bytes, stream, false);
 }
 
 int aq_check_workspace(aq_handle_t h, const void* workspace, void* stream_) {
