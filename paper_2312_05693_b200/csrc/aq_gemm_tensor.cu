@@ -15,7 +15,8 @@
 // One persistent CTA per SM walks a static list of (channel tile, token tile) pairs.
 // Warp roles: 0 and 2 = TMA producers (activations / weights), 1 and 3 = MMA issuers (warp 1
 // also owns the TMEM allocation; warp 3 only works in per-group mode), 4-11 = weight unpack
-// (two groups of four taking alternate k blocks), 12-19 = epilogue; registers are moved from
+// (two groups of four taking alternate k blocks; only the first group works in per-group mode),
+// 12-19 = epilogue; registers are moved from
 // the first two roles to the epilogue with setmaxnreg. One thread spends about 55 cycles per
 // MMA instruction and about 100 per TMA instruction, which is why issue is spread over
 // threads and why the tile is 256 tokens wide where tensor memory allows it. Two (one scale per channel)
@@ -411,7 +412,12 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         const uint32_t total_iters = (uint32_t)my_tiles * (uint32_t)(kb_last - kb_first);
         int pending = -1;                             // slice whose store has been issued but not published
-        for (uint32_t it = group; it < total_iters; it += kUnpackGroups) {
+        // With per-group rescaling the epilogue sets the pace (about four times the MMA time per k block) and
+        // one group of unpack warps keeps up; the second group would only poll barriers on the schedulers
+        // the epilogue warps issue from (measured: 1-2 % slower with it), so it leaves at once.
+        constexpr int kActiveGroups = GROUPED ? 1 : kUnpackGroups;
+        if (group >= kActiveGroups) goto role_done;
+        for (uint32_t it = group; it < total_iters; it += kActiveGroups) {
             const int s = (int)(it % kNumStages);
             const int ai = (int)(it % kNumASlices);
             if (!mbar_wait_warp(&sm.tma_full[s], (it / kNumStages) & 1u, abort_flag, 6u)) goto role_done;
