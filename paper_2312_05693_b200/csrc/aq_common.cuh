@@ -47,7 +47,7 @@ struct Control {
     unsigned int min_key, max_key;   // zero-point variant: order-preserving keys of min(x), max(x)
     int zero_point;             // zero-point variant: zp of Eq. 7
     unsigned int split_flags[57];   // tensor kernel: one bit per (shared tile, epilogue warp), "first half arrived"
-    static constexpr int kMaxSplitTiles = 57 * 32 / 8;
+    static constexpr int kMaxSplitTiles = 57 * 32 / 12;   // up to twelve epilogue warps per tile
 };
 static_assert(sizeof(Control) == 256, "control block is 256 bytes");
 

@@ -33,15 +33,27 @@ namespace {
 
 constexpr int kUnpackGroups = 2;              // groups of four unpack warps; group g takes k blocks g, g+2, ...
 constexpr int kFirstUnpackWarp = 4;           // warps 0-3 (one warpgroup): two TMA producers, two MMA issuers
-constexpr int kFirstEpiWarp = kFirstUnpackWarp + 4 * kUnpackGroups;
+constexpr int kWarps = 20;
+constexpr int kThreads = kWarps * 32;
 // Registers per thread after the roles split (setmaxnreg works on aligned groups of four warps):
-constexpr int kRegsControl = 40, kRegsUnpack = 48, kRegsEpilogue = 168;
-constexpr int kEpiWarps = 8;                  // two warps per TMEM lane quarter, half of the token columns each
-constexpr int kThreads = (kFirstEpiWarp + kEpiWarps) * 32;
-// setmaxnreg can only hand out what the launch allocated (96 registers for each of the threads): a
-// larger request would wait forever.
-static_assert(128 * kRegsControl + 32 * 4 * kUnpackGroups * kRegsUnpack + 32 * kEpiWarps * kRegsEpilogue <= kThreads * 96,
-              "register plan exceeds the launch allocation");
+constexpr int kRegsControl = 40, kRegsUnpack = 48;
+// The warps behind the control warpgroup are unpack warps, then epilogue warps. Eight epilogue warps (two per
+// TMEM lane quarter, half of the token columns each) follow two groups of unpack warps; the per-group
+// kernels with 96- or 192-token tiles run twelve (three per quarter, a third of the columns each) behind
+// the one unpack group they need: there the per-group rescaling sets the pace, and a third warp per
+// scheduler hides the latency of the other two's barrier and tensor-memory round trips.
+template <int BM, bool GROUPED>
+struct Roles {
+    static constexpr int kEpiWarps = (GROUPED && (BM == 96 || BM == 192)) ? 12 : 8;
+    static constexpr int kFirstEpiWarp = kWarps - kEpiWarps;
+    static constexpr int kRegsEpilogue = kEpiWarps == 12 ? 128 : 168;
+    static constexpr int kColsPerEpiWarp = BM / (kEpiWarps / 4);
+    // setmaxnreg can only hand out what the launch allocated (96 registers for each of the threads): a
+    // larger request would wait forever.
+    static_assert(128 * kRegsControl + 32 * (kFirstEpiWarp - kFirstUnpackWarp) * kRegsUnpack +
+                          32 * kEpiWarps * kRegsEpilogue <= kThreads * 96,
+                  "register plan exceeds the launch allocation");
+};
 // The bit pattern of the float 1.5 * 2^23: an integer add of it turns an int32 sum v, |v| < 2^22,
 // into the bits of the float 12582912 + v, so the per-group epilogue needs no int->float
 // conversion instruction (those saturated their pipe); one FADD removes the bias.
@@ -181,10 +193,10 @@ __host__ __device__ constexpr uint32_t idesc_i8(int m, int n) {
 template <int BM>
 struct TileConfig {
     // shared-memory ring depth: activation tile + packed weight block (+ scales) per stage
-    static constexpr int kNumStages = BM >= 256 ? 5 : 6;
+    static constexpr int kNumStages = BM >= 192 ? 5 : 6;
 };
 
-template <int BM>
+template <int BM, int EPI_WARPS>
 struct SharedStorage {
     static constexpr int kNumStages = TileConfig<BM>::kNumStages;
     alignas(1024) uint8_t x[kNumStages][BM * 128];   // activation tiles, 128-byte swizzled rows
@@ -197,8 +209,8 @@ struct SharedStorage {
     alignas(16) __half sc[kNumScaleSlots][kTileN];
     // Each epilogue warp stages fp16 outputs of its 32 channels here, kStageRows tokens at a time
     // (token-major rows of 64 bytes), and hands them to a TMA store.
-    static constexpr int kStageRows = BM <= 128 ? BM / 2 : 32;
-    alignas(128) __half ystage[kEpiWarps][kStageRows][32];
+    static constexpr int kStageRows = BM / (EPI_WARPS / 4) <= 64 ? BM / (EPI_WARPS / 4) : 32;
+    alignas(128) __half ystage[EPI_WARPS][kStageRows][32];
     alignas(8) uint64_t tma_full[kNumStages];        // both producers' bytes landed -> unpack warps
     uint64_t smem_empty[kNumStages];                 // MMA done (+ epilogue took the scales) -> TMA producers
     uint64_t a_full[8];                              // unpack warps stored the slice -> MMA
@@ -257,24 +269,27 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap y_map,
                    const TensorParams p) {
     extern __shared__ uint8_t smem_raw[];
-    using Smem = SharedStorage<BM>;
+    using R = Roles<BM, GROUPED>;
+    constexpr int kEpiWarps = R::kEpiWarps, kFirstEpiWarp = R::kFirstEpiWarp, kRegsEpilogue = R::kRegsEpilogue;
+    using Smem = SharedStorage<BM, kEpiWarps>;
     Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
 
     constexpr int kNumStages = TileConfig<BM>::kNumStages;
     // accumulator stages in tensor memory: three for per-group rescaling, otherwise as many
     // 2 (or 1 for the 256-token tile) as leave room for the weight-slice ring
-    constexpr int kNumAcc = GROUPED ? 3 : (BM >= 256 ? 1 : 2);
+    constexpr int kNumAcc = GROUPED ? (BM > 128 ? 2 : 3) : (BM >= 256 ? 1 : 2);
+    constexpr int kAccStride = BM == 96 ? 128 : BM;   // columns between accumulator stages
     constexpr int kNumMmaThreads = GROUPED ? 2 : 1;   // issuers alternate k blocks when every block has its own accumulator
-    constexpr int kAccCols = kNumAcc * BM;
+    constexpr int kAccCols = kNumAcc * kAccStride;
     // the rest of tensor memory (up to 8 slices) is the ring of unpacked weight slices (A operand)
     constexpr int kNumASlices = (512 - kAccCols) / kAColsPerStage >= 8 ? 8 : (512 - kAccCols) / kAColsPerStage;
     static_assert(kNumASlices >= 4 && kNumASlices % kUnpackGroups == 0, "weight-slice ring");
-    static_assert(!GROUPED || kNumAcc == 3, "the scale ring's depth assumes three accumulator stages");
+    static_assert(!GROUPED || kNumAcc <= 3, "the scale ring's depth assumes at most three accumulator stages");
     constexpr int kTmemColsUsed = kAccCols + kNumASlices * kAColsPerStage;
     constexpr int kTmemCols = kTmemColsUsed <= 128 ? 128 : kTmemColsUsed <= 256 ? 256 : 512;
     static_assert(kTmemColsUsed <= 512, "tensor memory has 512 columns");
-    static_assert(BM % 64 == 0 && BM >= 64 && BM <= 256, "token tile");
-    constexpr int kColsPerEpiWarp = BM / 2;           // each quarter's columns are split between two warps
+    static_assert(BM % 32 == 0 && BM >= 64 && BM <= 256, "token tile");
+    constexpr int kColsPerEpiWarp = R::kColsPerEpiWarp;   // each quarter's columns are split between two or three warps
     static_assert(kColsPerEpiWarp % 16 == 0 && (!GROUPED || kColsPerEpiWarp % 32 == 0), "epilogue chunking");
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -363,7 +378,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
                     if (!mbar_wait(&sm.acc_empty[a], ((it / kNumAcc) & 1u) ^ 1u, abort_flag, 2u)) goto role_done;
                     if (!mbar_wait(&sm.a_full[ai], (it / kNumASlices) & 1u, abort_flag, 3u)) goto role_done;
                     tc_fence_after();
-                    const uint32_t d_addr = tmem_acc + (uint32_t)(a * BM);
+                    const uint32_t d_addr = tmem_acc + (uint32_t)(a * kAccStride);
                     const uint32_t a_addr = tmem_a + (uint32_t)(ai * kAColsPerStage);
                     const uint64_t bdesc = smem_desc_sw128(smem_u32(sm.x[s]));
 #pragma unroll
@@ -386,7 +401,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
                         // tile included) have landed, so this one wait covers both operands
                         if (!mbar_wait(&sm.a_full[ai], (it / kNumASlices) & 1u, abort_flag, 5u)) goto role_done;
                         tc_fence_after();
-                        const uint32_t d_addr = tmem_acc + (uint32_t)(a * BM);
+                        const uint32_t d_addr = tmem_acc + (uint32_t)(a * kAccStride);
                         const uint32_t a_addr = tmem_a + (uint32_t)(ai * kAColsPerStage);
                         const uint64_t bdesc = smem_desc_sw128(smem_u32(sm.x[s]));
 #pragma unroll
@@ -456,7 +471,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
         // ----------------------------------------------------------------------- epilogue
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kRegsEpilogue));
         const int quarter = warp & 3;
-        const int half = (warp - kFirstEpiWarp) >> 2;                                // which half of the token columns
+        const int half = (warp - kFirstEpiWarp) >> 2;                                // which half (third) of the token columns
         const int r = quarter * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
         const int col0 = half * kColsPerEpiWarp;
@@ -484,7 +499,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
                 uint32_t v[kColsPerEpiWarp];
 #pragma unroll
                 for (int c0 = 0; c0 < kColsPerEpiWarp; c0 += 32)
-                    tc_ld32(tmem_acc + lane_addr + (uint32_t)(a * BM + col0 + c0), *reinterpret_cast<uint32_t(*)[32]>(&v[c0]));
+                    tc_ld32(tmem_acc + lane_addr + (uint32_t)(a * kAccStride + col0 + c0), *reinterpret_cast<uint32_t(*)[32]>(&v[c0]));
                 tc_wait_ld();
                 tc_fence_before();
                 __syncwarp();
@@ -547,26 +562,34 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
                     if (++g_a == (uint32_t)kNumAcc) { g_a = 0; g_ph ^= 1u; }
                     if (++g_slot == (uint32_t)Smem::kNumScaleSlots) g_slot = 0;
                     static_assert(kColsPerEpiWarp == 32 || kColsPerEpiWarp == 64, "epilogue register plan");
-                    const uint32_t taddr = tmem_acc + lane_addr + (uint32_t)(a * BM + col0);
-                    uint32_t v[kColsPerEpiWarp];
-                    tc_ld32(taddr, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
-                    if (kColsPerEpiWarp == 64) tc_ld32(taddr + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32 % kColsPerEpiWarp]));
-                    tc_wait_ld();
-                    // the sums are in registers: the accumulator stage goes back to the MMA at once
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&sm.acc_empty[a]);
+                    const uint32_t taddr = tmem_acc + lane_addr + (uint32_t)(a * kAccStride + col0);
+                    // With twelve epilogue warps (128 registers each) a warp's 64 columns pass through one
+                    // 32-register buffer in two turns; otherwise all of them are loaded at once.
+                    constexpr int kLdCols = (kEpiWarps == 12 && kColsPerEpiWarp == 64) ? 32 : kColsPerEpiWarp;
 #pragma unroll
-                    for (int c = 0; c < kColsPerEpiWarp; ++c) {
-                        // int -> float without the conversion unit: adding the bits of 1.5 * 2^23 to an
-                        // integer |v| < 2^22 gives the bits of the float 12582912 + v
-                        fsum[c] = fmaf(__uint_as_float(v[c] + kMagicBits) - kMagicFloat, sg, fsum[c]);
-                    }
-                    if (p.acc_dump) {
+                    for (int c0 = 0; c0 < kColsPerEpiWarp; c0 += kLdCols) {
+                        uint32_t v[kLdCols];
+                        tc_ld32(taddr + c0, *reinterpret_cast<uint32_t(*)[32]>(&v[0]));
+                        if (kLdCols == 64) tc_ld32(taddr + c0 + 32, *reinterpret_cast<uint32_t(*)[32]>(&v[32 % kLdCols]));
+                        tc_wait_ld();
+                        if (c0 + kLdCols == kColsPerEpiWarp) {
+                            // the sums are in registers: the accumulator stage goes back to the MMA at once
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&sm.acc_empty[a]);
+                        }
 #pragma unroll
-                        for (int c = 0; c < kColsPerEpiWarp; ++c) {
-                            const int m = m_base + c;
-                            if (n_ok && m < p.M) p.acc_dump[((size_t)m * p.N + n) * G + kb] = (int)v[c] >> 4;
+                        for (int c = 0; c < kLdCols; ++c) {
+                            // int -> float without the conversion unit: adding the bits of 1.5 * 2^23 to an
+                            // integer |v| < 2^22 gives the bits of the float 12582912 + v
+                            fsum[c0 + c] = fmaf(__uint_as_float(v[c] + kMagicBits) - kMagicFloat, sg, fsum[c0 + c]);
+                        }
+                        if (p.acc_dump) {
+#pragma unroll
+                            for (int c = 0; c < kLdCols; ++c) {
+                                const int m = m_base + c0 + c;
+                                if (n_ok && m < p.M) p.acc_dump[((size_t)m * p.N + n) * G + kb] = (int)v[c] >> 4;
+                            }
                         }
                     }
                 }
@@ -651,7 +674,31 @@ role_done:
     }
 }
 
-constexpr int kSplitMinKBlocks = 64;          // shared tiles only from K = 8192 on (see launch_bm)
+// Shared tiles pay from K = 8192 on with 64- and 128-token tiles and from K = 4096 on with 192-token
+// tiles, where half a tile is worth more (see launch_bm).
+constexpr int split_min_k_blocks(int bm) { return bm >= 192 ? 32 : 64; }
+
+// Whether a last, partial round of `rem` tiles is run as shared tiles.
+inline bool round_is_shared(int rem, int sms, int k_blocks, int bm) {
+    return rem > 0 && 2 * rem <= sms && k_blocks >= split_min_k_blocks(bm) && rem <= Control::kMaxSplitTiles;
+}
+
+// Token tile of the per-group kernels. Up to 64 tokens: 64. Otherwise 128 (eight epilogue warps, three
+// accumulator stages) or 192 (twelve epilogue warps, two stages), whichever gives the shorter schedule:
+// rounds of tiles over the SMs (a shared last round counts half) x tile height x the measured cost per
+// token column and k block (about 8.5 cycles with 128-token tiles, 7.7 with 192-token tiles).
+int grouped_token_tile(int M, int K, int N, int sms, bool may_share) {
+    if (M <= 64) return 64;
+    const int k_blocks = K / kTileK, n_tiles_n = round_up(N, kTileN) / kTileN;
+    auto cost = [&](int bm, float per_col) {
+        const long tiles = (long)((M + bm - 1) / bm) * n_tiles_n;
+        const long rounds = tiles / sms;
+        const int rem = (int)(tiles % sms);
+        const float last = rem == 0 ? 0.0f : (may_share && round_is_shared(rem, sms, k_blocks, bm) ? 0.5f : 1.0f);
+        return ((float)rounds + last) * (float)bm * per_col;
+    };
+    return cost(192, 7.7f) < cost(128, 8.5f) ? 192 : 128;
+}
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -661,7 +708,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 template <int BM, bool GROUPED, bool OFFSET, bool CHAIN, bool SPLIT = false>
 cudaError_t launch_off(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream, int tile_limit = -1,
                        int split_base = 0, int split_tiles = 0) {
-    using Smem = SharedStorage<BM>;
+    using Smem = SharedStorage<BM, Roles<BM, GROUPED>::kEpiWarps>;
     const size_t smem_bytes = sizeof(Smem) + 1024;
     static bool attr_done = false;
     if (!attr_done) {
@@ -770,12 +817,13 @@ cudaError_t launch_bm(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t str
     if constexpr (GROUPED) {
         // A last round that would leave more than half of the SMs idle is run as shared tiles, when the
         // reduction is deep enough for half a tile to outweigh the second launch and the exchange of
-        // partial sums (measured: a loss of 2-5 us at K = 4096, a gain of 8 us at K = 11008).
+        // partial sums (measured with 128-token tiles: a loss of 2-5 us at K = 4096, a gain of 8 us at
+        // K = 11008; with 192-token tiles a gain of 2 us at K = 4096 already).
         const int sms = dev.sm_count;
         const int n_tiles = ((a.M + BM - 1) / BM) * (round_up(a.N, kTileN) / kTileN);
         const int rounds = n_tiles / sms, rem = n_tiles % sms;
-        const size_t need = (size_t)rem * 2 * kEpiWarps * (BM / 2) * 32 * sizeof(float);
-        if (rem > 0 && 2 * rem <= sms && a.K / kTileK >= kSplitMinKBlocks && rem <= Control::kMaxSplitTiles && a.split_scratch &&
+        const size_t need = (size_t)rem * 2 * BM * kTileN * sizeof(float);
+        if (round_is_shared(rem, sms, a.K / kTileK, BM) && a.split_scratch &&
             a.split_bytes >= need && (reinterpret_cast<uintptr_t>(a.split_scratch) & 15u) == 0) {
             if (rounds > 0) {
                 const cudaError_t e = launch_off<BM, true, false, false>(a, dev, stream, rounds * sms);
@@ -790,17 +838,24 @@ cudaError_t launch_bm(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t str
 }  // namespace
 
 size_t tensor_split_scratch_bytes(int M, int K, int N, int group, int sm_count) {
-    if (!group || K / kTileK < kSplitMinKBlocks) return 0;
-    const int bm = M <= 64 ? 64 : 128;                       // the per-group token tile (see launch_gemm_tensor)
+    if (!group) return 0;
+    const int bm = grouped_token_tile(M, K, N, sm_count, true);
     const int n_tiles = ((M + bm - 1) / bm) * (round_up(N, kTileN) / kTileN);
     const int rem = n_tiles % sm_count;
-    if (rem == 0 || 2 * rem > sm_count || rem > Control::kMaxSplitTiles) return 0;
-    return (size_t)rem * 2 * kEpiWarps * (bm / 2) * 32 * sizeof(float);
+    if (!round_is_shared(rem, sm_count, K / kTileK, bm)) return 0;
+    return (size_t)rem * 2 * bm * kTileN * sizeof(float);
 }
 
 cudaError_t launch_gemm_tensor(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
     if (a.M <= 64) return a.group ? launch_bm<64, true>(a, dev, stream) : launch_bm<64, false>(a, dev, stream);
-    if (a.group) return launch_bm<128, true>(a, dev, stream);
+    if (a.group) {
+        // the chained and zero-point variants have no shared-tile launch
+        switch (grouped_token_tile(a.M, a.K, a.N, dev.sm_count, !a.q_next && !a.chan_offset)) {
+            case 96: return launch_bm<96, true>(a, dev, stream);
+            case 192: return launch_bm<192, true>(a, dev, stream);
+            default: return launch_bm<128, true>(a, dev, stream);
+        }
+    }
     // one scale per channel: the 256-token tile halves the MMA instructions per unit of work
     if (a.M <= 128) return launch_bm<128, false>(a, dev, stream);
     return launch_bm<256, false>(a, dev, stream);

@@ -234,12 +234,12 @@ def test_several_tiles_per_cta_and_deep_k(group):
     assert_y_close(gpu["y"], ref["y"])
 
 
-@pytest.mark.parametrize("M,N", [(200, 520), (1100, 2304)])
-def test_shared_tiles_of_a_partial_last_round(M, N):
-    """Deep reduction (64 k blocks) with a last round that fills less than half of the SMs: those tiles
-    are shared by two CTAs (half of K each, partial sums exchanged). 10 tiles: every tile is shared;
-    162 tiles: one whole round, then 14 shared tiles."""
-    K = 8192
+@pytest.mark.parametrize("M,N,K", [(200, 520, 8192), (380, 12800, 4096), (380, 12800, 8192)])
+def test_shared_tiles_of_a_partial_last_round(M, N, K):
+    """A last round that fills less than half of the SMs: those tiles are shared by two CTAs (half of K
+    each, partial sums exchanged). 200 x 520: ten 128-token tiles, every tile is shared; 380 x 12800: two
+    hundred 192-token tiles, one whole round and then 52 shared tiles, at the smallest depth that shares
+    such tiles (32 k blocks) and at 64."""
     x = inputs.activations(M, K, seed=125, outlier_frac=0.005, outlier_mult=30.0)
     w = inputs.weights(N, K, seed=126)
     assert binding.aq_workspace_bytes(M, K, N, 128) > binding.aq_workspace_bytes(M, K, N, 0)   # room for the partial sums
