@@ -54,11 +54,6 @@ struct Roles {
                           32 * kEpiWarps * kRegsEpilogue <= kThreads * 96,
                   "register plan exceeds the launch allocation");
 };
-// The bit pattern of the float 1.5 * 2^23: an integer add of it turns an int32 sum v, |v| < 2^22,
-// into the bits of the float 12582912 + v, so the per-group epilogue needs no int->float
-// conversion instruction (those saturated their pipe); one FADD removes the bias.
-constexpr uint32_t kMagicBits = 0x4B400000u;
-constexpr float kMagicFloat = 12582912.0f;
 constexpr int kAColsPerStage = 32;            // 128 k of int8 = 32 TMEM columns per lane
 constexpr unsigned long long kWaitCycles = 4000000000ull;   // ~2 s
 
@@ -580,9 +575,11 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
                         }
 #pragma unroll
                         for (int c = 0; c < kLdCols; ++c) {
-                            // int -> float without the conversion unit: adding the bits of 1.5 * 2^23 to an
-                            // integer |v| < 2^22 gives the bits of the float 12582912 + v
-                            fsum[c0 + c] = fmaf(__uint_as_float(v[c] + kMagicBits) - kMagicFloat, sg, fsum[c0 + c]);
+                            // One conversion and one FMA per element. (An integer add of the bits of
+                            // 1.5 * 2^23 plus a float subtract also converts, on the FMA and ALU pipes, but
+                            // costs a third instruction; measured 8-16 % slower: issue slots are what this
+                            // loop runs out of, not the conversion unit.)
+                            fsum[c0 + c] = fmaf((float)(int)v[c], sg, fsum[c0 + c]);
                         }
                         if (p.acc_dump) {
 #pragma unroll
@@ -686,7 +683,7 @@ inline bool round_is_shared(int rem, int sms, int k_blocks, int bm) {
 // Token tile of the per-group kernels. Up to 64 tokens: 64. Otherwise 128 (eight epilogue warps, three
 // accumulator stages) or 192 (twelve epilogue warps, two stages), whichever gives the shorter schedule:
 // rounds of tiles over the SMs (a shared last round counts half) x tile height x the measured cost per
-// token column and k block (about 8.5 cycles with 128-token tiles, 7.7 with 192-token tiles).
+// token column and k block (about 7.6 cycles with 128-token tiles, 6.6 with 192-token tiles).
 int grouped_token_tile(int M, int K, int N, int sms, bool may_share) {
     if (M <= 64) return 64;
     const int k_blocks = K / kTileK, n_tiles_n = round_up(N, kTileN) / kTileN;
@@ -697,7 +694,7 @@ int grouped_token_tile(int M, int K, int N, int sms, bool may_share) {
         const float last = rem == 0 ? 0.0f : (may_share && round_is_shared(rem, sms, k_blocks, bm) ? 0.5f : 1.0f);
         return ((float)rounds + last) * (float)bm * per_col;
     };
-    return cost(192, 7.7f) < cost(128, 8.5f) ? 192 : 128;
+    return cost(192, 6.6f) < cost(128, 7.6f) ? 192 : 128;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
