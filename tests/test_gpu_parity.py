@@ -136,6 +136,8 @@ SHAPES = [
     (260, 1152, 520, 128),
     (130, 256, 203, 128),      # N not a multiple of 8: outputs take direct stores instead of TMA stores
     (70, 256, 77, 0),
+    (950, 256, 2556, 128),     # 192-token tiles (5 x 20 tiles in one round), ragged last tile, direct stores
+    (950, 384, 2560, 128),     # the same tiles with TMA stores
 ]
 
 
