@@ -253,6 +253,26 @@ def test_shared_tiles_of_a_partial_last_round(M, N, K):
     assert np.array_equal(gpu["y"].view(np.uint16), gpu2["y"].view(np.uint16))     # whichever half arrives second
 
 
+@pytest.mark.parametrize("seed", range(10))
+def test_seeded_random_shapes_per_group_scales(seed):
+    """Shapes drawn from a seeded generator: token counts that leave ragged 128- and 192-token tiles,
+    channel counts that are not multiples of 128 (some not of 8), 1 to 12 k blocks; with and without
+    int4 activations."""
+    rng = np.random.default_rng(1000 + seed)
+    M = int(rng.integers(129, 1400))
+    K = 128 * int(rng.integers(1, 13))
+    N = int(rng.integers(1, 700)) * (4 if seed % 3 == 0 else 8)
+    bits = 4 if seed % 2 else 8
+    x = inputs.activations(M, K, seed=seed, outlier_frac=0.01, outlier_mult=25.0)
+    w = inputs.weights(N, K, seed=seed + 50)
+    gpu, ref = run_layer_both(x, w, bits, 128, TENSOR, clip=4 if bits == 4 else 0)
+    assert gpu["e"] == ref["e"] and np.array_equal(gpu["q"], ref["q"])
+    assert np.array_equal(gpu["acc"], ref["acc"])
+    assert_y_close(gpu["y"], ref["y"])
+    gpu2, _ = run_layer_both(x, w, bits, 128, TENSOR, clip=4 if bits == 4 else 0, want_acc=False)
+    assert np.array_equal(gpu["y"].view(np.uint16), gpu2["y"].view(np.uint16))
+
+
 def test_results_are_deterministic_run_to_run():
     M, K, N = 260, 1152, 520
     x = inputs.activations(M, K, seed=9, outlier_frac=0.01, outlier_mult=20.0)
