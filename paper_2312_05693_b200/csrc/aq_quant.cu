@@ -189,6 +189,20 @@ quantize_small_kernel(const uint4* __restrict__ x, int M, int vec_per_row, const
     }
     if (rank == 0 && threadIdx.x < 57) ctl->split_flags[threadIdx.x] = 0;    // the product kernel's shared-tile bits
     const float lo = -(float)(1 << (bits - 1)), hi = (float)((1 << (bits - 1)) - 1);
+    if (alpha == nullptr && e >= -14 && e <= 14) {           // 2^-e is a normal half: codes in half2 arithmetic
+        const __half2 inv2 = __float2half2_rn(__int_as_float((127 - e) << 23));
+        const __half2 lo2 = __float2half2_rn(lo), hi2 = __float2half2_rn(hi);
+#pragma unroll
+        for (int i = 0; i < kSmallVecs; ++i) {
+            const int v = (i * kSmallCtas + rank) * kSmallThreads + (int)threadIdx.x;
+            if (v < total) {
+                uint2 w;
+                quantize8_half2(buf[i], inv2, lo2, hi2, w.x, w.y);
+                q[v] = w;
+            }
+        }
+        return;
+    }
 #pragma unroll
     for (int i = 0; i < kSmallVecs; ++i) {
         const int v = (i * kSmallCtas + rank) * kSmallThreads + (int)threadIdx.x;

@@ -49,6 +49,28 @@ def test_quantize_act_dynamic(bits, M, K):
         assert np.array_equal(q.cpu().numpy(), oracle.quantize_act(x, bits, e_ref))
 
 
+@pytest.mark.parametrize("bits", [8, 4])
+def test_quantize_act_small_dynamic_ties_over_the_exponent_range(bits):
+    """The one-launch kernel for small activations: exact ties (x = (j + 1/2) * 2^e), clamped values and
+    NaN, with the layer exponent swept over both of its code routes (half2 arithmetic while 2^-e is a
+    normal half, fp32 otherwise)."""
+    M, K = 8, 256
+    qmax = (1 << (bits - 1)) - 1
+    j = (np.arange(M * K) % (2 * qmax)) - qmax
+    base = (j + 0.5).astype(np.float64).reshape(M, K)          # ties; the largest magnitude sets the exponent
+    base[0, 0] = qmax
+    h = handle()
+    for s in range(-20, 9):
+        x = np.ldexp(base, s).astype(np.float16)
+        x[1, 1] = np.nan
+        q, e = h.aq_quantize_act(dev(x), bits, binding.AQ_SCALE_DYNAMIC, 0)
+        e_ref = oracle.layer_exponent(x, bits)
+        assert int(e.item()) == e_ref, s
+        assert np.array_equal(q.cpu().numpy(), oracle.quantize_act(x, bits, e_ref)), s
+        q, e = h.aq_quantize_act(dev(x), bits, binding.AQ_SCALE_DYNAMIC, 2)     # lower exponent: values clamp
+        assert np.array_equal(q.cpu().numpy(), oracle.quantize_act(x, bits, e_ref - 2)), s
+
+
 def test_quantize_act_static_rowidx_and_nonfinite():
     M, K = 40, 256
     x = inputs.activations(M, K, seed=5, outlier_frac=0.01, outlier_mult=20.0)
