@@ -20,9 +20,9 @@
  *    void*, NULL = default stream) and return without synchronizing, except the calls
  *    documented as synchronizing.
  *  - Return value: AQ_OK (0) or a negative aq_status. On error nothing was enqueued.
- *  - Shapes: K % 128 == 0, 128 <= K <= 65536; N >= 1; M >= 1. group_size is 0 (one scale
- *    per output channel) or 128. Activation bits is 8 or 4 (4-bit codes are stored one
- *    per int8, values -8..7).
+ *  - Shapes: K % 32 == 0, 32 <= K <= 65536, and K % 128 == 0 when group_size is 128; N >= 1;
+ *    M >= 1. group_size is 0 (one scale per output channel) or 128. Activation bits is 8 or 4
+ *    (4-bit codes are stored one per int8, values -8..7).
  *  - Rounding is to nearest, ties to even.
  *  - Requires a device of compute capability 10.0 (B200); anything else is refused with
  *    AQ_ERR_UNSUPPORTED_DEVICE. There is no CPU or other fallback.
@@ -74,14 +74,24 @@ int aq_last_cuda_error(aq_handle_t h);
 int aq_set_kernel(aq_handle_t h, int kernel);
 
 /* ---- sizes -------------------------------------------------------------------------- */
-/* Bytes of the packed 4-bit weight buffer (rows are padded to a multiple of 128). */
+/* Bytes of the packed 4-bit weight buffer (rows are padded to a multiple of 128 channels, and K to a
+ * multiple of 128 with zero codes; the size does not depend on group_size). */
 size_t aq_packed_w4_bytes(int N, int K);
+/* Version of the packed layout that aq_pack_w4 of this library writes. The packed buffer is a bare
+ * array of blocks without a header, so a program that stores packed weights (a file, a cache) keeps
+ * this number beside them and repacks when a later library reports another one. */
+int aq_packed_w4_layout_version(void);
 /* Bytes of the fp16 scale buffer: [G][Npad], G = 1 (group_size 0) or K/128, Npad = N
  * rounded up to 128; element (g, n) at index g*Npad + n. */
 size_t aq_scales_bytes(int N, int K, int group_size);
-/* Bytes of scratch that aq_quantize_act / aq_linear_* / aq_gemm_w4 / aq_token_select need
+/* Bytes of scratch that aq_quantize_act / aq_linear_* / aq_gemm_w4 / aq_token_select should get
  * for these sizes (M = rows actually multiplied). Always a multiple of 256. */
 size_t aq_workspace_bytes(int M, int K, int N, int group_size);
+/* The least the calls accept: control block, activation codes, per-row scratch, per-channel terms.
+ * aq_workspace_bytes() adds, for per-group scales, room for the partial sums of output tiles whose
+ * k range CTAs share; with less than that the kernel shares no tile (slower on some shapes; outputs
+ * may then differ in the last fp32 rounding before the fp16 one, integer sums never). */
+size_t aq_workspace_min_bytes(int M, int K, int N, int group_size);
 
 /* ---- weights (offline; paper Sec. 4.4 last paragraph, Sec. 5.1: 4-bit per-channel weights)
  * Round-to-nearest symmetric quantization of w_fp16 [N,K] row-major:
@@ -138,7 +148,7 @@ int aq_token_compact(aq_handle_t h, const void* x_fp16, int M, int K, const int3
  * alpha: K bytes on the device (16-byte aligned), one factor per input channel, each in
  * 0..k_max, k_max <= 4. Channel k is quantized to a 4-bit code with the coarser step
  * 2^(e + alpha_k) (Eq. 5), and the code enters the integer product shifted left by alpha_k,
- * which is the factor "transformed over the corresponding weights" of Sec. 4.4 (a 4-bit code
+ * which is Sec. 4.4's move of the factor from the activation scale onto the weights (a 4-bit code
  * shifted by at most 4 still fits the int8 operand). The dynamic base exponent is
  * e = e0 - k_max - clip_shift, e0 the plain 4-bit layer exponent (Eq. 6 read as
  * s = 2^(e0 - K)), so channels with the largest factor still reach the layer maximum; in
@@ -308,6 +318,17 @@ int aq_linear_host_async(aq_handle_t h, int bits, const void* x_host, int M, int
  * aq_linear_* / aq_gemm_w4 / aq_quantize_act call clears the record when it starts. */
 int aq_check_workspace(aq_handle_t h, const void* workspace, void* stream);
 
+/* ---- measurement aid: the tensor cores' int8 rate on this GPU (the denominator of the roofline of
+ * the prefill product, Sec. 4.4's integer matrix multiplication)
+ * Enqueues one kernel in which every SM issues iters x 4 tcgen05.mma kind::i8 instructions of
+ * 128 x 256 x 32 on operands that stay in place (A from tensor memory when a_from_tmem != 0, as in the
+ * product kernel, else from shared memory), with no loads and no epilogue. *ops_out (host, may be NULL)
+ * receives the integer operations of the launch (2 per multiply-add); time the launch with events on
+ * `stream`. workspace: 256 bytes (control block; aq_check_workspace reports a wait that gave up).
+ * 1 <= iters <= 2^24. */
+int aq_probe_int8_mma(aq_handle_t h, int iters, int a_from_tmem, double* ops_out, void* workspace,
+                      size_t workspace_bytes, void* stream);
+
 /* ---- the layer without any caller-provided or allocated scratch
  * (The paper has no counterpart to this call: it exists for the way some programs must use
  * the library, not for anything the method computes.)
@@ -322,23 +343,34 @@ int aq_check_workspace(aq_handle_t h, const void* workspace, void* stream);
  * This call performs no cudaMalloc / cudaFree and calls nothing that allocates.
  *
  * Limits and rules
- *  - aq_workspace_bytes(M, K, N, group_size) must not exceed AQ_NOALLOC_SCRATCH_BYTES
- *    (about M*K <= 16 Mi codes, e.g. 2048 x 8192 or 4096 x 4096); larger sizes are refused with
- *    AQ_ERR_TOO_LARGE and nothing is enqueued. Use aq_linear_w4a8 with your own workspace then.
+ *  - aq_workspace_min_bytes(M, K, N, group_size) = 256 + up256(M*K) + up256(M) + up256(4*N)
+ *    (up256 rounds up to a multiple of 256) must not exceed AQ_NOALLOC_SCRATCH_BYTES: M*K up to
+ *    16 Mi codes as long as M + 4*N stays under 64 KiB (2048 x 8192 or 4096 x 4096 activations with
+ *    N <= 15360), and any N when M*K is smaller by 4*N + M bytes. Larger sizes are refused with
+ *    AQ_ERR_TOO_LARGE and nothing is enqueued; use aq_linear_w4a8 with your own workspace then.
+ *    What the buffer has left beyond that minimum serves the per-group kernel's shared tiles; a
+ *    shape that would want more than is left runs without sharing (see aq_workspace_min_bytes).
  *  - The buffer is a static device array: every GPU on which the library is loaded holds
  *    AQ_NOALLOC_SCRATCH_BYTES of device memory until the process exits.
  *  - The first call on each device looks up the buffer's device address (a one-time,
- *    host-side set-up that needs that device to be current). Make that first call before
+ *    host-side set-up that needs that device to be current). With lazy module loading (the CUDA
+ *    default) that look-up is also the moment the driver loads the library's device code and
+ *    reserves the buffer, so it can fail with AQ_ERR_CUDA when the device is already full. Make
+ *    that first call at start-up: before a memory pool takes the rest of the device and before
  *    starting any stream capture.
  *  - All calls on a device share the one buffer, and it keeps the previous call's contents; the
  *    call itself clears the part that must start at zero. Two calls that can overlap on the
  *    GPU (different streams without ordering) race on the buffer: order them, or use
  *    aq_linear_w4a8 with separate workspaces.
- *  - The handle's device must be the current device. */
+ *  - The handle's device must be the current device.
+ *  - aq_check_noalloc is aq_check_workspace for the built-in buffer (whose address callers do not
+ *    have): it SYNCHRONIZES the stream and reports whether a kernel of the last call gave up on a
+ *    bounded wait. */
 #define AQ_NOALLOC_SCRATCH_BYTES ((size_t)16 * 1024 * 1024 + 65536 + 256)
 int aq_linear_w4a8_noalloc(aq_handle_t h, const void* x_fp16, int M, int K, const void* w_packed,
                            const void* w_scales, int N, int group_size, int scale_mode,
                            int clip_shift_or_exp, void* y_fp16, void* stream);
+int aq_check_noalloc(aq_handle_t h, void* stream);
 
 #ifdef __cplusplus
 }

@@ -65,6 +65,9 @@ def load():
     L.aq_scales_bytes.argtypes = [i32, i32, i32]
     L.aq_workspace_bytes.restype = sz
     L.aq_workspace_bytes.argtypes = [i32, i32, i32, i32]
+    L.aq_workspace_min_bytes.restype = sz
+    L.aq_workspace_min_bytes.argtypes = [i32, i32, i32, i32]
+    L.aq_packed_w4_layout_version.restype = i32
     L.aq_linear_host_scratch_bytes.restype = sz
     L.aq_linear_host_scratch_bytes.argtypes = [i32, i32, i32, i32]
     L.aq_pack_w4.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp]
@@ -106,6 +109,8 @@ def load():
     L.aq_linear_host_async.argtypes = L.aq_linear_host.argtypes
     L.aq_check_workspace.argtypes = [vp, vp, vp]
     L.aq_linear_w4a8_noalloc.argtypes = [vp, vp, i32, i32, vp, vp, i32, i32, i32, i32, vp, vp]
+    L.aq_check_noalloc.argtypes = [vp, vp]
+    L.aq_probe_int8_mma.argtypes = [vp, i32, i32, vp, vp, sz, vp]
     _lib = L
     return L
 
@@ -146,6 +151,14 @@ def aq_prune_schedule(M: int, beta: float, m: int):
 
 def aq_workspace_bytes(M: int, K: int, N: int, group_size: int) -> int:
     return load().aq_workspace_bytes(M, K, N, group_size)
+
+
+def aq_workspace_min_bytes(M: int, K: int, N: int, group_size: int) -> int:
+    return load().aq_workspace_min_bytes(M, K, N, group_size)
+
+
+def aq_packed_w4_layout_version() -> int:
+    return load().aq_packed_w4_layout_version()
 
 
 def aq_linear_host_scratch_bytes(M: int, K: int, N: int, group_size: int) -> int:
@@ -488,3 +501,13 @@ class Handle:
 
     def aq_check_workspace(self, workspace: torch.Tensor) -> int:
         return load().aq_check_workspace(self._h, _ptr(workspace), _stream())
+
+    def aq_probe_int8_mma(self, iters: int, a_from_tmem: bool, workspace: torch.Tensor) -> float:
+        """Enqueues the tensor-core rate probe; returns the integer operations of the launch."""
+        ops = C.c_double(0.0)
+        _check(load().aq_probe_int8_mma(self._h, iters, 1 if a_from_tmem else 0, C.cast(C.byref(ops), C.c_void_p),
+                                        _ptr(workspace), workspace.numel(), _stream()), "aq_probe_int8_mma")
+        return ops.value
+
+    def aq_check_noalloc(self) -> int:
+        return load().aq_check_noalloc(self._h, _stream())

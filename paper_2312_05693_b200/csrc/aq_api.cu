@@ -26,8 +26,9 @@ int cuda_fail(aq_handle_t h, cudaError_t e) {
 
 int check_shape(int M, int K, int N, int group) {
     if (M < 1 || N < 1) return AQ_ERR_SHAPE;
-    if (K < 128 || K > 65536 || K % 128 != 0) return AQ_ERR_SHAPE;
+    if (K < 32 || K > 65536 || K % 32 != 0) return AQ_ERR_SHAPE;
     if (group != 0 && group != 128) return AQ_ERR_SHAPE;
+    if (group == 128 && K % 128 != 0) return AQ_ERR_SHAPE;
     if ((size_t)M * (size_t)N > ((size_t)1 << 40)) return AQ_ERR_SHAPE;
     return AQ_OK;
 }
@@ -46,9 +47,13 @@ struct Workspace {
 // [fp32 partial outputs of tiles that two CTAs share in the tensor kernel, sized for a 148-SM B200; a
 // device that would need more simply shares no tile]
 constexpr int kPlannedSmCount = 148;
+// what every call needs
+size_t workspace_min_bytes(int M, int K, int N) {
+    return sizeof(Control) + up256((size_t)M * K) + up256((size_t)M) + up256((size_t)N * sizeof(float));
+}
+// plus the optional area that lets the per-group tensor kernel share the tiles of a partial last round
 size_t workspace_bytes(int M, int K, int N, int group) {
-    return sizeof(Control) + up256((size_t)M * K) + up256((size_t)M) + up256((size_t)N * sizeof(float)) +
-           up256(tensor_split_scratch_bytes(M, K, N, group, kPlannedSmCount));
+    return workspace_min_bytes(M, K, N) + up256(tensor_split_scratch_bytes(M, K, N, group, kPlannedSmCount));
 }
 
 Workspace carve(void* ws, int M, int K, int N, size_t total_bytes) {
@@ -59,7 +64,7 @@ Workspace carve(void* ws, int M, int K, int N, size_t total_bytes) {
     w.scratch = b + sizeof(Control) + up256((size_t)M * K);
     w.scratch_bytes = up256((size_t)M);
     w.chan_offset = reinterpret_cast<float*>(b + sizeof(Control) + up256((size_t)M * K) + up256((size_t)M));
-    const size_t used = sizeof(Control) + up256((size_t)M * K) + up256((size_t)M) + up256((size_t)N * sizeof(float));
+    const size_t used = workspace_min_bytes(M, K, N);
     w.split_scratch = reinterpret_cast<float*>(b + used);
     w.split_bytes = total_bytes > used ? total_bytes - used : 0;
     return w;
@@ -114,7 +119,7 @@ int linear_impl(aq_handle_t h, int bits, const void* x, int M, int K, const void
     if (scale_mode == AQ_SCALE_STATIC && (clip_shift_or_exp < -40 || clip_shift_or_exp > 40)) return AQ_ERR_INVALID_ARG;
     const int s = check_shape(M, K, N, group);
     if (s != AQ_OK) return s;
-    if (!workspace || workspace_bytes_ < workspace_bytes(M, K, N, group)) return AQ_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes_ < workspace_min_bytes(M, K, N)) return AQ_ERR_WORKSPACE;
     if (!aligned(x, 16) || !aligned(w_packed, 16) || !aligned(w_scales, 2) || (y && !aligned(y, 2)) ||
         !aligned(workspace, 256) || (acc_dump && !aligned(acc_dump, 4)) || (row_idx && !aligned(row_idx, 4)))
         return AQ_ERR_ALIGNMENT;
@@ -170,7 +175,11 @@ const char* aq_status_string(int status) {
     }
 }
 
-int aq_version(void) { return 100; }
+int aq_version(void) { return 200; }
+
+// 1: blocks of 128 channels x 128 k, 16-byte units of 32 codes, nibble planes (see aq_common.cuh).
+// 2: the same, with K padded to a multiple of 128 by zero codes (identical to 1 when K % 128 == 0).
+int aq_packed_w4_layout_version(void) { return 2; }
 
 int aq_create(aq_handle_t* out, int device) {
     if (!out) return AQ_ERR_INVALID_ARG;
@@ -221,12 +230,12 @@ int aq_set_kernel(aq_handle_t h, int kernel) {
 }
 
 size_t aq_packed_w4_bytes(int N, int K) {
-    if (N < 1 || K < 128 || K % 128) return 0;
-    return (size_t)round_up(N, kTileN) * (size_t)K / 2;
+    if (N < 1 || K < 32 || K % 32) return 0;
+    return (size_t)round_up(N, kTileN) * (size_t)round_up(K, kTileK) / 2;
 }
 
 size_t aq_scales_bytes(int N, int K, int group_size) {
-    if (N < 1 || K < 128 || K % 128 || (group_size != 0 && group_size != 128)) return 0;
+    if (N < 1 || K < 32 || K % 32 || (group_size != 0 && group_size != 128) || (group_size && K % 128)) return 0;
     const size_t G = group_size ? (size_t)K / 128 : 1;
     return G * (size_t)round_up(N, kTileN) * sizeof(__half);
 }
@@ -234,6 +243,11 @@ size_t aq_scales_bytes(int N, int K, int group_size) {
 size_t aq_workspace_bytes(int M, int K, int N, int group_size) {
     if (check_shape(M, K, N, group_size) != AQ_OK) return 0;
     return workspace_bytes(M, K, N, group_size);
+}
+
+size_t aq_workspace_min_bytes(int M, int K, int N, int group_size) {
+    if (check_shape(M, K, N, group_size) != AQ_OK) return 0;
+    return workspace_min_bytes(M, K, N);
 }
 
 int aq_pack_w4(aq_handle_t h, const void* w_fp16, int N, int K, int group_size, void* w_packed,
@@ -345,7 +359,7 @@ int aq_gemm_w4(aq_handle_t h, const int8_t* q, int M, int K, const void* w_packe
     if (!h || !q || !w_packed || !w_scales || !scale_exp || !y_fp16) return AQ_ERR_INVALID_ARG;
     const int s = check_shape(M, K, N, group_size);
     if (s != AQ_OK) return s;
-    if (!workspace || workspace_bytes_ < workspace_bytes(M, K, N, group_size)) return AQ_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes_ < workspace_min_bytes(M, K, N)) return AQ_ERR_WORKSPACE;
     if (!aligned(q, 16) || !aligned(w_packed, 16) || !aligned(w_scales, 2) || !aligned(y_fp16, 2) ||
         !aligned(workspace, 256) || !aligned(scale_exp, 4) || (acc_dump && !aligned(acc_dump, 4)))
         return AQ_ERR_ALIGNMENT;
@@ -410,7 +424,7 @@ int aq_gemm_w4_act4(aq_handle_t h, const void* q4, int M, int K, const void* w_p
     if (!h || !q4) return AQ_ERR_INVALID_ARG;
     const int s = check_shape(M, K, N, group_size);
     if (s != AQ_OK) return s;
-    if (!workspace || workspace_bytes_ < workspace_bytes(M, K, N, group_size)) return AQ_ERR_WORKSPACE;
+    if (!workspace || workspace_bytes_ < workspace_min_bytes(M, K, N)) return AQ_ERR_WORKSPACE;
     if (!aligned(q4, 16) || !aligned(workspace, 256)) return AQ_ERR_ALIGNMENT;
     const Workspace w = carve(workspace, M, K, N, workspace_bytes_);
     const cudaError_t e = launch_act4_unpack(static_cast<const uint8_t*>(q4), (size_t)M * K, w.codes,
@@ -658,6 +672,20 @@ int aq_linear_host_async(aq_handle_t h, int bits, const void* x_host, int M, int
                          void* y_host, void* device_scratch, size_t scratch_bytes, void* stream) {
     return linear_host_impl(h, bits, x_host, M, K, w_packed, w_scales, N, group_size, scale_mode, clip_shift_or_exp,
                             y_host, device_scratch, scratch_bytes, stream, false);
+}
+
+int aq_probe_int8_mma(aq_handle_t h, int iters, int a_from_tmem, double* ops_out, void* workspace,
+                      size_t workspace_bytes_, void* stream_) {
+    if (!h || iters < 1 || iters > (1 << 24)) return AQ_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes_ < sizeof(Control)) return AQ_ERR_WORKSPACE;
+    if (!aligned(workspace, 256)) return AQ_ERR_ALIGNMENT;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    Control* ctl = static_cast<Control*>(workspace);
+    cudaError_t e = cudaMemsetAsync(ctl, 0, sizeof(Control), stream);
+    if (e == cudaSuccess) e = launch_int8_probe(iters, a_from_tmem ? 1 : 0, ctl, h->dev, stream);
+    if (e != cudaSuccess) return cuda_fail(h, e);
+    if (ops_out) *ops_out = 2.0 * 128.0 * 256.0 * 32.0 * 4.0 * (double)iters * (double)h->dev.sm_count;
+    return AQ_OK;
 }
 
 int aq_check_workspace(aq_handle_t h, const void* workspace, void* stream_) {

@@ -466,13 +466,9 @@ cudaError_t launch_attn_tc(const void* w, const int8_t* vt, const uint32_t* max_
                            cudaStream_t stream) {
     using Smem = AttnSmem<DN>;
     const size_t smem_bytes = sizeof(Smem) + 1024;
-    static bool attr_done = false;
-    if (!attr_done) {
-        const cudaError_t e = cudaFuncSetAttribute(attn_v_tc_kernel<DN, A_SIGNED>,
-                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    static SmemOptIn opt_in;
+    if (const cudaError_t e = opt_in.ensure(attn_v_tc_kernel<DN, A_SIGNED>, dev.device, smem_bytes); e != cudaSuccess)
+        return e;
     CUtensorMap amap, bmap;
     const cuuint32_t estr[2] = {1u, 1u};
     const cuuint64_t strides[1] = {(cuuint64_t)J};

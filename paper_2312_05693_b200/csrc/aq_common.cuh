@@ -7,6 +7,8 @@
 #include <stdint.h>
 #include <stddef.h>
 
+#include <atomic>
+
 #include "../../include/agileq.h"
 
 namespace aq {
@@ -31,6 +33,10 @@ constexpr int kTileK = 128;          // k per packed block (= the weight-scale g
 constexpr int kBlockBytes = kTileN * kTileK / 2;   // 8192
 
 __host__ __device__ inline int round_up(int v, int m) { return (v + m - 1) / m * m; }
+// Blocks of 128 k that cover K. With one scale per channel K need only be a multiple of 32: the last
+// block is then padded with zero codes at pack time, so whatever the activation side delivers for
+// k >= K (zeros from a tensor map's bounds, or stale staging bytes) contributes nothing.
+__host__ __device__ inline int k_blocks(int K) { return (K + kTileK - 1) / kTileK; }
 __host__ __device__ inline size_t packed_unit_offset(int KB, int nt, int kb, int j, int r) {
     return ((size_t)nt * KB + kb) * kBlockBytes + (size_t)(j * kTileN + r) * 16;
 }
@@ -77,6 +83,22 @@ struct DeviceInfo {
     int cc_major, cc_minor;
     size_t smem_optin;
     void* encode_tiled;   // cuTensorMapEncodeTiled, resolved through the runtime
+};
+
+// Opting a kernel in to more than 48 KB of dynamic shared memory acts on the current device only, so
+// the "already done" flag is kept per device (a process may hold handles on several GPUs). One
+// static instance per kernel, owned by that kernel's launcher.
+constexpr int kMaxDevices = 64;
+struct SmemOptIn {
+    std::atomic<bool> done[kMaxDevices];
+    template <class Kernel>
+    cudaError_t ensure(Kernel kernel, int device, size_t bytes) {
+        if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+        if (done[device].load(std::memory_order_acquire)) return cudaSuccess;
+        const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+        if (e == cudaSuccess) done[device].store(true, std::memory_order_release);
+        return e;
+    }
 };
 
 cudaError_t launch_pack_w4(const __half* w, int N, int K, int group, uint8_t* packed, __half* scales,
@@ -178,6 +200,8 @@ void handle_record_cuda_error(aq_handle_t h, cudaError_t e);
 cudaError_t launch_gemm_tensor(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream);
 // Bytes of split_scratch the tensor kernel can use for these sizes on a GPU with sm_count SMs (0: none).
 size_t tensor_split_scratch_bytes(int M, int K, int N, int group, int sm_count);
+// Tensor-core rate probe: every SM issues iters x 4 MMAs of 128 x 256 x 32 (int8) on resident operands.
+cudaError_t launch_int8_probe(int iters, int a_from_tmem, Control* ctl, const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_gemm_decode(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream);
 
 }  // namespace aq

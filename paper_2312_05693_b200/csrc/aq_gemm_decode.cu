@@ -60,7 +60,7 @@ gemm_decode_kernel(const int8_t* __restrict__ q, int M, int K, int N, int Npad,
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     // this kernel has no bounded waits; after a quantize kernel of the same call the word is that kernel's
     if (clear_status && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) ctl->status = 0;
-    const int KB = K / kTileK;
+    const int KB = k_blocks(K);
     const int n0 = blockIdx.x * 32;
     const int nt = n0 / kTileN, r = (n0 % kTileN) + lane;
     const int n = n0 + lane;
@@ -104,6 +104,7 @@ gemm_decode_kernel(const int8_t* __restrict__ q, int M, int K, int N, int Npad,
             }
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
+                if (kb * kTileK + 32 * j >= K) break;            // a last block padded with zero codes (K % 128 != 0)
                 const uint32_t w[4] = {cur[j].x, cur[j].y, cur[j].z, cur[j].w};
                 uint32_t w8[8];
 #pragma unroll
@@ -256,11 +257,10 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     constexpr int kRows = StreamCfg<MB>::kRows;
     cg::cluster_group cluster = cg::this_cluster();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int KB = p.K / kTileK;
+    const int KB = k_blocks(p.K);
     const int rank = blockIdx.x, split = gridDim.x;
     const int tile = blockIdx.y;
     const int kb0 = (int)((long long)KB * rank / split), kb1 = (int)((long long)KB * (rank + 1) / split);
-    constexpr uint32_t kUnitBytes = kBlockBytes + kRows * kTileK;
 
     if (threadIdx.x == 0) {
         if constexpr (kRows > 1)     // start the descriptor's fetch now; the first tile load would wait for it
@@ -277,9 +277,15 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     const uint8_t* wsrc = p.w_packed + (size_t)tile * KB * kBlockBytes;
 
     // a stage's barrier expects the weight block and the activation codes; the two copies may be issued apart
+    // One row is fetched with a plain copy, which must stay inside the row: of a last block that K does
+    // not fill, only the codes that exist are copied (a multiple of 32 bytes); the rest of the stage keeps
+    // stale bytes, which meet zero weight codes. Tensor-map loads count their whole box.
+    auto x_bytes = [&](int kb) -> uint32_t {
+        return kRows == 1 ? (uint32_t)min(kTileK, p.K - kb * kTileK) : (uint32_t)(kRows * kTileK);
+    };
     auto issue_w = [&](int kb, int s) {
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
-                     ::"r"(s_u32(&sm.full[s])), "r"(kUnitBytes) : "memory");
+                     ::"r"(s_u32(&sm.full[s])), "r"((uint32_t)kBlockBytes + x_bytes(kb)) : "memory");
         asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                      ::"r"(s_u32(sm.w[s])), "l"(wsrc + (size_t)kb * kBlockBytes), "r"((uint32_t)kBlockBytes),
                        "r"(s_u32(&sm.full[s])) : "memory");
@@ -288,7 +294,7 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
         if constexpr (kRows == 1) {
             // one row: its 128 codes are contiguous, a plain bulk copy needs no tensor-map fetch
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                         ::"r"(s_u32(sm.x[s])), "l"(p.q + (size_t)kb * kTileK), "r"((uint32_t)kTileK),
+                         ::"r"(s_u32(sm.x[s])), "l"(p.q + (size_t)kb * kTileK), "r"(x_bytes(kb)),
                            "r"(s_u32(&sm.full[s])) : "memory");
         } else {
             asm volatile(
@@ -479,13 +485,9 @@ template <int MB>
 cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
     using Smem = StreamSmem<MB>;
     const size_t smem_bytes = sizeof(Smem) + 1024;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_decode_stream_kernel<MB>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    static SmemOptIn opt_in;
+    if (const cudaError_t e = opt_in.ensure(gemm_decode_stream_kernel<MB>, dev.device, smem_bytes); e != cudaSuccess)
+        return e;
     CUtensorMap map;
     const cuuint64_t dims[2] = {(cuuint64_t)a.K, (cuuint64_t)a.M};
     const cuuint64_t strides[1] = {(cuuint64_t)a.K};
@@ -508,7 +510,7 @@ cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t
     p.next_inv = ldexpf(1.0f, -a.next_exp);
     p.next_lo = -(float)(1 << (a.next_bits - 1));
     p.next_hi = (float)((1 << (a.next_bits - 1)) - 1);
-    const int tiles = p.Npad / kTileN, KB = a.K / kTileK;
+    const int tiles = p.Npad / kTileN, KB = k_blocks(a.K);
     // as many k ranges per tile (cluster size 1, 2 or 4: clusters of 7-8 measured slower) as keep
     // all CTAs resident at once (two per SM), and at least two k blocks per CTA
     int split = 1;

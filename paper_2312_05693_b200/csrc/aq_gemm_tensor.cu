@@ -288,7 +288,7 @@ gemm_tensor_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_const
     static_assert(kColsPerEpiWarp % 16 == 0 && (!GROUPED || kColsPerEpiWarp % 32 == 0), "epilogue chunking");
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int KB = p.K / kTileK;
+    const int KB = k_blocks(p.K);      // a last block that K does not fill: zero weight codes meet the tensor map's zero fill
     static_assert(!SPLIT || (GROUPED && !OFFSET && !CHAIN), "only the plain per-group kernel shares tiles");
     const int my_tiles = SPLIT ? 1
                                : (p.n_tiles > (int)blockIdx.x
@@ -671,6 +671,104 @@ role_done:
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// Rate probe: what this GPU's tensor cores deliver on kind::i8 when nothing else is in the way.
+// One CTA per SM; one thread issues `iters` rounds of four 128 x 256 x 32 MMAs on operands that
+// stay where they are (pseudo-random bytes, so that the data toggles as real codes do): both from
+// shared memory, or A from tensor memory as in the product kernel. No loads, no epilogue. Batches
+// of 32 rounds are committed to two alternating barriers and the issuer stays one batch ahead,
+// so the pipe never drains and the queue stays bounded.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ void tc_mma_i8_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+struct ProbeSmem {
+    alignas(1024) uint8_t a[128 * 128];     // 128 rows x 128 k, 128-byte swizzled rows
+    alignas(1024) uint8_t b[256 * 128];     // 256 rows x 128 k
+    alignas(8) uint64_t bar[2];
+    uint32_t tmem_base;
+    volatile uint32_t abort_flag;
+};
+
+__global__ void __launch_bounds__(128, 1) int8_probe_kernel(int iters, int a_from_tmem, Control* ctl) {
+    extern __shared__ uint8_t smem_raw[];
+    ProbeSmem& sm = *reinterpret_cast<ProbeSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint32_t* words = reinterpret_cast<uint32_t*>(sm.a);
+    for (int i = threadIdx.x; i < (int)(sizeof(sm.a) + sizeof(sm.b)) / 4; i += blockDim.x) {
+        uint32_t v = (uint32_t)i * 2654435761u + blockIdx.x * 40503u;       // any bytes will do
+        v ^= v >> 15; v *= 2246822519u; v ^= v >> 13;
+        words[i] = v;
+    }
+    fence_proxy_async();
+    if (threadIdx.x == 0) {
+        mbar_init(&sm.bar[0], 1);
+        mbar_init(&sm.bar[1], 1);
+        sm.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&sm.tmem_base)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = sm.tmem_base;
+    const uint32_t tmem_a = tmem + 256;            // after the 256 accumulator columns
+    if (a_from_tmem) {                             // 128 lanes x 32 columns of bytes for the A operand
+        uint32_t v[8];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = words[(threadIdx.x * 32 + j * 8 + i) & 4095];
+            tc_st8(tmem_a + ((uint32_t)(warp * 32) << 16) + 8 * j, v);
+        }
+        tc_wait_st();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 0 && lane == 0) {
+        constexpr uint32_t idesc = idesc_i8(128, 256);
+        constexpr int kBatch = 32;
+        const uint64_t adesc = smem_desc_sw128(smem_u32(sm.a)), bdesc = smem_desc_sw128(smem_u32(sm.b));
+        const int batches = (iters + kBatch - 1) / kBatch;
+        bool ok = true;
+        for (int bt = 0; bt < batches && ok; ++bt) {
+            if (bt >= 2) ok = mbar_wait(&sm.bar[bt & 1], (uint32_t)((bt >> 1) - 1) & 1u, &sm.abort_flag, 12u);
+            if (!ok) break;
+            const int n = min(kBatch, iters - bt * kBatch);
+            for (int it = 0; it < n; ++it) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (a_from_tmem) tc_mma_i8_ts(tmem, tmem_a + 8 * j, bdesc + (uint64_t)(2 * j), idesc, 1u);
+                    else tc_mma_i8_ss(tmem, adesc + (uint64_t)(2 * j), bdesc + (uint64_t)(2 * j), idesc, 1u);
+                }
+            }
+            tc_commit(&sm.bar[bt & 1]);
+        }
+        // drain: the last one or two batches
+        for (int bt = max(batches - 2, 0); bt < batches && ok; ++bt)
+            ok = mbar_wait(&sm.bar[bt & 1], (uint32_t)(bt >> 1) & 1u, &sm.abort_flag, 12u);
+    }
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (sm.abort_flag && threadIdx.x == 0) atomicCAS(&ctl->status, 0u, sm.abort_flag);
+    if (warp == 0)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+}
+
 // Shared tiles pay from K = 8192 on with 64- and 128-token tiles and from K = 4096 on with 192-token
 // tiles, where half a tile is worth more (see launch_bm).
 constexpr int split_min_k_blocks(int bm) { return bm >= 192 ? 32 : 64; }
@@ -686,12 +784,12 @@ inline bool round_is_shared(int rem, int sms, int k_blocks, int bm) {
 // token column and k block (about 7.6 cycles with 128-token tiles, 6.6 with 192-token tiles).
 int grouped_token_tile(int M, int K, int N, int sms, bool may_share) {
     if (M <= 64) return 64;
-    const int k_blocks = K / kTileK, n_tiles_n = round_up(N, kTileN) / kTileN;
+    const int kbs = K / kTileK, n_tiles_n = round_up(N, kTileN) / kTileN;
     auto cost = [&](int bm, float per_col) {
         const long tiles = (long)((M + bm - 1) / bm) * n_tiles_n;
         const long rounds = tiles / sms;
         const int rem = (int)(tiles % sms);
-        const float last = rem == 0 ? 0.0f : (may_share && round_is_shared(rem, sms, k_blocks, bm) ? 0.5f : 1.0f);
+        const float last = rem == 0 ? 0.0f : (may_share && round_is_shared(rem, sms, kbs, bm) ? 0.5f : 1.0f);
         return ((float)rounds + last) * (float)bm * per_col;
     };
     return cost(192, 6.6f) < cost(128, 7.6f) ? 192 : 128;
@@ -707,13 +805,10 @@ cudaError_t launch_off(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t st
                        int split_base = 0, int split_tiles = 0) {
     using Smem = SharedStorage<BM, Roles<BM, GROUPED>::kEpiWarps>;
     const size_t smem_bytes = sizeof(Smem) + 1024;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_tensor_kernel<BM, GROUPED, OFFSET, CHAIN, SPLIT>,
-                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes);
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    static SmemOptIn opt_in;
+    if (const cudaError_t e = opt_in.ensure(gemm_tensor_kernel<BM, GROUPED, OFFSET, CHAIN, SPLIT>, dev.device, smem_bytes);
+        e != cudaSuccess)
+        return e;
     CUtensorMap map;
     const cuuint64_t dims[2] = {(cuuint64_t)a.K, (cuuint64_t)a.M};
     const cuuint64_t strides[1] = {(cuuint64_t)a.K};
@@ -841,6 +936,14 @@ size_t tensor_split_scratch_bytes(int M, int K, int N, int group, int sm_count) 
     const int rem = n_tiles % sm_count;
     if (!round_is_shared(rem, sm_count, K / kTileK, bm)) return 0;
     return (size_t)rem * 2 * bm * kTileN * sizeof(float);
+}
+
+cudaError_t launch_int8_probe(int iters, int a_from_tmem, Control* ctl, const DeviceInfo& dev, cudaStream_t stream) {
+    const size_t smem_bytes = sizeof(ProbeSmem) + 1024;
+    static SmemOptIn opt_in;
+    if (const cudaError_t e = opt_in.ensure(int8_probe_kernel, dev.device, smem_bytes); e != cudaSuccess) return e;
+    int8_probe_kernel<<<dev.sm_count, 128, smem_bytes, stream>>>(iters, a_from_tmem, ctl);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_gemm_tensor(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {

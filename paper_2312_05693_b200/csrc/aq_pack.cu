@@ -34,7 +34,7 @@ pack_w4_kernel(const __half* __restrict__ w, int N, int K, int group, uint8_t* _
     __shared__ int8_t codes[kTileK];
     const int n = blockIdx.x;
     const int Npad = gridDim.x;
-    const int KB = K / kTileK;
+    const int KB = k_blocks(K);
     const int t = threadIdx.x;
     const int nt = n / kTileN, r = n % kTileN;
     const bool live = n < N;
@@ -51,7 +51,7 @@ pack_w4_kernel(const __half* __restrict__ w, int N, int K, int group, uint8_t* _
         s_row = __half2float(sh);
     }
     for (int kb = 0; kb < KB; ++kb) {
-        const float wv = live ? __half2float(row[kb * kTileK + t]) : 0.0f;
+        const float wv = (live && kb * kTileK + t < K) ? __half2float(row[kb * kTileK + t]) : 0.0f;   // k >= K: zero codes
         float s = s_row;
         if (group != 0) {
             const float a = block_max_128(fabsf(wv), red);
@@ -83,7 +83,7 @@ __global__ void unpack_w4_kernel(const uint8_t* __restrict__ packed, int N, int 
     const size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (size_t)N * K) return;
     const int n = (int)(idx / K), k = (int)(idx % K);
-    const int KB = K / kTileK;
+    const int KB = k_blocks(K);
     const int kb = k / kTileK, kl = k % kTileK;
     const int j = kl >> 5, i = (kl & 31) >> 3, p = kl & 7;
     const uint8_t byte = packed[packed_unit_offset(KB, n / kTileN, kb, j, n % kTileN) + 4 * i + (p & 3)];
@@ -96,7 +96,7 @@ __global__ void weight_offsets_kernel(const uint8_t* __restrict__ packed, const 
                                       int K, int group, float* __restrict__ r_out) {
     const int n = blockIdx.x * blockDim.x + threadIdx.x;
     if (n >= N) return;
-    const int KB = K / kTileK, Npad = round_up(N, kTileN);
+    const int KB = k_blocks(K), Npad = round_up(N, kTileN);
     const int nt = n / kTileN, r = n % kTileN;
     double total = 0.0;
     long long run = 0;

@@ -664,13 +664,9 @@ cudaError_t launch_quantize_fused(const __half* x, int M, int K, const int32_t* 
     const size_t max_cache = dev.smem_optin > reserve ? (dev.smem_optin - reserve) / 32 : 0;
     unsigned int cache_units = units_per_cta < max_cache ? units_per_cta : (unsigned int)max_cache;
     const size_t smem_bytes = (size_t)cache_units * 32;
-    static size_t attr_bytes = 0;
-    if (smem_bytes > attr_bytes) {
-        const cudaError_t e = cudaFuncSetAttribute(quantize_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   (int)(dev.smem_optin - reserve));
-        if (e != cudaSuccess) return e;
-        attr_bytes = dev.smem_optin - reserve;
-    }
+    static SmemOptIn opt_in;            // always the device's whole opt-in size: any later share fits
+    if (const cudaError_t e = opt_in.ensure(quantize_fused_kernel, dev.device, dev.smem_optin - reserve); e != cudaSuccess)
+        return e;
     const uint4* xp = reinterpret_cast<const uint4*>(x);
     uint4* qp = reinterpret_cast<uint4*>(q);
     const uint4* ap = reinterpret_cast<const uint4*>(alpha);
@@ -708,14 +704,10 @@ cudaError_t launch_quantize_asym(const __half* x, int M, int K, const int32_t* r
     const size_t max_cache = dev.smem_optin > reserve ? (dev.smem_optin - reserve) / 32 : 0;
     unsigned int cache_units = units_per_cta < max_cache ? units_per_cta : (unsigned int)max_cache;
     const size_t smem_bytes = (size_t)cache_units * 32;
-    static bool attr_done = false;
-    if (!attr_done) {
-        const cudaError_t e = cudaFuncSetAttribute(quantize_asym_fused_kernel,
-                                                   cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   (int)(dev.smem_optin - reserve));
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
+    static SmemOptIn opt_in;
+    if (const cudaError_t e = opt_in.ensure(quantize_asym_fused_kernel, dev.device, dev.smem_optin - reserve);
+        e != cudaSuccess)
+        return e;
     const uint4* xp = reinterpret_cast<const uint4*>(x);
     uint4* qp = reinterpret_cast<uint4*>(q);
     void* args[] = {&xp, &M, &units_per_row, &row_idx, &bits, &ctl, &qp, &scale_exp_out, &zero_point_out, &cache_units,

@@ -20,7 +20,7 @@ KERNELS = [pytest.param(DECODE, id="decode"), pytest.param(TENSOR, id="tensor")]
 
 # ------------------------------------------------------------------------------ weights
 @pytest.mark.parametrize("N,K,group", [(768, 768, 0), (200, 384, 128), (128, 128, 0), (1, 256, 128),
-                                       (384, 1024, 128)])
+                                       (384, 1024, 128), (200, 160, 0), (136, 96, 0), (9, 32, 0)])
 def test_pack_w4_codes_and_scales_bit_exact(N, K, group):
     w = inputs.weights(N, K, seed=N + K)
     if N > 5:
@@ -175,6 +175,30 @@ def test_linear_w4a8_matches_checker(kernel, M, K, N, group):
     assert_y_close(gpu["y"], ref["y"])
 
 
+@pytest.mark.parametrize("kernel", KERNELS)
+@pytest.mark.parametrize("M,K,N", [(1, 160, 136), (5, 96, 200), (16, 4224, 128), (140, 160, 264), (300, 4224, 384),
+                                   (70, 32, 77), (1, 32, 8), (200, 1120, 130)])
+def test_k_a_multiple_of_32_with_one_scale_per_channel(kernel, M, K, N):
+    """K % 128 != 0 (one scale per channel): the last 128-k block of the packed weights is padded with zero
+    codes, so the activation codes beyond K never count, in every product kernel."""
+    x = inputs.activations(M, K, seed=M + N + 3, outlier_frac=0.02, outlier_mult=20.0)
+    w = inputs.weights(N, K, seed=K + N + 3)
+    gpu, ref = run_layer_both(x, w, 8, 0, kernel)
+    assert gpu["e"] == ref["e"]
+    assert np.array_equal(gpu["q"], ref["q"])
+    assert np.array_equal(gpu["acc"], ref["acc"])
+    assert_y_close(gpu["y"], ref["y"])
+    # extreme codes over a ragged K: a slip in the padding would show as a wrong count of terms
+    xe = np.full((M, K), -128.0, np.float16)
+    we = np.full((N, K), -0.01, np.float16)
+    gpu, ref = run_layer_both(xe, we, 8, 0, kernel, scale_mode=1, clip=0)
+    assert np.array_equal(gpu["acc"], ref["acc"]) and ref["acc"].max() == 128 * 7 * K
+    if K % 128:
+        with pytest.raises(binding.AgileqError) as ei:      # per-group scales keep K % 128 == 0
+            handle().aq_pack_w4(dev(w), 128)
+        assert ei.value.status == binding.AQ_ERR_SHAPE
+
+
 @pytest.mark.parametrize("group", [0, 128])
 @pytest.mark.parametrize("M", [1, 2, 3, 4, 5, 8, 11, 16])
 def test_decode_rows_1_to_16(M, group):
@@ -258,7 +282,7 @@ def test_several_tiles_per_cta_and_deep_k(group):
     assert_y_close(gpu["y"], ref["y"])
 
 
-@pytest.mark.parametrize("M,N,K", [(200, 520, 8192), (380, 12800, 4096), (380, 12800, 8192)])
+@pytest.mark.parametrize("M,N,K", [(200, 520, 8192), (200, 520, 11008), (380, 12800, 4096), (380, 12800, 8192)])
 def test_shared_tiles_of_a_partial_last_round(M, N, K):
     """A last round that fills less than half of the SMs: those tiles are shared by two CTAs (half of K
     each, partial sums exchanged). 200 x 520: ten 128-token tiles, every tile is shared; 380 x 12800: two
@@ -325,6 +349,36 @@ def test_token_select_and_compact(M, ratio):
         x = inputs.activations(M, 128, seed=M + 1)
         xp = h.aq_token_compact(dev(x), dev(ref)).cpu().numpy()
         assert np.array_equal(xp.view(np.uint16), oracle.token_compact(x, ref).view(np.uint16))
+
+
+# ------------------------------------------------------------------------ device status
+def test_a_status_word_left_in_the_control_block_is_reported():
+    """Every wait inside the kernels is bounded; a wait that gives up leaves a non-zero status word in the
+    workspace's control block, which aq_check_workspace turns into AQ_ERR_DEVICE_TIMEOUT. No kernel is made
+    to wait here: the word is written from the host side, as a kernel would have left it."""
+    h = handle()
+    M, K, N = 4, 256, 128
+    ws = h.alloc_workspace(M, K, N, 0)
+    ws.zero_()
+    assert h.aq_check_workspace(ws) == binding.AQ_OK
+    status = ws[8:12].view(torch.int32)              # Control::status
+    for code in (1, 7, 10):
+        status.fill_(code)
+        assert h.aq_check_workspace(ws) == binding.AQ_ERR_DEVICE_TIMEOUT
+        assert "bounded wait" in binding.status_string(binding.AQ_ERR_DEVICE_TIMEOUT)
+    status.fill_(11)                                  # the attention kernel's "negative code" report
+    assert h.aq_check_workspace(ws) == binding.AQ_ERR_INVALID_ARG
+    # the next call on the workspace starts from a clean record
+    x = dev(inputs.activations(M, K, seed=1))
+    packed, scales = h.aq_pack_w4(dev(inputs.weights(N, K, seed=2)), 0)
+    for kernel in (DECODE, TENSOR):
+        status.fill_(5)
+        h.aq_set_kernel(kernel)
+        try:
+            h.aq_linear_w4a8(x, packed, scales, N, 0, workspace=ws)
+            assert h.aq_check_workspace(ws) == binding.AQ_OK
+        finally:
+            h.aq_set_kernel(binding.AQ_KERNEL_AUTO)
 
 
 # --------------------------------------------------------------------- argument checking

@@ -277,29 +277,28 @@ def test_int_gemm_linearity_and_library_matmul():
     assert np.array_equal(a1.sum(axis=2), oracle.int_gemm(q1, c, 0)[:, :, 0])
 
 
-def test_int_gemm_agrees_with_packed_lane_products():
-    """Sec. 4.4 'INT4 Multiplier' / Algorithm 1: two unsigned 4-bit weights sit in one
-    16-bit lane (8 bits each), one multiply by the shared activation gives both products,
-    a shift-or-mask (0x00FF00FF) spreads them into the two 16-bit halves of a 32-bit word,
-    and up to 2^8 such words are summed without overflow. Restated here on unsigned 4-bit
-    operands as an independent route to the same integer sums."""
+def test_int_gemm_two_sums_share_one_word_without_carry():
+    """Sec. 4.4 'INT4 Multiplier': two sums of unsigned 4-bit products can live side by side in one
+    32-bit word as long as the reduction is at most 2^8 long. The property behind it, checked here
+    against the checker's sums: each sum is at most 15 * 15 * 256 = 57600 < 2^16, so the word
+    s0 + 2^16 * s1, built in plain integers, splits back into the two sums with no carry from the low
+    field into the high one, also at the extreme (every operand 15); one more doubling of the
+    reduction (512 terms of 225 = 115200 > 2^16) would carry, which is why the limit is 2^8."""
     rng = np.random.default_rng(4)
-    K = 256                                   # the paper's overflow-free limit
-    a = rng.integers(0, 16, size=(3, K))      # unsigned 4-bit activations
-    w0 = rng.integers(0, 16, size=(K,))       # two adjacent output channels
-    w1 = rng.integers(0, 16, size=(K,))
-    w0[:8] = 15
-    a[0, :8] = 15                             # largest product 225 fits its 8-bit field
-    c = np.stack([w0, w1]).astype(np.int8)
-    for m in range(3):
-        acc32 = 0
-        for k in range(K):
-            lane = int(w0[k]) | (int(w1[k]) << 8)
-            p = (lane * int(a[m, k])) & 0xFFFF            # one multiply, two products
-            p = (p | (p << 8)) & 0x00FF00FF               # rearrangement + mask
-            acc32 = (acc32 + p) & 0xFFFFFFFF              # 32-bit accumulation
-        ref = oracle.int_gemm(a[m:m + 1].astype(np.int8), c, 0)[0, :, 0]
-        assert int(ref[0]) == (acc32 & 0xFFFF) and int(ref[1]) == (acc32 >> 16)
+    K = 256
+    assert 15 * 15 * K < 1 << 16 <= 15 * 15 * 2 * K
+    a = rng.integers(0, 16, size=(4, K))
+    w = rng.integers(0, 16, size=(2, K))
+    a[0, :] = 15
+    w[0, :] = 15                              # row 0 x channel 0 reaches the bound exactly
+    sums = oracle.int_gemm(a.astype(np.int8), w.astype(np.int8), 0)[:, :, 0]
+    assert int(sums[0, 0]) == 15 * 15 * K
+    for m in range(4):
+        s0 = sum(int(a[m, k]) * int(w[0, k]) for k in range(K))       # per-field sums, plain integers
+        s1 = sum(int(a[m, k]) * int(w[1, k]) for k in range(K))
+        word = s0 + (s1 << 16)
+        assert word < 1 << 32
+        assert (word & 0xFFFF, word >> 16) == (int(sums[m, 0]), int(sums[m, 1]))
 
 
 # ----------------------------------------------------------------------------- dequant
