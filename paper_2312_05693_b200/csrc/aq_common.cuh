@@ -198,9 +198,6 @@ int handle_device(aq_handle_t h);
 void handle_record_cuda_error(aq_handle_t h, cudaError_t e);
 
 cudaError_t launch_gemm_tensor(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream);
-// Per-group scales (aq_gemm_grouped.cu); split_scratch / split_bytes hold the partial outputs of shared tiles.
-cudaError_t launch_gemm_grouped(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream);
-size_t grouped_scratch_bytes(int M, int K, int N, int sm_count);
 // Bytes of split_scratch the tensor kernel can use for these sizes on a GPU with sm_count SMs (0: none).
 size_t tensor_split_scratch_bytes(int M, int K, int N, int group, int sm_count);
 // Tensor-core rate probe: every SM issues iters x 4 MMAs of 128 x 256 x 32 (int8) on resident operands.

@@ -801,7 +801,6 @@ cudaError_t launch_bm(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t str
 
 size_t tensor_split_scratch_bytes(int M, int K, int N, int group, int sm_count) {
     if (!group) return 0;
-    return grouped_scratch_bytes(M, K, N, sm_count);
     const int bm = grouped_token_tile(M, K, N, sm_count, true);
     const int n_tiles = ((M + bm - 1) / bm) * (round_up(N, kTileN) / kTileN);
     const int rem = n_tiles % sm_count;
@@ -818,7 +817,6 @@ cudaError_t launch_int8_probe(int iters, int a_from_tmem, Control* ctl, const De
 }
 
 cudaError_t launch_gemm_tensor(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
-    if (a.group) return launch_gemm_grouped(a, dev, stream);
     if (a.M <= 64) return a.group ? launch_bm<64, true>(a, dev, stream) : launch_bm<64, false>(a, dev, stream);
     if (a.group) {
         // the chained and zero-point variants have no shared-tile launch
