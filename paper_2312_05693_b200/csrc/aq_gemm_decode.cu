@@ -223,7 +223,8 @@ struct StreamSmem {
     alignas(1024) int8_t x[kStrStages][kRows * kTileK];    // activation codes of the unit's k block
     alignas(128) uint8_t w[kStrStages][kBlockBytes];       // packed weight block of the unit
     int part[4][kRows][32];                                // the odd-k-block warp's partial sums
-    int sum[kRows][kTileN];                                // this CTA's sums over its k range
+    alignas(16) int sum[kRows][kTileN];                    // this CTA's sums over its k range
+    alignas(16) int recv[kRows][kTileN];                               // the other CTAs' sums for this CTA's channel slice, by sender
     alignas(8) uint64_t full[kStrStages];
     uint64_t empty[kStrStages];
     volatile uint32_t abort_flag;
@@ -262,6 +263,9 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     const int tile = blockIdx.y;
     const int kb0 = (int)((long long)KB * rank / split), kb1 = (int)((long long)KB * (rank + 1) / split);
 
+    // First meeting of the cluster, arrival only: by the time a CTA writes into another's shared memory
+    // (after its k range) every CTA of the cluster has started. The wait comes just before those writes.
+    if (split > 1) asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
     if (threadIdx.x == 0) {
         if constexpr (kRows > 1)     // start the descriptor's fetch now; the first tile load would wait for it
             asm volatile("prefetch.tensormap [%0];" ::"l"(&x_map) : "memory");
@@ -305,12 +309,16 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     // The weights do not depend on the kernel before this one: the first ring of weight blocks is on its
     // way before this grid waits for that kernel (a no-op unless the launch allowed the overlap), and only
     // then are the status word, the codes, the exponent and the offsets touched.
+    // Launched with programmatic stream serialization: this grid may have been set up while the kernel
+    // before it on the stream still ran. Nothing written before this launch is read, and nothing is written,
+    // until that kernel has completed; only behind the call's own quantize kernel (which was launched
+    // normally, after everything before it, weight packing included) the weights are fetched first.
     int issued = 0;
     if (!p.clear_status) {                            // launched behind this call's own quantize kernel
         if (warp == 0 && lane == 0)
             for (; issued < kStrStages && kb0 + issued < kb1; ++issued) issue_w(kb0 + issued, issued);
-        asm volatile("griddepcontrol.wait;" ::: "memory");
     }
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (p.clear_status && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) p.ctl->status = 0;   // nothing has given up yet
     if (warp == 0) {
         if (lane == 0) {
@@ -436,9 +444,11 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
             }
         }
     }
-    // Every CTA of the cluster now holds the tile's sums over its own k range. After the cluster meets,
-    // CTA `rank` finishes a slice of 128 / split channels: it reads that slice of every CTA's sums over
-    // distributed shared memory (integer addition is exact in any order), scales and writes the outputs.
+    // Every CTA of the cluster now holds the tile's sums over its own k range, and CTA `rank` finishes the
+    // slice of 128 / split channels [rank, rank + 1) * cw: every CTA writes its sums of the other slices into
+    // their owners' shared memory (slot = sender), the cluster meets once, and every CTA adds what it received
+    // to its own sums (integer addition is exact in any order), scales and writes its outputs. After the
+    // meeting nobody touches another CTA's memory, so a CTA may leave as soon as it is done.
     // The scale is fetched before the cluster meets so that its latency overlaps the wait.
     const int cw = kTileN / split;                            // split is 1, 2 or 4
     const int ft = (int)threadIdx.x - 32;                     // the 256 consumer threads finish; cw divides 256
@@ -450,16 +460,30 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
         sc = __half2float(p.w_scales[out_n]) * pe;
         if (p.chan_offset) off = p.chan_offset[out_n] * pe;
     }
-    if (split > 1) cluster.sync(); else __syncthreads();
+    const int rows = p.M < kRows ? p.M : kRows;
+    if (split > 1) {
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");     // everybody has started (arrival at the top)
+        __syncthreads();                                      // this CTA's sums are complete
+        if (ft >= 0) {
+            // four consecutive channels at a time (16-byte remote stores) go to the CTA that owns them
+            for (int e = ft; e < rows * (kTileN / 4); e += kStrConsumerWarps * 32) {
+                const int m = e / (kTileN / 4), ch = 4 * (e % (kTileN / 4));
+                const int owner = ch / cw;
+                if (owner != rank)
+                    *reinterpret_cast<int4*>(cluster.map_shared_rank(&sm.recv[0][0], owner) + m * kTileN + rank * cw + (ch % cw)) =
+                        *reinterpret_cast<const int4*>(&sm.sum[m][ch]);
+            }
+        }
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    } else {
+        __syncthreads();
+    }
     if (ft >= 0 && out_n < p.N) {
-        const int* src[4];
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-            src[c] = (split > 1 && c < split) ? cluster.map_shared_rank(&sm.sum[0][0], c) : &sm.sum[0][0];
-        for (int m = ft / cw; m < p.M && m < kRows; m += (kStrConsumerWarps * 32) / cw) {
-            int a = src[0][m * kTileN + out_r];
-            if (split > 1) a += src[1][m * kTileN + out_r];
-            if (split > 2) a += src[2][m * kTileN + out_r] + src[3][m * kTileN + out_r];
+        for (int m = ft / cw; m < rows; m += (kStrConsumerWarps * 32) / cw) {
+            int a = sm.sum[m][out_r];
+            for (int c = 0; c < split; ++c)
+                if (c != rank) a += sm.recv[m][c * cw + (out_r % cw)];
             a >>= 4;                                              // sums carry a factor 16
             if (p.acc_dump) p.acc_dump[(size_t)m * p.N + out_n] = a;
             const __half hv = __float2half_rn(fmaf((float)a, sc, off));
@@ -470,7 +494,6 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
             else p.y[(size_t)m * p.N + out_n] = hv;
         }
     }
-    if (split > 1) cluster.sync();                            // nobody leaves while its sums may still be read
     if (sm.abort_flag) {
         for (int i = 0; i < 64; ++i) __nanosleep(1000);          // let copies in flight land
         if (threadIdx.x == 0) atomicOr(&p.ctl->status, 1u);
@@ -528,7 +551,7 @@ cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = a.after_quantize ? 2 : 1;
+    cfg.numAttrs = 2;       // the kernel reads and writes nothing before the kernel ahead of it has completed
     return cudaLaunchKernelEx(&cfg, gemm_decode_stream_kernel<MB>, map, p);
 }
 
