@@ -127,8 +127,12 @@ int linear_impl(aq_handle_t h, int bits, const void* x, int M, int K, const void
     const Workspace w = carve(workspace, M, K, N, workspace_bytes_);
     const __half* xh = static_cast<const __half*>(x);
     if (alpha && !aligned(alpha, 16)) return AQ_ERR_ALIGNMENT;
-    cudaError_t e;
-    if (w_offsets) {
+    cudaError_t e = cudaSuccess;
+    // a single row on the few-row kernel: that kernel finds the scale and makes the codes itself
+    const bool fuse = !w_offsets && !alpha && kernel_for(h, M) == AQ_KERNEL_DECODE &&
+                      decode_can_fuse_quantize(M, K, N, group, h->dev.sm_count);
+    if (fuse) {
+    } else if (w_offsets) {
         // zero-point variant: min / max, then e, zp and codes; then the per-channel term -(zp - 2^(b-1)) * r[n]
         if (!aligned(w_offsets, 4)) return AQ_ERR_ALIGNMENT;
         e = cudaMemsetAsync(w.ctl, 0, sizeof(Control), stream);
@@ -152,7 +156,11 @@ int linear_impl(aq_handle_t h, int bits, const void* x, int M, int K, const void
     g.chan_offset = w_offsets ? w.chan_offset : nullptr;
     g.q_next = q_next; g.next_bits = next_bits; g.next_exp = next_exp;
     g.next_packed = next_packed;
-    g.after_quantize = true;
+    g.after_quantize = !fuse;
+    if (fuse) {
+        g.fuse_x = xh; g.fuse_row_idx = row_idx; g.fuse_bits = bits; g.fuse_scale_mode = scale_mode;
+        g.fuse_clip_shift_or_exp = clip_shift_or_exp;
+    }
     return run_gemm(h, g, stream);
 }
 

@@ -190,6 +190,11 @@ struct GemmArgs {
     // fp32 partial outputs of tiles whose k range two CTAs share (tensor kernel, per-group scales)
     float* split_scratch = nullptr;
     size_t split_bytes = 0;
+    // One row (M = 1): the few-row streaming kernel quantizes the activations itself (no quantize kernel runs
+    // ahead); q then receives the codes, the control block the exponent.
+    const __half* fuse_x = nullptr;
+    const int32_t* fuse_row_idx = nullptr;
+    int fuse_bits = 8, fuse_scale_mode = 0, fuse_clip_shift_or_exp = 0;
     void* scratch;          // beyond control block + codes
     size_t scratch_bytes;
 };
@@ -203,5 +208,6 @@ size_t tensor_split_scratch_bytes(int M, int K, int N, int group, int sm_count);
 // Tensor-core rate probe: every SM issues iters x 4 MMAs of 128 x 256 x 32 (int8) on resident operands.
 cudaError_t launch_int8_probe(int iters, int a_from_tmem, Control* ctl, const DeviceInfo& dev, cudaStream_t stream);
 cudaError_t launch_gemm_decode(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream);
+bool decode_can_fuse_quantize(int M, int K, int N, int group, int sm_count);
 
 }  // namespace aq

@@ -17,6 +17,7 @@
 #include <cuda.h>
 
 #include "aq_common.cuh"
+#include "aq_quant_math.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -184,6 +185,7 @@ constexpr int kStrStages = 8;
 constexpr int kStrConsumerWarps = 8;
 constexpr int kStrThreads = (1 + kStrConsumerWarps) * 32;
 constexpr unsigned long long kStrWaitCycles = 4000000000ull;
+constexpr int kFuseMaxBlocks = 64;        // k blocks per CTA up to which a single row is quantized inside the product kernel
 
 __device__ __forceinline__ uint32_t s_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ bool str_try_wait(uint64_t* bar, uint32_t parity) {
@@ -224,6 +226,9 @@ struct StreamSmem {
     alignas(128) uint8_t w[kStrStages][kBlockBytes];       // packed weight block of the unit
     int part[4][kRows][32];                                // the odd-k-block warp's partial sums
     alignas(16) int sum[kRows][kTileN];                    // this CTA's sums over its k range
+    // one row quantized by the kernel itself: the codes of this CTA's k range (up to kFuseMaxBlocks blocks)
+    alignas(16) int8_t xq[MB == 1 ? kFuseMaxBlocks * kTileK : 16];
+    unsigned int warp_max[kStrThreads / 32];
     alignas(16) int recv[kRows][kTileN];                               // the other CTAs' sums for this CTA's channel slice, by sender
     alignas(8) uint64_t full[kStrStages];
     uint64_t empty[kStrStages];
@@ -244,13 +249,20 @@ struct StreamParams {
     float next_inv, next_lo, next_hi;
     int clear_status;
     int next_packed;
+    // FUSEQ (one row): the activations themselves; the kernel finds the layer scale, writes the codes of
+    // its k range to shared memory (and, from the first channel tile, to q_out) and fills the control block
+    const __half* x_row;           // the row's K halves
+    const int32_t* row_idx;        // NULL or one index: the row is x_row + row_idx[0] * K
+    int8_t* q_out;                 // [K] codes
+    int bits, scale_mode, clip_shift_or_exp;
 };
 
 // grid = (split, channel tiles), cluster = (split, 1, 1): the CTAs of a cluster share a channel
 // tile and take consecutive k ranges; CTA r adds up and writes channels [r, r+1) * 128 / split.
-template <int MB>
+template <int MB, bool FUSEQ = false>
 __global__ void __launch_bounds__(kStrThreads, 2)
 gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const StreamParams p) {
+    static_assert(!FUSEQ || MB == 1, "only a single row is quantized inside the product kernel");
     extern __shared__ uint8_t smem_raw[];
     using Smem = StreamSmem<MB>;
     Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -285,6 +297,7 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     // not fill, only the codes that exist are copied (a multiple of 32 bytes); the rest of the stage keeps
     // stale bytes, which meet zero weight codes. Tensor-map loads count their whole box.
     auto x_bytes = [&](int kb) -> uint32_t {
+        if (FUSEQ) return 0u;                          // the codes are made here, not copied
         return kRows == 1 ? (uint32_t)min(kTileK, p.K - kb * kTileK) : (uint32_t)(kRows * kTileK);
     };
     auto issue_w = [&](int kb, int s) {
@@ -295,7 +308,8 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
                        "r"(s_u32(&sm.full[s])) : "memory");
     };
     auto issue_x = [&](int kb, int s) {
-        if constexpr (kRows == 1) {
+        if constexpr (FUSEQ) {
+        } else if constexpr (kRows == 1) {
             // one row: its 128 codes are contiguous, a plain bulk copy needs no tensor-map fetch
             asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                          ::"r"(s_u32(sm.x[s])), "l"(p.q + (size_t)kb * kTileK), "r"(x_bytes(kb)),
@@ -320,6 +334,83 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (p.clear_status && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) p.ctl->status = 0;   // nothing has given up yet
+    [[maybe_unused]] int fused_exp = 0;
+    if constexpr (FUSEQ) {
+        // ---- the layer scale and this CTA's codes (Eq. 1, Eq. 2 / Eq. 5 with zp = 0; one scale for the layer)
+        if (warp == 0 && lane == 0)
+            for (; issued < kStrStages && kb0 + issued < kb1; ++issued) issue_w(kb0 + issued, issued);   // weights on their way meanwhile
+        const uint4* xv = reinterpret_cast<const uint4*>(p.x_row + (p.row_idx ? (size_t)p.row_idx[0] * p.K : 0));
+        int e = p.clip_shift_or_exp;
+        // up to kKeep vectors per thread stay in registers between the two passes (K <= 18432); longer rows
+        // are read again (from L2) for the codes
+        constexpr int kKeep = 8;
+        uint4 keep[kKeep];
+        const int n_vec = p.K / 8;
+        const bool kept = n_vec <= kKeep * kStrThreads;
+        if (p.scale_mode == AQ_SCALE_DYNAMIC || kept) {
+            __half2 m2 = __float2half2_rn(0.0f);
+            if (kept) {
+#pragma unroll
+                for (int i = 0; i < kKeep; ++i) {
+                    const int v = (int)threadIdx.x + i * kStrThreads;
+                    keep[i] = v < n_vec ? __ldg(xv + v) : make_uint4(0, 0, 0, 0);
+                }
+#pragma unroll
+                for (int i = 0; i < kKeep; ++i) {
+                    const __half2* h = reinterpret_cast<const __half2*>(&keep[i]);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) m2 = __hmax2(m2, __habs2(h[k]));   // NaN operands are dropped
+                }
+            } else {
+                for (int v = (int)threadIdx.x; v < n_vec; v += kStrThreads) {
+                    const uint4 d = __ldg(xv + v);
+                    const __half2* h = reinterpret_cast<const __half2*>(&d);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) m2 = __hmax2(m2, __habs2(h[k]));
+                }
+            }
+            unsigned int bmax = max((unsigned int)__half_as_ushort(__low2half(m2)), (unsigned int)__half_as_ushort(__high2half(m2)));
+            if (bmax > 0x7C00u) bmax = 0;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) bmax = max(bmax, __shfl_xor_sync(0xFFFFFFFFu, bmax, o));
+            if (lane == 0) sm.warp_max[warp] = bmax;
+            __syncthreads();
+            unsigned int all = 0;
+#pragma unroll
+            for (int w = 0; w < kStrThreads / 32; ++w) all = max(all, sm.warp_max[w]);
+            if (p.scale_mode == AQ_SCALE_DYNAMIC) {
+                e = layer_exponent_from_bits(all, p.bits) - p.clip_shift_or_exp;
+                if (tile == 0 && rank == 0 && threadIdx.x == 0) p.ctl->absmax_bits = all;
+            }
+        }
+        if (tile == 0 && rank == 0) {
+            if (threadIdx.x == 0) { p.ctl->scale_exp = e; p.ctl->status = 0; p.ctl->counter = 0; }
+            if (threadIdx.x < 57) p.ctl->split_flags[threadIdx.x] = 0;
+        }
+        const float lo = -(float)(1 << (p.bits - 1)), hi = (float)((1 << (p.bits - 1)) - 1);
+        const int v0 = kb0 * (kTileK / 8), v1 = min(kb1 * (kTileK / 8), p.K / 8);       // 8-element vectors of this k range
+        const bool fast = e >= -14 && e <= 14;             // 2^-e is a normal half: codes in half2 arithmetic
+        const __half2 inv2 = __float2half2_rn(fast ? __int_as_float((127 - e) << 23) : 1.0f);
+        const __half2 lo2 = __float2half2_rn(lo), hi2 = __float2half2_rn(hi);
+        auto code8 = [&](const uint4& d, int v) {
+            uint2 c;
+            if (fast) quantize8_half2(d, inv2, lo2, hi2, c.x, c.y);
+            else c = quantize8_fp32(d, e, lo, hi, nullptr);
+            reinterpret_cast<uint2*>(sm.xq)[v - v0] = c;
+            if (tile == 0) reinterpret_cast<uint2*>(p.q_out)[v] = c;
+        };
+        if (kept) {
+#pragma unroll
+            for (int i = 0; i < kKeep; ++i) {
+                const int v = (int)threadIdx.x + i * kStrThreads;
+                if (v >= v0 && v < v1) code8(keep[i], v);
+            }
+        } else {
+            for (int v = v0 + (int)threadIdx.x; v < v1; v += kStrThreads) code8(__ldg(xv + v), v);
+        }
+        fused_exp = e;
+        __syncthreads();
+    }
     if (warp == 0) {
         if (lane == 0) {
             for (int i = 0; i < issued; ++i) issue_x(kb0 + i, i);
@@ -355,7 +446,8 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
                     }
 #pragma unroll
                     for (int m = 0; m < MB; ++m) {
-                        const uint4* xp = reinterpret_cast<const uint4*>(sm.x[s] + m * kTileK + 32 * j);
+                        const uint4* xp = FUSEQ ? reinterpret_cast<const uint4*>(sm.xq + (size_t)(kb - kb0) * kTileK + 32 * j)
+                                                : reinterpret_cast<const uint4*>(sm.x[s] + m * kTileK + 32 * j);
                         const uint4 x0 = xp[0], x1 = xp[1];              // same address in every lane: broadcast
                         int a = acc[m];
                         a = __dp4a((int)w8[0], (int)x0.x, a);
@@ -448,7 +540,9 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     // slice of 128 / split channels [rank, rank + 1) * cw: every CTA writes its sums of the other slices into
     // their owners' shared memory (slot = sender), the cluster meets once, and every CTA adds what it received
     // to its own sums (integer addition is exact in any order), scales and writes its outputs. After the
-    // meeting nobody touches another CTA's memory, so a CTA may leave as soon as it is done.
+    // meeting nobody touches another CTA's memory, so a CTA may leave as soon as it is done. (Reading the
+    // other CTAs' sums over distributed shared memory instead, with a second meeting before anybody leaves,
+    // measured 0.1-0.5 us slower at every row count.)
     // The scale is fetched before the cluster meets so that its latency overlaps the wait.
     const int cw = kTileN / split;                            // split is 1, 2 or 4
     const int ft = (int)threadIdx.x - 32;                     // the 256 consumer threads finish; cw divides 256
@@ -456,7 +550,7 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     const int out_n = tile * kTileN + out_r;
     float sc = 0.0f, off = 0.0f;
     if (ft >= 0 && out_n < p.N) {
-        const float pe = __int_as_float((127 + *p.scale_exp) << 23);
+        const float pe = __int_as_float((127 + (FUSEQ ? fused_exp : *p.scale_exp)) << 23);
         sc = __half2float(p.w_scales[out_n]) * pe;
         if (p.chan_offset) off = p.chan_offset[out_n] * pe;
     }
@@ -504,12 +598,12 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-template <int MB>
+template <int MB, bool FUSEQ = false>
 cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
     using Smem = StreamSmem<MB>;
     const size_t smem_bytes = sizeof(Smem) + 1024;
     static SmemOptIn opt_in;
-    if (const cudaError_t e = opt_in.ensure(gemm_decode_stream_kernel<MB>, dev.device, smem_bytes); e != cudaSuccess)
+    if (const cudaError_t e = opt_in.ensure(gemm_decode_stream_kernel<MB, FUSEQ>, dev.device, smem_bytes); e != cudaSuccess)
         return e;
     CUtensorMap map;
     const cuuint64_t dims[2] = {(cuuint64_t)a.K, (cuuint64_t)a.M};
@@ -533,6 +627,9 @@ cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t
     p.next_inv = ldexpf(1.0f, -a.next_exp);
     p.next_lo = -(float)(1 << (a.next_bits - 1));
     p.next_hi = (float)((1 << (a.next_bits - 1)) - 1);
+    p.x_row = a.fuse_x; p.row_idx = a.fuse_row_idx; p.q_out = const_cast<int8_t*>(a.q);
+    p.bits = a.fuse_bits; p.scale_mode = a.fuse_scale_mode; p.clip_shift_or_exp = a.fuse_clip_shift_or_exp;
+    if (FUSEQ) p.clear_status = 1;       // no quantize kernel of this call runs ahead: nothing is fetched before the wait
     const int tiles = p.Npad / kTileN, KB = k_blocks(a.K);
     // as many k ranges per tile (cluster size 1, 2 or 4: clusters of 7-8 measured slower) as keep
     // all CTAs resident at once (two per SM), and at least two k blocks per CTA
@@ -552,7 +649,7 @@ cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;       // the kernel reads and writes nothing before the kernel ahead of it has completed
-    return cudaLaunchKernelEx(&cfg, gemm_decode_stream_kernel<MB>, map, p);
+    return cudaLaunchKernelEx(&cfg, gemm_decode_stream_kernel<MB, FUSEQ>, map, p);
 }
 
 template <int MB>
@@ -574,10 +671,21 @@ cudaError_t launch_mb(const GemmArgs& a, cudaStream_t stream) {
 
 }  // namespace
 
+// One row, one scale per channel, and a k range per CTA that fits the kernel's code buffer: the product
+// kernel can quantize the row itself (one launch for the layer).
+bool decode_can_fuse_quantize(int M, int K, int N, int group, int sm_count) {
+    if (M != 1 || group) return false;
+    const int tiles = round_up(N, kTileN) / kTileN, KB = k_blocks(K);
+    int split = 1;
+    while (split < 4 && tiles * split * 2 <= 2 * sm_count && KB / (split * 2) >= 2) split *= 2;
+    return (KB + split - 1) / split + 1 <= kFuseMaxBlocks;
+}
+
 cudaError_t launch_gemm_decode(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
     if (!a.group && a.M <= 16) {
         // one row: dp4a; 2..16 rows: the warp MMA on a 16-row tile (fewer instructions per weight
         // chunk than dp4a from two rows on; measured faster at M = 4)
+        if (a.M <= 1 && a.fuse_x) return launch_stream<1, true>(a, dev, stream);
         if (a.M <= 1) return launch_stream<1>(a, dev, stream);
         return launch_stream<16>(a, dev, stream);
     }
