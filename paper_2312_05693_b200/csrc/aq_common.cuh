@@ -203,6 +203,9 @@ int handle_device(aq_handle_t h);
 void handle_record_cuda_error(aq_handle_t h, cudaError_t e);
 
 cudaError_t launch_gemm_tensor(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream);
+// One scale per channel on tiles of 256 channels x 128 tokens (aq_gemm_wide.cu), for shapes it applies to.
+bool gemm_wide_applies(const GemmArgs& a);
+cudaError_t launch_gemm_wide(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream);
 // Bytes of split_scratch the tensor kernel can use for these sizes on a GPU with sm_count SMs (0: none).
 size_t tensor_split_scratch_bytes(int M, int K, int N, int group, int sm_count);
 // Tensor-core rate probe: every SM issues iters x 4 MMAs of 128 x 256 x 32 (int8) on resident operands.

@@ -826,6 +826,8 @@ cudaError_t launch_gemm_tensor(const GemmArgs& a, const DeviceInfo& dev, cudaStr
             default: return launch_bm<128, true>(a, dev, stream);
         }
     }
+    // one scale per channel: two channel blocks share a 128-token activation tile where the shape allows it
+    if (gemm_wide_applies(a)) return launch_gemm_wide(a, dev, stream);
     // one scale per channel: the 256-token tile halves the MMA instructions per unit of work
     if (a.M <= 128) return launch_bm<128, false>(a, dev, stream);
     return launch_bm<256, false>(a, dev, stream);
