@@ -1,12 +1,13 @@
-// Integer product with one scale per output channel (Sec. 4.4) on tiles of 256 channels x 128 tokens.
+// Integer product with one scale per output channel (Sec. 4.4) on tiles of 256 channels x 128 or 192 tokens.
 //
 // The per-channel kernel of aq_gemm_tensor.cu moves 40 KB from L2 per 128-k block and SM (a 256-token
 // activation tile and one packed 128-channel weight block) and runs within 20 % of what the L2 -> SM path
 // delivers for that pattern. Here a CTA's tile covers TWO adjacent 128-channel blocks that share one
-// 128-token activation tile: 32 KB per k block for the same number of products, so the same path feeds a
-// fifth more work. The two channel halves are two accumulators of 128 columns in tensor memory, each fed
-// by its own MMA-issuing thread (N = 128 instructions) from its own weight slices, which its own group of
-// four unpack warps writes; the activation tile in shared memory is the B operand of both.
+// activation tile of 128 or 192 tokens: 32 KB per k block for the products of 40 KB there, or 40 KB for one
+// and a half times as many, so the same path feeds a fifth to a half more work. The two channel halves are
+// two accumulators in tensor memory, each fed by its own MMA-issuing thread from its own weight slices, which
+// its own group of four unpack warps writes; the activation tile in shared memory is the B operand of both.
+// Each half has its own pair of accumulator barriers: the epilogue takes the halves one after the other.
 // Roles: warp 0 = TMA producer of the activation tiles, warp 2 = of the two weight blocks, warps 1 and 3 =
 // MMA issuers (half 0 / half 1), warps 4-7 and 8-11 = unpack (half 0 / half 1), warps 12-19 = epilogue.
 // Needs an even number of 128-channel blocks; other shapes take the kernel of aq_gemm_tensor.cu.
@@ -24,22 +25,28 @@ constexpr int kWFirstUnpack = 4, kWFirstEpi = 12, kWEpiWarps = 8;
 constexpr int kWRegsControl = 40, kWRegsUnpack = 48, kWRegsEpi = 168;     // of the 96 x 640 the launch allocates
 static_assert(128 * kWRegsControl + 256 * kWRegsUnpack + 256 * kWRegsEpi <= kWThreads * 96,
               "register plan exceeds the launch allocation");
-constexpr int kWBM = 128;                 // tokens per tile
-constexpr int kWStages = 6;               // shared-memory ring: activation tile + two packed weight blocks per stage
-constexpr int kWSlices = 8;               // weight slices in tensor memory: (k block, half) pairs, four k blocks deep
-constexpr int kWAccCols = 2 * kWBM;       // two accumulators (one per channel half)
 constexpr int kWStageRows = 32;           // tokens per TMA store of an epilogue warp
+template <int BM>
+struct WCfg {
+    static constexpr int kStages = BM == 128 ? 6 : 5;          // shared-memory ring: activation tile + two packed weight blocks per stage
+    static constexpr int kSlices = (512 - 2 * BM) / 32;        // weight slices in tensor memory: (k block, half) pairs: 8 or 4
+    static constexpr int kAccCols = 2 * BM;                    // two accumulators (one per channel half)
+    static constexpr int kCols = BM / 2;                       // token columns of one epilogue warp (per half)
+    static_assert(kCols % kWStageRows == 0 && kCols <= 96, "epilogue register plan");
+};
 
+template <int BM>
 struct WSmem {
-    alignas(1024) uint8_t x[kWStages][kWBM * 128];             // activation tiles, 128-byte swizzled rows
-    alignas(128) uint8_t w[kWStages][2][kBlockBytes];          // the two packed weight blocks of a k block
+    static constexpr int kStages = WCfg<BM>::kStages;
+    alignas(1024) uint8_t x[kStages][BM * 128];                // activation tiles, 128-byte swizzled rows
+    alignas(128) uint8_t w[kStages][2][kBlockBytes];           // the two packed weight blocks of a k block
     alignas(128) __half ystage[kWEpiWarps][kWStageRows][32];
-    alignas(8) uint64_t tma_full[kWStages];                    // both producers' bytes landed -> unpack warps
-    uint64_t smem_empty[kWStages];                             // both halves' MMAs done -> TMA producers
-    uint64_t a_full[kWSlices];                                 // a half's unpack warps stored the slice -> its MMA issuer
-    uint64_t a_empty[kWSlices];                                // MMA done with the slice -> unpack warps
-    uint64_t acc_full;                                         // both issuers' last MMAs of the tile done -> epilogue
-    uint64_t acc_empty;                                        // epilogue has the sums in registers -> issuers
+    alignas(8) uint64_t tma_full[kStages];                     // both producers' bytes landed -> unpack warps
+    uint64_t smem_empty[kStages];                              // both halves' MMAs done -> TMA producers
+    uint64_t a_full[8];                                        // a half's unpack warps stored the slice -> its MMA issuer
+    uint64_t a_empty[8];                                       // MMA done with the slice -> unpack warps
+    uint64_t acc_full[2];                                      // a half's last MMAs of the tile done -> epilogue
+    uint64_t acc_empty[2];                                     // epilogue has the half's sums in registers -> its issuer
     uint32_t tmem_base;
     volatile uint32_t abort_flag;
 };
@@ -76,11 +83,14 @@ __device__ __forceinline__ void w_stage_code(__half* stage, int c, int lane, int
 
 // OFFSET: add the per-channel term of the zero-point variant. CHAIN: write the next layer's codes instead
 // of fp16 outputs.
-template <bool OFFSET, bool CHAIN>
+template <int BM, bool OFFSET, bool CHAIN>
 __global__ void __launch_bounds__(kWThreads, 1)
 gemm_wide_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constant__ CUtensorMap y_map, const WParams p) {
     extern __shared__ uint8_t smem_raw[];
-    WSmem& sm = *reinterpret_cast<WSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    using Smem = WSmem<BM>;
+    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    constexpr int kWBM = BM, kWStages = WCfg<BM>::kStages, kWSlices = WCfg<BM>::kSlices, kWAccCols = WCfg<BM>::kAccCols;
+    constexpr int kCols = WCfg<BM>::kCols;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KB = p.KB;
     const int my_tiles = p.n_tiles > (int)blockIdx.x ? (p.n_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
@@ -95,8 +105,10 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
             mbar_init(&sm.a_full[i], 4);
             mbar_init(&sm.a_empty[i], 1);
         }
-        mbar_init(&sm.acc_full, 2);
-        mbar_init(&sm.acc_empty, kWEpiWarps);
+        for (int h = 0; h < 2; ++h) {
+            mbar_init(&sm.acc_full[h], 1);
+            mbar_init(&sm.acc_empty[h], kWEpiWarps);
+        }
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -109,8 +121,8 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
-    const uint32_t tmem_acc = tmem;                 // columns [0, 256): half h at h * 128
-    const uint32_t tmem_a = tmem + kWAccCols;       // then eight slices of 32 columns
+    const uint32_t tmem_acc = tmem;                 // half h at column h * BM
+    const uint32_t tmem_a = tmem + kWAccCols;       // then the slices of 32 columns
     volatile uint32_t* abort_flag = &sm.abort_flag;
 
     if (warp < kWFirstUnpack) {
@@ -148,7 +160,7 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
                 constexpr uint32_t idesc = idesc_i8(128, kWBM);
                 uint32_t it = 0;
                 for (int tl = 0; tl < my_tiles; ++tl) {
-                    if (!mbar_wait(&sm.acc_empty, ((uint32_t)tl & 1u) ^ 1u, abort_flag, 4u)) goto role_done;
+                    if (!mbar_wait(&sm.acc_empty[h], ((uint32_t)tl & 1u) ^ 1u, abort_flag, 4u)) goto role_done;
                     for (int kb = 0; kb < KB; ++kb, ++it) {
                         const int s = (int)(it % kWStages);
                         const uint32_t u = it * 2u + (uint32_t)h;            // this half's slice of the block
@@ -166,7 +178,7 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
                         tc_commit(&sm.a_empty[ai]);
                         tc_commit(&sm.smem_empty[s]);
                     }
-                    tc_commit(&sm.acc_full);
+                    tc_commit(&sm.acc_full[h]);
                 }
             }
         }
@@ -219,10 +231,10 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
         asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kWRegsEpi));
         const int ew = warp - kWFirstEpi;
         const int quarter = warp & 3;
-        const int chalf = ew >> 2;                    // which 64 of the tile's 128 token columns
+        const int chalf = ew >> 2;                    // which half of the tile's token columns
         const int r = quarter * 32 + lane;
         const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
-        const int col0 = chalf * 64;
+        const int col0 = chalf * kCols;
         asm volatile("griddepcontrol.wait;" ::: "memory");               // see the activation producer
         const float pe = __int_as_float((127 + *p.scale_exp) << 23);     // 2^e
         __half* stage = &sm.ystage[ew][0][0];
@@ -239,33 +251,31 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
                 sc[h] = __half2float(p.w_scales[n]) * 0.0625f * pe;      // sums carry a factor 16 (n < Npad: the scale array is padded)
                 off_pe[h] = (OFFSET && n_ok[h]) ? p.chan_offset[n] * pe : 0.0f;
             }
-            if (!mbar_wait_warp(&sm.acc_full, (uint32_t)tl & 1u, abort_flag, 8u)) goto role_done;
-            tc_fence_after();
-            // all of this warp's sums (64 columns of both halves) go to registers and the accumulators return
-            // to the MMA at once, so that the conversion and the stores below overlap the next tile's MMAs
-            uint32_t v[2][64];
+            // One half after the other: the half's sums (this warp's columns) go to registers and its
+            // accumulator returns to its issuer at once, so that conversion and stores overlap the next tile's MMAs.
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                tc_ld32(tmem_acc + lane_addr + (uint32_t)(h * kWBM + col0), *reinterpret_cast<uint32_t(*)[32]>(&v[h][0]));
-                tc_ld32(tmem_acc + lane_addr + (uint32_t)(h * kWBM + col0 + 32), *reinterpret_cast<uint32_t(*)[32]>(&v[h][32]));
-            }
-            tc_wait_ld();
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.acc_empty);
+                if (!mbar_wait_warp(&sm.acc_full[h], (uint32_t)tl & 1u, abort_flag, 8u)) goto role_done;
+                tc_fence_after();
+                uint32_t v[kCols];
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
+                for (int c0 = 0; c0 < kCols; c0 += 32)
+                    tc_ld32(tmem_acc + lane_addr + (uint32_t)(h * kWBM + col0 + c0), *reinterpret_cast<uint32_t(*)[32]>(&v[c0]));
+                tc_wait_ld();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.acc_empty[h]);
                 const int n = (2 * np + h) * kTileN + r;
                 const int n0 = (2 * np + h) * kTileN + quarter * 32;
                 if (p.y_tma) {
 #pragma unroll
-                    for (int r0 = 0; r0 < 64; r0 += kWStageRows) {
+                    for (int r0 = 0; r0 < kCols; r0 += kWStageRows) {
                         if (lane == 0) tma_store_wait_read();     // the previous store has read the staging rows
                         __syncwarp();
 #pragma unroll
                         for (int c = 0; c < kWStageRows; ++c) {
-                            const __half hv = __float2half_rn(OFFSET ? fmaf((float)(int)v[h][r0 + c], sc[h], off_pe[h])
-                                                                     : (float)(int)v[h][r0 + c] * sc[h]);
+                            const __half hv = __float2half_rn(OFFSET ? fmaf((float)(int)v[r0 + c], sc[h], off_pe[h])
+                                                                     : (float)(int)v[r0 + c] * sc[h]);
                             if constexpr (CHAIN)
                                 w_stage_code(stage, c, lane, w_chain_code(hv, p.next_inv, p.next_lo, p.next_hi), p.next_packed);
                             else
@@ -278,11 +288,11 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
                     }
                 } else {
 #pragma unroll
-                    for (int c = 0; c < 64; ++c) {
+                    for (int c = 0; c < kCols; ++c) {
                         const int m = m_base + c;
                         if (n_ok[h] && m < p.M) {
-                            const __half hv = __float2half_rn(OFFSET ? fmaf((float)(int)v[h][c], sc[h], off_pe[h])
-                                                                     : (float)(int)v[h][c] * sc[h]);
+                            const __half hv = __float2half_rn(OFFSET ? fmaf((float)(int)v[c], sc[h], off_pe[h])
+                                                                     : (float)(int)v[c] * sc[h]);
                             if constexpr (CHAIN)
                                 p.q_next[(size_t)m * p.N + n] = (int8_t)w_chain_code(hv, p.next_inv, p.next_lo, p.next_hi);
                             else
@@ -292,9 +302,9 @@ gemm_wide_kernel(const __grid_constant__ CUtensorMap x_map, const __grid_constan
                 }
                 if (p.acc_dump) {
 #pragma unroll
-                    for (int c = 0; c < 64; ++c) {
+                    for (int c = 0; c < kCols; ++c) {
                         const int m = m_base + c;
-                        if (n_ok[h] && m < p.M) p.acc_dump[(size_t)m * p.N + n] = (int)v[h][c] >> 4;
+                        if (n_ok[h] && m < p.M) p.acc_dump[(size_t)m * p.N + n] = (int)v[c] >> 4;
                     }
                 }
             }
@@ -321,11 +331,12 @@ typedef CUresult (*WEncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-template <bool OFFSET, bool CHAIN>
+template <int BM, bool OFFSET, bool CHAIN>
 cudaError_t launch_wide_t(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
-    const size_t smem_bytes = sizeof(WSmem) + 1024;
+    constexpr int kWBM = BM;
+    const size_t smem_bytes = sizeof(WSmem<BM>) + 1024;
     static SmemOptIn opt_in;
-    if (const cudaError_t e = opt_in.ensure(gemm_wide_kernel<OFFSET, CHAIN>, dev.device, smem_bytes); e != cudaSuccess)
+    if (const cudaError_t e = opt_in.ensure(gemm_wide_kernel<BM, OFFSET, CHAIN>, dev.device, smem_bytes); e != cudaSuccess)
         return e;
     WEncodeTiledFn enc = reinterpret_cast<WEncodeTiledFn>(dev.encode_tiled);
     CUtensorMap map;
@@ -385,7 +396,7 @@ cudaError_t launch_wide_t(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = a.after_quantize ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, gemm_wide_kernel<OFFSET, CHAIN>, map, ymap, p);
+    return cudaLaunchKernelEx(&cfg, gemm_wide_kernel<BM, OFFSET, CHAIN>, map, ymap, p);
 }
 
 }  // namespace
@@ -394,13 +405,33 @@ bool gemm_wide_applies(const GemmArgs& a) {
     return !a.group && a.M > 128 && (round_up(a.N, kTileN) / kTileN) % 2 == 0;
 }
 
-cudaError_t launch_gemm_wide(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
+namespace {
+template <int BM>
+cudaError_t launch_wide_bm(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
     if (a.q_next) {
         if (a.chan_offset) return cudaErrorInvalidValue;       // the two variants are not combined
-        return launch_wide_t<false, true>(a, dev, stream);
+        return launch_wide_t<BM, false, true>(a, dev, stream);
     }
-    if (a.chan_offset) return launch_wide_t<true, false>(a, dev, stream);
-    return launch_wide_t<false, false>(a, dev, stream);
+    if (a.chan_offset) return launch_wide_t<BM, true, false>(a, dev, stream);
+    return launch_wide_t<BM, false, false>(a, dev, stream);
+}
+}  // namespace
+
+// Token tile: rounds of tiles over the SMs x k blocks x the time of a k block, which the L2 -> SM path sets
+// (about 36 bytes per clock and SM measured in this kernel: 32 KB per k block on 128-token tiles, 40 KB on
+// 192-token tiles) unless the tensor pipe's 512 / 768 cycles are longer.
+int wide_token_tile(int M, int N, int sm_count) {
+    const long pairs = round_up(N, kTileN) / (2 * kTileN);
+    auto cost = [&](int bm, long unit_cycles) {
+        const long tiles = (long)((M + bm - 1) / bm) * pairs;
+        return ((tiles + sm_count - 1) / sm_count) * unit_cycles;
+    };
+    return cost(192, 1138) < cost(128, 910) ? 192 : 128;
+}
+
+cudaError_t launch_gemm_wide(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
+    return wide_token_tile(a.M, a.N, dev.sm_count) == 192 ? launch_wide_bm<192>(a, dev, stream)
+                                                          : launch_wide_bm<128>(a, dev, stream);
 }
 
 }  // namespace aq

@@ -94,7 +94,7 @@ def test_chained_layers_with_packed_intermediate_codes():
 @pytest.mark.parametrize("kernel", [binding.AQ_KERNEL_DECODE, binding.AQ_KERNEL_TENSOR])
 @pytest.mark.parametrize("bits", [8, 4])
 @pytest.mark.parametrize("M,K,N,group", [(1, 256, 128, 0), (16, 768, 768, 0), (129, 384, 224, 128), (300, 1024, 384, 0),
-                                         (260, 1152, 544, 128)])
+                                         (260, 1152, 544, 128), (300, 1024, 512, 0), (900, 256, 5120, 0)])
 def test_chained_epilogue_writes_packed_codes(kernel, bits, M, K, N, group):
     x = inputs.activations(M, K, seed=65, outlier_frac=0.01, outlier_mult=20.0)
     h = handle()

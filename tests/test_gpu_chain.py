@@ -18,7 +18,7 @@ KERNELS = [binding.AQ_KERNEL_DECODE, binding.AQ_KERNEL_TENSOR]
 @pytest.mark.parametrize("kernel", KERNELS)
 @pytest.mark.parametrize("next_bits", [8, 4])
 @pytest.mark.parametrize("M,K,N,group", [(16, 768, 768, 0), (129, 384, 200, 128), (300, 1024, 384, 0),
-                                         (260, 1152, 520, 128), (130, 256, 203, 128)])
+                                         (260, 1152, 520, 128), (130, 256, 203, 128), (300, 1024, 512, 0), (900, 256, 5120, 0)])
 def test_chain_codes_equal_quantized_plain_output(kernel, next_bits, M, K, N, group):
     x = inputs.activations(M, K, seed=41, outlier_frac=0.01, outlier_mult=20.0)
     w = inputs.weights(N, K, 41)

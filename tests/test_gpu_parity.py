@@ -269,6 +269,30 @@ def test_linear_with_row_idx_equals_compacted_input(kernel):
     assert_y_close(gpu["y"], ref["y"])
 
 
+@pytest.mark.parametrize("M,K,N", [(300, 1024, 512), (257, 384, 250), (129, 4224, 256), (1000, 256, 5120), (1400, 640, 6400),
+                                   (700, 2048, 1024), (193, 160, 1536)])
+def test_one_scale_per_channel_on_tiles_of_two_channel_blocks(M, K, N):
+    """More than 128 tokens and an even number of 128-channel blocks: the tensor-core kernel whose tile is two
+    channel blocks sharing an activation tile of 128 or 192 tokens. Ragged token and channel edges, K not a
+    multiple of 128, more tiles than SMs (several tiles per CTA), both tile heights, with the zero-point term
+    and with chaining."""
+    x = inputs.activations(M, K, seed=M + N + 9, outlier_frac=0.01, outlier_mult=20.0)
+    w = inputs.weights(N, K, seed=K + N + 9)
+    for bits, clip in ((8, 0), (4, 4)):
+        gpu, ref = run_layer_both(x, w, bits, 0, TENSOR, clip=clip)
+        assert gpu["e"] == ref["e"] and np.array_equal(gpu["q"], ref["q"])
+        assert np.array_equal(gpu["acc"], ref["acc"])
+        assert_y_close(gpu["y"], ref["y"])
+    gpu2, _ = run_layer_both(x, w, 8, 0, TENSOR, want_acc=False)          # as the benchmark calls it
+    gpu1, _ = run_layer_both(x, w, 8, 0, TENSOR)
+    assert np.array_equal(gpu1["y"].view(np.uint16), gpu2["y"].view(np.uint16))
+    # extreme codes: the largest sums
+    xe = np.full((M, K), -128.0, np.float16)
+    we = np.full((N, K), -0.01, np.float16)
+    gpu, ref = run_layer_both(xe, we, 8, 0, TENSOR, scale_mode=1, clip=0)
+    assert np.array_equal(gpu["acc"], ref["acc"]) and ref["acc"].max() == 128 * 7 * K
+
+
 @pytest.mark.parametrize("group", [0, 128])
 def test_several_tiles_per_cta_and_deep_k(group):
     """More tiles than SMs and more k blocks than any ring is deep: every ring and every

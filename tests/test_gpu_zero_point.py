@@ -58,7 +58,7 @@ def test_weight_offsets_match_exact_sums(N, K, group):
 @pytest.mark.parametrize("kernel", [binding.AQ_KERNEL_DECODE, binding.AQ_KERNEL_TENSOR])
 @pytest.mark.parametrize("bits", [8, 4])
 @pytest.mark.parametrize("M,K,N,group", [(16, 768, 768, 0), (129, 384, 200, 128), (300, 1024, 384, 0),
-                                         (260, 1152, 520, 128)])
+                                         (260, 1152, 520, 128), (300, 1024, 512, 0), (900, 256, 5120, 0)])
 def test_linear_asym_matches_checker(kernel, bits, M, K, N, group):
     x = _acts(M, K, 34, 2.5)
     w = inputs.weights(N, K, 34)
