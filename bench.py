@@ -831,6 +831,19 @@ def main():
                 line[key] = fn(h)
             except Exception as ex:  # report, do not hide
                 line[key] = {"error": repr(ex)}
+    if isinstance(line.get("pruned_prefill"), list):
+        # the per-channel prefill product of the token-pruned workload (tiles of 256 channels), as a roofline entry
+        pr = line["pruned_prefill"]
+        ach = statistics.mean(r["product_only"]["TOPS"] for r in pr)
+        ent = {"kernel": "gemm_wide_kernel<192> (one scale per channel, 256-channel tiles)", "bound": "tensor", "unit": "TFLOP/s",
+               "workload": "opt30b_pruned_prefill_w4a8, product kernel, mean of the two shapes", "achieved": ach,
+               "peak": burst_peak, "frac": ach / burst_peak, "frac_of_nominal_4500": ach / 4500.0,
+               "per_shape_TOPS": [r["product_only"]["TOPS"] for r in pr],
+               "timing": "event-timed back-to-back launches (a fraction of a second at full clock: burst peak)"}
+        probe = line.get("int8_peak_measured", {})
+        if "a_from_tmem" in probe:
+            ent["frac_of_int8_probe_burst"] = ach / probe["a_from_tmem"]["burst_TOPS"]
+        line["perchannel_roofline"] = ent
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(wl, xs_np, ws_np, M)
     if rank == 0:
