@@ -615,7 +615,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-decode", action="store_true", help="skip the extra keys (decode, w4a4, pruned_prefill)")
+    ap.add_argument("--no-decode", action="store_true", help="skip the extra keys (rate probe, sustained leg, decode, w4a4, pruned_prefill, ...)")
     ap.add_argument("--case", default=None, help="M,K,N,group[,bits[,kernel]]: time one product kernel")
     ap.add_argument("--rotate-mb", type=float, default=0.0,
                     help="with --case: rotate through this many MB of weight copies (defeats L2)")
@@ -792,7 +792,7 @@ def main():
         "clocks": clocks,
         "roofline": roofline,
     }
-    if rank == 0 and world == 1:
+    if rank == 0 and world == 1 and not args.no_decode:
         try:
             probe = bench_int8_probe(h, local_rank)
             line["int8_peak_measured"] = probe
