@@ -408,6 +408,10 @@ def bench_attention(h, reps=5):
     t_av = _event_ms(lambda: h.aq_attn_v_log2(pc, pmax, vq, ev, 4, y=y), reps)
     _, ws = h.aq_attn_v_log2_tc(pc, pmax, vq, ev, y=y)
     t_tc = _event_ms(lambda: h.aq_attn_v_log2_tc(pc, pmax, vq, ev, y=y, workspace=ws), 4 * reps)
+    # the same with the byte factors written by the log2 kernel itself: no conversion pass over P
+    pf, pfmax, _ = h.aq_log2_quantize_factors(p)
+    t_qf = _event_ms(lambda: h.aq_log2_quantize_factors(p, factors=pf), reps)
+    t_tcf = _event_ms(lambda: h.aq_attn_v_factors_tc(pf, pfmax, vq, ev, y=y, workspace=ws), 4 * reps)
     macs = float(H) * M * J * D
     # query x key scores on int8 codes (reduction over the head dimension); the fp16 score matrix is the traffic
     qa = torch.from_numpy(inputs.activations(H * M, D, 8, 0.01, 6.0)).cuda()
@@ -425,7 +429,9 @@ def bench_attention(h, reps=5):
             "attn_v_shift": {"us": t_av * 1e3, "Gproducts_per_s": macs / (t_av * 1e-3) / 1e9,
                              "note": "CUDA-core kernel: one shift and one add per product"},
             "attn_v_tensor": {"us": t_tc * 1e3, "TOPS": 2.0 * macs / (t_tc * 1e-3) / 1e12,
-                              "note": "factor conversion + value transpose + tcgen05 u8 x s8 kernel"}}
+                              "note": "factor conversion + value transpose + tcgen05 u8 x s8 kernel"},
+            "attn_v_tensor_on_factors": {"us": t_tcf * 1e3, "TOPS": 2.0 * macs / (t_tcf * 1e-3) / 1e12, "log2_quantize_factors_us": t_qf * 1e3,
+                                         "note": "byte factors from aq_log2_quantize_factors: value transpose + tcgen05 kernel"}}
 
 
 def bench_pruned(h, reps=10):

@@ -280,6 +280,17 @@ int aq_attn_v_log2(aq_handle_t h, const int8_t* p_codes, const uint32_t* p_max_b
 int aq_attn_qk_tc(aq_handle_t h, const int8_t* q_codes, const int32_t* q_scale_exp, const int8_t* k_codes,
                   const int32_t* k_scale_exp, int H, int M, int J, int D, void* s_fp16, void* workspace,
                   size_t workspace_bytes, void* stream);
+/* The two calls that spare the tensor-core route its conversion pass over P (Eq. 3 with 4-bit codes of a
+ * non-negative input): aq_log2_quantize_factors writes, instead of the code, the byte 2^(kmax - k) =
+ * 128 >> k that multiplies the value code (0 for an exact zero or NaN; a negative input is an error that
+ * aq_check_workspace on this workspace reports as AQ_ERR_INVALID_ARG, its factor is 0), i.e. exactly what
+ * aq_attn_v_log2_tc derives from the codes of aq_log2_quantize(bits = 4); aq_attn_v_factors_tc is
+ * aq_attn_v_log2_tc on those bytes (p_factors [H,M,J], 16-byte aligned). Same results bit for bit. */
+int aq_log2_quantize_factors(aq_handle_t h, const void* x_fp16, long long count, uint8_t* factors,
+                             uint32_t* max_bits_out, void* workspace, size_t workspace_bytes, void* stream);
+int aq_attn_v_factors_tc(aq_handle_t h, const uint8_t* p_factors, const uint32_t* p_max_bits, const int8_t* v_codes,
+                         const int32_t* v_scale_exp, int H, int M, int J, int D, void* y_fp16, void* workspace,
+                         size_t workspace_bytes, void* stream);
 size_t aq_attn_workspace_bytes(int H, int M, int J, int D);
 int aq_attn_v_log2_tc(aq_handle_t h, const int8_t* p_codes, const uint32_t* p_max_bits, const int8_t* v_codes,
                       const int32_t* v_scale_exp, int H, int M, int J, int D, void* y_fp16, void* workspace,

@@ -98,6 +98,8 @@ def load():
     L.aq_attn_workspace_bytes.restype = sz
     L.aq_attn_workspace_bytes.argtypes = [i32, i32, i32, i32]
     L.aq_attn_v_log2_tc.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, sz, vp]
+    L.aq_log2_quantize_factors.argtypes = [vp, vp, C.c_longlong, vp, vp, vp, sz, vp]
+    L.aq_attn_v_factors_tc.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, sz, vp]
     L.aq_attn_qk_tc.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, vp, vp, sz, vp]
     L.aq_prune_schedule.argtypes = [i32, C.c_double, i32, vp, vp]
     L.aq_trip_calibrate.argtypes = [vp, vp, i32, i32, i32, vp, vp, vp, vp, sz, vp]
@@ -284,6 +286,29 @@ class Handle:
         _check(load().aq_attn_v_log2_tc(self._h, _ptr(p_codes), _ptr(p_max_bits), _ptr(v_codes), _ptr(v_scale_exp), H, M,
                                         J, D, _ptr(y), _ptr(workspace), workspace.numel(), _stream()),
                "aq_attn_v_log2_tc")
+        return y, workspace
+
+    def aq_log2_quantize_factors(self, x: torch.Tensor, factors: Optional[torch.Tensor] = None,
+                                 workspace: Optional[torch.Tensor] = None):
+        """(uint8 byte factors 128 >> k of x's shape, uint32[1] holding the fp16 bits of max|x|, workspace)."""
+        if factors is None:
+            factors = torch.empty(x.shape, dtype=torch.uint8, device=x.device)
+        mx = torch.zeros(1, dtype=torch.int32, device=x.device)
+        ws = workspace if workspace is not None else torch.empty(256, dtype=torch.uint8, device=x.device)
+        _check(load().aq_log2_quantize_factors(self._h, _ptr(x), x.numel(), _ptr(factors), _ptr(mx), _ptr(ws), ws.numel(),
+                                               _stream()), "aq_log2_quantize_factors")
+        return factors, mx, ws
+
+    def aq_attn_v_factors_tc(self, p_factors, p_max_bits, v_codes, v_scale_exp, y=None, workspace=None):
+        H, M, J = p_factors.shape
+        D = v_codes.shape[2]
+        if y is None:
+            y = torch.empty((H, M, D), dtype=torch.float16, device=p_factors.device)
+        if workspace is None:
+            workspace = torch.empty(load().aq_attn_workspace_bytes(H, M, J, D), dtype=torch.uint8, device=p_factors.device)
+        _check(load().aq_attn_v_factors_tc(self._h, _ptr(p_factors), _ptr(p_max_bits), _ptr(v_codes), _ptr(v_scale_exp), H,
+                                           M, J, D, _ptr(y), _ptr(workspace), workspace.numel(), _stream()),
+               "aq_attn_v_factors_tc")
         return y, workspace
 
     def aq_attn_qk_tc(self, q_codes, q_exp, k_codes, k_exp, s=None, workspace=None):

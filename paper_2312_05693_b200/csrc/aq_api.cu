@@ -566,6 +566,21 @@ int aq_log2_quantize(aq_handle_t h, const void* x_fp16, long long count, int bit
     return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
 }
 
+int aq_log2_quantize_factors(aq_handle_t h, const void* x_fp16, long long count, uint8_t* factors,
+                             uint32_t* max_bits_out, void* workspace, size_t workspace_bytes_, void* stream_) {
+    if (!h || !x_fp16 || !factors || count < 1) return AQ_ERR_INVALID_ARG;
+    if (!workspace || workspace_bytes_ < sizeof(Control)) return AQ_ERR_WORKSPACE;
+    if (!aligned(x_fp16, 2) || !aligned(workspace, 256) || (max_bits_out && !aligned(max_bits_out, 4)))
+        return AQ_ERR_ALIGNMENT;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    Control* ctl = static_cast<Control*>(workspace);
+    cudaError_t e = cudaMemsetAsync(ctl, 0, sizeof(Control), stream);
+    if (e == cudaSuccess)
+        e = launch_log2_quantize(static_cast<const __half*>(x_fp16), count, 4, ctl, reinterpret_cast<int8_t*>(factors),
+                                 max_bits_out, h->dev, stream, true);
+    return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
 int aq_attn_v_log2(aq_handle_t h, const int8_t* p_codes, const uint32_t* p_max_bits, const int8_t* v_codes,
                    const int32_t* v_scale_exp, int H, int M, int J, int D, int bits, void* y_fp16, int32_t* acc_dump,
                    void* stream) {
@@ -586,14 +601,14 @@ size_t aq_attn_workspace_bytes(int H, int M, int J, int D) {
     return sizeof(Control) + attn_tc_scratch_bytes(H, M, J, D);
 }
 
-int aq_attn_v_log2_tc(aq_handle_t h, const int8_t* p_codes, const uint32_t* p_max_bits, const int8_t* v_codes,
+static int attn_v_tc_impl(aq_handle_t h, bool p_is_factors, const int8_t* p_codes, const uint32_t* p_max_bits, const int8_t* v_codes,
                       const int32_t* v_scale_exp, int H, int M, int J, int D, void* y_fp16, void* workspace,
                       size_t workspace_bytes_, void* stream_) {
     if (!h || !p_codes || !p_max_bits || !v_codes || !v_scale_exp || !y_fp16) return AQ_ERR_INVALID_ARG;
     if (H < 1 || H > 65535 || M < 1 || J < 16 || J > 65536 || J % 16 != 0 || (D != 64 && D != 128)) return AQ_ERR_SHAPE;
     if ((long long)H * M > 0x7FFFFFFFll || (long long)H * D > 0x7FFFFFFFll) return AQ_ERR_SHAPE;
     if (!workspace || workspace_bytes_ < aq_attn_workspace_bytes(H, M, J, D)) return AQ_ERR_WORKSPACE;
-    if (!aligned(p_codes, 4) || !aligned(v_codes, 1) || !aligned(y_fp16, 16) || !aligned(p_max_bits, 4) ||
+    if (!aligned(p_codes, p_is_factors ? 16 : 4) || !aligned(v_codes, 1) || !aligned(y_fp16, 16) || !aligned(p_max_bits, 4) ||
         !aligned(v_scale_exp, 4) || !aligned(workspace, 256))
         return AQ_ERR_ALIGNMENT;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
@@ -601,8 +616,22 @@ int aq_attn_v_log2_tc(aq_handle_t h, const int8_t* p_codes, const uint32_t* p_ma
     cudaError_t e = cudaMemsetAsync(ctl, 0, sizeof(Control), stream);
     if (e == cudaSuccess)
         e = launch_attn_v_log2_tc(p_codes, p_max_bits, v_codes, v_scale_exp, H, M, J, D, static_cast<__half*>(y_fp16), ctl,
-                                  static_cast<uint8_t*>(workspace) + sizeof(Control), h->dev, stream);
+                                  static_cast<uint8_t*>(workspace) + sizeof(Control), h->dev, stream, p_is_factors);
     return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
+}
+
+int aq_attn_v_log2_tc(aq_handle_t h, const int8_t* p_codes, const uint32_t* p_max_bits, const int8_t* v_codes,
+                      const int32_t* v_scale_exp, int H, int M, int J, int D, void* y_fp16, void* workspace,
+                      size_t workspace_bytes_, void* stream_) {
+    return attn_v_tc_impl(h, false, p_codes, p_max_bits, v_codes, v_scale_exp, H, M, J, D, y_fp16, workspace,
+                          workspace_bytes_, stream_);
+}
+
+int aq_attn_v_factors_tc(aq_handle_t h, const uint8_t* p_factors, const uint32_t* p_max_bits, const int8_t* v_codes,
+                         const int32_t* v_scale_exp, int H, int M, int J, int D, void* y_fp16, void* workspace,
+                         size_t workspace_bytes_, void* stream_) {
+    return attn_v_tc_impl(h, true, reinterpret_cast<const int8_t*>(p_factors), p_max_bits, v_codes, v_scale_exp, H, M, J, D,
+                          y_fp16, workspace, workspace_bytes_, stream_);
 }
 
 int aq_attn_qk_tc(aq_handle_t h, const int8_t* q_codes, const int32_t* q_scale_exp, const int8_t* k_codes,

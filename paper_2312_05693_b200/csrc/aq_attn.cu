@@ -89,9 +89,25 @@ __device__ __forceinline__ int log2_code(unsigned int raw, unsigned int mb_bits,
     return none ? 0 : ((raw & 0x8000u) ? -k : k);
 }
 
+// codes -> weights: c > 0 -> 128 >> (c - 1); 0 -> 0; a negative code is not representable here:
+// it is recorded in the status word (11) and treated as 0.
+__device__ __forceinline__ uint32_t log2_factors4(uint32_t c4, bool& bad) {
+    uint32_t o = 0;
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+        const int c = (int)(int8_t)((c4 >> (8 * t)) & 0xFFu);
+        bad |= c < 0;
+        o |= (c > 0 ? (128u >> (c - 1)) : 0u) << (8 * t);
+    }
+    return o;
+}
+
 __global__ void __launch_bounds__(256)
-log2_codes_kernel(const __half* __restrict__ x, long long count, int bits, const Control* __restrict__ ctl,
-                  int8_t* __restrict__ codes, uint32_t* __restrict__ max_bits_out) {
+log2_codes_kernel(const __half* __restrict__ x, long long count, int bits, Control* __restrict__ ctl,
+                  int8_t* __restrict__ codes, uint32_t* __restrict__ max_bits_out, int as_factors) {
+    // as_factors (4-bit codes of a non-negative input): instead of the code c the byte 2^(kmax - k) = 128 >> (c - 1)
+    // is written (0 for a zero), the form the tensor-core product takes; a negative value is reported (status 11)
+    bool bad = false;
     const unsigned int mb_bits = ctl->absmax_bits;
     if (blockIdx.x == 0 && threadIdx.x == 0 && max_bits_out) *max_bits_out = mb_bits;
     const int kmax = (1 << (bits - 1)) - 1;
@@ -112,11 +128,16 @@ log2_codes_kernel(const __half* __restrict__ x, long long count, int bits, const
             const uint32_t c1 = (uint32_t)log2_code(w[t] >> 16, mb_bits, eb, t_up, t_down, kmax) & 0xFFu;
             out[t >> 1] |= (c0 | (c1 << 8)) << (16 * (t & 1));
         }
+        if (as_factors) { out[0] = log2_factors4(out[0], bad); out[1] = log2_factors4(out[1], bad); }
         *reinterpret_cast<uint2*>(codes + 8 * i) = make_uint2(out[0], out[1]);
     }
     if (blockIdx.x == 0 && threadIdx.x == 0)
-        for (long long i = nvec * 8; i < count; ++i)
-            codes[i] = (int8_t)log2_code(__half_as_ushort(x[i]), mb_bits, eb, t_up, t_down, kmax);
+        for (long long i = nvec * 8; i < count; ++i) {
+            const int c = log2_code(__half_as_ushort(x[i]), mb_bits, eb, t_up, t_down, kmax);
+            bad |= as_factors && c < 0;
+            codes[i] = as_factors ? (int8_t)(uint8_t)(c > 0 ? (128u >> (c - 1)) : 0u) : (int8_t)c;
+        }
+    if (bad) atomicCAS(&ctl->status, 0u, 11u);
 }
 
 // ---- attention x value on the codes -----------------------------------------------------------
@@ -163,19 +184,6 @@ attn_v_log2_kernel(const int8_t* __restrict__ pcodes, const uint32_t* __restrict
 // u8 x s8 -> s32 contraction over the key index j: acc[m][d] = sum_j w[m][j] * v[d][j], with both
 // operands stored j-major. tcgen05.mma kind::i8 reads both from shared memory (128-byte swizzle,
 // staged by TMA); the accumulator [128 query rows x D] lives in tensor memory.
-
-// codes -> weights: c > 0 -> 128 >> (c - 1); 0 -> 0; a negative code is not representable here:
-// it is recorded in the status word (11) and treated as 0.
-__device__ __forceinline__ uint32_t log2_factors4(uint32_t c4, bool& bad) {
-    uint32_t o = 0;
-#pragma unroll
-    for (int t = 0; t < 4; ++t) {
-        const int c = (int)(int8_t)((c4 >> (8 * t)) & 0xFFu);
-        bad |= c < 0;
-        o |= (c > 0 ? (128u >> (c - 1)) : 0u) << (8 * t);
-    }
-    return o;
-}
 
 __global__ void __launch_bounds__(256)
 log2_weights_kernel(const int8_t* __restrict__ codes, long long count, uint8_t* __restrict__ w, Control* __restrict__ ctl) {
@@ -507,9 +515,10 @@ size_t attn_tc_scratch_bytes(int H, int M, int J, int D) {
 }
 
 // scratch: [weights H*M*J, padded to 256][transposed value codes H*D*J]
+// p_is_factors: pcodes already holds the byte factors (written by the log2 kernel), no conversion pass.
 cudaError_t launch_attn_v_log2_tc(const int8_t* pcodes, const uint32_t* max_bits, const int8_t* vq, const int32_t* e_v,
                                   int H, int M, int J, int D, __half* y, Control* ctl, void* scratch,
-                                  const DeviceInfo& dev, cudaStream_t stream) {
+                                  const DeviceInfo& dev, cudaStream_t stream, bool p_is_factors) {
     uint8_t* w = static_cast<uint8_t*>(scratch);
     int8_t* vt = reinterpret_cast<int8_t*>(w + ((size_t)H * M * J + 255) / 256 * 256);
     const long long count = (long long)H * M * J;
@@ -517,9 +526,14 @@ cudaError_t launch_attn_v_log2_tc(const int8_t* pcodes, const uint32_t* max_bits
     const long long cap = (long long)dev.sm_count * 16;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
-    log2_weights_kernel<<<(unsigned int)blocks, 256, 0, stream>>>(pcodes, count, w, ctl);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return e;
+    cudaError_t e = cudaSuccess;
+    if (p_is_factors) {
+        w = const_cast<uint8_t*>(reinterpret_cast<const uint8_t*>(pcodes));
+    } else {
+        log2_weights_kernel<<<(unsigned int)blocks, 256, 0, stream>>>(pcodes, count, w, ctl);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
     transpose_i8_kernel<<<dim3((J + 31) / 32, (D + 31) / 32, H), 256, 0, stream>>>(vq, J, D, vt);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
@@ -534,7 +548,7 @@ cudaError_t launch_attn_qk_tc(const int8_t* qc, const int32_t* e_q, const int8_t
 }
 
 cudaError_t launch_log2_quantize(const __half* x, long long count, int bits, Control* ctl, int8_t* codes,
-                                 uint32_t* max_bits_out, const DeviceInfo& dev, cudaStream_t stream) {
+                                 uint32_t* max_bits_out, const DeviceInfo& dev, cudaStream_t stream, bool as_factors) {
     long long blocks = (count / 8 + 255) / 256;
     const long long cap = (long long)dev.sm_count * 8;
     if (blocks > cap) blocks = cap;
@@ -542,7 +556,7 @@ cudaError_t launch_log2_quantize(const __half* x, long long count, int bits, Con
     log2_absmax_kernel<<<(unsigned int)blocks, 256, 0, stream>>>(x, count, ctl);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    log2_codes_kernel<<<(unsigned int)blocks, 256, 0, stream>>>(x, count, bits, ctl, codes, max_bits_out);
+    log2_codes_kernel<<<(unsigned int)blocks, 256, 0, stream>>>(x, count, bits, ctl, codes, max_bits_out, as_factors ? 1 : 0);
     return cudaGetLastError();
 }
 

@@ -146,12 +146,12 @@ cudaError_t launch_chan_offsets(const float* r, int N, int bits, const Control* 
 
 // Log2 codes of Eq. 3 (two kernels: layer maximum, codes) and attention x value on them (aq_attn.cu).
 cudaError_t launch_log2_quantize(const __half* x, long long count, int bits, Control* ctl, int8_t* codes,
-                                 uint32_t* max_bits_out, const DeviceInfo& dev, cudaStream_t stream);
+                                 uint32_t* max_bits_out, const DeviceInfo& dev, cudaStream_t stream, bool as_factors = false);
 // The same product on the tensor cores, for non-negative P; scratch holds attn_tc_scratch_bytes().
 size_t attn_tc_scratch_bytes(int H, int M, int J, int D);
 cudaError_t launch_attn_v_log2_tc(const int8_t* pcodes, const uint32_t* max_bits, const int8_t* vq, const int32_t* e_v,
                                   int H, int M, int J, int D, __half* y, Control* ctl, void* scratch,
-                                  const DeviceInfo& dev, cudaStream_t stream);
+                                  const DeviceInfo& dev, cudaStream_t stream, bool p_is_factors = false);
 // Query x key product on int8 codes (head dimension 128), same tensor-core kernel.
 cudaError_t launch_attn_qk_tc(const int8_t* qc, const int32_t* e_q, const int8_t* kc, const int32_t* e_k, int H, int M,
                               int J, int D, __half* s_out, Control* ctl, const DeviceInfo& dev, cudaStream_t stream);

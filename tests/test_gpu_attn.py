@@ -101,6 +101,38 @@ def test_attn_v_log2_tensor_core_path_matches_checker(H, M, J, D):
     assert torch.equal(y, y_shift)
 
 
+@pytest.mark.parametrize("H,M,J,D", [(2, 33, 80, 128), (3, 300, 1040, 64), (1, 5, 16, 64)])
+def test_byte_factors_from_the_log2_kernel_feed_the_tensor_core_path(H, M, J, D):
+    """aq_log2_quantize_factors writes 128 >> k where aq_log2_quantize writes the code k + 1: the bytes must be that
+    function of the checker's codes, and the product on them must be the product on the codes, bit for bit."""
+    h = handle()
+    p = _softmax_rows(H, M, J, 59)
+    p[0, 0, :3] = 0.0                                        # exact zeros: code 0, factor 0
+    f, fmax, ws_q = h.aq_log2_quantize_factors(dev(p))
+    assert h.aq_check_workspace(ws_q) == binding.AQ_OK
+    pc_ref, pmax_ref = oracle.log2_quantize(p, 4)
+    assert np.float16(pmax_ref).view(np.uint16) == (int(fmax.item()) & 0xFFFF)
+    expect = np.where(pc_ref > 0, 128 >> np.maximum(pc_ref.astype(np.int32) - 1, 0), 0).astype(np.uint8)
+    assert np.array_equal(f.cpu().numpy(), expect)
+    v = inputs.activations(H * J, 128, seed=60, outlier_frac=0.01, outlier_mult=8.0)[:, :D].copy()
+    vq, ev = h.aq_quantize_act(dev(v.reshape(-1, 128)), 8)
+    vq = vq.reshape(H, J, D)
+    y_f, ws = h.aq_attn_v_factors_tc(f, fmax, vq, ev)
+    assert h.aq_check_workspace(ws) == binding.AQ_OK
+    pc, pmax = h.aq_log2_quantize(dev(p), 4)
+    y_c, _ = h.aq_attn_v_log2_tc(pc, pmax, vq, ev)
+    assert torch.equal(y_f, y_c)
+    e_ref = oracle.layer_exponent(v.reshape(-1, 128), 8)
+    vq_ref = oracle.quantize_act(v.reshape(-1, 128), 8, e_ref).reshape(H, J, D)
+    _, y_ref = oracle.attn_v_log2(pc_ref, pmax_ref, vq_ref, e_ref, 4)
+    assert_y_close(y_f.cpu().numpy().reshape(H * M, D), y_ref.reshape(H * M, D))
+    # a negative input has no byte factor: reported, not silently dropped
+    pn = p.copy()
+    pn[0, 1, 2] = -0.25
+    _, _, ws_n = h.aq_log2_quantize_factors(dev(pn))
+    assert h.aq_check_workspace(ws_n) == binding.AQ_ERR_INVALID_ARG
+
+
 def test_attn_tensor_core_path_reports_negative_codes():
     h = handle()
     pc = torch.ones((1, 8, 16), dtype=torch.int8, device="cuda")
