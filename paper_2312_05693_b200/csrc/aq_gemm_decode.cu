@@ -544,6 +544,9 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     // other CTAs' sums over distributed shared memory instead, with a second meeting before anybody leaves,
     // measured 0.1-0.5 us slower at every row count.)
     // The scale is fetched before the cluster meets so that its latency overlaps the wait.
+    // This CTA's k range is done: a launch behind this one that allows it may be scheduled and set up now
+    // (it reads and writes nothing before this grid has completed).
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int cw = kTileN / split;                            // split is 1, 2 or 4
     const int ft = (int)threadIdx.x - 32;                     // the 256 consumer threads finish; cw divides 256
     const int out_r = rank * cw + (ft >= 0 ? ft % cw : 0);
