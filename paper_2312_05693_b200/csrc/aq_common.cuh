@@ -184,8 +184,9 @@ struct GemmArgs {
     // The launch directly before this one on the stream is this call's own quantize (or offset) kernel: the
     // status word is already initialised, and the product kernels may be set up (the few-row streaming
     // kernel also starts streaming weights) while that kernel still runs (programmatic dependent launch;
-    // they wait for that grid before they touch the codes). Weights cannot be in flight then: the preceding kernel
-    // was launched normally, after everything before it had completed.
+    // they wait for that grid before they touch the codes). Weights cannot be in flight then: the quantize
+    // kernels allow the dependent launch only once everything before them on the stream has completed (the
+    // cooperative one is launched normally, the small one signals after its own wait for the kernel ahead).
     bool after_quantize = false;
     // fp32 partial outputs of tiles whose k range two CTAs share (tensor kernel, per-group scales)
     float* split_scratch = nullptr;

@@ -325,8 +325,8 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     // then are the status word, the codes, the exponent and the offsets touched.
     // Launched with programmatic stream serialization: this grid may have been set up while the kernel
     // before it on the stream still ran. Nothing written before this launch is read, and nothing is written,
-    // until that kernel has completed; only behind the call's own quantize kernel (which was launched
-    // normally, after everything before it, weight packing included) the weights are fetched first.
+    // until that kernel has completed; only behind the call's own quantize kernel (which allows this
+    // launch only once everything before it, weight packing included, has completed) the weights are fetched first.
     int issued = 0;
     if (!p.clear_status) {                            // launched behind this call's own quantize kernel
         if (warp == 0 && lane == 0)

@@ -92,13 +92,19 @@ quantize_small_kernel(const uint4* __restrict__ x, int M, int vec_per_row, const
     cg::cluster_group cluster = cg::this_cluster();
     __shared__ unsigned int warp_max[kSmallThreads / 32];
     __shared__ unsigned int slots[kSmallCtas];
-    // A product kernel launched with programmatic stream serialization may be set up on the idle SMs
-    // while this one runs (it waits for this grid before it reads the codes); no effect otherwise.
+    // The launch allows programmatic stream serialization, so this grid may be set up while the kernel
+    // ahead of it drains; nothing is read or written before that kernel has completed. Only then is the
+    // dependent launch allowed: a product kernel launched the same way behind this one may be set up on
+    // the idle SMs and fetch its weights while this one runs (it waits for this grid before it reads the
+    // codes), and by then everything that preceded this kernel on the stream is complete.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int rank = (int)cluster.block_rank();
     const int total = M * vec_per_row;
     uint4 buf[kSmallVecs];
     __half2 m2 = __float2half2_rn(0.0f);
+    // all loads first, then the maximum: the loads of a thread are in flight together (one memory round
+    // trip for the whole activation instead of one per vector)
 #pragma unroll
     for (int i = 0; i < kSmallVecs; ++i) {
         const int v = (i * kSmallCtas + rank) * kSmallThreads + (int)threadIdx.x;
@@ -106,10 +112,13 @@ quantize_small_kernel(const uint4* __restrict__ x, int M, int vec_per_row, const
         if (v < total) {
             const int m = v / vec_per_row, c = v % vec_per_row;
             buf[i] = __ldg(x + (size_t)(row_idx ? row_idx[m] : m) * vec_per_row + c);
-            const __half2* h = reinterpret_cast<const __half2*>(&buf[i]);
-#pragma unroll
-            for (int k = 0; k < 4; ++k) m2 = __hmax2(m2, __habs2(h[k]));   // NaN operands are dropped
         }
+    }
+#pragma unroll
+    for (int i = 0; i < kSmallVecs; ++i) {
+        const __half2* h = reinterpret_cast<const __half2*>(&buf[i]);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) m2 = __hmax2(m2, __habs2(h[k]));   // NaN operands are dropped; absent vectors are zero
     }
     unsigned int bits_max = max((unsigned int)__half_as_ushort(__low2half(m2)),
                                 (unsigned int)__half_as_ushort(__high2half(m2)));
@@ -196,17 +205,34 @@ quantize_fused_kernel(const uint4* __restrict__ x, int M, int units_per_row /* 1
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     __half2 m2 = __float2half2_rn(0.0f);
-#pragma unroll 2
-    for (size_t u = u0 + threadIdx.x; u < u1; u += kFusedThreads) {
-        const int m = (int)(u / units_per_row), c = (int)(u % units_per_row);
-        const size_t src = ((size_t)(row_idx ? row_idx[m] : m) * units_per_row + c) * 2;
-        const uint4 d0 = __ldg(x + src), d1 = __ldg(x + src + 1);
-        const unsigned int local = (unsigned int)(u - u0);
-        if (local < cache_units) { fused_cache[local] = d0; fused_cache[cache_units + local] = d1; }
-        const __half2* h0 = reinterpret_cast<const __half2*>(&d0);
-        const __half2* h1 = reinterpret_cast<const __half2*>(&d1);
+    // four units (eight 16-byte loads) in flight per thread before the first is used: a CTA's share is a few
+    // units per thread, so the pass is one or two memory round trips rather than one per unit
+    constexpr int kInFlight = 4;
+    for (size_t ub = u0 + threadIdx.x; ub < u1; ub += (size_t)kFusedThreads * kInFlight) {
+        uint4 d0[kInFlight], d1[kInFlight];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) m2 = __hmax2(m2, __hmax2(__habs2(h0[i]), __habs2(h1[i])));   // NaN operands are dropped
+        for (int i = 0; i < kInFlight; ++i) {
+            const size_t u = ub + (size_t)i * kFusedThreads;
+            if (u < u1) {
+                const int m = (int)(u / units_per_row), c = (int)(u % units_per_row);
+                const size_t src = ((size_t)(row_idx ? row_idx[m] : m) * units_per_row + c) * 2;
+                d0[i] = __ldg(x + src); d1[i] = __ldg(x + src + 1);
+            } else {
+                d0[i] = make_uint4(0u, 0u, 0u, 0u); d1[i] = d0[i];
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < kInFlight; ++i) {
+            const size_t u = ub + (size_t)i * kFusedThreads;
+            if (u < u1) {
+                const unsigned int local = (unsigned int)(u - u0);
+                if (local < cache_units) { fused_cache[local] = d0[i]; fused_cache[cache_units + local] = d1[i]; }
+            }
+            const __half2* h0 = reinterpret_cast<const __half2*>(&d0[i]);
+            const __half2* h1 = reinterpret_cast<const __half2*>(&d1[i]);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) m2 = __hmax2(m2, __hmax2(__habs2(h0[k]), __habs2(h1[k])));   // NaN operands are dropped
+        }
     }
     unsigned int bmax = max((unsigned int)__half_as_ushort(__low2half(m2)),
                             (unsigned int)__half_as_ushort(__high2half(m2)));
@@ -509,66 +535,128 @@ trip_calibrate_kernel(const __half* __restrict__ x, int M, int K, const int32_t*
     alpha_out[k] = (uint8_t)best;
 }
 
-// ---- token selection: rank every score, keep rank < n_keep, then compact the flags ------
-// rank(i) = #{ j : s_j > s_i  or (s_j == s_i and j < i) }, so equal scores resolve toward
-// the lower index and exactly n_keep tokens have rank < n_keep.
-// A CTA ranks 32 tokens: lane = token, and each of the 8 warps counts over one eighth of the scores
-// (a warp reads one score at a time, the same address in every lane).
-constexpr int kRankWarps = 8;
-__global__ void __launch_bounds__(32 * kRankWarps)
-token_rank_kernel(const float* __restrict__ scores, int M, int n_keep, uint8_t* __restrict__ keep) {
-    __shared__ int ranks[32];
-    const int lane = threadIdx.x & 31, part = threadIdx.x >> 5;
-    const int i = blockIdx.x * 32 + lane;
-    if (part == 0) ranks[lane] = 0;
-    __syncthreads();
-    const float si = i < M ? scores[i] : 0.0f;
-    const int per = (M + kRankWarps - 1) / kRankWarps;
-    const int j0 = part * per, j1 = min(M, j0 + per);
-    int rank = 0;
-#pragma unroll 4
-    for (int j = j0; j < j1; ++j) {
-        const float sj = __ldg(scores + j);
-        rank += (sj > si) || (sj == si && j < i);
-    }
-    atomicAdd(&ranks[lane], rank);
-    __syncthreads();
-    if (part == 0 && i < M) keep[i] = ranks[lane] < n_keep ? 1 : 0;
+// ---- token selection: the n_keep highest scores, equal scores toward the lower index, ascending indices out ----
+// One CTA. Scores become 32-bit keys whose unsigned order is the scores' order (-0 and +0 share a key, so
+// they tie as they do in a float comparison). The key T of the n_keep-th highest score is built from the top,
+// two bits per pass: a digit is the largest one for which at least n_keep keys are >= the candidate (16
+// counting passes, one block-wide sum of three counts each). Every key above T is kept, and of the keys equal to T the first
+// n_keep - #{key > T} in index order; one block scan over (greater, equal) counts gives each kept token its
+// place in the output. Exactly n_keep indices are written whatever the scores hold (NaNs order by their bit
+// patterns: positive ones above +inf, negative ones below -inf).
+// REGS: M <= 4 * kSelThreads and each thread keeps its four consecutive tokens' keys in registers for all
+// passes (a counting pass is then twelve compares, two rounds of warp reductions and one barrier).
+constexpr int kSelThreads = 1024;
+constexpr int kSelStage = 8192;           // keys held in shared memory up to this M; beyond it every pass reads the scores
+
+__device__ __forceinline__ uint32_t score_key(float s) {
+    uint32_t u = __float_as_uint(s);
+    if (u == 0x80000000u) u = 0u;
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// One CTA of 1024 threads: exclusive scan of the keep flags, ascending indices out.
-__global__ void __launch_bounds__(1024)
-token_compact_idx_kernel(const uint8_t* __restrict__ keep, int M, int32_t* __restrict__ idx) {
-    __shared__ int warp_sums[32];
-    __shared__ int running;
-    if (threadIdx.x == 0) running = 0;
+template <bool REGS>
+__global__ void __launch_bounds__(kSelThreads)
+token_select_kernel(const float* __restrict__ scores, int M, int n_keep, int32_t* __restrict__ idx) {
+    __shared__ uint32_t skeys[REGS ? 1 : kSelStage];
+    __shared__ int wsum[2][3][32];
+    __shared__ unsigned long long wscan[32];
+    __shared__ unsigned long long running;
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const bool staged = !REGS && M <= kSelStage;
+    uint32_t kreg[4] = {0u, 0u, 0u, 0u};                 // key 0 is below every candidate of the passes
+    if (REGS) {
+#pragma unroll
+        for (int b = 0; b < 4; ++b)
+            if (4 * tid + b < M) kreg[b] = score_key(__ldg(scores + 4 * tid + b));
+    } else if (staged) {
+        for (int j = tid; j < M; j += kSelThreads) skeys[j] = score_key(__ldg(scores + j));
+    }
+    if (tid == 0) running = 0ull;
     __syncthreads();
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    for (int base = 0; base < M; base += 1024) {
-        const int i = base + threadIdx.x;
-        const int f = i < M ? keep[i] : 0;
-        int incl = f;
+    auto key_at = [&](int j) -> uint32_t { return staged ? skeys[j] : score_key(__ldg(scores + j)); };
+    // One pass settles two bits of T: the counts of keys >= T | (v << shift) for v = 1, 2, 3, the same values
+    // in every thread; T takes the largest v whose count still reaches n_keep. buf alternates so that a pass
+    // never overwrites sums a slower warp is still reading.
+    uint32_t T = 0u;
+    int above = 0;            // #{ key >= T + (1 << settled digits' lowest bit) }: 0 while nothing is settled
+    for (int shift = 30; shift >= 0; shift -= 2) {
+        const uint32_t c1 = T | (1u << shift), c2 = T | (2u << shift), c3 = T | (3u << shift);
+        int n1 = 0, n2 = 0, n3 = 0;
+        if (REGS) {
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                n1 += (int)(kreg[b] >= c1); n2 += (int)(kreg[b] >= c2); n3 += (int)(kreg[b] >= c3);
+            }
+        } else {
+            for (int j = tid; j < M; j += kSelThreads) {
+                const uint32_t k = key_at(j);
+                n1 += (int)(k >= c1); n2 += (int)(k >= c2); n3 += (int)(k >= c3);
+            }
+        }
+        n1 = __reduce_add_sync(0xFFFFFFFFu, n1);
+        n2 = __reduce_add_sync(0xFFFFFFFFu, n2);
+        n3 = __reduce_add_sync(0xFFFFFFFFu, n3);
+        const int buf = (shift >> 1) & 1;
+        if (lane == 0) { wsum[buf][0][wid] = n1; wsum[buf][1][wid] = n2; wsum[buf][2][wid] = n3; }
+        __syncthreads();
+        n1 = __reduce_add_sync(0xFFFFFFFFu, wsum[buf][0][lane]);
+        n2 = __reduce_add_sync(0xFFFFFFFFu, wsum[buf][1][lane]);
+        n3 = __reduce_add_sync(0xFFFFFFFFu, wsum[buf][2][lane]);
+        // counts fall with v. The candidate one digit step above the chosen one is the next v, or, for
+        // v = 3, the previous pass's upper neighbour, whose count `above` already holds.
+        if (n3 >= n_keep)      { T = c3; }
+        else if (n2 >= n_keep) { T = c2; above = n3; }
+        else if (n1 >= n_keep) { T = c1; above = n2; }
+        else                   { above = n1; }
+    }
+    const int greater = above;                          // after the last pass the step is 1: #{ key > T }
+    const int need = n_keep - greater;                  // ties at T to keep, lowest indices first
+
+    // four consecutive tokens per thread; counts packed as (equal << 32) | greater
+    for (int base = 0; base < M; base += 4 * kSelThreads) {
+        const int j0 = base + 4 * tid;
+        uint32_t gt = 0u, eq = 0u;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            if (j0 + b < M) {
+                const uint32_t k = REGS ? kreg[b] : key_at(j0 + b);
+                gt |= (uint32_t)(k > T) << b;
+                eq |= (uint32_t)(k == T) << b;
+            }
+        }
+        const unsigned long long own = ((unsigned long long)__popc(eq) << 32) | (unsigned long long)__popc(gt);
+        unsigned long long incl = own;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
-            const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            const unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
             if (lane >= o) incl += t;
         }
-        if (lane == 31) warp_sums[wid] = incl;
+        if (lane == 31) wscan[wid] = incl;
         __syncthreads();
         if (wid == 0) {
-            int ws = warp_sums[lane];
+            unsigned long long ws = wscan[lane];
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
-                const int t = __shfl_up_sync(0xFFFFFFFFu, ws, o);
+                const unsigned long long t = __shfl_up_sync(0xFFFFFFFFu, ws, o);
                 if (lane >= o) ws += t;
             }
-            warp_sums[lane] = ws;   // inclusive over warps
+            wscan[lane] = ws;   // inclusive over warps
         }
         __syncthreads();
-        const int before = running + (wid ? warp_sums[wid - 1] : 0) + incl - f;
-        if (f) idx[before] = i;
+        const unsigned long long before = running + (wid ? wscan[wid - 1] : 0ull) + incl - own;
+        int gt_before = (int)(uint32_t)before, eq_before = (int)(before >> 32);
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+            if ((gt >> b) & 1u) {
+                idx[gt_before + min(eq_before, need)] = j0 + b;
+                ++gt_before;
+            } else if ((eq >> b) & 1u) {
+                if (eq_before < need) idx[gt_before + eq_before] = j0 + b;
+                ++eq_before;
+            }
+        }
         __syncthreads();
-        if (threadIdx.x == 0) running += warp_sums[31];
+        if (tid == 0) running += wscan[31];
         __syncthreads();
     }
 }
@@ -675,19 +763,29 @@ bool quantize_small_fits(int M, int K) { return (size_t)M * (size_t)K <= kSmallM
 cudaError_t launch_quantize_small(const __half* x, int M, int K, const int32_t* row_idx, int bits, int scale_mode,
                                   int clip_shift_or_exp, Control* ctl, int8_t* q, int32_t* scale_exp_out,
                                   cudaStream_t stream, const uint8_t* alpha, int k_max) {
-    quantize_small_kernel<<<kSmallCtas, kSmallThreads, 0, stream>>>(
-        reinterpret_cast<const uint4*>(x), M, K / 8, row_idx, bits, scale_mode, clip_shift_or_exp, ctl,
-        reinterpret_cast<uint2*>(q), scale_exp_out, reinterpret_cast<const uint2*>(alpha), k_max);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(kSmallCtas);
+    cfg.blockDim = dim3(kSmallThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;       // the kernel touches no memory before the kernel ahead of it has completed
+    return cudaLaunchKernelEx(&cfg, quantize_small_kernel, reinterpret_cast<const uint4*>(x), M, K / 8, row_idx, bits,
+                              scale_mode, clip_shift_or_exp, ctl, reinterpret_cast<uint2*>(q), scale_exp_out,
+                              reinterpret_cast<const uint2*>(alpha), k_max);
 }
 
 cudaError_t launch_token_select(const float* scores, int M, int n_keep, int32_t* idx, void* scratch,
                                 cudaStream_t stream) {
-    uint8_t* keep = static_cast<uint8_t*>(scratch);
-    token_rank_kernel<<<(M + 31) / 32, 32 * kRankWarps, 0, stream>>>(scores, M, n_keep, keep);
-    cudaError_t err = cudaGetLastError();
-    if (err != cudaSuccess) return err;
-    token_compact_idx_kernel<<<1, 1024, 0, stream>>>(keep, M, idx);
+    (void)scratch;
+    if (n_keep == 0) return cudaSuccess;
+    if (M <= 4 * kSelThreads)
+        token_select_kernel<true><<<1, kSelThreads, 0, stream>>>(scores, M, n_keep, idx);
+    else
+        token_select_kernel<false><<<1, kSelThreads, 0, stream>>>(scores, M, n_keep, idx);
     return cudaGetLastError();
 }
 

@@ -359,7 +359,8 @@ def test_results_are_deterministic_run_to_run():
 
 
 # ------------------------------------------------------------------------ token pruning
-@pytest.mark.parametrize("M,ratio", [(1, 1.0), (7, 0.5), (257, 0.6), (4096, 0.6), (1000, 0.0)])
+@pytest.mark.parametrize("M,ratio", [(1, 1.0), (7, 0.5), (257, 0.6), (4096, 0.6), (1000, 0.0), (4097, 1.0), (8192, 0.3),
+                                     (10000, 0.6), (65536, 0.41)])
 def test_token_select_and_compact(M, ratio):
     h = handle()
     scores = inputs.token_scores(M, seed=M)
@@ -373,6 +374,28 @@ def test_token_select_and_compact(M, ratio):
         x = inputs.activations(M, 128, seed=M + 1)
         xp = h.aq_token_compact(dev(x), dev(ref)).cpu().numpy()
         assert np.array_equal(xp.view(np.uint16), oracle.token_compact(x, ref).view(np.uint16))
+
+
+@pytest.mark.parametrize("M", [64, 5000, 9001])
+def test_token_select_on_signed_scores_zeros_and_infinities(M):
+    """Scores of both signs with -0 and +0 (equal in a float comparison, so they tie by index), infinities,
+    subnormals and long runs of equal values; every n_keep that cuts inside a run of ties."""
+    h = handle()
+    rng = np.random.default_rng(M)
+    scores = rng.standard_normal(M).astype(np.float32)
+    scores[rng.integers(0, M, M // 4)] = 0.0
+    scores[rng.integers(0, M, M // 4)] = -0.0
+    scores[rng.integers(0, M, M // 8)] = np.float32(1e-42)
+    scores[rng.integers(0, M, M // 8)] = np.float32(-1e-42)
+    scores[rng.integers(0, M, 3)] = np.inf
+    scores[rng.integers(0, M, 3)] = -np.inf
+    scores[rng.integers(0, M, M // 8)] = scores[0]
+    sd = dev(scores)
+    n_zero_or_more = int((scores >= 0).sum())
+    for n_keep in sorted({1, 2, 3, M // 2, n_zero_or_more - 1, n_zero_or_more, int((scores > 0).sum()) + 1, M - 1, M}):
+        if 0 < n_keep <= M:
+            idx = h.aq_token_select(sd, n_keep).cpu().numpy()
+            assert np.array_equal(idx, oracle.token_select(scores, n_keep)), n_keep
 
 
 # ------------------------------------------------------------------------ device status
