@@ -181,7 +181,6 @@ gemm_decode_kernel(const int8_t* __restrict__ q, int M, int K, int N, int Npad,
 // ---------------------------------------------------------------------------------------
 // Streaming kernel (one scale per channel, M <= 16)
 // ---------------------------------------------------------------------------------------
-constexpr int kStrStages = 8;
 constexpr int kStrConsumerWarps = 8;
 constexpr int kStrThreads = (1 + kStrConsumerWarps) * 32;
 constexpr unsigned long long kStrWaitCycles = 4000000000ull;
@@ -214,24 +213,34 @@ __device__ __forceinline__ bool str_wait(uint64_t* bar, uint32_t parity, volatil
 // One row uses dp4a with one lane per channel; more rows use the warp-level int8 MMA
 // (m16n8k32) on 16 rows, with the activation tile stored 128-byte swizzled so that fragment
 // loads are free of bank conflicts.
+// Ring depth 8 (64 KB of weights in flight per CTA, two CTAs per SM): 9 stages for 16 rows and 12 for one
+// row, which shared memory would allow, measured no faster.
+// Producer lanes: a wait, an expect and two copies per block are four shared-memory-pipe instructions of a
+// hundred cycles and more each next to the working consumers, so one lane cannot issue faster than a block
+// per ~500 cycles, which bounds a CTA that streams alone on its SM. With two lanes of the warp in lockstep
+// (lane l takes the blocks l, l + 2, ... of the k range) the single-row kernel gains 0.3-1.1 us per launch;
+// four lanes gain no more, eight lose, and with 16 rows (tensor-map copies of the codes) two lanes measured
+// 0.1-0.3 us slower than one.
 template <int MB> struct StreamCfg {
     static constexpr bool kUseMma = MB > 4;
     static constexpr int kRows = kUseMma ? 16 : MB;
+    static constexpr int kStages = 8;
+    static constexpr int kProdLanes = kUseMma ? 1 : 2;
 };
 
 template <int MB>
 struct StreamSmem {
     static constexpr int kRows = StreamCfg<MB>::kRows;
-    alignas(1024) int8_t x[kStrStages][kRows * kTileK];    // activation codes of the unit's k block
-    alignas(128) uint8_t w[kStrStages][kBlockBytes];       // packed weight block of the unit
-    int part[4][kRows][32];                                // the odd-k-block warp's partial sums
+    static constexpr int kStages = StreamCfg<MB>::kStages;
+    alignas(1024) int8_t x[kStages][kRows * kTileK];       // activation codes of the unit's k block
+    alignas(128) uint8_t w[kStages][kBlockBytes];          // packed weight block of the unit
     alignas(16) int sum[kRows][kTileN];                    // this CTA's sums over its k range
     // one row quantized by the kernel itself: the codes of this CTA's k range (up to kFuseMaxBlocks blocks)
     alignas(16) int8_t xq[MB == 1 ? kFuseMaxBlocks * kTileK : 16];
     unsigned int warp_max[kStrThreads / 32];
     alignas(16) int recv[kRows][kTileN];                               // the other CTAs' sums for this CTA's channel slice, by sender
-    alignas(8) uint64_t full[kStrStages];
-    uint64_t empty[kStrStages];
+    alignas(8) uint64_t full[kStages];
+    uint64_t empty[kStages];
     volatile uint32_t abort_flag;
 };
 
@@ -268,6 +277,7 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     constexpr bool kUseMma = StreamCfg<MB>::kUseMma;
     constexpr int kRows = StreamCfg<MB>::kRows;
+    constexpr int kStrStages = StreamCfg<MB>::kStages;
     cg::cluster_group cluster = cg::this_cluster();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KB = k_blocks(p.K);
@@ -327,18 +337,24 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     // before it on the stream still ran. Nothing written before this launch is read, and nothing is written,
     // until that kernel has completed; only behind the call's own quantize kernel (which allows this
     // launch only once everything before it, weight packing included, has completed) the weights are fetched first.
+    // The producer is kProdLanes lanes of warp 0 in lockstep, lane l taking the blocks l, l + kProdLanes, ...
+    constexpr int kProdLanes = StreamCfg<MB>::kProdLanes;
+    const bool producer = warp == 0 && lane < kProdLanes;
+    const int ring = min(kStrStages, kb1 - kb0);      // blocks of the first ring
     int issued = 0;
     if (!p.clear_status) {                            // launched behind this call's own quantize kernel
-        if (warp == 0 && lane == 0)
-            for (; issued < kStrStages && kb0 + issued < kb1; ++issued) issue_w(kb0 + issued, issued);
+        if (producer)
+            for (int i = lane; i < ring; i += kProdLanes) issue_w(kb0 + i, i);
+        issued = ring;
     }
     asm volatile("griddepcontrol.wait;" ::: "memory");
     if (p.clear_status && blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) p.ctl->status = 0;   // nothing has given up yet
     [[maybe_unused]] int fused_exp = 0;
     if constexpr (FUSEQ) {
         // ---- the layer scale and this CTA's codes (Eq. 1, Eq. 2 / Eq. 5 with zp = 0; one scale for the layer)
-        if (warp == 0 && lane == 0)
-            for (; issued < kStrStages && kb0 + issued < kb1; ++issued) issue_w(kb0 + issued, issued);   // weights on their way meanwhile
+        if (producer)
+            for (int i = issued + lane; i < ring; i += kProdLanes) issue_w(kb0 + i, i);   // weights on their way meanwhile
+        issued = ring;
         const uint4* xv = reinterpret_cast<const uint4*>(p.x_row + (p.row_idx ? (size_t)p.row_idx[0] * p.K : 0));
         int e = p.clip_shift_or_exp;
         // up to kKeep vectors per thread stay in registers between the two passes (K <= 18432); longer rows
@@ -412,9 +428,9 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
         __syncthreads();
     }
     if (warp == 0) {
-        if (lane == 0) {
-            for (int i = 0; i < issued; ++i) issue_x(kb0 + i, i);
-            for (int kb = kb0 + issued; kb < kb1; ++kb) {
+        if (producer) {
+            for (int i = lane; i < issued; i += kProdLanes) issue_x(kb0 + i, i);
+            for (int kb = kb0 + issued + lane; kb < kb1; kb += kProdLanes) {
                 const uint32_t i = (uint32_t)(kb - kb0);
                 const int s = (int)(i % kStrStages);
                 if (!str_wait(&sm.empty[s], ((i / kStrStages) & 1u) ^ 1u, abort_flag)) break;
@@ -464,15 +480,16 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
                 __syncwarp();
                 if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s_u32(&sm.empty[s])) : "memory");
             }
-            // the two k-halves of a channel meet in shared memory: this CTA's sums over its k range
-            if (half == 1) {
-#pragma unroll
-                for (int m = 0; m < MB; ++m) sm.part[quarter][m][lane] = acc[m];
-            }
-            asm volatile("bar.sync 1, %0;" ::"n"(kStrConsumerWarps * 32) : "memory");
+            // the two k-halves of a channel meet in shared memory: this CTA's sums over its k range (the same
+            // thread position owns an element in both warps: one stores, then the other adds)
             if (half == 0) {
 #pragma unroll
-                for (int m = 0; m < MB; ++m) sm.sum[m][r] = acc[m] + sm.part[quarter][m][lane];
+                for (int m = 0; m < MB; ++m) sm.sum[m][r] = acc[m];
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(kStrConsumerWarps * 32) : "memory");
+            if (half == 1) {
+#pragma unroll
+                for (int m = 0; m < MB; ++m) sm.sum[m][r] += acc[m];
             }
         } else {
             // Warp-level int8 MMA, D[16 rows x 8 channels] += A[16 x 32 k] * B[32 k x 8 channels].
@@ -518,21 +535,18 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
                 if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s_u32(&sm.empty[s])) : "memory");
             }
             // D fragment: acc[i][0..1] = row g, channels 8i+2t, +1; acc[i][2..3] = row g+8
-            if (half == 1) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) sm.part[quarter][g + 8 * (c >> 1)][8 * i + 2 * t + (c & 1)] = acc[i][c];
-            }
-            asm volatile("bar.sync 1, %0;" ::"n"(kStrConsumerWarps * 32) : "memory");
             if (half == 0) {
 #pragma unroll
                 for (int i = 0; i < 4; ++i)
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const int m = g + 8 * (c >> 1), ch = 8 * i + 2 * t + (c & 1);
-                        sm.sum[m][quarter * 32 + ch] = acc[i][c] + sm.part[quarter][m][ch];
-                    }
+                    for (int c = 0; c < 4; ++c) sm.sum[g + 8 * (c >> 1)][quarter * 32 + 8 * i + 2 * t + (c & 1)] = acc[i][c];
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(kStrConsumerWarps * 32) : "memory");
+            if (half == 1) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) sm.sum[g + 8 * (c >> 1)][quarter * 32 + 8 * i + 2 * t + (c & 1)] += acc[i][c];
             }
         }
     }
@@ -547,9 +561,11 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     // This CTA's k range is done: a launch behind this one that allows it may be scheduled and set up now
     // (it reads and writes nothing before this grid has completed).
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const int cw = kTileN / split;                            // split is 1, 2 or 4
+    const int cw = kTileN / split;                            // split is 1, 2 or 4: a power of two, so
+    const int cw_log = 7 - (31 - __clz(split));               // divisions by cw are shifts
     const int ft = (int)threadIdx.x - 32;                     // the 256 consumer threads finish; cw divides 256
-    const int out_r = rank * cw + (ft >= 0 ? ft % cw : 0);
+    const int rc = ft & (cw - 1);                             // channel inside the slice (only used when ft >= 0)
+    const int out_r = rank * cw + rc;
     const int out_n = tile * kTileN + out_r;
     float sc = 0.0f, off = 0.0f;
     if (ft >= 0 && out_n < p.N) {
@@ -564,10 +580,10 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
         if (ft >= 0) {
             // four consecutive channels at a time (16-byte remote stores) go to the CTA that owns them
             for (int e = ft; e < rows * (kTileN / 4); e += kStrConsumerWarps * 32) {
-                const int m = e / (kTileN / 4), ch = 4 * (e % (kTileN / 4));
-                const int owner = ch / cw;
+                const int m = e >> 5, ch = 4 * (e & 31);
+                const int owner = ch >> cw_log;
                 if (owner != rank)
-                    *reinterpret_cast<int4*>(cluster.map_shared_rank(&sm.recv[0][0], owner) + m * kTileN + rank * cw + (ch % cw)) =
+                    *reinterpret_cast<int4*>(cluster.map_shared_rank(&sm.recv[0][0], owner) + m * kTileN + rank * cw + (ch & (cw - 1))) =
                         *reinterpret_cast<const int4*>(&sm.sum[m][ch]);
             }
         }
@@ -577,18 +593,45 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
         __syncthreads();
     }
     if (ft >= 0 && out_n < p.N) {
-        for (int m = ft / cw; m < rows; m += (kStrConsumerWarps * 32) / cw) {
-            int a = sm.sum[m][out_r];
-            for (int c = 0; c < split; ++c)
-                if (c != rank) a += sm.recv[m][c * cw + (out_r % cw)];
-            a >>= 4;                                              // sums carry a factor 16
-            if (p.acc_dump) p.acc_dump[(size_t)m * p.N + out_n] = a;
-            const __half hv = __float2half_rn(fmaf((float)a, sc, off));
-            // (a warp's lanes hold consecutive channels and run this loop together: 128 / split >= 32)
-            if (p.q_next)
-                store_next_code(p.q_next, (size_t)m * p.N + out_n, next_code(hv, p.next_inv, p.next_lo, p.next_hi),
-                                p.next_packed, true, lane);
-            else p.y[(size_t)m * p.N + out_n] = hv;
+        // All shared-memory reads of this thread's outputs are issued before the first is used and without
+        // branches around them (rows that do not exist read the last row of the buffer and are dropped):
+        // taken one after the other, each behind its own test, they were the longest part of the finish at
+        // 16 rows.
+        constexpr int kIt = kRows >= 16 ? 8 : (kRows + 1) / 2;    // a pass of the 256 threads covers 256 / cw >= 2 rows
+        const int stride = (kStrConsumerWarps * 32) >> cw_log, m0 = ft >> cw_log;
+        int av[kIt];
+#pragma unroll
+        for (int i = 0; i < kIt; ++i) av[i] = sm.sum[min(m0 + i * stride, kRows - 1)][out_r];
+#pragma unroll
+        for (int k = 1; k < 4; ++k) {
+            if (k < split) {
+                const int col = ((rank + k) & (split - 1)) * cw + rc;         // the k-th other CTA's slot
+#pragma unroll
+                for (int i = 0; i < kIt; ++i) av[i] += sm.recv[min(m0 + i * stride, kRows - 1)][col];
+            }
+        }
+        if (!p.acc_dump && !p.q_next) {
+#pragma unroll
+            for (int i = 0; i < kIt; ++i) {
+                const int m = m0 + i * stride;
+                const __half hv = __float2half_rn(fmaf((float)(av[i] >> 4), sc, off));     // sums carry a factor 16
+                if (m < rows) p.y[(size_t)m * p.N + out_n] = hv;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < kIt; ++i) {
+                const int m = m0 + i * stride;
+                if (m < rows) {
+                    const int a = av[i] >> 4;
+                    if (p.acc_dump) p.acc_dump[(size_t)m * p.N + out_n] = a;
+                    const __half hv = __float2half_rn(fmaf((float)a, sc, off));
+                    // (a warp's lanes hold consecutive channels and run this loop together: 128 / split >= 32)
+                    if (p.q_next)
+                        store_next_code(p.q_next, (size_t)m * p.N + out_n, next_code(hv, p.next_inv, p.next_lo, p.next_hi),
+                                        p.next_packed, true, lane);
+                    else p.y[(size_t)m * p.N + out_n] = hv;
+                }
+            }
         }
     }
     if (sm.abort_flag) {
