@@ -181,8 +181,6 @@ gemm_decode_kernel(const int8_t* __restrict__ q, int M, int K, int N, int Npad,
 // ---------------------------------------------------------------------------------------
 // Streaming kernel (one scale per channel, M <= 16)
 // ---------------------------------------------------------------------------------------
-constexpr int kStrConsumerWarps = 8;
-constexpr int kStrThreads = (1 + kStrConsumerWarps) * 32;
 constexpr unsigned long long kStrWaitCycles = 4000000000ull;
 constexpr int kFuseMaxBlocks = 64;        // k blocks per CTA up to which a single row is quantized inside the product kernel
 
@@ -226,6 +224,14 @@ template <int MB> struct StreamCfg {
     static constexpr int kRows = kUseMma ? 16 : MB;
     static constexpr int kStages = 8;
     static constexpr int kProdLanes = kUseMma ? 1 : 2;
+    // Consumer warps: a channel quarter each, kPhases warps per quarter taking the k blocks in turn. A third
+    // warp per quarter measured slower with 16 rows (7.6 / 11.4 / 13.6 -> 8.5 / 12.0 / 14.4 us on the 13B
+    // shapes) although a warp holds a block for 600-700 cycles there: the stream slows with the amount of
+    // consumer work in flight, not with the time a block waits (with the consumers' arithmetic taken out the
+    // same launches take 6.6 / 9.1 / 10.1 us, and the ring is never full either way).
+    static constexpr int kPhases = 2;
+    static constexpr int kConsumerWarps = 4 * kPhases;
+    static constexpr int kThreads = (1 + kConsumerWarps) * 32;
 };
 
 template <int MB>
@@ -237,7 +243,7 @@ struct StreamSmem {
     alignas(16) int sum[kRows][kTileN];                    // this CTA's sums over its k range
     // one row quantized by the kernel itself: the codes of this CTA's k range (up to kFuseMaxBlocks blocks)
     alignas(16) int8_t xq[MB == 1 ? kFuseMaxBlocks * kTileK : 16];
-    unsigned int warp_max[kStrThreads / 32];
+    unsigned int warp_max[StreamCfg<MB>::kThreads / 32];
     alignas(16) int recv[kRows][kTileN];                               // the other CTAs' sums for this CTA's channel slice, by sender
     alignas(8) uint64_t full[kStages];
     uint64_t empty[kStages];
@@ -269,7 +275,7 @@ struct StreamParams {
 // grid = (split, channel tiles), cluster = (split, 1, 1): the CTAs of a cluster share a channel
 // tile and take consecutive k ranges; CTA r adds up and writes channels [r, r+1) * 128 / split.
 template <int MB, bool FUSEQ = false>
-__global__ void __launch_bounds__(kStrThreads, 2)
+__global__ void __launch_bounds__(StreamCfg<MB>::kThreads, 2)
 gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const StreamParams p) {
     static_assert(!FUSEQ || MB == 1, "only a single row is quantized inside the product kernel");
     extern __shared__ uint8_t smem_raw[];
@@ -278,6 +284,9 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     constexpr bool kUseMma = StreamCfg<MB>::kUseMma;
     constexpr int kRows = StreamCfg<MB>::kRows;
     constexpr int kStrStages = StreamCfg<MB>::kStages;
+    constexpr int kPhases = StreamCfg<MB>::kPhases;
+    constexpr int kStrConsumerWarps = StreamCfg<MB>::kConsumerWarps;
+    constexpr int kStrThreads = StreamCfg<MB>::kThreads;
     cg::cluster_group cluster = cg::this_cluster();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int KB = k_blocks(p.K);
@@ -293,7 +302,7 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
             asm volatile("prefetch.tensormap [%0];" ::"l"(&x_map) : "memory");
         for (int s = 0; s < kStrStages; ++s) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(s_u32(&sm.full[s])) : "memory");
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s_u32(&sm.empty[s])), "r"(kStrConsumerWarps / 2) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s_u32(&sm.empty[s])), "r"(4) : "memory");   // the four quarter warps of the block's phase
         }
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -440,56 +449,76 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
         }
     } else {
         const int cw = warp - 1;
-        const int quarter = cw & 3, half = cw >> 2;
+        const int quarter = cw & 3, phase = cw >> 2;
         if constexpr (!kUseMma) {
-            const int r = quarter * 32 + lane;                       // channel inside the tile
-            int acc[MB];
+            // A lane takes one 32-k chunk of the block (t = lane / 8) and eight channels per pass (g = lane % 8,
+            // four passes cover the warp's 32 channels): per block it reads four 16-byte weight units (chunk t
+            // of channels 8i + g; the eight lanes of a quarter warp read eight consecutive units) and the 32
+            // activation bytes of its chunk, six 16-byte shared-memory loads where one lane per channel, every
+            // lane reading every activation byte, took twelve. The sum over k does not care which lane adds
+            // which k; the lanes' partial sums meet once, after the k range.
+            const int g = lane & 7, t = lane >> 3;
+            int acc[MB][4];
 #pragma unroll
-            for (int m = 0; m < MB; ++m) acc[m] = 0;
-            for (int kb = kb0 + half; kb < kb1; kb += 2) {       // the two warps of a quarter take alternate k blocks
-                const uint32_t i = (uint32_t)(kb - kb0);
-                const int s = (int)(i % kStrStages);
-                if (!__all_sync(0xFFFFFFFFu, str_wait(&sm.full[s], (i / kStrStages) & 1u, abort_flag) ? 1 : 0)) break;
+            for (int m = 0; m < MB; ++m)
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint4 d = reinterpret_cast<const uint4*>(sm.w[s])[j * kTileN + r];
-                    const uint32_t w[4] = {d.x, d.y, d.z, d.w};
-                    uint32_t w8[8];
+                for (int i = 0; i < 4; ++i) acc[m][i] = 0;
+            for (int kb = kb0 + phase; kb < kb1; kb += kPhases) {       // the warps of a quarter take the k blocks in turn
+                const uint32_t it = (uint32_t)(kb - kb0);
+                const int s = (int)(it % kStrStages);
+                if (!__all_sync(0xFFFFFFFFu, str_wait(&sm.full[s], (it / kStrStages) & 1u, abort_flag) ? 1 : 0)) break;
+                uint4 wv[4];
 #pragma unroll
-                    for (int t = 0; t < 4; ++t) {
-                        w8[2 * t] = (w[t] << 4) & 0xF0F0F0F0u;           // 16*code for k0..k0+3
-                        w8[2 * t + 1] = w[t] & 0xF0F0F0F0u;              // 16*code for k0+4..k0+7
-                    }
+                for (int i = 0; i < 4; ++i)
+                    wv[i] = reinterpret_cast<const uint4*>(sm.w[s])[t * kTileN + quarter * 32 + 8 * i + g];
 #pragma unroll
-                    for (int m = 0; m < MB; ++m) {
-                        const uint4* xp = FUSEQ ? reinterpret_cast<const uint4*>(sm.xq + (size_t)(kb - kb0) * kTileK + 32 * j)
-                                                : reinterpret_cast<const uint4*>(sm.x[s] + m * kTileK + 32 * j);
-                        const uint4 x0 = xp[0], x1 = xp[1];              // same address in every lane: broadcast
-                        int a = acc[m];
-                        a = __dp4a((int)w8[0], (int)x0.x, a);
-                        a = __dp4a((int)w8[1], (int)x0.y, a);
-                        a = __dp4a((int)w8[2], (int)x0.z, a);
-                        a = __dp4a((int)w8[3], (int)x0.w, a);
-                        a = __dp4a((int)w8[4], (int)x1.x, a);
-                        a = __dp4a((int)w8[5], (int)x1.y, a);
-                        a = __dp4a((int)w8[6], (int)x1.z, a);
-                        a = __dp4a((int)w8[7], (int)x1.w, a);
-                        acc[m] = a;
+                for (int m = 0; m < MB; ++m) {
+                    const uint4* xp = FUSEQ ? reinterpret_cast<const uint4*>(sm.xq + (size_t)(kb - kb0) * kTileK + 32 * t)
+                                            : reinterpret_cast<const uint4*>(sm.x[s] + m * kTileK + 32 * t);
+                    const uint4 x0 = xp[0], x1 = xp[1];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        // word u of a unit: k 8u..8u+3 of the chunk in its low nibbles, k 8u+4..8u+7 in its high ones
+                        const uint32_t w[4] = {wv[i].x, wv[i].y, wv[i].z, wv[i].w};
+                        int a = acc[m][i];
+                        a = __dp4a((int)((w[0] << 4) & 0xF0F0F0F0u), (int)x0.x, a);      // 16*code
+                        a = __dp4a((int)(w[0] & 0xF0F0F0F0u), (int)x0.y, a);
+                        a = __dp4a((int)((w[1] << 4) & 0xF0F0F0F0u), (int)x0.z, a);
+                        a = __dp4a((int)(w[1] & 0xF0F0F0F0u), (int)x0.w, a);
+                        a = __dp4a((int)((w[2] << 4) & 0xF0F0F0F0u), (int)x1.x, a);
+                        a = __dp4a((int)(w[2] & 0xF0F0F0F0u), (int)x1.y, a);
+                        a = __dp4a((int)((w[3] << 4) & 0xF0F0F0F0u), (int)x1.z, a);
+                        a = __dp4a((int)(w[3] & 0xF0F0F0F0u), (int)x1.w, a);
+                        acc[m][i] = a;
                     }
                 }
                 __syncwarp();
                 if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s_u32(&sm.empty[s])) : "memory");
             }
-            // the two k-halves of a channel meet in shared memory: this CTA's sums over its k range (the same
-            // thread position owns an element in both warps: one stores, then the other adds)
-            if (half == 0) {
+            // the four chunks of a channel meet (two exchange steps), then lane (g, t) keeps pass t's channel
+            // 8t + g; the warps of a quarter meet in the sum buffer, one after the other (the same thread
+            // position owns an element in each of them: the first stores, the others add)
+            int mine[MB];
 #pragma unroll
-                for (int m = 0; m < MB; ++m) sm.sum[m][r] = acc[m];
+            for (int m = 0; m < MB; ++m) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    acc[m][i] += __shfl_xor_sync(0xFFFFFFFFu, acc[m][i], 8);
+                    acc[m][i] += __shfl_xor_sync(0xFFFFFFFFu, acc[m][i], 16);
+                }
+                mine[m] = t == 0 ? acc[m][0] : t == 1 ? acc[m][1] : t == 2 ? acc[m][2] : acc[m][3];
             }
-            asm volatile("bar.sync 1, %0;" ::"n"(kStrConsumerWarps * 32) : "memory");
-            if (half == 1) {
+            const int r = quarter * 32 + 8 * t + g;                  // channel inside the tile
 #pragma unroll
-                for (int m = 0; m < MB; ++m) sm.sum[m][r] += acc[m];
+            for (int ph = 0; ph < kPhases; ++ph) {
+                if (ph > 0) asm volatile("bar.sync 1, %0;" ::"n"(kStrConsumerWarps * 32) : "memory");
+                if (phase == ph) {
+#pragma unroll
+                    for (int m = 0; m < MB; ++m) {
+                        if (ph == 0) sm.sum[m][r] = mine[m];
+                        else sm.sum[m][r] += mine[m];
+                    }
+                }
             }
         } else {
             // Warp-level int8 MMA, D[16 rows x 8 channels] += A[16 x 32 k] * B[32 k x 8 channels].
@@ -501,7 +530,7 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
             for (int i = 0; i < 4; ++i)
 #pragma unroll
                 for (int c = 0; c < 4; ++c) acc[i][c] = 0;
-            for (int kb = kb0 + half; kb < kb1; kb += 2) {       // the two warps of a quarter take alternate k blocks
+            for (int kb = kb0 + phase; kb < kb1; kb += kPhases) {       // the warps of a quarter take the k blocks in turn
                 const uint32_t it = (uint32_t)(kb - kb0);
                 const int s = (int)(it % kStrStages);
                 if (!__all_sync(0xFFFFFFFFu, str_wait(&sm.full[s], (it / kStrStages) & 1u, abort_flag) ? 1 : 0)) break;
@@ -535,18 +564,21 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
                 if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s_u32(&sm.empty[s])) : "memory");
             }
             // D fragment: acc[i][0..1] = row g, channels 8i+2t, +1; acc[i][2..3] = row g+8
-            if (half == 0) {
+            // the warps of a quarter meet in the sum buffer, one after the other (the same thread position
+            // owns an element in each of them: the first stores, the others add)
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
+            for (int ph = 0; ph < kPhases; ++ph) {
+                if (ph > 0) asm volatile("bar.sync 1, %0;" ::"n"(kStrConsumerWarps * 32) : "memory");
+                if (phase == ph) {
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) sm.sum[g + 8 * (c >> 1)][quarter * 32 + 8 * i + 2 * t + (c & 1)] = acc[i][c];
-            }
-            asm volatile("bar.sync 1, %0;" ::"n"(kStrConsumerWarps * 32) : "memory");
-            if (half == 1) {
+                    for (int i = 0; i < 4; ++i)
 #pragma unroll
-                for (int i = 0; i < 4; ++i)
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) sm.sum[g + 8 * (c >> 1)][quarter * 32 + 8 * i + 2 * t + (c & 1)] += acc[i][c];
+                        for (int c = 0; c < 4; ++c) {
+                            int& dst = sm.sum[g + 8 * (c >> 1)][quarter * 32 + 8 * i + 2 * t + (c & 1)];
+                            if (ph == 0) dst = acc[i][c];
+                            else dst += acc[i][c];
+                        }
+                }
             }
         }
     }
@@ -563,7 +595,7 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int cw = kTileN / split;                            // split is 1, 2 or 4: a power of two, so
     const int cw_log = 7 - (31 - __clz(split));               // divisions by cw are shifts
-    const int ft = (int)threadIdx.x - 32;                     // the 256 consumer threads finish; cw divides 256
+    const int ft = (int)threadIdx.x - 32;                     // the consumer threads finish (a multiple of 128 = 4 cw at most)
     const int rc = ft & (cw - 1);                             // channel inside the slice (only used when ft >= 0)
     const int out_r = rank * cw + rc;
     const int out_n = tile * kTileN + out_r;
@@ -597,7 +629,7 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
         // branches around them (rows that do not exist read the last row of the buffer and are dropped):
         // taken one after the other, each behind its own test, they were the longest part of the finish at
         // 16 rows.
-        constexpr int kIt = kRows >= 16 ? 8 : (kRows + 1) / 2;    // a pass of the 256 threads covers 256 / cw >= 2 rows
+        constexpr int kIt = (kRows + kPhases - 1) / kPhases;      // a pass of the consumer threads covers at least kPhases rows
         const int stride = (kStrConsumerWarps * 32) >> cw_log, m0 = ft >> cw_log;
         int av[kIt];
 #pragma unroll
@@ -683,7 +715,7 @@ cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t
     while (split < 4 && tiles * split * 2 <= 2 * dev.sm_count && KB / (split * 2) >= 2) split *= 2;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(split, tiles, 1);
-    cfg.blockDim = dim3(kStrThreads);
+    cfg.blockDim = dim3(StreamCfg<MB>::kThreads);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
@@ -730,7 +762,8 @@ bool decode_can_fuse_quantize(int M, int K, int N, int group, int sm_count) {
 cudaError_t launch_gemm_decode(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
     if (!a.group && a.M <= 16) {
         // one row: dp4a; 2..16 rows: the warp MMA on a 16-row tile (fewer instructions per weight
-        // chunk than dp4a from two rows on; measured faster at M = 4)
+        // chunk than dp4a from two rows on; measured faster at M = 4: 7.5 / 11.1 / 13.3 us against
+        // 8.1 / 12.8 / 15.2 us on the three 13B shapes)
         if (a.M <= 1 && a.fuse_x) return launch_stream<1, true>(a, dev, stream);
         if (a.M <= 1) return launch_stream<1>(a, dev, stream);
         return launch_stream<16>(a, dev, stream);
