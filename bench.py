@@ -250,10 +250,20 @@ def bench_decode(h, peaks, iters=40):
                 for i in range(copies):
                     h.aq_linear_w4a8(x, packs[i][0], packs[i][1], s.N, 0, y=y, workspace=ws)
             layer_ms = graph_replay_ms(launch_layer, max(2, iters // copies)) / copies
+            # the same two sequences with the caller's promise that nothing in flight writes the weights
+            # (aq_set_weights_stable): consecutive launches overlap; reported beside the default, not instead
+            h.aq_set_weights_stable(True)
+            try:
+                ms_st = graph_replay_ms(launch, max(2, iters // copies)) / copies
+                layer_ms_st = graph_replay_ms(launch_layer, max(2, iters // copies)) / copies
+            finally:
+                h.aq_set_weights_stable(False)
             algo = wbytes + 2 * s.N + M * s.K + 2 * M * s.N
             gbs = algo / (ms * 1e-3) / 1e9
             out.append({"K": s.K, "N": s.N, "M": M, "us": ms * 1e3, "layer_us": layer_ms * 1e3, "GBps": gbs,
-                        "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]})
+                        "frac_of_hbm_peak": gbs / peaks["hbm_gbs"],
+                        "weights_stable": {"us": ms_st * 1e3, "layer_us": layer_ms_st * 1e3,
+                                           "frac_of_hbm_peak": algo / (ms_st * 1e-3) / 1e9 / peaks["hbm_gbs"]}})
         del packs
     return out
 

@@ -72,6 +72,15 @@ int aq_destroy(aq_handle_t h);
 int aq_last_cuda_error(aq_handle_t h);
 /* Force a kernel choice for subsequent calls on this handle (AQ_KERNEL_*). */
 int aq_set_kernel(aq_handle_t h, int kernel);
+/* A scheduling promise, not part of the paper's method; off by default. enabled != 0 tells the library that,
+ * for every later call on this handle, no work still in flight on the call's stream when the call is enqueued
+ * writes the packed weights or weight scales the call reads (the usual case: weights are packed once, before
+ * inference starts). The few-row kernels (M <= 16, one scale per channel) then let the launch behind them be
+ * set up from their start and fetch their first 64 KB of weights per CTA before they wait for the kernel ahead
+ * of them; everything else a call reads or writes still waits for that kernel. Results are the same bit for
+ * bit; consecutive few-row calls on one stream overlap by a microsecond or two. With the promise broken (a
+ * kernel that writes the weights is still running when the call starts) the call may read stale weights. */
+int aq_set_weights_stable(aq_handle_t h, int enabled);
 
 /* ---- sizes -------------------------------------------------------------------------- */
 /* Bytes of the packed 4-bit weight buffer (rows are padded to a multiple of 128 channels, and K to a

@@ -58,6 +58,7 @@ def load():
     L.aq_destroy.argtypes = [vp]
     L.aq_last_cuda_error.argtypes = [vp]
     L.aq_set_kernel.argtypes = [vp, i32]
+    L.aq_set_weights_stable.argtypes = [vp, i32]
     for f in ("aq_packed_w4_bytes",):
         getattr(L, f).restype = sz
         getattr(L, f).argtypes = [i32, i32]
@@ -199,6 +200,9 @@ class Handle:
 
     def aq_set_kernel(self, kernel: int):
         _check(load().aq_set_kernel(self._h, kernel), "aq_set_kernel")
+
+    def aq_set_weights_stable(self, enabled: bool):
+        _check(load().aq_set_weights_stable(self._h, 1 if enabled else 0), "aq_set_weights_stable")
 
     def aq_last_cuda_error(self) -> int:
         return load().aq_last_cuda_error(self._h)

@@ -10,6 +10,7 @@ struct aq_context {
     aq::DeviceInfo dev;
     int last_cuda_error;
     int kernel_choice;
+    int weights_stable;
 };
 
 namespace {
@@ -77,8 +78,10 @@ int kernel_for(aq_handle_t h, int M) {
 
 int run_gemm(aq_handle_t h, const GemmArgs& g, cudaStream_t stream) {
     const int choice = kernel_for(h, g.M);
-    const cudaError_t e = choice == AQ_KERNEL_DECODE ? launch_gemm_decode(g, h->dev, stream)
-                                                     : launch_gemm_tensor(g, h->dev, stream);
+    GemmArgs a = g;
+    a.weights_stable = h->weights_stable != 0;
+    const cudaError_t e = choice == AQ_KERNEL_DECODE ? launch_gemm_decode(a, h->dev, stream)
+                                                     : launch_gemm_tensor(a, h->dev, stream);
     return e == cudaSuccess ? AQ_OK : cuda_fail(h, e);
 }
 
@@ -91,7 +94,7 @@ cudaError_t quantize_dispatch(aq_handle_t h, const __half* xh, int M, int K, con
         // small activations (decode): one kernel finds the scale, writes the codes and initialises
         // the control block
         return launch_quantize_small(xh, M, K, row_idx, bits, scale_mode, clip_shift_or_exp, ctl, q, scale_exp_out,
-                                     stream, alpha, k_max);
+                                     stream, alpha, k_max, h->weights_stable != 0);
     const cudaError_t e = cudaMemsetAsync(ctl, 0, sizeof(Control), stream);
     if (e != cudaSuccess) return e;
     if (scale_mode == AQ_SCALE_DYNAMIC)
@@ -210,6 +213,7 @@ int aq_create(aq_handle_t* out, int device) {
     c->dev.encode_tiled = fn;
     c->last_cuda_error = 0;
     c->kernel_choice = AQ_KERNEL_AUTO;
+    c->weights_stable = 0;
     *out = c;
     return AQ_OK;
 }
@@ -230,6 +234,12 @@ void handle_record_cuda_error(aq_handle_t h, cudaError_t e) {
 }  // namespace aq
 
 extern "C" {
+
+int aq_set_weights_stable(aq_handle_t h, int enabled) {
+    if (!h) return AQ_ERR_INVALID_ARG;
+    h->weights_stable = enabled ? 1 : 0;
+    return AQ_OK;
+}
 
 int aq_set_kernel(aq_handle_t h, int kernel) {
     if (!h || kernel < AQ_KERNEL_AUTO || kernel > AQ_KERNEL_DECODE) return AQ_ERR_INVALID_ARG;

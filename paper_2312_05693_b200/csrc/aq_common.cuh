@@ -118,7 +118,8 @@ cudaError_t launch_quantize(const __half* x, int M, int K, const int32_t* row_id
 bool quantize_small_fits(int M, int K);
 cudaError_t launch_quantize_small(const __half* x, int M, int K, const int32_t* row_idx, int bits, int scale_mode,
                                   int clip_shift_or_exp, Control* ctl, int8_t* q, int32_t* scale_exp_out,
-                                  cudaStream_t stream, const uint8_t* alpha = nullptr, int k_max = 0);
+                                  cudaStream_t stream, const uint8_t* alpha = nullptr, int k_max = 0,
+                                  bool early_dependents = false);
 
 // Dynamic scale, any size: one cooperative kernel (absmax, exponent, codes). The control block must
 // have been cleared (absmax_bits, counter) on the same stream before.
@@ -188,6 +189,10 @@ struct GemmArgs {
     // kernels allow the dependent launch only once everything before them on the stream has completed (the
     // cooperative one is launched normally, the small one signals after its own wait for the kernel ahead).
     bool after_quantize = false;
+    // The caller's promise (aq_set_weights_stable) that nothing in flight on the stream writes the packed
+    // weights or their scales: the few-row kernel then allows the launch behind it at its very start and puts
+    // its own first ring of weight copies in flight before it waits for the kernel ahead of it.
+    bool weights_stable = false;
     // fp32 partial outputs of tiles whose k range two CTAs share (tensor kernel, per-group scales)
     float* split_scratch = nullptr;
     size_t split_bytes = 0;

@@ -266,6 +266,8 @@ struct StreamParams {
     int8_t* q_next;
     float next_inv, next_lo, next_hi;
     int clear_status;
+    int early_weights;             // the first ring of weight copies may be issued before the wait for the kernel ahead
+    int early_dependents;          // the launch behind this one may be set up from this kernel's start
     int next_packed;
     // FUSEQ (one row): the activations themselves; the kernel finds the layer scale, writes the codes of
     // its k range to shared memory (and, from the first channel tile, to q_out) and fills the control block
@@ -348,13 +350,17 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     // Launched with programmatic stream serialization: this grid may have been set up while the kernel
     // before it on the stream still ran. Nothing written before this launch is read, and nothing is written,
     // until that kernel has completed; only behind the call's own quantize kernel (which allows this
-    // launch only once everything before it, weight packing included, has completed) the weights are fetched first.
+    // launch only once everything before it, weight packing included, has completed), or on the caller's
+    // promise that nothing in flight writes the weights, the weights are fetched first. With that promise
+    // the launch behind this one is also allowed from the start, so that its CTAs take the places of this
+    // grid's CTAs as they leave and have their first ring on the way while this grid finishes.
     // The producer is kProdLanes lanes of warp 0 in lockstep, lane l taking the blocks l, l + kProdLanes, ...
     constexpr int kProdLanes = StreamCfg<MB>::kProdLanes;
     const bool producer = warp == 0 && lane < kProdLanes;
     const int ring = min(kStrStages, kb1 - kb0);      // blocks of the first ring
     int issued = 0;
-    if (!p.clear_status) {                            // launched behind this call's own quantize kernel
+    if (p.early_dependents) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (p.early_weights) {     // behind this call's own quantize kernel, or the caller has promised stable weights
         if (producer)
             for (int i = lane; i < ring; i += kProdLanes) issue_w(kb0 + i, i);
         issued = ring;
@@ -604,7 +610,7 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     // The scale is fetched before the cluster meets so that its latency overlaps the wait.
     // This CTA's k range is done: a launch behind this one that allows it may be scheduled and set up now
     // (it reads and writes nothing before this grid has completed).
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (!p.early_dependents) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int cw = kTileN / split;                            // split is 1, 2 or 4: a power of two, so
     const int cw_log = 7 - (31 - __clz(split));               // divisions by cw are shifts
     const int ft = (int)threadIdx.x - 32;                     // the consumer threads finish (a multiple of 128 = 4 cw at most)
@@ -719,7 +725,11 @@ cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t
     p.next_hi = (float)((1 << (a.next_bits - 1)) - 1);
     p.x_row = a.fuse_x; p.row_idx = a.fuse_row_idx; p.q_out = const_cast<int8_t*>(a.q);
     p.bits = a.fuse_bits; p.scale_mode = a.fuse_scale_mode; p.clip_shift_or_exp = a.fuse_clip_shift_or_exp;
-    if (FUSEQ) p.clear_status = 1;       // no quantize kernel of this call runs ahead: nothing is fetched before the wait
+    if (FUSEQ) p.clear_status = 1;       // no quantize kernel of this call runs ahead
+    // Weights ahead of the wait: behind the call's own quantize kernel (which allows this launch only once
+    // everything before it has completed), or on the caller's promise that nothing in flight writes them.
+    p.early_weights = (!p.clear_status || a.weights_stable) ? 1 : 0;
+    p.early_dependents = a.weights_stable ? 1 : 0;
     const int tiles = p.Npad / kTileN, KB = k_blocks(a.K);
     // as many k ranges per tile (cluster size 1, 2 or 4: clusters of 7-8 measured slower) as keep
     // all CTAs resident at once (two per SM), and at least two k blocks per CTA

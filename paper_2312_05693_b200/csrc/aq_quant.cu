@@ -88,7 +88,7 @@ __global__ void __cluster_dims__(kSmallCtas, 1, 1) __launch_bounds__(kSmallThrea
 quantize_small_kernel(const uint4* __restrict__ x, int M, int vec_per_row, const int32_t* __restrict__ row_idx,
                       int bits, int scale_mode, int clip_shift_or_exp, Control* __restrict__ ctl,
                       uint2* __restrict__ q, int32_t* __restrict__ scale_exp_out, const uint2* __restrict__ alpha,
-                      int k_max) {
+                      int k_max, int early_dependents) {
     cg::cluster_group cluster = cg::this_cluster();
     __shared__ unsigned int warp_max[kSmallThreads / 32];
     __shared__ unsigned int slots[kSmallCtas];
@@ -97,8 +97,11 @@ quantize_small_kernel(const uint4* __restrict__ x, int M, int vec_per_row, const
     // dependent launch allowed: a product kernel launched the same way behind this one may be set up on
     // the idle SMs and fetch its weights while this one runs (it waits for this grid before it reads the
     // codes), and by then everything that preceded this kernel on the stream is complete.
+    // early_dependents: the caller has promised that nothing in flight writes the weights the product kernel
+    // fetches ahead of its own wait, so that kernel may be set up before this one's wait ends as well.
+    if (early_dependents) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (!early_dependents) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int rank = (int)cluster.block_rank();
     const int total = M * vec_per_row;
     uint4 buf[kSmallVecs];
@@ -762,7 +765,7 @@ bool quantize_small_fits(int M, int K) { return (size_t)M * (size_t)K <= kSmallM
 
 cudaError_t launch_quantize_small(const __half* x, int M, int K, const int32_t* row_idx, int bits, int scale_mode,
                                   int clip_shift_or_exp, Control* ctl, int8_t* q, int32_t* scale_exp_out,
-                                  cudaStream_t stream, const uint8_t* alpha, int k_max) {
+                                  cudaStream_t stream, const uint8_t* alpha, int k_max, bool early_dependents) {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(kSmallCtas);
     cfg.blockDim = dim3(kSmallThreads);
@@ -775,7 +778,7 @@ cudaError_t launch_quantize_small(const __half* x, int M, int K, const int32_t* 
     cfg.numAttrs = 1;       // the kernel touches no memory before the kernel ahead of it has completed
     return cudaLaunchKernelEx(&cfg, quantize_small_kernel, reinterpret_cast<const uint4*>(x), M, K / 8, row_idx, bits,
                               scale_mode, clip_shift_or_exp, ctl, reinterpret_cast<uint2*>(q), scale_exp_out,
-                              reinterpret_cast<const uint2*>(alpha), k_max);
+                              reinterpret_cast<const uint2*>(alpha), k_max, early_dependents ? 1 : 0);
 }
 
 cudaError_t launch_token_select(const float* scores, int M, int n_keep, int32_t* idx, void* scratch,

@@ -68,3 +68,60 @@ def test_chain_bad_arguments_are_refused():
         h.aq_linear_chain(8, x, p, s, 128, 0, 5, 0)            # next_bits must be 8 or 4
     with pytest.raises(binding.AgileqError):
         h.aq_linear_chain(8, x, p, s, 128, 0, 8, 41)           # exponent out of range
+
+
+@pytest.mark.parametrize("M", [1, 4, 16])
+def test_three_layers_in_graph_replay_with_the_stable_weights_promise(M):
+    """aq_set_weights_stable lets consecutive few-row calls overlap (the next launch is set up early and fetches
+    weights before it waits). Three layers x -> y1 -> y2 -> y3, each reading the previous one's fp16 output,
+    captured in a CUDA graph and replayed several times: outputs equal bit for bit with the promise on and
+    off, every replay gives the same bits, and each layer matches the CPU checker run on its actual input."""
+    dims = [(768, 1280), (1280, 640), (640, 896)]          # (K, N) per layer
+    h = handle()
+    x = inputs.activations(M, dims[0][0], seed=77, outlier_frac=0.01, outlier_mult=20.0)
+    ws, layers = [], []
+    for li, (K, N) in enumerate(dims):
+        w = inputs.weights(N, K, 78 + li) * 8.0             # keeps the activations of later layers well scaled
+        packed, scales = h.aq_pack_w4(dev(w), 0)
+        layers.append((w, packed, scales, K, N))
+        ws.append(h.alloc_workspace(M, K, N, 0))
+    xd = dev(x)
+    ys = [torch.empty((M, N), dtype=torch.float16, device="cuda") for _, N in dims]
+
+    def run():
+        src = xd
+        for li, (_, packed, scales, K, N) in enumerate(layers):
+            h.aq_linear_w4a8(src, packed, scales, N, 0, y=ys[li], workspace=ws[li])
+            src = ys[li]
+
+    results = {}
+    try:
+        for promise in (False, True):
+            h.aq_set_weights_stable(promise)
+            run()
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                run()
+            outs = []
+            for _ in range(4):
+                for y in ys:
+                    y.zero_()
+                g.replay()
+                torch.cuda.synchronize()
+                outs.append([y.cpu().numpy().copy() for y in ys])
+            for o in outs[1:]:
+                for a, b in zip(o, outs[0]):
+                    assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
+            for wsp in ws:
+                assert h.aq_check_workspace(wsp) == binding.AQ_OK
+            results[promise] = outs[0]
+    finally:
+        h.aq_set_weights_stable(False)
+    for a, b in zip(results[False], results[True]):
+        assert np.array_equal(a.view(np.uint16), b.view(np.uint16))
+    src = x
+    for li, (w, _, _, K, N) in enumerate(layers):
+        codes, sc = oracle.quantize_weights(w, 0)
+        assert_y_close(results[True][li], oracle.linear(src, codes, sc, 8, 0)["y"])
+        src = results[True][li]

@@ -68,6 +68,7 @@ def test_which_shapes_fit_the_built_in_scratch_buffer():
 def test_null_handle_is_rejected_without_touching_a_device():
     L = binding.load()
     assert L.aq_set_kernel(None, 0) == binding.AQ_ERR_INVALID_ARG
+    assert L.aq_set_weights_stable(None, 1) == binding.AQ_ERR_INVALID_ARG
     assert L.aq_pack_w4(None, None, 128, 128, 0, None, None, None) == binding.AQ_ERR_INVALID_ARG
     assert L.aq_create(None, 0) == binding.AQ_ERR_INVALID_ARG
 
