@@ -230,6 +230,10 @@ template <int MB> struct StreamCfg {
     // consumer work in flight, not with the time a block waits (with the consumers' arithmetic taken out the
     // same launches take 6.6 / 9.1 / 10.1 us, and the ring is never full either way).
     static constexpr int kPhases = 2;
+    // Two CTAs per SM for both routes. Three single-row CTAs would fit (with 128-byte instead of 1024-byte
+    // alignment slack), so that under the stable-weights promise the next launch's CTAs sit, fetching, beside
+    // two CTAs of this one; measured slower (M = 1 layer 5.8 / 9.1 / 9.7 -> 6.6 / 9.7 / 11.8 us): what the
+    // early CTAs fetch is taken from the grid that has to finish first.
     static constexpr int kConsumerWarps = 4 * kPhases;
     static constexpr int kThreads = (1 + kConsumerWarps) * 32;
 };
