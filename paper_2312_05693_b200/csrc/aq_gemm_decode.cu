@@ -326,7 +326,8 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     // stale bytes, which meet zero weight codes. Tensor-map loads count their whole box.
     auto x_bytes = [&](int kb) -> uint32_t {
         if (FUSEQ) return 0u;                          // the codes are made here, not copied
-        return kRows == 1 ? (uint32_t)min(kTileK, p.K - kb * kTileK) : (uint32_t)(kRows * kTileK);
+        return kRows == 1 ? (uint32_t)min(kTileK, p.K - kb * kTileK)
+                          : (uint32_t)((kRows == 16 && p.M <= 8 ? 8 : kRows) * kTileK);   // the tensor map's box: 8 rows when M <= 8
     };
     auto issue_w = [&](int kb, int s) {
         asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
@@ -708,7 +709,8 @@ cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t
     CUtensorMap map;
     const cuuint64_t dims[2] = {(cuuint64_t)a.K, (cuuint64_t)a.M};
     const cuuint64_t strides[1] = {(cuuint64_t)a.K};
-    const cuuint32_t box[2] = {128u, (cuuint32_t)StreamCfg<MB>::kRows};
+    // 16-row route: rows 8..15 are neither copied nor read when M <= 8
+    const cuuint32_t box[2] = {128u, (cuuint32_t)(StreamCfg<MB>::kRows == 16 && a.M <= 8 ? 8 : StreamCfg<MB>::kRows)};
     const cuuint32_t estr[2] = {1u, 1u};
     const CUresult r = reinterpret_cast<EncodeTiledFn>(dev.encode_tiled)(
         &map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(a.q), dims, strides, box, estr,
