@@ -238,7 +238,7 @@ template <int MB> struct StreamCfg {
     static constexpr int kThreads = (1 + kConsumerWarps) * 32;
 };
 
-template <int MB>
+template <int MB, bool WIDE = false>
 struct StreamSmem {
     static constexpr int kRows = StreamCfg<MB>::kRows;
     static constexpr int kStages = StreamCfg<MB>::kStages;
@@ -251,7 +251,10 @@ struct StreamSmem {
     // one row quantized by the kernel itself: the codes of this CTA's k range (up to kFuseMaxBlocks blocks)
     alignas(16) int8_t xq[MB == 1 ? kFuseMaxBlocks * kTileK : 16];
     unsigned int warp_max[StreamCfg<MB>::kThreads / 32];
-    alignas(16) int recv[kRows][kTileN];                               // the other CTAs' sums for this CTA's channel slice, by sender
+    // the other CTAs' sums for this CTA's channel slice, by sender: `split` slots of 128 / split channels, or
+    // (clusters of 5 to 8) eight slots of 32
+    static constexpr int kRecvStride = WIDE ? 256 : kTileN;
+    alignas(16) int recv[kRows][kRecvStride];
     alignas(8) uint64_t full[kStages];
     uint64_t empty[kStages];
     volatile uint32_t abort_flag;
@@ -283,12 +286,13 @@ struct StreamParams {
 
 // grid = (split, channel tiles), cluster = (split, 1, 1): the CTAs of a cluster share a channel
 // tile and take consecutive k ranges; CTA r adds up and writes channels [r, r+1) * 128 / split.
-template <int MB, bool FUSEQ = false>
+template <int MB, bool FUSEQ = false, bool WIDE = false>
 __global__ void __launch_bounds__(StreamCfg<MB>::kThreads, 2)
 gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const StreamParams p) {
     static_assert(!FUSEQ || MB == 1, "only a single row is quantized inside the product kernel");
+    static_assert(!WIDE || MB == 16, "clusters of 5 to 8 are for the 16-row route");
     extern __shared__ uint8_t smem_raw[];
-    using Smem = StreamSmem<MB>;
+    using Smem = StreamSmem<MB, WIDE>;
     Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     constexpr bool kUseMma = StreamCfg<MB>::kUseMma;
     constexpr int kRows = StreamCfg<MB>::kRows;
@@ -616,14 +620,21 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     // This CTA's k range is done: a launch behind this one that allows it may be scheduled and set up now
     // (it reads and writes nothing before this grid has completed).
     if (!p.early_dependents) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const int cw = kTileN / split;                            // split is 1, 2 or 4: a power of two, so
-    const int cw_log = 7 - (31 - __clz(split));               // divisions by cw are shifts
+    // Channel slices: 128 / split channels each for split 1, 2, 4 (divisions are shifts). Clusters of 5 to 8
+    // (16-row route on long k ranges) cut the tile's 32 groups of four channels into `split` nearly equal
+    // runs, slice r = groups [32 r / split, 32 (r + 1) / split): at most 28 channels, handled by the first
+    // lanes of 32-thread rows.
+    constexpr bool wide = WIDE;                                // this instantiation is launched with clusters of 5 to 8
+    const int cw = wide ? 32 : kTileN / split;                // slot width in the receive buffer
+    const int cw_log = wide ? 5 : 7 - (31 - __clz(split));
+    const int g_first = (32 * rank) / split, g_count = (32 * (rank + 1)) / split - g_first;   // this CTA's groups (wide)
     const int ft = (int)threadIdx.x - 32;                     // the consumer threads finish (a multiple of 128 = 4 cw at most)
     const int rc = ft & (cw - 1);                             // channel inside the slice (only used when ft >= 0)
-    const int out_r = rank * cw + rc;
+    const int out_r = wide ? 4 * g_first + rc : rank * cw + rc;
     const int out_n = tile * kTileN + out_r;
+    const bool mine = ft >= 0 && out_n < p.N && (!wide || rc < 4 * g_count);
     float sc = 0.0f, off = 0.0f;
-    if (ft >= 0 && out_n < p.N) {
+    if (mine) {
         const float pe = __int_as_float((127 + (FUSEQ ? fused_exp : *p.scale_exp)) << 23);
         sc = __half2float(p.w_scales[out_n]) * pe;
         if (p.chan_offset) off = p.chan_offset[out_n] * pe;
@@ -635,10 +646,11 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
         if (ft >= 0) {
             // four consecutive channels at a time (16-byte remote stores) go to the CTA that owns them
             for (int e = ft; e < rows * (kTileN / 4); e += kStrConsumerWarps * 32) {
-                const int m = e >> 5, ch = 4 * (e & 31);
-                const int owner = ch >> cw_log;
+                const int m = e >> 5, g4 = e & 31, ch = 4 * g4;
+                const int owner = wide ? (((g4 + 1) * split + 31) >> 5) - 1 : ch >> cw_log;
+                const int at = wide ? ch - 4 * ((32 * owner) / split) : ch & (cw - 1);   // place inside the owner's slice
                 if (owner != rank)
-                    *reinterpret_cast<int4*>(cluster.map_shared_rank(&sm.recv[0][0], owner) + m * kTileN + rank * cw + (ch & (cw - 1))) =
+                    *reinterpret_cast<int4*>(cluster.map_shared_rank(&sm.recv[0][0], owner) + m * Smem::kRecvStride + rank * cw + at) =
                         *reinterpret_cast<const int4*>(&sm.sum[m][ch]);
             }
         }
@@ -647,7 +659,7 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
     } else {
         __syncthreads();
     }
-    if (ft >= 0 && out_n < p.N) {
+    if (mine) {
         // All shared-memory reads of this thread's outputs are issued before the first is used and without
         // branches around them (rows that do not exist read the last row of the buffer and are dropped):
         // taken one after the other, each behind its own test, they were the longest part of the finish at
@@ -656,13 +668,16 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
         const int stride = (kStrConsumerWarps * 32) >> cw_log, m0 = ft >> cw_log;
         int av[kIt];
 #pragma unroll
-        for (int i = 0; i < kIt; ++i) av[i] = sm.sum[min(m0 + i * stride, kRows - 1)][out_r];
+        for (int i = 0; i < kIt; ++i) av[i] = i * stride < kRows ? sm.sum[min(m0 + i * stride, kRows - 1)][out_r] : 0;
 #pragma unroll
-        for (int k = 1; k < 4; ++k) {
+        for (int k = 1; k < (WIDE ? 8 : 4); ++k) {
             if (k < split) {
-                const int col = ((rank + k) & (split - 1)) * cw + rc;         // the k-th other CTA's slot
+                int c = rank + k;                                             // the k-th other CTA's slot
+                if (c >= split) c -= split;
+                const int col = c * cw + rc;
 #pragma unroll
-                for (int i = 0; i < kIt; ++i) av[i] += sm.recv[min(m0 + i * stride, kRows - 1)][col];
+                for (int i = 0; i < kIt; ++i)
+                    if (i * stride < kRows) av[i] += sm.recv[min(m0 + i * stride, kRows - 1)][col];   // the same test in every thread
             }
         }
         if (!p.acc_dump && !p.q_next) {
@@ -680,7 +695,8 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
                     const int a = av[i] >> 4;
                     if (p.acc_dump) p.acc_dump[(size_t)m * p.N + out_n] = a;
                     const __half hv = __float2half_rn(fmaf((float)a, sc, off));
-                    // (a warp's lanes hold consecutive channels and run this loop together: 128 / split >= 32)
+                    // (a warp's lanes hold consecutive channels and run this loop together: slices of 32 and
+                    // more channels; clusters of 5 to 8 are not used with chained outputs)
                     if (p.q_next)
                         store_next_code(p.q_next, (size_t)m * p.N + out_n, next_code(hv, p.next_inv, p.next_lo, p.next_hi),
                                         p.next_packed, true, lane);
@@ -699,12 +715,20 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-template <int MB, bool FUSEQ = false>
-cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream) {
-    using Smem = StreamSmem<MB>;
+// k ranges per tile: 1, 2 or 4, as many as keep all CTAs resident at once (two per SM) with at least two k
+// blocks per CTA
+inline int decode_split(int tiles, int KB, int sm_count) {
+    int split = 1;
+    while (split < 4 && tiles * split * 2 <= 2 * sm_count && KB / (split * 2) >= 2) split *= 2;
+    return split;
+}
+
+template <int MB, bool FUSEQ = false, bool WIDE = false>
+cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t stream, int wide_split = 0) {
+    using Smem = StreamSmem<MB, WIDE>;
     const size_t smem_bytes = sizeof(Smem) + 1024;
     static SmemOptIn opt_in;
-    if (const cudaError_t e = opt_in.ensure(gemm_decode_stream_kernel<MB, FUSEQ>, dev.device, smem_bytes); e != cudaSuccess)
+    if (const cudaError_t e = opt_in.ensure(gemm_decode_stream_kernel<MB, FUSEQ, WIDE>, dev.device, smem_bytes); e != cudaSuccess)
         return e;
     CUtensorMap map;
     const cuuint64_t dims[2] = {(cuuint64_t)a.K, (cuuint64_t)a.M};
@@ -737,25 +761,69 @@ cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t
     p.early_weights = (!p.clear_status || a.weights_stable) ? 1 : 0;
     p.early_dependents = a.weights_stable ? 1 : 0;
     const int tiles = p.Npad / kTileN, KB = k_blocks(a.K);
-    // as many k ranges per tile (cluster size 1, 2 or 4: clusters of 7-8 measured slower) as keep
-    // all CTAs resident at once (two per SM), and at least two k blocks per CTA
-    int split = 1;
-    while (split < 4 && tiles * split * 2 <= 2 * dev.sm_count && KB / (split * 2) >= 2) split *= 2;
+    // as many k ranges per tile (cluster size 1, 2 or 4) as keep all CTAs resident at once (two per SM), and
+    // at least two k blocks per CTA
+    const int split = WIDE ? wide_split : decode_split(tiles, KB, dev.sm_count);
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(split, tiles, 1);
     cfg.blockDim = dim3(StreamCfg<MB>::kThreads);
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = split;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    cfg.gridDim = dim3(split, tiles, 1);
+    attr[0].val.clusterDim.x = split;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 2;       // the kernel reads and writes nothing before the kernel ahead of it has completed
-    return cudaLaunchKernelEx(&cfg, gemm_decode_stream_kernel<MB, FUSEQ>, map, p);
+    return cudaLaunchKernelEx(&cfg, gemm_decode_stream_kernel<MB, FUSEQ, WIDE>, map, p);
+}
+
+// 16-row route on long k ranges: its consumers, not the memory, set a CTA's pace, so more CTAs per tile pay
+// as long as each keeps a dozen blocks and all clusters still run at once (a GPC holds only so many clusters
+// of a size: the occupancy query says how many the device does). Measured with clusters of 8 on N = 4096,
+// K = 13824: 11.1 / 11.4 -> 9.2 / 9.5 us at M = 4 / 16; with five blocks per CTA (K = 5120) nothing is
+// gained, and a single row loses. Chained outputs keep slices of at least 32 channels. Returns the cluster
+// size (5 to 8), or 0 for the usual 1, 2 or 4.
+int wide_split_for(const GemmArgs& a, const DeviceInfo& dev) {
+    const int tiles = round_up(a.N, kTileN) / kTileN, KB = k_blocks(a.K);
+    if (a.q_next || decode_split(tiles, KB, dev.sm_count) != 4) return 0;
+    static std::atomic<int> fits[kMaxDevices][9];               // clusters of s that run at once, + 1 (0: not asked yet)
+    int s = (2 * dev.sm_count) / tiles;
+    if (s > 8) s = 8;
+    for (; s > 4; --s) {
+        if (KB / s < 12) continue;
+        int known = fits[dev.device][s].load(std::memory_order_relaxed);
+        if (known == 0) {
+            using Smem = StreamSmem<16, true>;
+            const size_t smem_bytes = sizeof(Smem) + 1024;
+            static SmemOptIn opt_in;
+            int n = 0;
+            if (opt_in.ensure(gemm_decode_stream_kernel<16, false, true>, dev.device, smem_bytes) == cudaSuccess) {
+                cudaLaunchConfig_t cfg = {};
+                cfg.gridDim = dim3(s, tiles, 1);
+                cfg.blockDim = dim3(StreamCfg<16>::kThreads);
+                cfg.dynamicSmemBytes = smem_bytes;
+                cudaLaunchAttribute attr[1];
+                attr[0].id = cudaLaunchAttributeClusterDimension;
+                attr[0].val.clusterDim.x = s;
+                attr[0].val.clusterDim.y = 1;
+                attr[0].val.clusterDim.z = 1;
+                cfg.attrs = attr;
+                cfg.numAttrs = 1;
+                if (cudaOccupancyMaxActiveClusters(&n, gemm_decode_stream_kernel<16, false, true>, &cfg) != cudaSuccess) {
+                    (void)cudaGetLastError();
+                    n = 0;
+                }
+            }
+            known = n + 1;
+            fits[dev.device][s].store(known, std::memory_order_relaxed);
+        }
+        if (known - 1 >= tiles) return s;
+    }
+    return 0;
 }
 
 template <int MB>
@@ -782,8 +850,7 @@ cudaError_t launch_mb(const GemmArgs& a, cudaStream_t stream) {
 bool decode_can_fuse_quantize(int M, int K, int N, int group, int sm_count) {
     if (M != 1 || group) return false;
     const int tiles = round_up(N, kTileN) / kTileN, KB = k_blocks(K);
-    int split = 1;
-    while (split < 4 && tiles * split * 2 <= 2 * sm_count && KB / (split * 2) >= 2) split *= 2;
+    const int split = decode_split(tiles, KB, sm_count);
     return (KB + split - 1) / split + 1 <= kFuseMaxBlocks;
 }
 
@@ -794,6 +861,7 @@ cudaError_t launch_gemm_decode(const GemmArgs& a, const DeviceInfo& dev, cudaStr
         // 8.1 / 12.8 / 15.2 us on the three 13B shapes)
         if (a.M <= 1 && a.fuse_x) return launch_stream<1, true>(a, dev, stream);
         if (a.M <= 1) return launch_stream<1>(a, dev, stream);
+        if (const int ws = wide_split_for(a, dev)) return launch_stream<16, false, true>(a, dev, stream, ws);
         return launch_stream<16>(a, dev, stream);
     }
     if (a.M <= 1) return launch_mb<1>(a, stream);

@@ -219,6 +219,28 @@ def test_decode_rows_1_to_16(M, group):
     assert_y_close(gpu["y"], ref["y"])
 
 
+@pytest.mark.parametrize("M,K,N", [(2, 12288, 4096), (16, 13824, 5120), (5, 7680, 6400), (9, 9216, 5700),
+                                   (16, 13824, 4000)])
+def test_decode_clusters_of_five_to_eight(M, K, N):
+    """Long k ranges with 2..16 rows take clusters of 8, 7, 5, 6 and 8 CTAs per channel tile (uneven channel
+    slices for 5 to 7; a ragged N twice): integer sums exact, outputs within tolerance, and the chained call,
+    which keeps clusters of at most 4, gives the codes of the quantizer applied to these outputs."""
+    x = inputs.activations(M, K, seed=M + K, outlier_frac=0.01, outlier_mult=20.0)
+    w = inputs.weights(N, K, seed=N + K)
+    gpu, ref = run_layer_both(x, w, 8, 0, binding.AQ_KERNEL_AUTO)
+    assert gpu["e"] == ref["e"] and np.array_equal(gpu["q"], ref["q"])
+    assert np.array_equal(gpu["acc"], ref["acc"])
+    assert_y_close(gpu["y"], ref["y"])
+    h = handle()
+    packed, scales = h.aq_pack_w4(dev(w), 0)
+    y = h.aq_linear_w4a8(dev(x), packed, scales, N, 0)            # without the dump of the sums: the plain-output loop
+    assert np.array_equal(y.cpu().numpy().view(np.uint16), gpu["y"].view(np.uint16))
+    if N % 32 == 0:
+        e_next = oracle.layer_exponent(gpu["y"], 8) - 1
+        q_next = h.aq_linear_chain(8, dev(x), packed, scales, N, 0, 8, e_next)
+        assert np.array_equal(q_next.cpu().numpy(), oracle.quantize_act(gpu["y"], 8, e_next))
+
+
 @pytest.mark.parametrize("kernel", KERNELS)
 @pytest.mark.parametrize("M,K,N,group", [(16, 768, 768, 0), (129, 384, 200, 128), (260, 1152, 520, 128)])
 def test_linear_w4a4_matches_checker(kernel, M, K, N, group):
