@@ -781,12 +781,12 @@ cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t
     return cudaLaunchKernelEx(&cfg, gemm_decode_stream_kernel<MB, FUSEQ, WIDE>, map, p);
 }
 
-// 16-row route on long k ranges: its consumers, not the memory, set a CTA's pace, so more CTAs per tile pay
-// as long as each keeps a dozen blocks and all clusters still run at once (a GPC holds only so many clusters
-// of a size: the occupancy query says how many the device does). Measured with clusters of 8 on N = 4096,
-// K = 13824: 11.1 / 11.4 -> 9.2 / 9.5 us at M = 4 / 16; with five blocks per CTA (K = 5120) nothing is
-// gained, and a single row loses. Chained outputs keep slices of at least 32 channels. Returns the cluster
-// size (5 to 8), or 0 for the usual 1, 2 or 4.
+// 16-row route: its consumers, not the memory, set a CTA's pace, so more CTAs per tile pay as long as each
+// keeps five k blocks and all clusters still run at once (a GPC holds only so many clusters of a size: the
+// occupancy query says how many the device does). Measured on the 13B shapes with N = 5120 (clusters of 7):
+// K = 13824 12.5 / 13.2 -> 9.8 / 10.4 us at M = 4 / 16, K = 5120 6.9 / 7.3 -> 6.0 / 6.5 us; a single row
+// loses with clusters of 8 (N = 4096, K = 5120: 5.1 -> 6.2 us). Chained outputs keep slices of at least 32
+// channels. Returns the cluster size (5 to 8), or 0 for the usual 1, 2 or 4.
 int wide_split_for(const GemmArgs& a, const DeviceInfo& dev) {
     const int tiles = round_up(a.N, kTileN) / kTileN, KB = k_blocks(a.K);
     if (a.q_next || decode_split(tiles, KB, dev.sm_count) != 4) return 0;
@@ -794,7 +794,7 @@ int wide_split_for(const GemmArgs& a, const DeviceInfo& dev) {
     int s = (2 * dev.sm_count) / tiles;
     if (s > 8) s = 8;
     for (; s > 4; --s) {
-        if (KB / s < 12) continue;
+        if (KB / s < 5) continue;
         int known = fits[dev.device][s].load(std::memory_order_relaxed);
         if (known == 0) {
             using Smem = StreamSmem<16, true>;
