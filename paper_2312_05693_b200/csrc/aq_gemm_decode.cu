@@ -285,7 +285,9 @@ struct StreamParams {
 };
 
 // grid = (split, channel tiles), cluster = (split, 1, 1): the CTAs of a cluster share a channel
-// tile and take consecutive k ranges; CTA r adds up and writes channels [r, r+1) * 128 / split.
+// tile and take consecutive k ranges; CTA r adds up and writes its slice of the tile's channels:
+// [r, r+1) * 128 / split for split 1, 2, 4; WIDE (split 5 to 8, 16-row route only) the groups of four
+// channels [32 r / split, 32 (r + 1) / split).
 template <int MB, bool FUSEQ = false, bool WIDE = false>
 __global__ void __launch_bounds__(StreamCfg<MB>::kThreads, 2)
 gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const StreamParams p) {
@@ -610,7 +612,7 @@ gemm_decode_stream_kernel(const __grid_constant__ CUtensorMap x_map, const Strea
         }
     }
     // Every CTA of the cluster now holds the tile's sums over its own k range, and CTA `rank` finishes the
-    // slice of 128 / split channels [rank, rank + 1) * cw: every CTA writes its sums of the other slices into
+    // tile's channel slice `rank`: every CTA writes its sums of the other slices into
     // their owners' shared memory (slot = sender), the cluster meets once, and every CTA adds what it received
     // to its own sums (integer addition is exact in any order), scales and writes its outputs. After the
     // meeting nobody touches another CTA's memory, so a CTA may leave as soon as it is done. (Reading the
@@ -715,8 +717,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-// k ranges per tile: 1, 2 or 4, as many as keep all CTAs resident at once (two per SM) with at least two k
-// blocks per CTA
+// k ranges per tile by the usual rule: 1, 2 or 4, as many as keep all CTAs resident at once (two per SM) with at
+// least two k blocks per CTA (wide_split_for may raise a 4 to 5..8 for the 16-row route)
 inline int decode_split(int tiles, int KB, int sm_count) {
     int split = 1;
     while (split < 4 && tiles * split * 2 <= 2 * sm_count && KB / (split * 2) >= 2) split *= 2;
@@ -761,8 +763,6 @@ cudaError_t launch_stream(const GemmArgs& a, const DeviceInfo& dev, cudaStream_t
     p.early_weights = (!p.clear_status || a.weights_stable) ? 1 : 0;
     p.early_dependents = a.weights_stable ? 1 : 0;
     const int tiles = p.Npad / kTileN, KB = k_blocks(a.K);
-    // as many k ranges per tile (cluster size 1, 2 or 4) as keep all CTAs resident at once (two per SM), and
-    // at least two k blocks per CTA
     const int split = WIDE ? wide_split : decode_split(tiles, KB, dev.sm_count);
     cudaLaunchConfig_t cfg = {};
     cfg.blockDim = dim3(StreamCfg<MB>::kThreads);
