@@ -273,9 +273,11 @@ struct AttnSmem {
 };
 
 // Batched int8 contraction y[h][m][n] = scale * sum_k A[h*M + m][k] * B[h*NB + n][k] (both operands
-// k-major). One CTA per (128 rows of A, head) walks all tiles of DN rows of B, with two accumulator
-// stages in tensor memory so that the epilogue of one tile overlaps the MMAs of the next. A is unsigned
-// or signed bytes, B signed.
+// k-major). A work item is (128 rows of A, head): all tiles of DN rows of B for those rows. The grid is
+// persistent: CTA c takes the items c, c + gridDim.x, ..., and the ring of operand stages and the two
+// accumulator stages in tensor memory run on across items, so the producer fetches the next item's tiles
+// while the epilogue of the last tile of this one still writes (a CTA's 16 k steps of one item alone were
+// mostly fill and drain). A is unsigned or signed bytes, B signed.
 // scale = (max_bits ? the half in its low 16 bits : 1) * 2^(*e1 + (e2 ? *e2 : 0) + e_off).
 // Used for attention x value (A = byte factors of the log2 codes, B = transposed value codes, k = key
 // index) and for the query x key product (A, B = int8 codes, k = head dimension).
@@ -283,14 +285,15 @@ template <int DN, bool A_SIGNED>
 __global__ void __launch_bounds__(kTcThreads, 1)
 attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__ CUtensorMap b_map,
                  const __grid_constant__ CUtensorMap y_map, const uint32_t* __restrict__ max_bits, const int32_t* __restrict__ e1, const int32_t* __restrict__ e2,
-                 int e_off, int M, int J /* length of k */, int NB, __half* __restrict__ y, Control* __restrict__ ctl) {
+                 int e_off, int H, int M, int J /* length of k */, int NB, __half* __restrict__ y, Control* __restrict__ ctl) {
     extern __shared__ uint8_t attn_smem_raw[];
     using Smem = AttnSmem<DN>;
     Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(attn_smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int h = blockIdx.y, m0 = blockIdx.x * 128;
+    const int MT = (M + 127) / 128;                                       // row tiles per head
+    const int items = MT * H;                                             // work items; item w = (head w / MT, row tile w % MT)
     const int JB = (J + 127) / 128;
-    const int NT = (NB + DN - 1) / DN;                                    // tiles of B rows this CTA walks
+    const int NT = (NB + DN - 1) / DN;                                    // tiles of B rows per item
     if (threadIdx.x == 0) {
         for (int s = 0; s < kTcStages; ++s) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(a_smem_u32(&sm.full[s])) : "memory");
@@ -316,11 +319,14 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
 
     if (warp == 0) {
         if (lane == 0) {
-            const int total = NT * JB;
-            for (int it = 0; it < total; ++it) {
-                const int nt = it / JB, jb = it % JB, n0 = nt * DN;
+            int it = 0;                                                   // stages filled so far, over all items
+            bool ok = true;
+            for (int w = blockIdx.x; w < items && ok; w += gridDim.x) {
+              const int h = w / MT, m0 = (w % MT) * 128;
+              for (int i = 0; i < NT * JB; ++i, ++it) {
+                const int nt = i / JB, jb = i % JB, n0 = nt * DN;
                 const int s = it % kTcStages;
-                if (!a_wait(&sm.empty[s], ((it / kTcStages) & 1) ^ 1, abort_flag)) break;
+                if (!a_wait(&sm.empty[s], ((it / kTcStages) & 1) ^ 1, abort_flag)) { ok = false; break; }
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
                              ::"r"(a_smem_u32(&sm.full[s])), "r"((uint32_t)((128 + DN) * 128)) : "memory");
                 asm volatile(
@@ -331,6 +337,7 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
                     "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                     ::"r"(a_smem_u32(sm.b[s])), "l"(&b_map), "r"(jb * 128), "r"(h * NB + n0), "r"(a_smem_u32(&sm.full[s]))
                     : "memory");
+              }
             }
         }
     } else if (warp == 1) {
@@ -340,10 +347,11 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
             constexpr uint32_t idesc = (2u << 4) | ((A_SIGNED ? 1u : 0u) << 7) | (1u << 10) | ((uint32_t)(DN >> 3) << 17) |
                                        ((uint32_t)(128 >> 4) << 24);
             bool ok = true;
-            int it = 0;
-            for (int nt = 0; nt < NT && ok; ++nt) {
-              const int a = nt & 1;
-              ok = a_wait(&sm.acc_empty[a], ((nt >> 1) & 1) ^ 1, abort_flag);      // the epilogue has drained this stage
+            int it = 0, tc = 0;                                           // stages and tiles consumed so far, over all items
+            for (int w = blockIdx.x; w < items && ok; w += gridDim.x)
+            for (int nt = 0; nt < NT && ok; ++nt, ++tc) {
+              const int a = tc & 1;
+              ok = a_wait(&sm.acc_empty[a], ((tc >> 1) & 1) ^ 1, abort_flag);      // the epilogue has drained this stage
               if (!ok) break;
               for (int jb = 0; jb < JB && ok; ++jb, ++it) {
                 const int s = it % kTcStages;
@@ -372,12 +380,16 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
         }
     } else {
         const int quarter = warp & 3;                                     // TMEM lanes this warp may read
-        const int row = quarter * 32 + lane, m = m0 + row;
         const float pmax = max_bits ? __half2float(__ushort_as_half((unsigned short)(*max_bits & 0xFFFFu))) : 1.0f;
         const float scale = pmax * __int_as_float((127 + *e1 + (e2 ? *e2 : 0) + e_off) << 23);
-        for (int nt = 0; nt < NT; ++nt) {
-            const int a = nt & 1, n0 = nt * DN;
-            if (!(__all_sync(0xFFFFFFFFu, a_wait(&sm.acc_full[a], (nt >> 1) & 1, abort_flag) ? 1 : 0) != 0)) break;
+        int tc = 0;                                                       // tiles drained so far, over all items
+        bool alive = true;
+        for (int w = blockIdx.x; w < items && alive; w += gridDim.x) {
+          const int h = w / MT, m0 = (w % MT) * 128;
+          const int row = quarter * 32 + lane, m = m0 + row;
+          for (int nt = 0; nt < NT; ++nt, ++tc) {
+            const int a = tc & 1, n0 = nt * DN;
+            if (!(__all_sync(0xFFFFFFFFu, a_wait(&sm.acc_full[a], (tc >> 1) & 1, abort_flag) ? 1 : 0) != 0)) { alive = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int ew = warp - 2;
 #pragma unroll 1
@@ -448,6 +460,7 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(a_smem_u32(&sm.acc_empty[a])) : "memory");
+          }
         }
     }
     if (warp >= 2 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // staging rows live until read
@@ -501,8 +514,9 @@ cudaError_t launch_attn_tc(const void* w, const int8_t* vt, const uint32_t* max_
     if (enc(&ymap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, y, ydims, ystrides, ybox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidValue;
-    dim3 grid((M + 127) / 128, H);
-    attn_v_tc_kernel<DN, A_SIGNED><<<grid, kTcThreads, smem_bytes, stream>>>(amap, bmap, ymap, max_bits, e1, e2, e_off, M,
+    const int items = ((M + 127) / 128) * H;
+    dim3 grid(items < dev.sm_count ? items : dev.sm_count);
+    attn_v_tc_kernel<DN, A_SIGNED><<<grid, kTcThreads, smem_bytes, stream>>>(amap, bmap, ymap, max_bits, e1, e2, e_off, H, M,
                                                                             J, NB, y, ctl);
     return cudaGetLastError();
 }
