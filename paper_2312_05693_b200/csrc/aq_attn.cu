@@ -257,9 +257,9 @@ __device__ __forceinline__ uint64_t a_desc_sw128(uint32_t saddr) {
     return d;
 }
 
-template <int DN>
+template <int DN, int RT>
 struct AttnSmem {
-    alignas(1024) uint8_t a[kTcStages][128 * 128];   // weights tile: 128 query rows x 128 j
+    alignas(1024) uint8_t a[kTcStages][RT * 128 * 128];   // weights tile: RT x 128 query rows x 128 j
     alignas(1024) uint8_t b[kTcStages][DN * 128];    // value tile: DN columns x 128 j
     // Output staging: each epilogue warp owns two boxes of 32 rows x 64 halves (128-byte rows, written
     // with the 128-byte swizzle of the store's tensor map), for alternate 64-column chunks.
@@ -277,20 +277,24 @@ struct AttnSmem {
 // persistent: CTA c takes the items c, c + gridDim.x, ..., and the ring of operand stages and the two
 // accumulator stages in tensor memory run on across items, so the producer fetches the next item's tiles
 // while the epilogue of the last tile of this one still writes (a CTA's 16 k steps of one item alone were
-// mostly fill and drain). A is unsigned or signed bytes, B signed.
+// mostly fill and drain). With RT = 2 an item is 256 rows of A, two accumulators of 128 rows that share
+// every tile of B: what limits this kernel is the L2 -> SM path, and the B tile is then fetched once for
+// twice the rows. A is unsigned or signed bytes, B signed.
 // scale = (max_bits ? the half in its low 16 bits : 1) * 2^(*e1 + (e2 ? *e2 : 0) + e_off).
 // Used for attention x value (A = byte factors of the log2 codes, B = transposed value codes, k = key
 // index) and for the query x key product (A, B = int8 codes, k = head dimension).
-template <int DN, bool A_SIGNED>
+template <int DN, bool A_SIGNED, int RT = 1>
 __global__ void __launch_bounds__(kTcThreads, 1)
 attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__ CUtensorMap b_map,
                  const __grid_constant__ CUtensorMap y_map, const uint32_t* __restrict__ max_bits, const int32_t* __restrict__ e1, const int32_t* __restrict__ e2,
                  int e_off, int H, int M, int J /* length of k */, int NB, __half* __restrict__ y, Control* __restrict__ ctl) {
     extern __shared__ uint8_t attn_smem_raw[];
-    using Smem = AttnSmem<DN>;
+    using Smem = AttnSmem<DN, RT>;
+    static_assert(2 * RT * DN <= 512, "two accumulator stages of RT x DN columns in tensor memory");
+    constexpr int kRows = RT * 128;                                       // rows of A per item
     Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(attn_smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int MT = (M + 127) / 128;                                       // row tiles per head
+    const int MT = (M + kRows - 1) / kRows;                               // row tiles per head
     const int items = MT * H;                                             // work items; item w = (head w / MT, row tile w % MT)
     const int JB = (J + 127) / 128;
     const int NT = (NB + DN - 1) / DN;                                    // tiles of B rows per item
@@ -308,7 +312,7 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
     }
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(a_smem_u32(&sm.tmem_base)), "r"((uint32_t)(2 * DN)) : "memory");
+                     ::"r"(a_smem_u32(&sm.tmem_base)), "r"((uint32_t)(2 * RT * DN)) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -322,13 +326,13 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
             int it = 0;                                                   // stages filled so far, over all items
             bool ok = true;
             for (int w = blockIdx.x; w < items && ok; w += gridDim.x) {
-              const int h = w / MT, m0 = (w % MT) * 128;
+              const int h = w / MT, m0 = (w % MT) * kRows;
               for (int i = 0; i < NT * JB; ++i, ++it) {
                 const int nt = i / JB, jb = i % JB, n0 = nt * DN;
                 const int s = it % kTcStages;
                 if (!a_wait(&sm.empty[s], ((it / kTcStages) & 1) ^ 1, abort_flag)) { ok = false; break; }
                 asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;"
-                             ::"r"(a_smem_u32(&sm.full[s])), "r"((uint32_t)((128 + DN) * 128)) : "memory");
+                             ::"r"(a_smem_u32(&sm.full[s])), "r"((uint32_t)((kRows + DN) * 128)) : "memory");
                 asm volatile(
                     "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                     ::"r"(a_smem_u32(sm.a[s])), "l"(&a_map), "r"(jb * 128), "r"(h * M + m0), "r"(a_smem_u32(&sm.full[s]))
@@ -361,14 +365,18 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
                 const uint64_t adesc = a_desc_sw128(a_smem_u32(sm.a[s]));
                 const uint64_t bdesc = a_desc_sw128(a_smem_u32(sm.b[s]));
 #pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                    const uint32_t accumulate = (jb == 0 && t == 0) ? 0u : 1u;
-                    asm volatile(
-                        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
-                        ::"r"(tmem + (uint32_t)(a * DN)), "l"(adesc + (uint64_t)(2 * t)), "l"(bdesc + (uint64_t)(2 * t)), "r"(idesc),
-                          "r"(accumulate)
-                        : "memory");
+                for (int r = 0; r < RT; ++r) {
+                    // the r-th 128 rows of the A tile start 16 KB (1024 in descriptor units of 16 bytes) further on
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const uint32_t accumulate = (jb == 0 && t == 0) ? 0u : 1u;
+                        asm volatile(
+                            "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                            "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+                            ::"r"(tmem + (uint32_t)((a * RT + r) * DN)), "l"(adesc + (uint64_t)(1024 * r + 2 * t)),
+                              "l"(bdesc + (uint64_t)(2 * t)), "r"(idesc), "r"(accumulate)
+                            : "memory");
+                    }
                 }
                 asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
                              ::"r"(a_smem_u32(&sm.empty[s])) : "memory");
@@ -385,13 +393,15 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
         int tc = 0;                                                       // tiles drained so far, over all items
         bool alive = true;
         for (int w = blockIdx.x; w < items && alive; w += gridDim.x) {
-          const int h = w / MT, m0 = (w % MT) * 128;
-          const int row = quarter * 32 + lane, m = m0 + row;
+          const int h = w / MT, m0_item = (w % MT) * kRows;
           for (int nt = 0; nt < NT; ++nt, ++tc) {
             const int a = tc & 1, n0 = nt * DN;
             if (!(__all_sync(0xFFFFFFFFu, a_wait(&sm.acc_full[a], (tc >> 1) & 1, abort_flag) ? 1 : 0) != 0)) { alive = false; break; }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const int ew = warp - 2;
+#pragma unroll 1
+            for (int r = 0; r < RT; ++r) {
+            const int m0 = m0_item + r * 128, m = m0 + quarter * 32 + lane;          // this accumulator's 128 rows
 #pragma unroll 1
             for (int c0 = 0; c0 < DN; c0 += 32) {
                 uint32_t v[32];
@@ -403,7 +413,7 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
                       "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
                       "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
                       "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-                    : "r"(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * DN + c0))
+                    : "r"(tmem + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((a * RT + r) * DN + c0))
                     : "memory");
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
                 // 32 columns of this thread's row -> 64 bytes of its 128-byte staging row; 16-byte chunk j of
@@ -456,6 +466,7 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
                     }
                 }
             }
+            }
             // this warp's part of the accumulator stage is in registers / written: hand the stage back
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
@@ -474,27 +485,27 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
     }
     __syncthreads();
     if (warp == 1)
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)(2 * DN)) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)(2 * RT * DN)) : "memory");
 }
 
 typedef CUresult (*AttnEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-template <int DN, bool A_SIGNED>
+template <int DN, bool A_SIGNED, int RT = 1>
 cudaError_t launch_attn_tc(const void* w, const int8_t* vt, const uint32_t* max_bits, const int32_t* e1, const int32_t* e2,
                            int e_off, int H, int M, int J, int NB, __half* y, Control* ctl, const DeviceInfo& dev,
                            cudaStream_t stream) {
-    using Smem = AttnSmem<DN>;
+    using Smem = AttnSmem<DN, RT>;
     const size_t smem_bytes = sizeof(Smem) + 1024;
     static SmemOptIn opt_in;
-    if (const cudaError_t e = opt_in.ensure(attn_v_tc_kernel<DN, A_SIGNED>, dev.device, smem_bytes); e != cudaSuccess)
+    if (const cudaError_t e = opt_in.ensure(attn_v_tc_kernel<DN, A_SIGNED, RT>, dev.device, smem_bytes); e != cudaSuccess)
         return e;
     CUtensorMap amap, bmap;
     const cuuint32_t estr[2] = {1u, 1u};
     const cuuint64_t strides[1] = {(cuuint64_t)J};
     const cuuint64_t adims[2] = {(cuuint64_t)J, (cuuint64_t)H * M};
-    const cuuint32_t abox[2] = {128u, 128u};
+    const cuuint32_t abox[2] = {128u, (cuuint32_t)(RT * 128)};
     const cuuint64_t bdims[2] = {(cuuint64_t)J, (cuuint64_t)H * NB};
     const cuuint32_t bbox[2] = {128u, (cuuint32_t)DN};
     AttnEncodeFn enc = reinterpret_cast<AttnEncodeFn>(dev.encode_tiled);
@@ -514,9 +525,9 @@ cudaError_t launch_attn_tc(const void* w, const int8_t* vt, const uint32_t* max_
     if (enc(&ymap, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, y, ydims, ystrides, ybox, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
         return cudaErrorInvalidValue;
-    const int items = ((M + 127) / 128) * H;
+    const int items = ((M + RT * 128 - 1) / (RT * 128)) * H;
     dim3 grid(items < dev.sm_count ? items : dev.sm_count);
-    attn_v_tc_kernel<DN, A_SIGNED><<<grid, kTcThreads, smem_bytes, stream>>>(amap, bmap, ymap, max_bits, e1, e2, e_off, H, M,
+    attn_v_tc_kernel<DN, A_SIGNED, RT><<<grid, kTcThreads, smem_bytes, stream>>>(amap, bmap, ymap, max_bits, e1, e2, e_off, H, M,
                                                                             J, NB, y, ctl);
     return cudaGetLastError();
 }
@@ -552,7 +563,9 @@ cudaError_t launch_attn_v_log2_tc(const int8_t* pcodes, const uint32_t* max_bits
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     return D == 64 ? launch_attn_tc<64, false>(w, vt, max_bits, e_v, nullptr, -7, H, M, J, D, y, ctl, dev, stream)
-                   : launch_attn_tc<128, false>(w, vt, max_bits, e_v, nullptr, -7, H, M, J, D, y, ctl, dev, stream);
+                   : (M % 256 == 0   // items of 256 query rows share every value tile; whole items only
+                          ? launch_attn_tc<128, false, 2>(w, vt, max_bits, e_v, nullptr, -7, H, M, J, D, y, ctl, dev, stream)
+                          : launch_attn_tc<128, false>(w, vt, max_bits, e_v, nullptr, -7, H, M, J, D, y, ctl, dev, stream));
 }
 
 // Query x key: s[h][m][j] = 2^(e_q + e_k) * sum_d q[h][m][d] * k[h][j][d], int8 codes, D = 128.
