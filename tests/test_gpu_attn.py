@@ -79,7 +79,9 @@ def test_attn_bad_shapes_are_refused():
         h.aq_attn_v_log2(pc, mx, torch.zeros((1, 8, 128), dtype=torch.int8, device="cuda"), ev, 8)   # 4-bit codes only
 
 
-@pytest.mark.parametrize("H,M,J,D", [(2, 33, 80, 128), (4, 128, 256, 128), (3, 300, 1040, 64), (1, 5, 16, 64)])
+# the last four: items of 256 query rows (M a multiple of 256, D = 128), and more items than SMs for both item sizes
+@pytest.mark.parametrize("H,M,J,D", [(2, 33, 80, 128), (4, 128, 256, 128), (3, 300, 1040, 64), (1, 5, 16, 64),
+                                     (2, 256, 384, 128), (5, 512, 1040, 128), (40, 1024, 256, 128), (20, 1000, 256, 128)])
 def test_attn_v_log2_tensor_core_path_matches_checker(H, M, J, D):
     h = handle()
     p = _softmax_rows(H, M, J, 55)
