@@ -102,6 +102,42 @@ __device__ __forceinline__ uint32_t log2_factors4(uint32_t c4, bool& bad) {
     return o;
 }
 
+// 4-bit codes in half2 arithmetic. k does not increase with |x|, so k = #{ j in 1..7 : |x| < B_j } with B_j the
+// smallest half whose k is below j. By the integer rule above, k <= j - 1 needs, at exponent Eb - j, a mantissa
+// from t_down on, and at exponent Eb - j + 1 a mantissa above t_up; one exponent lower nothing qualifies, one
+// higher everything does. So B_j = t_down * 2^(Eb - j) when t_down is a mantissa (<= 2047), else
+// (t_up + 1) * 2^(Eb - j + 1), rounded up to a half where it falls between subnormals (the inputs are halves,
+// so that keeps the comparison's outcome). Seven compares and adds for two elements replace the exponent and
+// mantissa arithmetic per element.
+struct Log2Fast {
+    __half2 bound[7];
+};
+__device__ __forceinline__ Log2Fast log2_fast_bounds(int mb, int eb, int t_up, int t_down) {
+    Log2Fast f;
+#pragma unroll
+    for (int j = 1; j <= 7; ++j) {
+        const float b = t_down <= 2047 ? ldexpf((float)t_down, eb - j) : ldexpf((float)max(t_up + 1, 1024), eb - j + 1);
+        f.bound[j - 1] = __half2half2(__float2half_ru(b));
+    }
+    (void)mb;
+    return f;
+}
+// Two halves -> (k + 1) * valid as halves (codes), or 2^(7 - k) * valid (factors); valid = 0 for zero and NaN.
+template <bool FACTORS>
+__device__ __forceinline__ __half2 log2_fast2(__half2 x2, const Log2Fast& f) {
+    const __half2 mag = __habs2(x2);
+    const __half2 valid = __hgt2(mag, __float2half2_rn(0.0f));                // 1 or 0; NaN compares false
+    const __half2 ax = __hmin2(mag, __float2half2_rn(65504.0f));              // Inf counts as the largest finite value (a NaN lane becomes 65504 here and is dropped by valid)
+    __half2 r = __float2half2_rn(FACTORS ? 128.0f : 1.0f);
+#pragma unroll
+    for (int j = 0; j < 7; ++j) {
+        const __half2 below = __hlt2(ax, f.bound[j]);                         // 1 or 0
+        if (FACTORS) r = __hfma2(below, __float2half2_rn(-(float)(64 >> j)), r);   // 128 - 64 - 32 - ... = 2^(7 - k)
+        else r = __hadd2(r, below);
+    }
+    return __hmul2(r, valid);
+}
+
 __global__ void __launch_bounds__(256)
 log2_codes_kernel(const __half* __restrict__ x, long long count, int bits, Control* __restrict__ ctl,
                   int8_t* __restrict__ codes, uint32_t* __restrict__ max_bits_out, int as_factors) {
@@ -117,6 +153,34 @@ log2_codes_kernel(const __half* __restrict__ x, long long count, int bits, Contr
     const bool vec = (reinterpret_cast<uintptr_t>(x) & 15u) == 0 && (reinterpret_cast<uintptr_t>(codes) & 7u) == 0;
     const long long nvec = vec ? count / 8 : 0;
     const uint4* xv = reinterpret_cast<const uint4*>(x);
+    if (bits == 4 && mb_bits != 0) {
+        const Log2Fast fast = log2_fast_bounds(mb, eb, t_up, t_down);
+#pragma unroll 4
+        for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
+            const uint4 d = __ldg(xv + i);
+            const uint32_t w[4] = {d.x, d.y, d.z, d.w};
+            uint32_t m[4];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const __half2 x2 = *reinterpret_cast<const __half2*>(&w[t]);
+                __half2 r;
+                if (as_factors) {
+                    r = log2_fast2<true>(x2, fast);
+                    // a negative input has no factor: recorded, its byte is 0
+                    const __half2 neg = __hlt2(x2, __float2half2_rn(0.0f));
+                    bad |= (*reinterpret_cast<const uint32_t*>(&neg) != 0u);
+                    r = __hfma2(neg, __hneg2(r), r);                                    // r * (1 - neg)
+                    r = __hadd2(r, __float2half2_rn(1024.0f));                           // the integer sits in the low bits
+                } else {
+                    r = log2_fast2<false>(x2, fast);
+                    uint32_t rb = *reinterpret_cast<uint32_t*>(&r) | (w[t] & 0x80008000u);   // Sign(x) * (k + 1)
+                    r = __hadd2(*reinterpret_cast<__half2*>(&rb), __float2half2_rn(1536.0f));   // two's complement in the low byte
+                }
+                m[t] = *reinterpret_cast<uint32_t*>(&r);
+            }
+            *reinterpret_cast<uint2*>(codes + 8 * i) = make_uint2(__byte_perm(m[0], m[1], 0x6420), __byte_perm(m[2], m[3], 0x6420));
+        }
+    } else
 #pragma unroll 4
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
         const uint4 d = __ldg(xv + i);

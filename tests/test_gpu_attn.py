@@ -43,6 +43,29 @@ def test_log2_quantize_matches_checker(bits):
     assert int(mx.item()) == 0 and not codes.any().item()
 
 
+@pytest.mark.parametrize("max_bits", [0x3C00, 0x3DA7, 0x3DA8, 0x3DA9, 0x3A00, 0x7BFF, 0x0400, 0x03FF, 0x0203, 0x0001,
+                                      0x2E66, 0x35A8])
+def test_log2_quantize_4bit_every_half_below_a_maximum(max_bits):
+    """The 4-bit route compares halves against seven bounds derived from the maximum: every half pattern of both
+    signs up to the maximum (normal, subnormal, around the sqrt(2) mantissa boundary 0x5A8 of the rounding rule,
+    and subnormal maxima), codes and byte factors, against the checker."""
+    h = handle()
+    mags = np.arange(0, max_bits + 1, dtype=np.uint16)
+    bits16 = np.concatenate([mags, mags | np.uint16(0x8000)])
+    pad = (-len(bits16)) % 8
+    bits16 = np.concatenate([bits16, np.zeros(pad, np.uint16)])
+    x = bits16.view(np.float16)
+    codes, mx = h.aq_log2_quantize(dev(x), 4)
+    ref, mref = oracle.log2_quantize(x, 4)
+    assert (int(mx.item()) & 0xFFFF) == max_bits == int(np.float16(mref).view(np.uint16))
+    assert np.array_equal(codes.cpu().numpy(), ref)
+    xp = np.concatenate([mags, np.zeros((-len(mags)) % 8, np.uint16)]).view(np.float16)      # non-negative only
+    f, _, _ = h.aq_log2_quantize_factors(dev(xp))
+    rp, _ = oracle.log2_quantize(xp, 4)
+    want = np.where(rp > 0, 128 >> np.maximum(rp.astype(np.int32) - 1, 0), 0).astype(np.uint8)
+    assert np.array_equal(f.cpu().numpy().view(np.uint8), want)
+
+
 @pytest.mark.parametrize("H,M,J,D", [(2, 33, 70, 128), (4, 128, 256, 128), (1, 5, 9, 256)])
 def test_attn_v_log2_matches_checker(H, M, J, D):
     bits = 4
