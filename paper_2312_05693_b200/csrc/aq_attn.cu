@@ -286,6 +286,33 @@ transpose_i8_kernel(const int8_t* __restrict__ in, int J, int D, int8_t* __restr
     }
 }
 
+// The same through a 64 x 64 tile with 4-byte accesses on both sides (D and J multiples of 4, 4-byte aligned
+// buffers): a warp reads and writes 64-byte row pieces as words instead of 32 single bytes.
+__global__ void __launch_bounds__(256)
+transpose_i8_words_kernel(const int8_t* __restrict__ in, int J, int D, int8_t* __restrict__ out) {
+    __shared__ __align__(4) int8_t tile[64][68];                      // [j][d], rows padded to 68 bytes
+    const int h = blockIdx.z, j0 = blockIdx.x * 64, d0 = blockIdx.y * 64;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int idx = (int)threadIdx.x + 256 * k, r = idx >> 4, c = 4 * (idx & 15);
+        const int j = j0 + r, d = d0 + c;
+        uint32_t w = 0u;
+        if (j < J && d < D) w = *reinterpret_cast<const uint32_t*>(in + ((size_t)h * J + j) * D + d);
+        *reinterpret_cast<uint32_t*>(&tile[r][c]) = w;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const int idx = (int)threadIdx.x + 256 * k, r = idx >> 4, c = 4 * (idx & 15);      // output row d0 + r, columns j0 + c..
+        const int d = d0 + r, j = j0 + c;
+        if (d < D && j < J) {
+            const uint32_t w = (uint32_t)(uint8_t)tile[c][r] | ((uint32_t)(uint8_t)tile[c + 1][r] << 8) |
+                               ((uint32_t)(uint8_t)tile[c + 2][r] << 16) | ((uint32_t)(uint8_t)tile[c + 3][r] << 24);
+            *reinterpret_cast<uint32_t*>(out + ((size_t)h * D + d) * J + j) = w;
+        }
+    }
+}
+
 constexpr int kTcStages = 4;
 constexpr int kTcThreads = 192;                      // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
 constexpr unsigned long long kTcWaitCycles = 4000000000ull;
@@ -623,7 +650,10 @@ cudaError_t launch_attn_v_log2_tc(const int8_t* pcodes, const uint32_t* max_bits
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
     }
-    transpose_i8_kernel<<<dim3((J + 31) / 32, (D + 31) / 32, H), 256, 0, stream>>>(vq, J, D, vt);
+    if (J % 4 == 0 && D % 4 == 0 && (reinterpret_cast<uintptr_t>(vq) & 3u) == 0 && (reinterpret_cast<uintptr_t>(vt) & 3u) == 0)
+        transpose_i8_words_kernel<<<dim3((J + 63) / 64, (D + 63) / 64, H), 256, 0, stream>>>(vq, J, D, vt);
+    else
+        transpose_i8_kernel<<<dim3((J + 31) / 32, (D + 31) / 32, H), 256, 0, stream>>>(vq, J, D, vt);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
     return D == 64 ? launch_attn_tc<64, false>(w, vt, max_bits, e_v, nullptr, -7, H, M, J, D, y, ctl, dev, stream)
