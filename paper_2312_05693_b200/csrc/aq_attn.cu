@@ -314,7 +314,9 @@ transpose_i8_words_kernel(const int8_t* __restrict__ in, int J, int D, int8_t* _
 }
 
 constexpr int kTcStages = 4;
-constexpr int kTcThreads = 192;                      // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2-5: epilogue
+// warp 0: TMA, warp 1: MMA + TMEM owner, then EW epilogue warps (4, or 8: two per quarter of the tensor-memory lanes,
+// each taking half of the columns, for products with one k step per tile, where the epilogue sets the pace)
+constexpr int tc_threads(int ew) { return (2 + ew) * 32; }
 constexpr unsigned long long kTcWaitCycles = 4000000000ull;
 
 __device__ __forceinline__ uint32_t a_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -348,13 +350,13 @@ __device__ __forceinline__ uint64_t a_desc_sw128(uint32_t saddr) {
     return d;
 }
 
-template <int DN, int RT>
+template <int DN, int RT, int EW>
 struct AttnSmem {
     alignas(1024) uint8_t a[kTcStages][RT * 128 * 128];   // weights tile: RT x 128 query rows x 128 j
     alignas(1024) uint8_t b[kTcStages][DN * 128];    // value tile: DN columns x 128 j
     // Output staging: each epilogue warp owns two boxes of 32 rows x 64 halves (128-byte rows, written
     // with the 128-byte swizzle of the store's tensor map), for alternate 64-column chunks.
-    alignas(1024) uint8_t ystage[4][2][32 * 128];
+    alignas(1024) uint8_t ystage[EW][2][32 * 128];
     alignas(8) uint64_t full[kTcStages];
     uint64_t empty[kTcStages];
     uint64_t acc_full[2];                            // MMA -> epilogue, one per accumulator stage
@@ -374,13 +376,15 @@ struct AttnSmem {
 // scale = (max_bits ? the half in its low 16 bits : 1) * 2^(*e1 + (e2 ? *e2 : 0) + e_off).
 // Used for attention x value (A = byte factors of the log2 codes, B = transposed value codes, k = key
 // index) and for the query x key product (A, B = int8 codes, k = head dimension).
-template <int DN, bool A_SIGNED, int RT = 1>
-__global__ void __launch_bounds__(kTcThreads, 1)
+template <int DN, bool A_SIGNED, int RT = 1, int EW = 4>
+__global__ void __launch_bounds__(tc_threads(EW), 1)
 attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__ CUtensorMap b_map,
                  const __grid_constant__ CUtensorMap y_map, const uint32_t* __restrict__ max_bits, const int32_t* __restrict__ e1, const int32_t* __restrict__ e2,
                  int e_off, int H, int M, int J /* length of k */, int NB, __half* __restrict__ y, Control* __restrict__ ctl) {
     extern __shared__ uint8_t attn_smem_raw[];
-    using Smem = AttnSmem<DN, RT>;
+    using Smem = AttnSmem<DN, RT, EW>;
+    static_assert(EW == 4 || (EW == 8 && DN % 64 == 0), "epilogue warps: one or two per lane quarter");
+    constexpr int kColsPerWarp = DN / (EW / 4);                          // columns an epilogue warp drains
     static_assert(2 * RT * DN <= 512, "two accumulator stages of RT x DN columns in tensor memory");
     constexpr int kRows = RT * 128;                                       // rows of A per item
     Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(attn_smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -396,7 +400,7 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
         }
         for (int a = 0; a < 2; ++a) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(a_smem_u32(&sm.acc_full[a])) : "memory");
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 4;" ::"r"(a_smem_u32(&sm.acc_empty[a])) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(a_smem_u32(&sm.acc_empty[a])), "r"(EW) : "memory");
         }
         sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -494,7 +498,7 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
             for (int r = 0; r < RT; ++r) {
             const int m0 = m0_item + r * 128, m = m0 + quarter * 32 + lane;          // this accumulator's 128 rows
 #pragma unroll 1
-            for (int c0 = 0; c0 < DN; c0 += 32) {
+            for (int c0 = ((warp - 2) >> 2) * kColsPerWarp; c0 < (((warp - 2) >> 2) + 1) * kColsPerWarp; c0 += 32) {
                 uint32_t v[32];
                 asm volatile(
                     "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -532,7 +536,7 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
                     // the box is about to be rewritten: the store that used it last must have read it (with two
                     // boxes in rotation one younger store may still be pending)
                     if (lane == 0) {
-                        if (DN > 64) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                        if (kColsPerWarp > 64) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                         else asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                     }
                     __syncwarp();
@@ -546,7 +550,7 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
                     const int chunk = half_of_box * 4 + q8;
                     *reinterpret_cast<uint4*>(srow + ((chunk ^ (lane & 7)) << 4)) = *reinterpret_cast<uint4*>(o);
                 }
-                if (half_of_box == 1 || c0 + 32 >= DN) {
+                if (half_of_box == 1 || c0 + 32 >= DN) {   // (a warp's column range ends on a box boundary or at DN)
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                     __syncwarp();
                     const int col = n0 + (c0 & ~63);
@@ -583,14 +587,14 @@ typedef CUresult (*AttnEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, 
                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-template <int DN, bool A_SIGNED, int RT = 1>
+template <int DN, bool A_SIGNED, int RT = 1, int EW = 4>
 cudaError_t launch_attn_tc(const void* w, const int8_t* vt, const uint32_t* max_bits, const int32_t* e1, const int32_t* e2,
                            int e_off, int H, int M, int J, int NB, __half* y, Control* ctl, const DeviceInfo& dev,
                            cudaStream_t stream) {
-    using Smem = AttnSmem<DN, RT>;
+    using Smem = AttnSmem<DN, RT, EW>;
     const size_t smem_bytes = sizeof(Smem) + 1024;
     static SmemOptIn opt_in;
-    if (const cudaError_t e = opt_in.ensure(attn_v_tc_kernel<DN, A_SIGNED, RT>, dev.device, smem_bytes); e != cudaSuccess)
+    if (const cudaError_t e = opt_in.ensure(attn_v_tc_kernel<DN, A_SIGNED, RT, EW>, dev.device, smem_bytes); e != cudaSuccess)
         return e;
     CUtensorMap amap, bmap;
     const cuuint32_t estr[2] = {1u, 1u};
@@ -618,7 +622,7 @@ cudaError_t launch_attn_tc(const void* w, const int8_t* vt, const uint32_t* max_
         return cudaErrorInvalidValue;
     const int items = ((M + RT * 128 - 1) / (RT * 128)) * H;
     dim3 grid(items < dev.sm_count ? items : dev.sm_count);
-    attn_v_tc_kernel<DN, A_SIGNED, RT><<<grid, kTcThreads, smem_bytes, stream>>>(amap, bmap, ymap, max_bits, e1, e2, e_off, H, M,
+    attn_v_tc_kernel<DN, A_SIGNED, RT, EW><<<grid, tc_threads(EW), smem_bytes, stream>>>(amap, bmap, ymap, max_bits, e1, e2, e_off, H, M,
                                                                             J, NB, y, ctl);
     return cudaGetLastError();
 }
@@ -665,7 +669,8 @@ cudaError_t launch_attn_v_log2_tc(const int8_t* pcodes, const uint32_t* max_bits
 // Query x key: s[h][m][j] = 2^(e_q + e_k) * sum_d q[h][m][d] * k[h][j][d], int8 codes, D = 128.
 cudaError_t launch_attn_qk_tc(const int8_t* qc, const int32_t* e_q, const int8_t* kc, const int32_t* e_k, int H, int M,
                               int J, int D, __half* s_out, Control* ctl, const DeviceInfo& dev, cudaStream_t stream) {
-    return launch_attn_tc<128, true>(qc, kc, nullptr, e_q, e_k, 0, H, M, D, J, s_out, ctl, dev, stream);
+    // one k step per tile (k = D = 128): the epilogue, 64 KB of scores per tile and row block, sets the pace
+    return launch_attn_tc<128, true, 1, 8>(qc, kc, nullptr, e_q, e_k, 0, H, M, D, J, s_out, ctl, dev, stream);
 }
 
 cudaError_t launch_log2_quantize(const __half* x, long long count, int bits, Control* ctl, int8_t* codes,
