@@ -838,6 +838,10 @@ def main():
                 "achieved": statistics.mean(d["GBps"] for d in line["decode"]), "frac": statistics.mean(fr),
                 "frac_min": min(fr), "frac_max": max(fr),
                 "algorithmic_bytes": "N*K/2 + 2*N + M*K + 2*M*N per launch", "cases": len(fr)}
+            fs = [d["weights_stable"]["frac_of_hbm_peak"] for d in line["decode"]]
+            # the same launches under the caller's promise that nothing in flight writes the weights (off by default)
+            line["decode_roofline"]["with_weights_stable_promise"] = {"frac": statistics.mean(fs), "frac_min": min(fs),
+                                                                      "frac_max": max(fs)}
         except Exception as ex:  # report, do not hide
             line["decode"] = {"error": repr(ex)}
     if rank == 0 and world == 1 and not args.no_decode:
