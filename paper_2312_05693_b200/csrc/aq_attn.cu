@@ -249,26 +249,6 @@ attn_v_log2_kernel(const int8_t* __restrict__ pcodes, const uint32_t* __restrict
 // operands stored j-major. tcgen05.mma kind::i8 reads both from shared memory (128-byte swizzle,
 // staged by TMA); the accumulator [128 query rows x D] lives in tensor memory.
 
-__global__ void __launch_bounds__(256)
-log2_weights_kernel(const int8_t* __restrict__ codes, long long count, uint8_t* __restrict__ w, Control* __restrict__ ctl) {
-    bool bad = false;
-    const bool vec = (reinterpret_cast<uintptr_t>(codes) & 15u) == 0;       // w is 256-byte aligned scratch
-    const long long nvec = vec ? count / 16 : 0;
-    const uint4* cv = reinterpret_cast<const uint4*>(codes);
-    uint4* wv = reinterpret_cast<uint4*>(w);
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (long long)gridDim.x * blockDim.x) {
-        const uint4 c = __ldg(cv + i);
-        wv[i] = make_uint4(log2_factors4(c.x, bad), log2_factors4(c.y, bad), log2_factors4(c.z, bad), log2_factors4(c.w, bad));
-    }
-    if (blockIdx.x == 0 && threadIdx.x == 0)
-        for (long long t = nvec * 16; t < count; ++t) {
-            const int c = codes[t];
-            w[t] = c > 0 ? (uint8_t)(128u >> (c - 1)) : 0;
-            bad |= c < 0;
-        }
-    if (bad) atomicCAS(&ctl->status, 0u, 11u);
-}
-
 // [H][J][D] int8 -> [H][D][J] int8 through a 32 x 32 shared-memory tile.
 __global__ void __launch_bounds__(256)
 transpose_i8_kernel(const int8_t* __restrict__ in, int J, int D, int8_t* __restrict__ out) {
@@ -316,7 +296,7 @@ transpose_i8_words_kernel(const int8_t* __restrict__ in, int J, int D, int8_t* _
 constexpr int kTcStages = 4;
 // warp 0: TMA, warp 1: MMA + TMEM owner, then EW epilogue warps (4, or 8: two per quarter of the tensor-memory lanes,
 // each taking half of the columns, for products with one k step per tile, where the epilogue sets the pace)
-constexpr int tc_threads(int ew) { return (2 + ew) * 32; }
+constexpr int tc_threads(int ew, bool convert = false) { return (2 + ew + (convert ? 4 : 0)) * 32; }
 constexpr unsigned long long kTcWaitCycles = 4000000000ull;
 
 __device__ __forceinline__ uint32_t a_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -359,6 +339,7 @@ struct AttnSmem {
     alignas(1024) uint8_t ystage[EW][2][32 * 128];
     alignas(8) uint64_t full[kTcStages];
     uint64_t empty[kTcStages];
+    uint64_t conv[kTcStages];                        // CONVERT: the A tile of the stage holds byte factors -> MMA
     uint64_t acc_full[2];                            // MMA -> epilogue, one per accumulator stage
     uint64_t acc_empty[2];                           // epilogue (4 warps) -> MMA
     uint32_t tmem_base;
@@ -372,12 +353,14 @@ struct AttnSmem {
 // while the epilogue of the last tile of this one still writes (a CTA's 16 k steps of one item alone were
 // mostly fill and drain). With RT = 2 an item is 256 rows of A, two accumulators of 128 rows that share
 // every tile of B: what limits this kernel is the L2 -> SM path, and the B tile is then fetched once for
-// twice the rows. A is unsigned or signed bytes, B signed.
+// twice the rows. A is unsigned or signed bytes, B signed. CONVERT: A arrives as 4-bit log2 codes (c = k + 1,
+// 0 for a zero) and four more warps turn every landed A tile into byte factors 128 >> k in place before the
+// MMA reads it, so that attention x value needs no conversion pass over the probabilities in memory.
 // scale = (max_bits ? the half in its low 16 bits : 1) * 2^(*e1 + (e2 ? *e2 : 0) + e_off).
 // Used for attention x value (A = byte factors of the log2 codes, B = transposed value codes, k = key
 // index) and for the query x key product (A, B = int8 codes, k = head dimension).
-template <int DN, bool A_SIGNED, int RT = 1, int EW = 4>
-__global__ void __launch_bounds__(tc_threads(EW), 1)
+template <int DN, bool A_SIGNED, int RT = 1, int EW = 4, bool CONVERT = false>
+__global__ void __launch_bounds__(tc_threads(EW, CONVERT), 1)
 attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constant__ CUtensorMap b_map,
                  const __grid_constant__ CUtensorMap y_map, const uint32_t* __restrict__ max_bits, const int32_t* __restrict__ e1, const int32_t* __restrict__ e2,
                  int e_off, int H, int M, int J /* length of k */, int NB, __half* __restrict__ y, Control* __restrict__ ctl) {
@@ -397,6 +380,7 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
         for (int s = 0; s < kTcStages; ++s) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(a_smem_u32(&sm.full[s])) : "memory");
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(a_smem_u32(&sm.empty[s])) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 4;" ::"r"(a_smem_u32(&sm.conv[s])) : "memory");
         }
         for (int a = 0; a < 2; ++a) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(a_smem_u32(&sm.acc_full[a])) : "memory");
@@ -454,7 +438,7 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
               if (!ok) break;
               for (int jb = 0; jb < JB && ok; ++jb, ++it) {
                 const int s = it % kTcStages;
-                ok = a_wait(&sm.full[s], (it / kTcStages) & 1, abort_flag);
+                ok = a_wait(CONVERT ? &sm.conv[s] : &sm.full[s], (it / kTcStages) & 1, abort_flag);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint64_t adesc = a_desc_sw128(a_smem_u32(sm.a[s]));
@@ -481,6 +465,47 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
                              ::"r"(a_smem_u32(&sm.acc_full[a])) : "memory");
             }
         }
+    } else if (CONVERT && warp >= 2 + EW) {
+        // ---- codes -> byte factors, in place, on every A tile that has landed (the map is bytewise, so the
+        // tile's swizzle does not matter). Per 32-bit word: a byte permute looks the factors of codes 1..7 up
+        // by the codes' low three bits, code 8 (k = 7) is added as 1, codes above 8 and negative codes give 0,
+        // and a negative code is recorded (status 11) as the conversion pass does.
+        const int cw = warp - (2 + EW);                                       // 0..3
+        bool bad = false;
+        int it = 0;
+        bool ok = true;
+        for (int w = blockIdx.x; w < items && ok; w += gridDim.x) {
+            for (int i = 0; i < NT * JB && ok; ++i, ++it) {
+                const int s = it % kTcStages;
+                ok = __all_sync(0xFFFFFFFFu, a_wait(&sm.full[s], (it / kTcStages) & 1, abort_flag) ? 1 : 0) != 0;
+                if (!ok) break;
+                uint4* tile = reinterpret_cast<uint4*>(sm.a[s]);
+#pragma unroll 4
+                for (int v = cw * 32 + lane; v < kRows * 128 / 16; v += 128) {
+                    uint4 c = tile[v];
+                    uint32_t* cwds = reinterpret_cast<uint32_t*>(&c);
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        const uint32_t x = cwds[t];
+                        const uint32_t neg = x & 0x80808080u;
+                        const uint32_t x7 = x & 0x7F7F7F7Fu;
+                        const uint32_t big = (x7 + 0x77777777u) & 0x80808080u;          // bytes from 9 up
+                        const uint32_t low = x & 0x07070707u;
+                        const uint32_t sel = __byte_perm(low | (low >> 4), 0u, 0x4420);   // four 3-bit indices as nibbles
+                        uint32_t r = __byte_perm(0x20408000u, 0x02040810u, sel);          // index 0..7 -> 0, 128, 64, ..., 2
+                        r |= (x7 >> 3) & 0x01010101u;                                     // code 8 -> 1 (9..15 are cleared below)
+                        const uint32_t kill = ((neg | big) >> 7) * 0xFFu;
+                        cwds[t] = r & ~kill;
+                        bad |= neg != 0u;
+                    }
+                    tile[v] = c;
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes before the tensor core's reads
+                __syncwarp();
+                if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(a_smem_u32(&sm.conv[s])) : "memory");
+            }
+        }
+        if (bad) atomicCAS(&ctl->status, 0u, 11u);
     } else {
         const int quarter = warp & 3;                                     // TMEM lanes this warp may read
         const float pmax = max_bits ? __half2float(__ushort_as_half((unsigned short)(*max_bits & 0xFFFFu))) : 1.0f;
@@ -569,7 +594,7 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
           }
         }
     }
-    if (warp >= 2 && lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // staging rows live until read
+    if (warp >= 2 && warp < 2 + EW && lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // staging rows live until read
     __syncwarp();
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -587,14 +612,14 @@ typedef CUresult (*AttnEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, 
                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-template <int DN, bool A_SIGNED, int RT = 1, int EW = 4>
+template <int DN, bool A_SIGNED, int RT = 1, int EW = 4, bool CONVERT = false>
 cudaError_t launch_attn_tc(const void* w, const int8_t* vt, const uint32_t* max_bits, const int32_t* e1, const int32_t* e2,
                            int e_off, int H, int M, int J, int NB, __half* y, Control* ctl, const DeviceInfo& dev,
                            cudaStream_t stream) {
     using Smem = AttnSmem<DN, RT, EW>;
     const size_t smem_bytes = sizeof(Smem) + 1024;
     static SmemOptIn opt_in;
-    if (const cudaError_t e = opt_in.ensure(attn_v_tc_kernel<DN, A_SIGNED, RT, EW>, dev.device, smem_bytes); e != cudaSuccess)
+    if (const cudaError_t e = opt_in.ensure(attn_v_tc_kernel<DN, A_SIGNED, RT, EW, CONVERT>, dev.device, smem_bytes); e != cudaSuccess)
         return e;
     CUtensorMap amap, bmap;
     const cuuint32_t estr[2] = {1u, 1u};
@@ -622,7 +647,7 @@ cudaError_t launch_attn_tc(const void* w, const int8_t* vt, const uint32_t* max_
         return cudaErrorInvalidValue;
     const int items = ((M + RT * 128 - 1) / (RT * 128)) * H;
     dim3 grid(items < dev.sm_count ? items : dev.sm_count);
-    attn_v_tc_kernel<DN, A_SIGNED, RT, EW><<<grid, tc_threads(EW), smem_bytes, stream>>>(amap, bmap, ymap, max_bits, e1, e2, e_off, H, M,
+    attn_v_tc_kernel<DN, A_SIGNED, RT, EW, CONVERT><<<grid, tc_threads(EW, CONVERT), smem_bytes, stream>>>(amap, bmap, ymap, max_bits, e1, e2, e_off, H, M,
                                                                             J, NB, y, ctl);
     return cudaGetLastError();
 }
@@ -647,23 +672,23 @@ cudaError_t launch_attn_v_log2_tc(const int8_t* pcodes, const uint32_t* max_bits
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
     cudaError_t e = cudaSuccess;
-    if (p_is_factors) {
-        w = const_cast<uint8_t*>(reinterpret_cast<const uint8_t*>(pcodes));
-    } else {
-        log2_weights_kernel<<<(unsigned int)blocks, 256, 0, stream>>>(pcodes, count, w, ctl);
-        e = cudaGetLastError();
-        if (e != cudaSuccess) return e;
-    }
+    // codes or byte factors: the product kernel reads either (codes are converted tile by tile in shared memory)
+    w = const_cast<uint8_t*>(reinterpret_cast<const uint8_t*>(pcodes));
+    (void)count; (void)blocks;
     if (J % 4 == 0 && D % 4 == 0 && (reinterpret_cast<uintptr_t>(vq) & 3u) == 0 && (reinterpret_cast<uintptr_t>(vt) & 3u) == 0)
         transpose_i8_words_kernel<<<dim3((J + 63) / 64, (D + 63) / 64, H), 256, 0, stream>>>(vq, J, D, vt);
     else
         transpose_i8_kernel<<<dim3((J + 31) / 32, (D + 31) / 32, H), 256, 0, stream>>>(vq, J, D, vt);
     e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    return D == 64 ? launch_attn_tc<64, false>(w, vt, max_bits, e_v, nullptr, -7, H, M, J, D, y, ctl, dev, stream)
-                   : (M % 256 == 0   // items of 256 query rows share every value tile; whole items only
-                          ? launch_attn_tc<128, false, 2>(w, vt, max_bits, e_v, nullptr, -7, H, M, J, D, y, ctl, dev, stream)
-                          : launch_attn_tc<128, false>(w, vt, max_bits, e_v, nullptr, -7, H, M, J, D, y, ctl, dev, stream));
+    const bool wide_items = M % 256 == 0;       // items of 256 query rows share every value tile; whole items only
+    if (p_is_factors)
+        return D == 64 ? launch_attn_tc<64, false>(w, vt, max_bits, e_v, nullptr, -7, H, M, J, D, y, ctl, dev, stream)
+               : wide_items ? launch_attn_tc<128, false, 2>(w, vt, max_bits, e_v, nullptr, -7, H, M, J, D, y, ctl, dev, stream)
+                            : launch_attn_tc<128, false>(w, vt, max_bits, e_v, nullptr, -7, H, M, J, D, y, ctl, dev, stream);
+    return D == 64 ? launch_attn_tc<64, false, 1, 4, true>(w, vt, max_bits, e_v, nullptr, -7, H, M, J, D, y, ctl, dev, stream)
+           : wide_items ? launch_attn_tc<128, false, 2, 4, true>(w, vt, max_bits, e_v, nullptr, -7, H, M, J, D, y, ctl, dev, stream)
+                        : launch_attn_tc<128, false, 1, 4, true>(w, vt, max_bits, e_v, nullptr, -7, H, M, J, D, y, ctl, dev, stream);
 }
 
 // Query x key: s[h][m][j] = 2^(e_q + e_k) * sum_d q[h][m][d] * k[h][j][d], int8 codes, D = 128.
