@@ -280,8 +280,8 @@ int aq_attn_v_log2(aq_handle_t h, const int8_t* p_codes, const uint32_t* p_max_b
 /* The same result on the tensor cores for a non-negative P (a softmax output), 4-bit codes: the factor
  * 2^(kmax - k) is then an unsigned byte and the sums are a u8 x s8 -> s32 contraction over j
  * (tcgen05.mma kind::i8, operands staged by TMA, accumulator in tensor memory). D is 64 or 128,
- * J % 16 == 0; y must be 16-byte aligned. The workspace (aq_attn_workspace_bytes) holds a control block,
- * the byte factors and the transposed value codes. A negative code in P is an error: it is counted as 0
+ * J % 16 == 0; y must be 16-byte aligned. The workspace (aq_attn_workspace_bytes) holds a control block
+ * and the transposed value codes (the codes of P become byte factors tile by tile inside the product kernel). A negative code in P is an error: it is counted as 0
  * and aq_check_workspace on this workspace then returns AQ_ERR_INVALID_ARG. */
 /* Query x key scores on int8 (or 4-bit, stored in int8) codes of aq_quantize_act, reduction over the head
  * dimension (Sec. 5.1): s[h,m,j] = fp16( 2^(e_q + e_k) * sum_d q[h,m,d] * k[h,j,d] ), q [H,M,D], k [H,J,D],

@@ -655,26 +655,20 @@ cudaError_t launch_attn_tc(const void* w, const int8_t* vt, const uint32_t* max_
 }  // namespace
 
 size_t attn_tc_scratch_bytes(int H, int M, int J, int D) {
-    const size_t a = ((size_t)H * M * J + 255) / 256 * 256, b = ((size_t)H * D * J + 255) / 256 * 256;
-    return a + b;
+    (void)M;
+    return ((size_t)H * D * J + 255) / 256 * 256;
 }
 
-// scratch: [weights H*M*J, padded to 256][transposed value codes H*D*J]
-// p_is_factors: pcodes already holds the byte factors (written by the log2 kernel), no conversion pass.
+// scratch: the transposed value codes, H*D*J bytes.
+// p_is_factors: pcodes already holds the byte factors (written by the log2 kernel); otherwise the product kernel
+// converts the codes tile by tile in shared memory.
 cudaError_t launch_attn_v_log2_tc(const int8_t* pcodes, const uint32_t* max_bits, const int8_t* vq, const int32_t* e_v,
                                   int H, int M, int J, int D, __half* y, Control* ctl, void* scratch,
                                   const DeviceInfo& dev, cudaStream_t stream, bool p_is_factors) {
-    uint8_t* w = static_cast<uint8_t*>(scratch);
-    int8_t* vt = reinterpret_cast<int8_t*>(w + ((size_t)H * M * J + 255) / 256 * 256);
-    const long long count = (long long)H * M * J;
-    long long blocks = (count / 16 + 255) / 256;
-    const long long cap = (long long)dev.sm_count * 16;
-    if (blocks > cap) blocks = cap;
-    if (blocks < 1) blocks = 1;
+    int8_t* vt = static_cast<int8_t*>(scratch);
     cudaError_t e = cudaSuccess;
-    // codes or byte factors: the product kernel reads either (codes are converted tile by tile in shared memory)
-    w = const_cast<uint8_t*>(reinterpret_cast<const uint8_t*>(pcodes));
-    (void)count; (void)blocks;
+    // codes or byte factors: the product kernel reads either
+    const uint8_t* w = reinterpret_cast<const uint8_t*>(pcodes);
     if (J % 4 == 0 && D % 4 == 0 && (reinterpret_cast<uintptr_t>(vq) & 3u) == 0 && (reinterpret_cast<uintptr_t>(vt) & 3u) == 0)
         transpose_i8_words_kernel<<<dim3((J + 63) / 64, (D + 63) / 64, H), 256, 0, stream>>>(vq, J, D, vt);
     else
