@@ -439,7 +439,7 @@ def bench_attention(h, reps=5):
             "attn_v_shift": {"us": t_av * 1e3, "Gproducts_per_s": macs / (t_av * 1e-3) / 1e9,
                              "note": "CUDA-core kernel: one shift and one add per product"},
             "attn_v_tensor": {"us": t_tc * 1e3, "TOPS": 2.0 * macs / (t_tc * 1e-3) / 1e12,
-                              "note": "factor conversion + value transpose + tcgen05 u8 x s8 kernel"},
+                              "note": "value transpose + tcgen05 u8 x s8 kernel that turns each tile of codes into byte factors in shared memory"},
             "attn_v_tensor_on_factors": {"us": t_tcf * 1e3, "TOPS": 2.0 * macs / (t_tcf * 1e-3) / 1e12, "log2_quantize_factors_us": t_qf * 1e3,
                                          "note": "byte factors from aq_log2_quantize_factors: value transpose + tcgen05 kernel"}}
 
