@@ -296,7 +296,8 @@ transpose_i8_words_kernel(const int8_t* __restrict__ in, int J, int D, int8_t* _
 constexpr int kTcStages = 4;
 // warp 0: TMA, warp 1: MMA + TMEM owner, then EW epilogue warps (4, or 8: two per quarter of the tensor-memory lanes,
 // each taking half of the columns, for products with one k step per tile, where the epilogue sets the pace)
-constexpr int tc_threads(int ew, bool convert = false) { return (2 + ew + (convert ? 4 : 0)) * 32; }
+constexpr int kConvWarps = 8;                        // warps that turn codes into byte factors (CONVERT)
+constexpr int tc_threads(int ew, bool convert = false) { return (2 + ew + (convert ? kConvWarps : 0)) * 32; }
 constexpr unsigned long long kTcWaitCycles = 4000000000ull;
 
 __device__ __forceinline__ uint32_t a_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -354,7 +355,7 @@ struct AttnSmem {
 // mostly fill and drain). With RT = 2 an item is 256 rows of A, two accumulators of 128 rows that share
 // every tile of B: what limits this kernel is the L2 -> SM path, and the B tile is then fetched once for
 // twice the rows. A is unsigned or signed bytes, B signed. CONVERT: A arrives as 4-bit log2 codes (c = k + 1,
-// 0 for a zero) and four more warps turn every landed A tile into byte factors 128 >> k in place before the
+// 0 for a zero) and kConvWarps more warps turn every landed A tile into byte factors 128 >> k in place before the
 // MMA reads it, so that attention x value needs no conversion pass over the probabilities in memory.
 // scale = (max_bits ? the half in its low 16 bits : 1) * 2^(*e1 + (e2 ? *e2 : 0) + e_off).
 // Used for attention x value (A = byte factors of the log2 codes, B = transposed value codes, k = key
@@ -380,7 +381,7 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
         for (int s = 0; s < kTcStages; ++s) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(a_smem_u32(&sm.full[s])) : "memory");
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(a_smem_u32(&sm.empty[s])) : "memory");
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], 4;" ::"r"(a_smem_u32(&sm.conv[s])) : "memory");
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(a_smem_u32(&sm.conv[s])), "r"(kConvWarps) : "memory");
         }
         for (int a = 0; a < 2; ++a) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(a_smem_u32(&sm.acc_full[a])) : "memory");
@@ -470,7 +471,7 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
         // tile's swizzle does not matter). Per 32-bit word: a byte permute looks the factors of codes 1..7 up
         // by the codes' low three bits, code 8 (k = 7) is added as 1, codes above 8 and negative codes give 0,
         // and a negative code is recorded (status 11) as the conversion pass does.
-        const int cw = warp - (2 + EW);                                       // 0..3
+        const int cw = warp - (2 + EW);                                       // 0..kConvWarps-1
         bool bad = false;
         int it = 0;
         bool ok = true;
@@ -481,7 +482,7 @@ attn_v_tc_kernel(const __grid_constant__ CUtensorMap a_map, const __grid_constan
                 if (!ok) break;
                 uint4* tile = reinterpret_cast<uint4*>(sm.a[s]);
 #pragma unroll 4
-                for (int v = cw * 32 + lane; v < kRows * 128 / 16; v += 128) {
+                for (int v = cw * 32 + lane; v < kRows * 128 / 16; v += kConvWarps * 32) {
                     uint4 c = tile[v];
                     uint32_t* cwds = reinterpret_cast<uint32_t*>(&c);
 #pragma unroll
